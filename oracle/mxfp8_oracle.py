@@ -1,0 +1,202 @@
+"""ctypes/numpy front end of the CPU oracle -- TEST INFRASTRUCTURE, not the product.
+
+The conversion arithmetic lives in ``mxfp8_oracle.c`` (scalar C, binary64); this file
+marshals numpy arrays to it and adds the two pieces that are plain definitions on top
+of it: the 128x4 scale-factor layout (an index permutation) and the block-scaled GEMM
+(two binary64 matrix products over the decoded operands, Sec. 2 and App. A.3).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+E4M3, E5M2 = 0, 1
+RULE_PAPER, RULE_OCP = 0, 1
+ROW, COL = 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mxfp8_oracle.c")
+_SO = os.path.join(_HERE, "libmxfp8_oracle.so")
+_lib = None
+_lock = threading.Lock()
+
+
+def build_oracle(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2, no fast-math) if the library is stale."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + ".%d.tmp" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build_oracle())
+            c_i, c_i64, c_p = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p
+            lib.orc_fp8_decode.restype = ctypes.c_double
+            lib.orc_fp8_decode.argtypes = [c_i, c_i]
+            lib.orc_fp8_encode.restype = c_i
+            lib.orc_fp8_encode.argtypes = [ctypes.c_double, c_i]
+            lib.orc_scale_byte.restype = c_i
+            lib.orc_scale_byte.argtypes = [ctypes.c_float, c_i, c_i]
+            lib.orc_quantize.restype = c_i
+            lib.orc_quantize.argtypes = [c_p, c_i64, c_i64, c_i, c_i, c_i, c_p, c_p]
+            lib.orc_dequantize.restype = c_i
+            lib.orc_dequantize.argtypes = [c_p, c_p, c_i64, c_i64, c_i, c_i, c_p]
+            lib.orc_round_to_f32.restype = None
+            lib.orc_round_to_f32.argtypes = [c_p, c_i64, c_p]
+            lib.orc_round_to_bf16.restype = None
+            lib.orc_round_to_bf16.argtypes = [c_p, c_i64, c_p]
+            _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def fp8_decode(code: int, elem: int = E4M3) -> float:
+    """Value of one FP8 code (Table 1)."""
+    return float(_load().orc_fp8_decode(int(code), elem))
+
+
+def fp8_encode(x: float, elem: int = E4M3) -> int:
+    """Quantize_to_fp8: RNE onto the element grid, saturating (Sec. 3.3, App. A.2)."""
+    return int(_load().orc_fp8_encode(float(x), elem))
+
+
+def scale_byte(amax, elem: int = E4M3, rule: int = RULE_PAPER) -> int:
+    """UE8M0 byte of a block with this amax (Algorithm 1 / App. A.1, or the OCP rule)."""
+    return int(_load().orc_scale_byte(np.float32(amax), elem, rule))
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bfloat16 bit patterns (uint16) to float32."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def quantize(src: np.ndarray, orientation: int, rule: int = RULE_PAPER, elem: int = E4M3):
+    """Convert a [rows, cols] float32 array to MXFP8.
+
+    Returns (q, s): q uint8 [rows, cols]; s uint8 in the linear layout, [rows, cols/32]
+    for ROW blocks and [rows/32, cols] for COL blocks.
+    """
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    rows, cols = src.shape
+    q = np.empty((rows, cols), dtype=np.uint8)
+    s = np.empty((rows, cols // 32) if orientation == ROW else (rows // 32, cols), dtype=np.uint8)
+    rc = _load().orc_quantize(_ptr(src), rows, cols, orientation, rule, elem, _ptr(q), _ptr(s))
+    if rc != 0:
+        raise ValueError("blocked dimension is not a multiple of 32")
+    return q, s
+
+
+def quantize_threads(src: np.ndarray, orientation: int, rule: int, elem: int, threads: int):
+    """The same conversion with row slabs handed to ``threads`` host threads.
+
+    Blocks are independent, so slabs of whole 32-row groups give the same bytes; the C
+    call releases the GIL.  Used by the benchmark's CPU-baseline leg only.
+    """
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    rows, cols = src.shape
+    q = np.empty((rows, cols), dtype=np.uint8)
+    s = np.empty((rows, cols // 32) if orientation == ROW else (rows // 32, cols), dtype=np.uint8)
+    lib = _load()
+    groups = rows // 32
+    bounds = [32 * (groups * t // threads) for t in range(threads + 1)]
+    bounds[-1] = rows
+
+    def work(t):
+        r0, r1 = bounds[t], bounds[t + 1]
+        if r1 <= r0:
+            return
+        s0 = r0 if orientation == ROW else r0 // 32
+        lib.orc_quantize(_ptr(src[r0:r1]), r1 - r0, cols, orientation, rule, elem,
+                         _ptr(q[r0:r1]), _ptr(s[s0:]))
+
+    ths = [threading.Thread(target=work, args=(t,)) for t in range(threads)]
+    for t in ths:
+        t.start()
+    for t in ths:
+        t.join()
+    return q, s
+
+
+def dequantize_f64(q: np.ndarray, s: np.ndarray, orientation: int, elem: int = E4M3) -> np.ndarray:
+    """Decoded values Q*X as float64 (exact), Sec. 2."""
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    s = np.ascontiguousarray(s, dtype=np.uint8)
+    rows, cols = q.shape
+    out = np.empty((rows, cols), dtype=np.float64)
+    rc = _load().orc_dequantize(_ptr(q), _ptr(s), rows, cols, orientation, elem, _ptr(out))
+    if rc != 0:
+        raise ValueError("blocked dimension is not a multiple of 32")
+    return out
+
+
+def dequantize(q, s, orientation: int, elem: int = E4M3, dst: str = "f32") -> np.ndarray:
+    """Decoded values rounded (RNE, once) to float32, or to bfloat16 bit patterns (uint16)."""
+    d = dequantize_f64(q, s, orientation, elem)
+    if dst == "f32":
+        out = np.empty(d.shape, dtype=np.float32)
+        _load().orc_round_to_f32(_ptr(d), d.size, _ptr(out))
+    elif dst == "bf16":
+        out = np.empty(d.shape, dtype=np.uint16)
+        _load().orc_round_to_bf16(_ptr(d), d.size, _ptr(out))
+    else:
+        raise ValueError(dst)
+    return out
+
+
+def sf_offset_swizzled(mn: int, kb: int, n_kblocks: int) -> int:
+    """Byte offset of the scale of (row-or-column mn, K-block kb) in the 128x4 layout.
+
+    The scale matrix, logically [MN, n_kblocks], is cut into atoms of 128 MN-indices by
+    4 K-blocks, 512 bytes each, atoms ordered MN-major-outer / K-inner.  Inside an atom
+    the byte of (mn, kb) sits at (mn % 32) * 16 + ((mn % 128) // 32) * 4 + kb % 4.
+    """
+    atoms_k = (n_kblocks + 3) // 4
+    return ((mn // 128) * atoms_k + kb // 4) * 512 + (mn % 32) * 16 + ((mn % 128) // 32) * 4 + kb % 4
+
+
+def swizzle_scales(s_logical: np.ndarray) -> np.ndarray:
+    """Lay a logical [MN, n_kblocks] scale matrix out in the 128x4 layout (pad bytes 0)."""
+    mn_n, nkb = s_logical.shape
+    out = np.zeros(((mn_n + 127) // 128) * ((nkb + 3) // 4) * 512, dtype=np.uint8)
+    for mn in range(mn_n):
+        for kb in range(nkb):
+            out[sf_offset_swizzled(mn, kb, nkb)] = s_logical[mn, kb]
+    return out
+
+
+def _operand_f64(q, s, major: str, elem: int) -> np.ndarray:
+    """Logical [MN, K] float64 operand.  'k': stored [MN, K], ROW blocks, scales [MN, K/32].
+    'mn': stored [K, MN], COL blocks (blocks run down K), scales [K/32, MN]."""
+    if major == "k":
+        return dequantize_f64(q, s, ROW, elem)
+    return np.ascontiguousarray(dequantize_f64(q, s, COL, elem).T)
+
+
+def gemm_f64(aq, a_s, bq, b_s, a_major: str = "k", b_major: str = "k",
+             a_elem: int = E4M3, b_elem: int = E4M3):
+    """Block-scaled product D[m,n] = sum_k A[m,k] * B[n,k] over the decoded operands.
+
+    Each decoded element is Q*X with X a power of two, so every product of two of them
+    is exact in binary64 and the block-wise application of the scales (Sec. 2, App. A.3)
+    equals the plain product of the decoded matrices.  Returns (D, S) with
+    S[m,n] = sum_k |A[m,k] * B[n,k]|, the magnitude sum the per-element bound uses.
+    """
+    a = _operand_f64(aq, a_s, a_major, a_elem)
+    b = _operand_f64(bq, b_s, b_major, b_elem)
+    with np.errstate(invalid="ignore", over="ignore"):
+        d = a @ b.T
+        sabs = np.abs(a) @ np.abs(b).T
+    return d, sabs
