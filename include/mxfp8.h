@@ -1,0 +1,179 @@
+/*
+ * mxfp8.h -- C ABI of the B200 (sm_100a) MXFP8 conversion + block-scaled GEMM library.
+ *
+ * The operations are those of "Recipes for Pre-training LLMs with MXFP8" (arXiv 2506.08027):
+ * conversion of FP32/BF16 tensors to MXFP8 (Sec. 2, Sec. 3.3, Algorithm 1, App. A.1, A.2),
+ * along rows and/or columns (Sec. 3.2), decoding (Sec. 2), and the block-scaled matrix
+ * product that consumes the result (Sec. 2, App. A.3), optionally re-quantizing its FP32
+ * output to MXFP8 (Sec. 2).
+ *
+ * Conventions shared by every call
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns
+ *     every buffer; the library never allocates, frees or keeps a pointer after returning.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream).  Nothing synchronises except mxfp8_device_status() and the *_host calls.
+ *   - Return value: MXFP8_OK or a negative mxfp8_status.  Nothing is printed, nothing aborts.
+ *   - Tensors are row-major.  A block is K = 32 consecutive elements (Sec. 2) along a row
+ *     (MXFP8_ROW) or down a column (MXFP8_COL).  Quantized data keeps the shape and the
+ *     row-major order of the source in both orientations: one byte per element.
+ *   - A scale is one UE8M0 byte b meaning X = 2^(b-127); b = 0xFF means NaN (Sec. 2).
+ *     mxfp8_quantize never produces 0xFF.
+ *
+ * Scale layouts (the paper leaves the memory layout of the scales open)
+ *   The scales of a tensor form a logical matrix S[mn, kb]: for MXFP8_ROW blocks mn = source
+ *   row and kb = column / 32; for MXFP8_COL blocks mn = source column and kb = row / 32.
+ *   MXFP8_SF_LINEAR   : ROW -> [rows, cols/32] row-major;  COL -> [rows/32, cols] row-major.
+ *   MXFP8_SF_SWIZZLED : what the tensor cores read.  S is cut into atoms of 128 mn x 4 kb
+ *                       (512 bytes); atoms are ordered mn-outer, kb-inner; inside an atom the
+ *                       byte of (mn, kb) is at (mn%32)*16 + ((mn%128)/32)*4 + kb%4.  mn is
+ *                       padded to a multiple of 128 and kb to a multiple of 4; pad bytes are 0.
+ *                       See mxfp8_sf_offset().
+ */
+#ifndef MXFP8_H_
+#define MXFP8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MXFP8_OK = 0,
+    MXFP8_ERR_NULL = -1,           /* a required pointer is NULL                         */
+    MXFP8_ERR_ENUM = -2,           /* an enum argument is out of range                   */
+    MXFP8_ERR_SHAPE = -3,          /* non-positive size, or blocked dimension % 32 != 0   */
+    MXFP8_ERR_ALIGN = -4,          /* a pointer or a row pitch misses its alignment       */
+    MXFP8_ERR_UNSUPPORTED = -5,    /* valid request this build does not implement         */
+    MXFP8_ERR_CUDA = -6,           /* a CUDA runtime/driver call or a launch failed       */
+    MXFP8_ERR_DEVICE_TIMEOUT = -7, /* a bounded wait inside a kernel ran out              */
+    MXFP8_ERR_WORKSPACE = -8       /* workspace missing or too small                      */
+} mxfp8_status;
+
+enum { MXFP8_FP32 = 0, MXFP8_BF16 = 1 };                 /* source / destination dtype   */
+enum { MXFP8_ROW = 1, MXFP8_COL = 2, MXFP8_BOTH = 3 };   /* block orientation (bit mask) */
+enum { MXFP8_RULE_PAPER = 0, MXFP8_RULE_OCP = 1 };       /* scale rounding rule          */
+enum { MXFP8_E4M3 = 0, MXFP8_E5M2 = 1 };                 /* element encoding (Table 1)   */
+enum { MXFP8_SF_LINEAR = 0, MXFP8_SF_SWIZZLED = 1 };     /* scale layout                 */
+enum { MXFP8_K_MAJOR = 0, MXFP8_MN_MAJOR = 1 };          /* GEMM operand storage         */
+
+/*
+ * mxfp8_quantize -- FP32/BF16 -> MXFP8 (Sec. 3.3, Algorithm 1, App. A.1, A.2; two
+ * orientations per Sec. 3.2).
+ *
+ * Per block of 32: amax = max |V_i| over the finite elements (0 if none); scale byte b by
+ *   MXFP8_RULE_PAPER: X = amax/destmax rounded UP to a power of two, at least 2^-127
+ *                     (Algorithm 1, App. A.1);  b = log2(X) + 127;
+ *   MXFP8_RULE_OCP  : exponent floor(log2 amax) - emax(elem), clamped to [-127, 127]
+ *                     (the OCP v1.0 suggestion Sec. 3.3 compares against);
+ * then Q_i = V_i / X rounded to nearest-even on the element grid and saturated to +-destmax
+ * (448 for E4M3, 57344 for E5M2).  NaN elements stay NaN, +-Inf become +-destmax, and neither
+ * enters amax.  FP32 subnormal inputs are honoured (no flush to zero).
+ *
+ *   src          [rows, cols] row-major, dtype MXFP8_FP32 or MXFP8_BF16, 16-byte aligned.
+ *   orientation  MXFP8_ROW (needs cols % 32 == 0), MXFP8_COL (needs rows % 32 == 0) or
+ *                MXFP8_BOTH (needs both); BOTH reads src once.
+ *   q_row, s_row outputs of the ROW orientation (ignored unless orientation & MXFP8_ROW):
+ *                q_row [rows, cols] bytes; s_row mxfp8_scale_bytes(rows, cols, ROW, layout).
+ *   q_col, s_col the same for the COL orientation.
+ *   q_* must be 16-byte aligned, s_* 16-byte aligned; outputs must not overlap src.
+ *   Errors: ERR_NULL, ERR_ENUM, ERR_SHAPE, ERR_ALIGN, ERR_CUDA (launch failure).
+ */
+int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                   int orientation, int scale_rule, int elem,
+                   void* q_row, void* s_row, void* q_col, void* s_col,
+                   int sf_layout, void* stream);
+
+/*
+ * mxfp8_dequantize -- decoded value Q_i * X (Sec. 2), written as FP32 or BF16 (one RNE
+ * rounding of the exact product; overflow gives +-Inf, scale byte 0xFF gives NaN).
+ *   q [rows, cols] bytes; s in `sf_layout` for `orientation` (MXFP8_ROW or MXFP8_COL only);
+ *   dst [rows, cols] of dst_dtype.  Same alignment rules and errors as mxfp8_quantize.
+ */
+int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int64_t cols,
+                     int orientation, int elem, int sf_layout,
+                     void* dst, int dst_dtype, void* stream);
+
+/*
+ * Optional fused epilogue of mxfp8_gemm: the FP32 accumulator tile is converted to MXFP8
+ * exactly as mxfp8_quantize would convert the FP32 output D[M, N] (Sec. 2: the FP32 output is
+ * quantized to MX format when its consumer needs it).  ROW blocks run along N, COL blocks
+ * along M.  Scales are written in MXFP8_SF_SWIZZLED layout.
+ */
+typedef struct {
+    int orientation;   /* MXFP8_ROW, MXFP8_COL or MXFP8_BOTH */
+    int scale_rule;
+    int elem;
+    void* q_row;       /* [M, N] bytes */
+    void* s_row;       /* mxfp8_scale_bytes(M, N, MXFP8_ROW, MXFP8_SF_SWIZZLED) */
+    void* q_col;
+    void* s_col;       /* mxfp8_scale_bytes(M, N, MXFP8_COL, MXFP8_SF_SWIZZLED) */
+} mxfp8_epilogue;
+
+/*
+ * mxfp8_gemm -- block-scaled product on the tensor cores (Sec. 2, App. A.3):
+ *     D[m, n] = sum over K-blocks kb of  2^(sa[m,kb]-127) * 2^(sb[n,kb]-127)
+ *                                        * sum_{k in kb} Aq[m,k] * Bq[n,k],
+ * accumulated in FP32.  A is logically [M, K], B logically [N, K].
+ *   a_major / b_major  MXFP8_K_MAJOR : stored [MN, K] row-major, quantized with ROW blocks;
+ *                      MXFP8_MN_MAJOR: stored [K, MN] row-major, quantized with COL blocks
+ *                      (blocks run down K).  fprop = (K,K), dgrad = (K,MN), wgrad = (MN,MN).
+ *   As, Bs             scales in MXFP8_SF_SWIZZLED layout, logically [MN, K/32] in both cases
+ *                      -- exactly what mxfp8_quantize writes for the matching orientation.
+ *   D                  [M, N] row-major, out_dtype MXFP8_FP32 or MXFP8_BF16 (RNE); may be NULL
+ *                      when `epi` is given and only the quantized output is wanted.
+ *   epi                NULL, or the fused MXFP8 output described above.
+ *   workspace          device scratch of at least mxfp8_gemm_workspace_bytes(); may be NULL
+ *                      when that is 0.  Contents are undefined afterwards.
+ * Requirements: K % 128 == 0, M % 128 == 0, N % 128 == 0 (else ERR_UNSUPPORTED); K % 32 != 0
+ * is ERR_SHAPE; all pointers 16-byte aligned (operands 128-byte aligned when MN-major).
+ * A bounded wait that expires inside the kernel sets the device status word; read it with
+ * mxfp8_device_status().  The result is deterministic (same inputs, same bytes).
+ */
+int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const void* Bs,
+               int64_t M, int64_t N, int64_t K,
+               int a_major, int b_major, int a_elem, int b_elem,
+               void* D, int out_dtype, const mxfp8_epilogue* epi,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of the scale buffer of a [rows, cols] tensor for one orientation (ROW or COL). */
+size_t mxfp8_scale_bytes(int64_t rows, int64_t cols, int orientation, int sf_layout);
+
+/* Byte offset of scale (mn, kblock) in a scale buffer with n_kblocks K-blocks per mn and
+ * (for LINEAR/COL only) mn_count columns.  LINEAR: ROW uses mn*n_kblocks + kblock; a COL
+ * buffer is addressed by the caller as kblock*mn_count + mn and is not handled here.
+ * SWIZZLED: the 128x4 atom formula in the header comment.  Host helper, no device work. */
+int64_t mxfp8_sf_offset(int64_t mn, int64_t kblock, int64_t n_kblocks, int sf_layout);
+
+/* Scratch bytes mxfp8_gemm needs for this problem (0 when none). */
+size_t mxfp8_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int out_dtype, int has_epilogue);
+
+/* Waits for `stream`, then returns and clears the device status word of the current device:
+ * MXFP8_OK, MXFP8_ERR_DEVICE_TIMEOUT, or MXFP8_ERR_CUDA if the wait itself failed.
+ * This is the only device-pointer call that synchronises. */
+int mxfp8_device_status(void* stream);
+
+/* Human-readable name of a status code (static string). */
+const char* mxfp8_status_string(int status);
+
+/* Number of kernels this library has launched in this process (for launch accounting). */
+int64_t mxfp8_launch_count(void);
+
+/*
+ * Host-buffer variants: the same operations with HOST pointers for inputs and outputs.  The
+ * caller provides a device staging buffer `dev_ws` of at least the returned *_host_ws_bytes;
+ * the call copies inputs host->device, runs the device path, copies results device->host,
+ * all on `stream`, and waits for the stream before returning.  Host buffers should be pinned
+ * for full PCIe bandwidth.  (No counterpart in the paper; provided for end-to-end use.)
+ */
+size_t mxfp8_quantize_host_ws_bytes(int src_dtype, int64_t rows, int64_t cols, int orientation);
+int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64_t cols,
+                        int orientation, int scale_rule, int elem,
+                        void* q_row_host, void* s_row_host, void* q_col_host, void* s_col_host,
+                        int sf_layout, void* dev_ws, size_t dev_ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXFP8_H_ */

@@ -1,0 +1,189 @@
+"""Thin ctypes binding of libmxfp8.so: argument marshalling only.
+
+Every function has the name and argument order of its C entry point in ``include/mxfp8.h``
+and takes torch tensors (device memory) where C takes device pointers.  Nothing here
+computes: a missing library or a non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+FP32, BF16 = 0, 1
+ROW, COL, BOTH = 1, 2, 3
+RULE_PAPER, RULE_OCP = 0, 1
+E4M3, E5M2 = 0, 1
+SF_LINEAR, SF_SWIZZLED = 0, 1
+K_MAJOR, MN_MAJOR = 0, 1
+
+EXPORTS = (
+    "mxfp8_quantize", "mxfp8_dequantize", "mxfp8_gemm", "mxfp8_scale_bytes", "mxfp8_sf_offset",
+    "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
+    "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
+)
+
+
+class Mxfp8Error(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__("%s failed: %d (%s)" % (what, status, status_string(status)))
+        self.status = status
+
+
+class _Epilogue(ctypes.Structure):
+    _fields_ = [("orientation", ctypes.c_int), ("scale_rule", ctypes.c_int), ("elem", ctypes.c_int),
+                ("q_row", ctypes.c_void_p), ("s_row", ctypes.c_void_p),
+                ("q_col", ctypes.c_void_p), ("s_col", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) the CUDA library; fail loudly."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if os.environ.get("MXFP8_NO_BUILD") != "1":
+            path = _build.build()
+        if not os.path.exists(path):
+            raise ImportError("libmxfp8.so is missing: run `python -m paper_2506_08027_b200.build`")
+        L = ctypes.CDLL(path)
+        i, i64, p, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+        L.mxfp8_quantize.restype = i
+        L.mxfp8_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p]
+        L.mxfp8_dequantize.restype = i
+        L.mxfp8_dequantize.argtypes = [p, p, i64, i64, i, i, i, p, i, p]
+        L.mxfp8_gemm.restype = i
+        L.mxfp8_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, p, i, ctypes.POINTER(_Epilogue), p, sz, p]
+        L.mxfp8_scale_bytes.restype = sz
+        L.mxfp8_scale_bytes.argtypes = [i64, i64, i, i]
+        L.mxfp8_sf_offset.restype = i64
+        L.mxfp8_sf_offset.argtypes = [i64, i64, i64, i]
+        L.mxfp8_gemm_workspace_bytes.restype = sz
+        L.mxfp8_gemm_workspace_bytes.argtypes = [i64, i64, i64, i, i]
+        L.mxfp8_device_status.restype = i
+        L.mxfp8_device_status.argtypes = [p]
+        L.mxfp8_status_string.restype = ctypes.c_char_p
+        L.mxfp8_status_string.argtypes = [i]
+        L.mxfp8_launch_count.restype = i64
+        L.mxfp8_launch_count.argtypes = []
+        L.mxfp8_quantize_host_ws_bytes.restype = sz
+        L.mxfp8_quantize_host_ws_bytes.argtypes = [i, i64, i64, i]
+        L.mxfp8_quantize_host.restype = i
+        L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().mxfp8_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise Mxfp8Error(status, what)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return FP32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("source must be float32 or bfloat16")
+
+
+def mxfp8_scale_bytes(rows: int, cols: int, orientation: int, sf_layout: int) -> int:
+    return int(lib().mxfp8_scale_bytes(rows, cols, orientation, sf_layout))
+
+
+def mxfp8_sf_offset(mn: int, kblock: int, n_kblocks: int, sf_layout: int) -> int:
+    return int(lib().mxfp8_sf_offset(mn, kblock, n_kblocks, sf_layout))
+
+
+def mxfp8_gemm_workspace_bytes(M: int, N: int, K: int, out_dtype: int, has_epilogue: bool) -> int:
+    return int(lib().mxfp8_gemm_workspace_bytes(M, N, K, out_dtype, int(has_epilogue)))
+
+
+def mxfp8_device_status(stream=None) -> int:
+    return int(lib().mxfp8_device_status(_stream(stream)))
+
+
+def mxfp8_launch_count() -> int:
+    return int(lib().mxfp8_launch_count())
+
+
+def alloc_quantize_outputs(rows: int, cols: int, orientation: int, sf_layout: int, device="cuda"):
+    """Caller-side allocation helper: (q_row, s_row, q_col, s_col), None where unused."""
+    out = []
+    for o in (ROW, COL):
+        if orientation & o:
+            out.append(torch.empty((rows, cols), dtype=torch.uint8, device=device))
+            out.append(torch.empty(mxfp8_scale_bytes(rows, cols, o, sf_layout), dtype=torch.uint8, device=device))
+        else:
+            out += [None, None]
+    return tuple(out)
+
+
+def mxfp8_quantize(src: torch.Tensor, orientation: int, scale_rule: int, elem: int,
+                   q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    rows, cols = src.shape
+    assert src.is_contiguous()
+    _check(lib().mxfp8_quantize(_ptr(src), _dtype_code(src), rows, cols, orientation, scale_rule, elem,
+                                _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
+                                _stream(stream)), "mxfp8_quantize")
+
+
+def mxfp8_dequantize(q: torch.Tensor, s: torch.Tensor, orientation: int, elem: int, sf_layout: int,
+                     dst: torch.Tensor, stream=None) -> None:
+    rows, cols = q.shape
+    _check(lib().mxfp8_dequantize(_ptr(q), _ptr(s), rows, cols, orientation, elem, sf_layout,
+                                  _ptr(dst), _dtype_code(dst), _stream(stream)), "mxfp8_dequantize")
+
+
+def make_epilogue(orientation: int, scale_rule: int, elem: int, q_row=None, s_row=None, q_col=None, s_col=None):
+    e = _Epilogue()
+    e.orientation, e.scale_rule, e.elem = orientation, scale_rule, elem
+    e.q_row = None if q_row is None else q_row.data_ptr()
+    e.s_row = None if s_row is None else s_row.data_ptr()
+    e.q_col = None if q_col is None else q_col.data_ptr()
+    e.s_col = None if s_col is None else s_col.data_ptr()
+    e._keep = (q_row, s_row, q_col, s_col)
+    return e
+
+
+def mxfp8_gemm(Aq, As, Bq, Bs, M: int, N: int, K: int, a_major: int, b_major: int, a_elem: int,
+               b_elem: int, D, epi=None, workspace=None, stream=None) -> None:
+    out_dtype = FP32 if D is None else _dtype_code(D)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mxfp8_gemm(_ptr(Aq), _ptr(As), _ptr(Bq), _ptr(Bs), M, N, K, a_major, b_major,
+                            a_elem, b_elem, _ptr(D), out_dtype,
+                            None if epi is None else ctypes.byref(epi),
+                            _ptr(workspace), ws_bytes, _stream(stream)), "mxfp8_gemm")
+
+
+def mxfp8_quantize_host_ws_bytes(src_dtype: int, rows: int, cols: int, orientation: int) -> int:
+    return int(lib().mxfp8_quantize_host_ws_bytes(src_dtype, rows, cols, orientation))
+
+
+def mxfp8_quantize_host(src_host: torch.Tensor, orientation: int, scale_rule: int, elem: int,
+                        q_row_host, s_row_host, q_col_host, s_col_host, sf_layout: int,
+                        dev_ws: torch.Tensor, stream=None) -> None:
+    rows, cols = src_host.shape
+    _check(lib().mxfp8_quantize_host(_ptr(src_host), _dtype_code(src_host), rows, cols, orientation,
+                                     scale_rule, elem, _ptr(q_row_host), _ptr(s_row_host),
+                                     _ptr(q_col_host), _ptr(s_col_host), sf_layout, _ptr(dev_ws),
+                                     dev_ws.numel() * dev_ws.element_size(), _stream(stream)),
+           "mxfp8_quantize_host")

@@ -1,0 +1,98 @@
+// Host helpers of the C ABI: sizes, layout offsets, status strings, host-buffer variant.
+#include "mxfp8_device.cuh"
+#include "mxfp8_host.h"
+
+extern "C" size_t mxfp8_scale_bytes(int64_t rows, int64_t cols, int orientation, int sf_layout)
+{
+    if (rows <= 0 || cols <= 0) return 0;
+    if (orientation != MXFP8_ROW && orientation != MXFP8_COL) return 0;
+    const int64_t mn = (orientation == MXFP8_ROW) ? rows : cols;
+    const int64_t nkb = ((orientation == MXFP8_ROW) ? cols : rows) / 32;
+    if (sf_layout == MXFP8_SF_LINEAR) return (size_t)(mn * nkb);
+    if (sf_layout == MXFP8_SF_SWIZZLED) return (size_t)(((mn + 127) / 128) * ((nkb + 3) / 4) * 512);
+    return 0;
+}
+
+extern "C" int64_t mxfp8_sf_offset(int64_t mn, int64_t kblock, int64_t n_kblocks, int sf_layout)
+{
+    if (mn < 0 || kblock < 0 || n_kblocks <= 0 || kblock >= n_kblocks) return -1;
+    if (sf_layout == MXFP8_SF_LINEAR) return mn * n_kblocks + kblock;
+    if (sf_layout == MXFP8_SF_SWIZZLED) return mxfp8::sf_swizzled_offset(mn, kblock, n_kblocks);
+    return -1;
+}
+
+extern "C" const char* mxfp8_status_string(int status)
+{
+    switch (status) {
+        case MXFP8_OK: return "ok";
+        case MXFP8_ERR_NULL: return "null pointer";
+        case MXFP8_ERR_ENUM: return "bad enum value";
+        case MXFP8_ERR_SHAPE: return "bad shape (non-positive, or blocked dimension not a multiple of 32)";
+        case MXFP8_ERR_ALIGN: return "misaligned pointer";
+        case MXFP8_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MXFP8_ERR_CUDA: return "CUDA error";
+        case MXFP8_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
+        case MXFP8_ERR_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int64_t mxfp8_launch_count(void) { return mxfp8::launches(); }
+
+extern "C" int mxfp8_device_status(void* stream)
+{
+    return mxfp8::read_and_clear_device_status(static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+}
+
+extern "C" size_t mxfp8_quantize_host_ws_bytes(int src_dtype, int64_t rows, int64_t cols, int orientation)
+{
+    if (rows <= 0 || cols <= 0) return 0;
+    const size_t esz = (src_dtype == MXFP8_BF16) ? 2 : 4;
+    size_t total = up256((size_t)rows * cols * esz);
+    for (int o = MXFP8_ROW; o <= MXFP8_COL; ++o)
+        if (orientation & o) total += up256((size_t)rows * cols) + up256(mxfp8_scale_bytes(rows, cols, o, MXFP8_SF_SWIZZLED));
+    return total;
+}
+
+extern "C" int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64_t cols,
+                                   int orientation, int scale_rule, int elem,
+                                   void* q_row_host, void* s_row_host, void* q_col_host, void* s_col_host,
+                                   int sf_layout, void* dev_ws, size_t dev_ws_bytes, void* stream)
+{
+    if (!src_host || !dev_ws) return MXFP8_ERR_NULL;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if (dev_ws_bytes < mxfp8_quantize_host_ws_bytes(src_dtype, rows, cols, orientation)) return MXFP8_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(dev_ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t esz = (src_dtype == MXFP8_BF16) ? 2 : 4;
+    const size_t n = (size_t)rows * cols;
+    char* p = static_cast<char*>(dev_ws);
+    void* d_src = p; p += up256(n * esz);
+    void *d_q[2] = {nullptr, nullptr}, *d_s[2] = {nullptr, nullptr};
+    size_t s_bytes[2] = {0, 0};
+    for (int o = 0; o < 2; ++o)
+        if (orientation & (o + 1)) {
+            s_bytes[o] = mxfp8_scale_bytes(rows, cols, o + 1, sf_layout);
+            d_q[o] = p; p += up256(n);
+            d_s[o] = p; p += up256(mxfp8_scale_bytes(rows, cols, o + 1, MXFP8_SF_SWIZZLED));
+        }
+    if (cudaMemcpyAsync(d_src, src_host, n * esz, cudaMemcpyHostToDevice, st) != cudaSuccess) return MXFP8_ERR_CUDA;
+    const int rc = mxfp8_quantize(d_src, src_dtype, rows, cols, orientation, scale_rule, elem,
+                                  d_q[0], d_s[0], d_q[1], d_s[1], sf_layout, stream);
+    if (rc != MXFP8_OK) return rc;
+    void* h_q[2] = {q_row_host, q_col_host};
+    void* h_s[2] = {s_row_host, s_col_host};
+    for (int o = 0; o < 2; ++o)
+        if (orientation & (o + 1)) {
+            if (!h_q[o] || !h_s[o]) return MXFP8_ERR_NULL;
+            if (cudaMemcpyAsync(h_q[o], d_q[o], n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXFP8_ERR_CUDA;
+            if (cudaMemcpyAsync(h_s[o], d_s[o], s_bytes[o], cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXFP8_ERR_CUDA;
+        }
+    return cudaStreamSynchronize(st) == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}

@@ -1,0 +1,136 @@
+// mxfp8_dequantize: decoded value Q_i * X (Sec. 2) written as FP32 or BF16.
+//
+// Every FP8 value times a power of two has at most 4 significant bits and magnitude at
+// least 2^-136, so the FP32 product below is exact (or overflows to infinity exactly where
+// the real product exceeds the FP32 range); the BF16 result is one RNE rounding of it.
+#include "mxfp8_device.cuh"
+#include "mxfp8_host.h"
+
+namespace mxfp8 {
+namespace {
+
+// X = 2^(b-127) as FP32: b = 0 is the subnormal 2^-127, b = 255 is NaN.
+__device__ __forceinline__ float scale_value(uint32_t b)
+{
+    if (b == 0xFFu) return __uint_as_float(0x7FC00000u);
+    return (b == 0u) ? __uint_as_float(0x00400000u) : __uint_as_float(b << 23);
+}
+
+template <int ELEM, int DST, int ORIENT>
+__global__ void __launch_bounds__(256)
+dequantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, int64_t rows, int64_t cols,
+                  int sf_layout, void* __restrict__ dst_v, int64_t chunks_per_row)
+{
+    // one thread = 16 consecutive elements of a row (or the ragged tail of the row)
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * chunks_per_row) return;
+    const int64_t r = idx / chunks_per_row;
+    const int64_t c0 = (idx % chunks_per_row) * 16;
+    const int n = (int)min((int64_t)16, cols - c0);
+    const bool vec = (n == 16) && ((cols & 15) == 0);
+
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    if (vec) {
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(q + r * cols + c0));
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else {
+        for (int i = 0; i < n; ++i) w[i >> 2] |= (uint32_t)q[r * cols + c0 + i] << (8 * (i & 3));
+    }
+
+    float out[16];
+    float row_scale = 0.f;
+    if (ORIENT == MXFP8_ROW) {
+        const int64_t ncb = cols >> 5, kb = c0 >> 5;
+        const int64_t off = (sf_layout == MXFP8_SF_SWIZZLED) ? sf_swizzled_offset(r, kb, ncb) : r * ncb + kb;
+        row_scale = scale_value(s[off]);
+    }
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        const float2 f = fp8x2_to_float2<ELEM>((w[p >> 1] >> (16 * (p & 1))) & 0xFFFFu);
+        float s0 = row_scale, s1 = row_scale;
+        if (ORIENT == MXFP8_COL) {
+            const int64_t nrb = rows >> 5, kb = r >> 5;
+            const int64_t ca = c0 + 2 * p, cb = c0 + 2 * p + 1;
+            if (2 * p < n)
+                s0 = scale_value(s[(sf_layout == MXFP8_SF_SWIZZLED) ? sf_swizzled_offset(ca, kb, nrb) : kb * cols + ca]);
+            if (2 * p + 1 < n)
+                s1 = scale_value(s[(sf_layout == MXFP8_SF_SWIZZLED) ? sf_swizzled_offset(cb, kb, nrb) : kb * cols + cb]);
+        }
+        out[2 * p] = f.x * s0;
+        out[2 * p + 1] = f.y * s1;
+    }
+
+    if (DST == MXFP8_FP32) {
+        float* d = static_cast<float*>(dst_v) + r * cols + c0;
+        if (vec) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                reinterpret_cast<float4*>(d)[i] = make_float4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+        } else {
+            for (int i = 0; i < n; ++i) d[i] = out[i];
+        }
+    } else {
+        __nv_bfloat16* d = static_cast<__nv_bfloat16*>(dst_v) + r * cols + c0;
+        if (vec) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(out[2 * i], out[2 * i + 1]);
+                pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            reinterpret_cast<uint4*>(d)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            reinterpret_cast<uint4*>(d)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        } else {
+            for (int i = 0; i < n; ++i) d[i] = __float2bfloat16_rn(out[i]);
+        }
+    }
+}
+
+template <int ELEM, int DST, int ORIENT>
+cudaError_t launch(const uint8_t* q, const uint8_t* s, int64_t rows, int64_t cols, int sf_layout,
+                   void* dst, cudaStream_t stream)
+{
+    const int64_t chunks = (cols + 15) / 16;
+    const int64_t blocks = (rows * chunks + 255) / 256;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    dequantize_kernel<ELEM, DST, ORIENT><<<(unsigned)blocks, 256, 0, stream>>>(q, s, rows, cols, sf_layout, dst, chunks);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+template <int ELEM, int DST>
+cudaError_t launch_o(int orient, const uint8_t* q, const uint8_t* s, int64_t rows, int64_t cols,
+                     int sf_layout, void* dst, cudaStream_t stream)
+{
+    return orient == MXFP8_ROW ? launch<ELEM, DST, MXFP8_ROW>(q, s, rows, cols, sf_layout, dst, stream)
+                               : launch<ELEM, DST, MXFP8_COL>(q, s, rows, cols, sf_layout, dst, stream);
+}
+
+}  // namespace
+}  // namespace mxfp8
+
+extern "C" int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int64_t cols,
+                                int orientation, int elem, int sf_layout,
+                                void* dst, int dst_dtype, void* stream)
+{
+    using namespace mxfp8;
+    if (orientation != MXFP8_ROW && orientation != MXFP8_COL) return MXFP8_ERR_ENUM;
+    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (dst_dtype != MXFP8_FP32 && dst_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (!q || !s || !dst) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if (orientation == MXFP8_ROW ? (cols % 32) : (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(s) || !aligned16(dst)) return MXFP8_ERR_ALIGN;
+    const uint8_t* qq = static_cast<const uint8_t*>(q);
+    const uint8_t* ss = static_cast<const uint8_t*>(s);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t err;
+    if (elem == MXFP8_E4M3)
+        err = dst_dtype == MXFP8_FP32 ? launch_o<MXFP8_E4M3, MXFP8_FP32>(orientation, qq, ss, rows, cols, sf_layout, dst, st)
+                                      : launch_o<MXFP8_E4M3, MXFP8_BF16>(orientation, qq, ss, rows, cols, sf_layout, dst, st);
+    else
+        err = dst_dtype == MXFP8_FP32 ? launch_o<MXFP8_E5M2, MXFP8_FP32>(orientation, qq, ss, rows, cols, sf_layout, dst, st)
+                                      : launch_o<MXFP8_E5M2, MXFP8_BF16>(orientation, qq, ss, rows, cols, sf_layout, dst, st);
+    return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}

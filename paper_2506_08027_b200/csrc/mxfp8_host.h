@@ -1,0 +1,26 @@
+// Host-side declarations shared by the translation units of the library (not public).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/mxfp8.h"
+
+namespace mxfp8 {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launch accounting (mxfp8_launch_count).
+int64_t launches();
+void count_launch(int n);
+
+// Device-pointer implementations behind the C entry points (arguments already validated).
+int quantize_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
+                    int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
+                    int sf_layout, cudaStream_t stream);
+
+// Device status word (bounded waits report here); defined in gemm.cu.
+int read_and_clear_device_status(cudaStream_t stream);
+
+}  // namespace mxfp8

@@ -1,0 +1,309 @@
+// mxfp8_quantize: FP32/BF16 -> MXFP8 in row and/or column blocks from ONE read of the source
+// (Sec. 3.2: every tensor is needed blocked along rows and along columns; Sec. 3.3,
+// Algorithm 1, App. A.1/A.2: amax -> UE8M0 scale -> RNE saturating cast).
+//
+// Work decomposition (HBM-bound streaming kernel):
+//   CTA tile  = 128 rows x 128 columns = exactly one 512-byte scale atom per orientation.
+//   warp tile = 32 rows x (32*VEC) columns held entirely in registers: lane l owns VEC
+//               adjacent columns of all 32 rows (VEC = 4 for BF16, 2 for FP32: 8-byte loads,
+//               32 of them in flight per thread).
+//   column blocks: the 32 rows of a column live in one thread -> amax needs no exchange.
+//   row blocks   : 32 columns = 32/VEC adjacent lanes -> amax by xor-shuffles.
+//   Q bytes go straight to global memory (each warp store covers whole 32-byte sectors);
+//   scale bytes are collected in shared memory in atom order and leave as one 512-byte
+//   copy (swizzled layout) or as per-row / per-block-row pieces (linear layout).
+#include <atomic>
+
+#include "mxfp8_device.cuh"
+#include "mxfp8_host.h"
+
+namespace mxfp8 {
+
+namespace {
+
+constexpr int TILE = 128;
+
+template <int DTYPE> struct Src;
+template <> struct Src<MXFP8_BF16> {
+    static constexpr int VEC = 4;
+    using Raw = uint2;
+    using Elem = __nv_bfloat16;
+    static __device__ __forceinline__ Raw zero() { return make_uint2(0u, 0u); }
+    static __device__ __forceinline__ void unpack(const Raw& r, float (&x)[4])
+    {
+        x[0] = __uint_as_float(r.x << 16);
+        x[1] = __uint_as_float(r.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(r.y << 16);
+        x[3] = __uint_as_float(r.y & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ Raw load_scalar(const Elem* p, int n_valid)
+    {
+        uint32_t h[4] = {0u, 0u, 0u, 0u};
+        for (int i = 0; i < 4; ++i)
+            if (i < n_valid) h[i] = (uint32_t)__bfloat16_as_ushort(p[i]);
+        return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+    }
+};
+template <> struct Src<MXFP8_FP32> {
+    static constexpr int VEC = 2;
+    using Raw = float2;
+    using Elem = float;
+    static __device__ __forceinline__ Raw zero() { return make_float2(0.f, 0.f); }
+    static __device__ __forceinline__ void unpack(const Raw& r, float (&x)[2])
+    {
+        x[0] = r.x;
+        x[1] = r.y;
+    }
+    static __device__ __forceinline__ Raw load_scalar(const Elem* p, int n_valid)
+    {
+        return make_float2(n_valid > 0 ? p[0] : 0.f, n_valid > 1 ? p[1] : 0.f);
+    }
+};
+
+template <int VEC>
+__device__ __forceinline__ void store_codes(uint8_t* dst, const uint32_t packed, bool vec_ok, int n_valid)
+{
+    if (vec_ok) {
+        if (VEC == 4) *reinterpret_cast<uint32_t*>(dst) = packed;
+        else *reinterpret_cast<uint16_t*>(dst) = (uint16_t)packed;
+    } else {
+        for (int i = 0; i < VEC; ++i)
+            if (i < n_valid) dst[i] = (uint8_t)(packed >> (8 * i));
+    }
+}
+
+template <int ELEM, int VEC>
+__device__ __forceinline__ uint32_t cast_vec(const float (&x)[VEC], const float (&inv)[VEC])
+{
+    if (VEC == 4) return cvt_fp8x4<ELEM>(x[0] * inv[0], x[1] * inv[1], x[2] * inv[2], x[3] * inv[3]);
+    return cvt_fp8x2<ELEM>(x[0] * inv[0], x[1] * inv[1]);
+}
+
+// Byte position of (mn, kb) inside one 512-byte scale atom, mn < 128, kb < 4.
+__device__ __forceinline__ int atom_pos(int mn, int kb) { return (mn & 31) * 16 + (mn >> 5) * 4 + kb; }
+
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool VEC_OK>
+__global__ void __launch_bounds__(128 * (TILE / (32 * Src<DTYPE>::VEC)))
+quantize_kernel(const void* __restrict__ src_v, int64_t rows, int64_t cols, int rule, int sf_layout,
+                uint8_t* __restrict__ q_row, uint8_t* __restrict__ s_row,
+                uint8_t* __restrict__ q_col, uint8_t* __restrict__ s_col, int64_t tiles_x)
+{
+    using S = Src<DTYPE>;
+    constexpr int VEC = S::VEC;
+    constexpr int WARP_COLS = 32 * VEC;
+    constexpr int WARPS_X = TILE / WARP_COLS;
+    constexpr int LPB = 32 / VEC;  // lanes per 32-column row block
+    constexpr int THREADS = 128 * WARPS_X;
+    const typename S::Elem* __restrict__ src = static_cast<const typename S::Elem*>(src_v);
+
+    __shared__ __align__(16) uint8_t sm_row[512];
+    __shared__ __align__(16) uint8_t sm_col[512];
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int wy = warp / WARPS_X;
+    const int wx = warp % WARPS_X;
+    const int64_t tile_y = (int64_t)blockIdx.x / tiles_x;
+    const int64_t tile_x = (int64_t)blockIdx.x % tiles_x;
+    const int64_t r0 = tile_y * TILE + wy * 32;
+    const int col_in_tile = wx * WARP_COLS + lane * VEC;
+    const int64_t c0 = tile_x * TILE + col_in_tile;
+
+    // zero both staging atoms (pad bytes of partial tiles must be 0)
+    for (int i = tid; i < 128; i += THREADS) {
+        reinterpret_cast<uint32_t*>(sm_row)[i] = 0u;
+        reinterpret_cast<uint32_t*>(sm_col)[i] = 0u;
+    }
+    __syncthreads();
+
+    const int n_valid = (int)max((int64_t)0, min((int64_t)VEC, cols - c0));  // columns this lane owns
+    const bool any_col = n_valid > 0;
+
+    // ---- one read of the source: 32 rows x VEC columns per lane ------------------------
+    typename S::Raw raw[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int64_t r = r0 + j;
+        raw[j] = S::zero();
+        if (r < rows && any_col) {
+            const typename S::Elem* p = src + r * cols + c0;
+            if (VEC_OK) raw[j] = __ldcs(reinterpret_cast<const typename S::Raw*>(p));
+            else raw[j] = S::load_scalar(p, n_valid);
+        }
+    }
+
+    // ---- column blocks: amax down the 32 rows, all inside this lane ---------------------
+    float col_inv[VEC];
+    if (DO_COL) {
+        float camax[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) camax[i] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float x[VEC];
+            S::unpack(raw[j], x);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) camax[i] = fmaxf(camax[i], fabsf(x[i]));  // NaN ignored
+        }
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            if (camax[i] == INFINITY) {  // rare: redo the maximum over finite elements only
+                float m = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float x[VEC];
+                    S::unpack(raw[j], x);
+                    const float a = fabsf(x[i]);
+                    if (a < INFINITY) m = fmaxf(m, a);
+                }
+                camax[i] = m;
+            }
+            const uint32_t b = scale_byte_from_amax_bits<ELEM>(__float_as_uint(camax[i]), rule);
+            col_inv[i] = inv_scale_from_byte(b);
+            if (i < n_valid && r0 < rows) sm_col[atom_pos(col_in_tile + i, wy)] = (uint8_t)b;
+        }
+    }
+
+    // ---- row by row: row-block amax across LPB lanes, then both casts --------------------
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int64_t r = r0 + j;
+        float x[VEC];
+        S::unpack(raw[j], x);
+        const bool live = (r < rows) && any_col;
+        if (DO_ROW) {
+            float m = 0.f;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) m = fmaxf(m, fabsf(x[i]));  // NaN ignored
+#pragma unroll
+            for (int off = 1; off < LPB; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+            if (__any_sync(0xFFFFFFFFu, m == INFINITY)) {  // rare: finite-only maximum
+                m = 0.f;
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                    const float a = fabsf(x[i]);
+                    if (a < INFINITY) m = fmaxf(m, a);
+                }
+#pragma unroll
+                for (int off = 1; off < LPB; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+            }
+            const uint32_t b = scale_byte_from_amax_bits<ELEM>(__float_as_uint(m), rule);
+            const float inv1 = inv_scale_from_byte(b);
+            float inv[VEC];
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) inv[i] = inv1;
+            if (live) {
+                store_codes<VEC>(q_row + r * cols + c0, cast_vec<ELEM, VEC>(x, inv), VEC_OK, n_valid);
+                if ((lane % LPB) == 0) sm_row[atom_pos(wy * 32 + j, col_in_tile >> 5)] = (uint8_t)b;
+            }
+        }
+        if (DO_COL && live)
+            store_codes<VEC>(q_col + r * cols + c0, cast_vec<ELEM, VEC>(x, col_inv), VEC_OK, n_valid);
+    }
+    __syncthreads();
+
+    // ---- scale bytes leave the CTA ----------------------------------------------------------
+    const int64_t tr0 = tile_y * TILE, tc0 = tile_x * TILE;
+    if (DO_ROW) {
+        const int64_t ncb = cols >> 5;
+        if (sf_layout == MXFP8_SF_SWIZZLED) {
+            const int64_t atom = tile_y * ((ncb + 3) >> 2) + tile_x;
+            if (tid < 32) reinterpret_cast<uint4*>(s_row + atom * 512)[tid] = reinterpret_cast<const uint4*>(sm_row)[tid];
+        } else if (tid < TILE && tr0 + tid < rows) {
+            uint8_t* d = s_row + (tr0 + tid) * ncb + (tc0 >> 5);
+            const int nkb = (int)min((int64_t)4, ncb - (tc0 >> 5));
+            if (nkb == 4 && (ncb & 3) == 0) {
+                *reinterpret_cast<uint32_t*>(d) = *reinterpret_cast<const uint32_t*>(sm_row + atom_pos(tid, 0));
+            } else {
+                for (int kb = 0; kb < nkb; ++kb) d[kb] = sm_row[atom_pos(tid, kb)];
+            }
+        }
+    }
+    if (DO_COL) {
+        const int64_t nrb = rows >> 5;
+        if (sf_layout == MXFP8_SF_SWIZZLED) {
+            const int64_t atom = tile_x * ((nrb + 3) >> 2) + tile_y;
+            if (tid < 32) reinterpret_cast<uint4*>(s_col + atom * 512)[tid] = reinterpret_cast<const uint4*>(sm_col)[tid];
+        } else if (tid < TILE && tc0 + tid < cols) {
+            const int nrb_here = (int)min((int64_t)4, nrb - (tr0 >> 5));
+            for (int w = 0; w < nrb_here; ++w) s_col[((tr0 >> 5) + w) * cols + tc0 + tid] = sm_col[atom_pos(tid, w)];
+        }
+    }
+}
+
+std::atomic<int64_t> g_launches{0};
+
+template <int DTYPE, int ELEM>
+cudaError_t launch_quantize(const void* src, int64_t rows, int64_t cols, int orientation, int rule,
+                            int sf_layout, uint8_t* q_row, uint8_t* s_row, uint8_t* q_col,
+                            uint8_t* s_col, cudaStream_t stream)
+{
+    constexpr int VEC = Src<DTYPE>::VEC;
+    constexpr int THREADS = 128 * (TILE / (32 * VEC));
+    const int64_t tiles_x = (cols + TILE - 1) / TILE;
+    const int64_t tiles_y = (rows + TILE - 1) / TILE;
+    const int64_t tiles = tiles_x * tiles_y;
+    if (tiles > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const dim3 grid((unsigned)tiles), block(THREADS);
+    const bool vec_ok = (cols % VEC) == 0;
+#define MXFP8_LAUNCH(R, C, V) \
+    quantize_kernel<DTYPE, ELEM, R, C, V><<<grid, block, 0, stream>>>(src, rows, cols, rule, sf_layout, q_row, s_row, q_col, s_col, tiles_x)
+    if (orientation == MXFP8_ROW) MXFP8_LAUNCH(true, false, true);
+    else if (orientation == MXFP8_BOTH) MXFP8_LAUNCH(true, true, true);
+    else if (vec_ok) MXFP8_LAUNCH(false, true, true);
+    else MXFP8_LAUNCH(false, true, false);
+#undef MXFP8_LAUNCH
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int64_t launches() { return g_launches.load(std::memory_order_relaxed); }
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int quantize_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
+                    int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
+                    int sf_layout, cudaStream_t stream)
+{
+    cudaError_t err;
+    uint8_t *qr = static_cast<uint8_t*>(q_row), *sr = static_cast<uint8_t*>(s_row);
+    uint8_t *qc = static_cast<uint8_t*>(q_col), *sc = static_cast<uint8_t*>(s_col);
+    if (src_dtype == MXFP8_BF16) {
+        err = (elem == MXFP8_E4M3)
+                  ? launch_quantize<MXFP8_BF16, MXFP8_E4M3>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream)
+                  : launch_quantize<MXFP8_BF16, MXFP8_E5M2>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream);
+    } else {
+        err = (elem == MXFP8_E4M3)
+                  ? launch_quantize<MXFP8_FP32, MXFP8_E4M3>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream)
+                  : launch_quantize<MXFP8_FP32, MXFP8_E5M2>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream);
+    }
+    return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}
+
+}  // namespace mxfp8
+
+extern "C" int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                              int orientation, int scale_rule, int elem,
+                              void* q_row, void* s_row, void* q_col, void* s_col,
+                              int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!src) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col || !s_col)) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(src)) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    return quantize_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
+                           q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
+}

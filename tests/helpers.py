@@ -1,0 +1,115 @@
+"""Shared test plumbing: run the CUDA library on numpy inputs, compare with the oracle."""
+import numpy as np
+
+import oracle as orc
+
+GUARD = 256          # sentinel bytes on each side of every output buffer
+SENTINEL = 0xA5
+
+
+def nan_code_mask(q: np.ndarray, elem: int) -> np.ndarray:
+    m = q & 0x7F
+    return (m == 0x7F) if elem == orc.E4M3 else (m > 0x7C)
+
+
+def assert_q_equal(got: np.ndarray, want: np.ndarray, elem: int, what=""):
+    """Bit-exact, except that any two NaN codes count as equal (several are valid)."""
+    gn, wn = nan_code_mask(got, elem), nan_code_mask(want, elem)
+    assert np.array_equal(gn, wn), "NaN positions differ " + what
+    bad = (got != want) & ~gn
+    if bad.any():
+        idx = np.argwhere(bad)[:5]
+        raise AssertionError("%d Q bytes differ %s; first at %s: got %s want %s" % (
+            bad.sum(), what, idx.tolist(), got[bad][:5], want[bad][:5]))
+
+
+def logical_scales_from_swizzled(buf: np.ndarray, mn: int, nkb: int) -> np.ndarray:
+    """Gather the logical [mn, nkb] scale matrix out of a 128x4-atom buffer (oracle's formula)."""
+    m_idx, k_idx = np.meshgrid(np.arange(mn), np.arange(nkb), indexing="ij")
+    atoms_k = (nkb + 3) // 4
+    off = ((m_idx // 128) * atoms_k + k_idx // 4) * 512 + (m_idx % 32) * 16 + ((m_idx % 128) // 32) * 4 + k_idx % 4
+    assert off[-1, -1] == orc.sf_offset_swizzled(mn - 1, nkb - 1, nkb)
+    assert off[mn // 2, nkb // 2] == orc.sf_offset_swizzled(mn // 2, nkb // 2, nkb)
+    return buf[off]
+
+
+def swizzled_pad_mask(mn: int, nkb: int) -> np.ndarray:
+    size = ((mn + 127) // 128) * ((nkb + 3) // 4) * 512
+    used = np.zeros(size, dtype=bool)
+    m_idx, k_idx = np.meshgrid(np.arange(mn), np.arange(nkb), indexing="ij")
+    atoms_k = (nkb + 3) // 4
+    off = ((m_idx // 128) * atoms_k + k_idx // 4) * 512 + (m_idx % 32) * 16 + ((m_idx % 128) // 32) * 4 + k_idx % 4
+    used[off.reshape(-1)] = True
+    return ~used
+
+
+class Guarded:
+    """A device byte buffer with sentinel bands before and after the payload."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        import torch
+        self.n = nbytes
+        self.buf = torch.full((nbytes + 2 * GUARD,), SENTINEL, dtype=torch.uint8, device=device)
+        self.view = self.buf[GUARD:GUARD + nbytes]
+
+    def check(self, what=""):
+        b = self.buf.cpu().numpy()
+        assert (b[:GUARD] == SENTINEL).all() and (b[GUARD + self.n:] == SENTINEL).all(), "guard band overwritten " + what
+
+    def numpy(self):
+        return self.view.cpu().numpy()
+
+
+def gpu_quantize(src_np, dtype: str, orientation: int, rule: int, elem: int, sf_layout: int):
+    """src_np: float32 array (dtype 'fp32') or uint16 bf16 bit patterns (dtype 'bf16').
+    Returns dict with 'q_row','s_row','q_col','s_col' numpy arrays (scales logical, linear
+    shape) plus the raw swizzled buffers when sf_layout is swizzled."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = src_np.shape
+    if dtype == "bf16":
+        src = torch.from_numpy(src_np.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        src = torch.from_numpy(src_np).cuda()
+    bufs = {}
+    args = []
+    for o, name in ((B.ROW, "row"), (B.COL, "col")):
+        if orientation & o:
+            q = Guarded(rows * cols)
+            s = Guarded(B.mxfp8_scale_bytes(rows, cols, o, sf_layout))
+            bufs[name] = (q, s)
+            args += [q.view.view(rows, cols), s.view]
+        else:
+            args += [None, None]
+    B.mxfp8_quantize(src, orientation, rule, elem, args[0], args[1], args[2], args[3], sf_layout)
+    torch.cuda.synchronize()
+    out = {}
+    for name, (q, s) in bufs.items():
+        q.check("q_" + name)
+        s.check("s_" + name)
+        out["q_" + name] = q.numpy().reshape(rows, cols)
+        raw = s.numpy()
+        if name == "row":
+            mn, nkb = rows, cols // 32
+        else:
+            mn, nkb = cols, rows // 32
+        if sf_layout == B.SF_SWIZZLED:
+            out["raw_s_" + name] = raw
+            logical = logical_scales_from_swizzled(raw, mn, nkb)
+            assert (raw[swizzled_pad_mask(mn, nkb)] == 0).all(), "pad bytes must be 0"
+        else:
+            logical = raw.reshape(rows, cols // 32) if name == "row" else raw.reshape(rows // 32, cols).T
+        out["s_" + name] = logical if name == "row" else np.ascontiguousarray(logical.T)
+    return out
+
+
+def check_against_oracle(src_np, dtype, orientation, rule, elem, sf_layout, what=""):
+    from paper_2506_08027_b200 import binding as B
+    x = orc.bf16_bits_to_f32(src_np) if dtype == "bf16" else src_np
+    got = gpu_quantize(src_np, dtype, orientation, rule, elem, sf_layout)
+    for o, name in ((B.ROW, "row"), (B.COL, "col")):
+        if orientation & o:
+            wq, ws = orc.quantize(x, orc.ROW if o == B.ROW else orc.COL, rule, elem)
+            assert np.array_equal(got["s_" + name], ws), "scale bytes differ (%s) %s" % (name, what)
+            assert_q_equal(got["q_" + name], wq, elem, "(%s) %s" % (name, what))
+    return got

@@ -1,0 +1,215 @@
+"""Parity of mxfp8_quantize / mxfp8_dequantize with the CPU oracle: bit-exact Q and scale bytes."""
+import os
+import struct
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2506_08027_b200 import synth
+from helpers import check_against_oracle, gpu_quantize, assert_q_equal
+
+pytestmark = pytest.mark.gpu
+
+ROW, COL, BOTH = 1, 2, 3
+LINEAR, SWIZZLED = 0, 1
+
+
+def as_dtype(x32, dtype):
+    return synth.f32_to_bf16_bits(x32) if dtype == "bf16" else x32
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("rule", [orc.RULE_PAPER, orc.RULE_OCP])
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+def test_pr1_reference_tensor(dtype, rule, elem):
+    # config 1: 256x512, row-scaled Gaussian with outliers, zero blocks, a block with amax 448
+    x = as_dtype(synth.pr1_tensor(0), dtype)
+    for orientation in (ROW, COL, BOTH):
+        for layout in (LINEAR, SWIZZLED):
+            check_against_oracle(x, dtype, orientation, rule, elem, layout, "pr1 o=%d l=%d" % (orientation, layout))
+
+
+SHAPES = [(32, 32), (1, 32), (7, 64), (32, 128), (160, 352), (128, 128), (160, 416),
+          (384, 8288), (96, 4096 + 128), (1024, 4096)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_shapes_and_ragged_tails(shape, dtype):
+    rows, cols = shape
+    x = as_dtype(synth.gaussian(shape, 1234 + rows + cols), dtype)
+    orients = [ROW]
+    if rows % 32 == 0:
+        orients += [COL, BOTH]
+    for o in orients:
+        for layout in (LINEAR, SWIZZLED):
+            check_against_oracle(x, dtype, o, orc.RULE_PAPER, orc.E4M3, layout, "%s o=%d l=%d" % (shape, o, layout))
+
+
+@pytest.mark.parametrize("cols", [100, 33, 2, 130])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_column_blocks_with_odd_width(cols, dtype):
+    x = as_dtype(synth.gaussian((64, cols), 99 + cols), dtype)
+    for layout in (LINEAR, SWIZZLED):
+        check_against_oracle(x, dtype, COL, orc.RULE_PAPER, orc.E4M3, layout, "cols=%d" % cols)
+
+
+@pytest.mark.parametrize("dist", synth.DISTRIBUTIONS)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+def test_distributions(dist, dtype, elem):
+    x = as_dtype(synth.draw(dist, (256, 1024), synth.seed_for(4, hash(dist) % 50)), dtype)
+    for rule in (orc.RULE_PAPER, orc.RULE_OCP):
+        check_against_oracle(x, dtype, BOTH, rule, elem, SWIZZLED, dist)
+
+
+def test_nonfinite_dense():
+    # many NaN / Inf, including whole blocks of them, in both orientations
+    rng = np.random.default_rng(5)
+    x = synth.gaussian((128, 256), 77)
+    pick = rng.random(x.shape)
+    x[pick < 0.05] = np.nan
+    x[(pick >= 0.05) & (pick < 0.10)] = np.inf
+    x[(pick >= 0.10) & (pick < 0.15)] = -np.inf
+    x[3, 32:64] = np.nan
+    x[32:64, 9] = np.inf
+    x[5, 64:96] = [np.inf, -np.inf] * 16
+    for dtype in ("fp32", "bf16"):
+        for elem in (orc.E4M3, orc.E5M2):
+            check_against_oracle(as_dtype(x, dtype), dtype, BOTH, orc.RULE_PAPER, elem, LINEAR, "nonfinite")
+
+
+def test_fp32_extremes_and_subnormals():
+    # FP32 subnormal inputs are honoured; the largest finite inputs do not overflow the scale
+    bits = np.array([0x00000001, 0x00000200, 0x00080000, 0x007FFFFF, 0x00800000, 0x03E00000, 0x04600000,
+                     0x04600001, 0x07E00001, 0x7F7FFFFF, 0x7F000000, 0x80000000, 0x80000001], dtype=np.uint32)
+    rng = np.random.default_rng(8)
+    x = np.zeros((64, 128), dtype=np.float32)
+    flat = x.reshape(-1)
+    pos = rng.choice(flat.size, size=bits.size * 8, replace=False)
+    flat[pos] = np.tile(bits, 8).view(np.float32)
+    # plus blocks made only of subnormals
+    x[10, 32:64] = np.frombuffer(struct.pack("<I", 0x00080000), np.float32)[0]
+    for rule in (orc.RULE_PAPER, orc.RULE_OCP):
+        for elem in (orc.E4M3, orc.E5M2):
+            check_against_oracle(x, "fp32", BOTH, rule, elem, LINEAR, "extremes")
+
+
+def test_handworked_blocks_on_gpu(golden_dir):
+    from test_oracle_pins import read_golden, ELEMS
+    rows_ = read_golden(os.path.join(golden_dir, "handworked_blocks.txt"))
+    for elem_name in ("e4m3", "e5m2"):
+        sel = [r for r in rows_ if r[0] == elem_name]
+        x = np.zeros((32, 32 * len(sel)), dtype=np.float32)
+        for i, r in enumerate(sel):
+            x[0, 32 * i + 3] = np.frombuffer(struct.pack("<I", int(r[1], 16)), np.float32)[0]
+        for rule, bi, qi in ((orc.RULE_PAPER, 2, 3), (orc.RULE_OCP, 4, 5)):
+            got = gpu_quantize(x, "fp32", ROW, rule, ELEMS[elem_name], LINEAR)
+            for i, r in enumerate(sel):
+                assert got["s_row"][0, i] == int(r[bi], 16), r
+                assert got["q_row"][0, 32 * i + 3] == int(r[qi], 16), r
+
+
+def test_deterministic_and_both_equals_separate():
+    x = synth.f32_to_bf16_bits(synth.gradient_like((512, 2048), 31))
+    a = gpu_quantize(x, "bf16", BOTH, orc.RULE_PAPER, orc.E4M3, SWIZZLED)
+    b = gpu_quantize(x, "bf16", BOTH, orc.RULE_PAPER, orc.E4M3, SWIZZLED)
+    r = gpu_quantize(x, "bf16", ROW, orc.RULE_PAPER, orc.E4M3, SWIZZLED)
+    c = gpu_quantize(x, "bf16", COL, orc.RULE_PAPER, orc.E4M3, SWIZZLED)
+    for k in ("q_row", "q_col", "raw_s_row", "raw_s_col"):
+        assert np.array_equal(a[k], b[k])
+    assert np.array_equal(a["q_row"], r["q_row"]) and np.array_equal(a["raw_s_row"], r["raw_s_row"])
+    assert np.array_equal(a["q_col"], c["q_col"]) and np.array_equal(a["raw_s_col"], c["raw_s_col"])
+
+
+def test_large_tensor_sampled():
+    # a benchmark-sized tensor (8192 x 8192 BF16, drawn on the device): the oracle checks a
+    # strided sample of 128-row slabs plus the first and last slab
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows = cols = 8192
+    src = synth.device_tensor("output_gradient", (rows, cols), synth.seed_for(2, 2))
+    qr, sr, qc, sc = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_LINEAR)
+    B.mxfp8_quantize(src, B.BOTH, B.RULE_PAPER, B.E4M3, qr, sr, qc, sc, B.SF_LINEAR)
+    torch.cuda.synchronize()
+    for r0 in (0, 1024 + 128, 4096 - 128, 8192 - 128):
+        sl = slice(r0, r0 + 128)
+        x = orc.bf16_bits_to_f32(src[sl].view(torch.int16).cpu().numpy().view(np.uint16))
+        wq, ws = orc.quantize(x, orc.ROW)
+        assert np.array_equal(sr.view(rows, cols // 32)[sl].cpu().numpy(), ws)
+        assert_q_equal(qr[sl].cpu().numpy(), wq, orc.E4M3)
+        wq, ws = orc.quantize(x, orc.COL)
+        assert np.array_equal(sc.view(rows // 32, cols)[r0 // 32:r0 // 32 + 4].cpu().numpy(), ws)
+        assert_q_equal(qc[sl].cpu().numpy(), wq, orc.E4M3)
+
+
+# ------------------------------------------------------------------------------- dequantize
+
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+@pytest.mark.parametrize("dst", ["f32", "bf16"])
+def test_dequantize_exhaustive_codes_and_scales(elem, dst):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    codes = np.arange(256, dtype=np.uint8)
+    q = np.tile(np.repeat(codes, 32)[None, :], (256, 1))            # [256, 8192]
+    s = np.repeat(np.arange(256, dtype=np.uint8)[:, None], 256, axis=1)
+    want = orc.dequantize(q, s, orc.ROW, elem, dst)
+    qd, sd = torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda()
+    out = torch.empty(q.shape, dtype=torch.float32 if dst == "f32" else torch.bfloat16, device="cuda")
+    B.mxfp8_dequantize(qd, sd.view(-1), B.ROW, elem, B.SF_LINEAR, out)
+    torch.cuda.synchronize()
+    if dst == "f32":
+        got = out.cpu().numpy()
+        nan = np.isnan(want)
+        assert np.array_equal(np.isnan(got), nan)
+        assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+    else:
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        nan = (want & 0x7FFF) > 0x7F80
+        assert np.array_equal((got & 0x7FFF) > 0x7F80, nan)
+        assert np.array_equal(got[~nan], want[~nan])
+
+
+@pytest.mark.parametrize("orientation", [ROW, COL])
+@pytest.mark.parametrize("layout", [LINEAR, SWIZZLED])
+@pytest.mark.parametrize("shape", [(256, 512), (96, 352), (64, 100)])
+def test_dequantize_roundtrip_layouts(orientation, layout, shape):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = shape
+    if orientation == ROW and cols % 32:
+        pytest.skip("row blocks need cols % 32 == 0")
+    x = synth.gradient_like(shape, 5 + rows)
+    src = torch.from_numpy(x).cuda()
+    outs = B.alloc_quantize_outputs(rows, cols, orientation, layout)
+    B.mxfp8_quantize(src, orientation, B.RULE_PAPER, B.E4M3, *outs, layout)
+    q, s = (outs[0], outs[1]) if orientation == ROW else (outs[2], outs[3])
+    for dst_dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        dst = torch.empty(shape, dtype=dst_dtype, device="cuda")
+        B.mxfp8_dequantize(q, s, orientation, B.E4M3, layout, dst)
+        torch.cuda.synchronize()
+        wq, ws = orc.quantize(x, orc.ROW if orientation == ROW else orc.COL)
+        want = orc.dequantize(wq, ws, orc.ROW if orientation == ROW else orc.COL, orc.E4M3, name)
+        if name == "f32":
+            assert np.array_equal(dst.cpu().numpy().view(np.uint32), want.view(np.uint32))
+        else:
+            assert np.array_equal(dst.view(torch.int16).cpu().numpy().view(np.uint16), want)
+
+
+def test_quantize_host_variant():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = 256, 384
+    x = synth.f32_to_bf16_bits(synth.gaussian((rows, cols), 3))
+    src = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
+    ws = torch.empty(B.mxfp8_quantize_host_ws_bytes(B.BF16, rows, cols, B.BOTH), dtype=torch.uint8, device="cuda")
+    host = [torch.empty(n, dtype=torch.uint8).pin_memory() for n in (
+        rows * cols, B.mxfp8_scale_bytes(rows, cols, B.ROW, B.SF_LINEAR),
+        rows * cols, B.mxfp8_scale_bytes(rows, cols, B.COL, B.SF_LINEAR))]
+    B.mxfp8_quantize_host(src, B.BOTH, B.RULE_PAPER, B.E4M3, host[0], host[1], host[2], host[3], B.SF_LINEAR, ws)
+    xf = orc.bf16_bits_to_f32(x)
+    wq, wsr = orc.quantize(xf, orc.ROW)
+    assert np.array_equal(host[0].numpy().reshape(rows, cols), wq) and np.array_equal(host[1].numpy().reshape(rows, -1), wsr)
+    wq, wsc = orc.quantize(xf, orc.COL)
+    assert np.array_equal(host[2].numpy().reshape(rows, cols), wq) and np.array_equal(host[3].numpy().reshape(-1, cols), wsc)
