@@ -113,3 +113,58 @@ def check_against_oracle(src_np, dtype, orientation, rule, elem, sf_layout, what
             assert np.array_equal(got["s_" + name], ws), "scale bytes differ (%s) %s" % (name, what)
             assert_q_equal(got["q_" + name], wq, elem, "(%s) %s" % (name, what))
     return got
+
+
+def swizzle_np(s_logical: np.ndarray) -> np.ndarray:
+    """Vectorised form of oracle.swizzle_scales (checked against it in the CPU tests)."""
+    mn, nkb = s_logical.shape
+    out = np.zeros(((mn + 127) // 128) * ((nkb + 3) // 4) * 512, dtype=np.uint8)
+    m_idx, k_idx = np.meshgrid(np.arange(mn), np.arange(nkb), indexing="ij")
+    atoms_k = (nkb + 3) // 4
+    off = ((m_idx // 128) * atoms_k + k_idx // 4) * 512 + (m_idx % 32) * 16 + ((m_idx % 128) // 32) * 4 + k_idx % 4
+    out[off.reshape(-1)] = s_logical.reshape(-1)
+    return out
+
+
+def gpu_gemm(aq, a_s, bq, b_s, a_major="k", b_major="k", a_elem=0, b_elem=0, out="fp32"):
+    """aq/bq: uint8 arrays as stored ([MN,K] for 'k', [K,MN] for 'mn'); a_s/b_s: linear scale
+    arrays as the oracle returns them for that storage.  Returns D as numpy (float32, or
+    uint16 bf16 bit patterns)."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    if a_major == "k":
+        M, K = aq.shape
+        sa_log = a_s
+    else:
+        K, M = aq.shape
+        sa_log = np.ascontiguousarray(a_s.T)
+    if b_major == "k":
+        N, _ = bq.shape
+        sb_log = b_s
+    else:
+        _, N = bq.shape
+        sb_log = np.ascontiguousarray(b_s.T)
+    dA, dB = torch.from_numpy(aq).cuda(), torch.from_numpy(bq).cuda()
+    dSA, dSB = torch.from_numpy(swizzle_np(sa_log)).cuda(), torch.from_numpy(swizzle_np(sb_log)).cuda()
+    D = torch.full((M, N), float("nan"), dtype=torch.float32 if out == "fp32" else torch.bfloat16, device="cuda")
+    B.mxfp8_gemm(dA, dSA, dB, dSB, M, N, K, B.MN_MAJOR if a_major == "mn" else B.K_MAJOR,
+                 B.MN_MAJOR if b_major == "mn" else B.K_MAJOR, a_elem, b_elem, D)
+    assert B.mxfp8_device_status() == 0, "device status word reports a timeout"
+    if out == "fp32":
+        return D.cpu().numpy()
+    return D.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def check_gemm_tolerance(d_gpu, d64, sabs, what=""):
+    """spec bounds: relative Frobenius error <= 1e-5 and every element within
+    2^-16 * sum_k |a_k b_k| (plus an absolute floor of 2^-126 at the edge of the FP32 range)."""
+    d = d_gpu.astype(np.float64)
+    assert np.array_equal(np.isnan(d), np.isnan(d64)), "NaN positions differ " + what
+    ok = ~np.isnan(d64)
+    err = np.abs(d[ok] - d64[ok])
+    bound = 2.0 ** -16 * sabs[ok] + 2.0 ** -126
+    worst = float((err / bound).max()) if err.size else 0.0
+    assert worst <= 1.0, "element bound exceeded %s: worst err/bound = %.3g" % (what, worst)
+    fro = np.sqrt((err ** 2).sum()) / max(np.sqrt((d64[ok] ** 2).sum()), 1e-300)
+    assert fro <= 1e-5, "relative Frobenius error %.3g %s" % (fro, what)
+    return worst, fro

@@ -1,0 +1,158 @@
+"""Parity of mxfp8_gemm with the FP64 oracle over decoded operands.
+
+Exact-integer cases must match exactly (every partial sum is an integer below 2^24, so any
+FP32 accumulation order gives the same result); everything else must meet the tolerance:
+relative Frobenius error <= 1e-5 and |D - D64| <= 2^-16 * sum_k |a_k b_k| per element.
+"""
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2506_08027_b200 import synth
+from helpers import gpu_gemm, check_gemm_tolerance
+
+pytestmark = pytest.mark.gpu
+
+INTS = np.array([-4, -3, -2, -1, 0, 1, 2, 3, 4])
+
+
+def int_operand(rng, mn, k):
+    vals = rng.choice(INTS, (mn, k))
+    enc = np.zeros(256, dtype=np.uint8)
+    for v in INTS:
+        enc[int(v) & 0xFF] = orc.fp8_encode(float(v))
+    return vals, enc[vals.astype(np.int64) & 0xFF]
+
+
+def stored(q_logical, s_logical, major):
+    """logical [MN,K] data and [MN,K/32] scales -> storage for 'k' or 'mn' majorness."""
+    if major == "k":
+        return q_logical, s_logical
+    return np.ascontiguousarray(q_logical.T), np.ascontiguousarray(s_logical.T)
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 128), (128, 256, 128), (256, 128, 256), (384, 512, 640), (128, 384, 1024)])
+@pytest.mark.parametrize("majors", [("k", "k"), ("k", "mn"), ("mn", "k"), ("mn", "mn")])
+def test_exact_integers(shape, majors):
+    m, n, k = shape
+    rng = np.random.default_rng(m + 3 * n + 7 * k)
+    ai, aq = int_operand(rng, m, k)
+    bi, bq = int_operand(rng, n, k)
+    a_s = np.full((m, k // 32), 127, np.uint8)
+    b_s = np.full((n, k // 32), 127, np.uint8)
+    want = (ai @ bi.T).astype(np.float64)
+    A, SA = stored(aq, a_s, majors[0])
+    B_, SB = stored(bq, b_s, majors[1])
+    d64, _ = orc.gemm_f64(A, SA, B_, SB, majors[0], majors[1])
+    assert np.array_equal(d64, want)
+    got = gpu_gemm(A, SA, B_, SB, majors[0], majors[1])
+    assert np.array_equal(got.astype(np.float64), want), "max |diff| = %g" % np.abs(got - want).max()
+
+
+@pytest.mark.parametrize("majors", [("k", "k"), ("mn", "mn")])
+def test_identity_b_returns_decoded_a(majors):
+    # B = identity (K = N): D equals the decoded A exactly
+    m, n = 256, 256
+    k = n
+    x = synth.gradient_like((m, k), 12)
+    if majors[0] == "k":
+        aq, a_s = orc.quantize(x, orc.ROW)
+        a_dec = orc.dequantize_f64(aq, a_s, orc.ROW)
+    else:
+        aq, a_s = orc.quantize(np.ascontiguousarray(x.T), orc.COL)
+        a_dec = orc.dequantize_f64(aq, a_s, orc.COL).T
+    eye_q = np.where(np.eye(n, dtype=bool), orc.fp8_encode(1.0), 0).astype(np.uint8)
+    eye_s = np.full((n, k // 32), 127, np.uint8)
+    Bq, Bs = stored(eye_q, eye_s, majors[1])
+    got = gpu_gemm(aq, a_s, Bq, Bs, majors[0], majors[1])
+    assert np.array_equal(got.astype(np.float64), a_dec.astype(np.float32).astype(np.float64))
+
+
+@pytest.mark.parametrize("majors", [("k", "k"), ("mn", "mn")])
+def test_one_hot_scales_pin_the_scale_layout(majors):
+    # all scale bytes 127 except one (mn, kb) = 128: exactly the products through that block
+    # double.  Sweeps rows across quadrants / tiles and K-blocks across atoms and stages.
+    m, n, k = 256, 256, 512
+    rng = np.random.default_rng(4)
+    ai, aq = int_operand(rng, m, k)
+    bi, bq = int_operand(rng, n, k)
+    base = (ai @ bi.T).astype(np.float64)
+    picks = [(0, 0), (1, 1), (31, 3), (32, 4), (77, 5), (127, 15), (128, 0), (200, 9), (255, 15), (96, 7)]
+    for which in ("a", "b"):
+        for (mn, kb) in picks:
+            a_s = np.full((m, k // 32), 127, np.uint8)
+            b_s = np.full((n, k // 32), 127, np.uint8)
+            extra = np.zeros((m, n))
+            if which == "a":
+                a_s[mn, kb] = 128
+                extra[mn, :] = ai[mn, kb * 32:(kb + 1) * 32] @ bi[:, kb * 32:(kb + 1) * 32].T
+            else:
+                b_s[mn, kb] = 129
+                extra[:, mn] = 3 * (ai[:, kb * 32:(kb + 1) * 32] @ bi[mn, kb * 32:(kb + 1) * 32])
+            A, SA = stored(aq, a_s, majors[0])
+            B_, SB = stored(bq, b_s, majors[1])
+            got = gpu_gemm(A, SA, B_, SB, majors[0], majors[1])
+            assert np.array_equal(got.astype(np.float64), base + extra), (which, mn, kb)
+
+
+def test_pr1_reference_gemm():
+    # config 1: both operands 256x512 FP32, quantized rowwise (paper rule), M=N=256, K=512;
+    # and the same product from column-quantized transposes (MN-major x MN-major).
+    a = synth.pr1_tensor(0)
+    b = synth.pr1_tensor(1)
+    aq, a_s = orc.quantize(a, orc.ROW)
+    bq, b_s = orc.quantize(b, orc.ROW)
+    d64, sabs = orc.gemm_f64(aq, a_s, bq, b_s)
+    got = gpu_gemm(aq, a_s, bq, b_s)
+    check_gemm_tolerance(got, d64, sabs, "pr1 k-major")
+    aqt, a_st = orc.quantize(np.ascontiguousarray(a.T), orc.COL)
+    bqt, b_st = orc.quantize(np.ascontiguousarray(b.T), orc.COL)
+    assert np.array_equal(aqt.T, aq) and np.array_equal(a_st.T, a_s)
+    got2 = gpu_gemm(aqt, a_st, bqt, b_st, "mn", "mn")
+    check_gemm_tolerance(got2, d64, sabs, "pr1 mn-major")
+
+
+@pytest.mark.parametrize("shape,majors", [((512, 768, 1024), ("k", "k")), ((256, 1280, 2048), ("k", "mn")),
+                                          ((640, 256, 4096), ("mn", "mn")), ((1024, 1024, 512), ("mn", "k"))])
+@pytest.mark.parametrize("elems", [(0, 0), (1, 0), (0, 1)])
+def test_random_operands_meet_tolerance(shape, majors, elems):
+    m, n, k = shape
+    a = synth.gaussian((m, k), 100 + m)
+    b = synth.output_gradient((n, k), 200 + n)
+    qa = orc.quantize(a, orc.ROW, orc.RULE_PAPER, elems[0])
+    qb = orc.quantize(b, orc.ROW, orc.RULE_PAPER, elems[1])
+    A, SA = stored(qa[0], qa[1], majors[0])
+    B_, SB = stored(qb[0], qb[1], majors[1])
+    d64, sabs = orc.gemm_f64(A, SA, B_, SB, majors[0], majors[1], elems[0], elems[1])
+    got = gpu_gemm(A, SA, B_, SB, majors[0], majors[1], elems[0], elems[1])
+    check_gemm_tolerance(got, d64, sabs, str((shape, majors, elems)))
+
+
+def test_bf16_output_is_rne_of_fp32_output_and_deterministic():
+    import torch
+    m, n, k = 384, 512, 1024
+    a = synth.gaussian((m, k), 1)
+    b = synth.gaussian((n, k), 2, 0.02)
+    aq, a_s = orc.quantize(a, orc.ROW)
+    bq, b_s = orc.quantize(b, orc.ROW)
+    d32 = gpu_gemm(aq, a_s, bq, b_s)
+    d32b = gpu_gemm(aq, a_s, bq, b_s)
+    assert np.array_equal(d32.view(np.uint32), d32b.view(np.uint32))
+    dbf = gpu_gemm(aq, a_s, bq, b_s, out="bf16")
+    want = torch.from_numpy(d32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(dbf, want)
+    d64, sabs = orc.gemm_f64(aq, a_s, bq, b_s)
+    check_gemm_tolerance(d32, d64, sabs)
+
+
+def test_nan_scale_byte_poisons_its_outputs():
+    m, n, k = 128, 128, 256
+    rng = np.random.default_rng(9)
+    _, aq = int_operand(rng, m, k)
+    _, bq = int_operand(rng, n, k)
+    a_s = np.full((m, k // 32), 127, np.uint8)
+    b_s = np.full((n, k // 32), 127, np.uint8)
+    b_s[5, 2] = 0xFF
+    d64, _ = orc.gemm_f64(aq, a_s, bq, b_s)
+    got = gpu_gemm(aq, a_s, bq, b_s)
+    assert np.array_equal(np.isnan(got), np.isnan(d64))
