@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the MXFP8 hot path on B200: one training step of a linear layer.
+
+A "step" is one pass of the whole path over one batch of synthetic input, for the
+~800M-parameter GPT-style linear layer (tokens 8192, hidden 2048, FFN 8192): the three BF16
+tensors X, W, dY are each converted to MXFP8-E4M3 in both block orientations (one read each),
+then FPROP, DGRAD and WGRAD run as block-scaled MXFP8 GEMMs with BF16 output.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.  `value` is the step's GEMM work (3 x 2MNK FLOP) divided by
+the whole step time (casts included), summed over ranks; `cast` and `gemm` give the two parts
+of the metric separately (GB/s and TFLOP/s from per-launch CUDA events); `roofline` describes
+the dominant kernel (the GEMM); `cpu_baseline` is the CPU oracle timed on a bounded sample.
+With --impl reference the oracle alone is timed (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+T, H, F = 8192, 2048, 8192          # tokens, hidden, FFN of the benchmarked linear layer
+METRIC = "MXFP8 cast GB/s (% HBM peak); MXFP8 GEMM TFLOP/s (% dense FP8 peak)"
+WORKLOAD = "linear layer of a ~800M-param GPT: tokens 8192, hidden 2048, FFN 8192; quantize X,W,dY (both orientations) + fprop/dgrad/wgrad MXFP8 GEMMs, BF16 out"
+NOMINAL_FP8_TFLOPS = 4500.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+STEP_FLOP = 3 * 2.0 * T * H * F                       # three GEMMs of 275 GFLOP
+CAST_BYTES = (T * H + F * H + T * F) * (2 + 2 * (1 + 1 / 32))   # src + two orientations x (q + scales)
+GEMM_SHAPES = {"fprop": (T, F, H), "dgrad": (T, H, F), "wgrad": (F, H, T)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples = []
+        self.proc = None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) >= 6:
+                    self.samples.append(parts)
+        except Exception:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+        self.join(timeout=2)
+        sm, smax, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                smax = max(smax, float(s[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, s[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # only the busiest half of the samples is "under load" (the sampler also sees idle gaps)
+        sm_sorted = sorted(sm)
+        under = sm_sorted[len(sm_sorted) // 2:] if sm_sorted else []
+        return {"sm_mhz": statistics.median(under) if under else None, "sm_max_mhz": smax or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample_seconds(sample_rows: int = 256):
+    """Time the oracle, as it stands, on a bounded sample of the step and scale to a full step.
+
+    Cast: `sample_rows` rows of each tensor in both orientations (all host threads, row slabs).
+    GEMM: `sample_rows` output rows of each product in FP64 over decoded operands (numpy/BLAS).
+    Returns (seconds for the sample, estimated seconds for the full step, description).
+    """
+    import numpy as np
+    import oracle as orc
+    from paper_2506_08027_b200 import synth
+
+    threads = os.cpu_count() or 1
+    r = sample_rows
+    x = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.gaussian((r, H), synth.seed_for(2, 0))))
+    w = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.gaussian((r, H), synth.seed_for(2, 1), 0.02)))
+    dy = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.output_gradient((r, F), synth.seed_for(2, 2))))
+    t0 = time.perf_counter()
+    q = {}
+    for name, t in (("x", x), ("w", w), ("dy", dy)):
+        q[name, "r"] = orc.quantize_threads(t, orc.ROW, orc.RULE_PAPER, orc.E4M3, threads)
+        q[name, "c"] = orc.quantize_threads(t, orc.COL, orc.RULE_PAPER, orc.E4M3, threads)
+    t_cast = time.perf_counter() - t0
+    cast_full = t_cast * (T * H + F * H + T * F) / float(r * H + r * H + r * F)
+    # GEMM sample: r x r outputs of fprop over the full K = H (decoded FP64 operands, two products)
+    t0 = time.perf_counter()
+    d, s = orc.gemm_f64(q["x", "r"][0], q["x", "r"][1], q["w", "r"][0], q["w", "r"][1])
+    t_gemm = time.perf_counter() - t0
+    gemm_full = t_gemm * STEP_FLOP / (2.0 * r * r * H)
+    desc = ("%d rows of X, W, dY quantized in both orientations on %d threads; %dx%dx%d FP64 product "
+            "(+|A||B| bound product) via numpy; scaled linearly to the full step" % (r, threads, r, r, H))
+    return t_cast + t_gemm, cast_full + gemm_full, desc, threads
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample_seconds(64)
+    times, full = [], []
+    desc, threads = "", 1
+    for _ in range(args.steps):
+        s, f, desc, threads = oracle_sample_seconds(1024)
+        times.append(s)
+        full.append(f)
+    est = statistics.mean(full)
+    value = STEP_FLOP / est / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sampled": True},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ GPU arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_08027_b200 import binding as B
+    from paper_2506_08027_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback exists)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()  # fail loudly if the CUDA library is missing
+
+    dev = "cuda"
+    # each rank draws its own batch (data parallel: per-GPU work is fixed, no exchange on the path)
+    X = synth.device_tensor("activation", (T, H), synth.seed_for(2, 0) + 1000 * rank)
+    W = synth.device_tensor("weight", (F, H), synth.seed_for(2, 1))
+    dY = synth.device_tensor("output_gradient", (T, F), synth.seed_for(2, 2) + 1000 * rank)
+    qX = B.alloc_quantize_outputs(T, H, B.BOTH, B.SF_SWIZZLED)
+    qW = B.alloc_quantize_outputs(F, H, B.BOTH, B.SF_SWIZZLED)
+    qdY = B.alloc_quantize_outputs(T, F, B.BOTH, B.SF_SWIZZLED)
+    Y = torch.empty((T, F), dtype=torch.bfloat16, device=dev)
+    dX = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
+    dW = torch.empty((F, H), dtype=torch.bfloat16, device=dev)
+    P, E, S = B.RULE_PAPER, B.E4M3, B.SF_SWIZZLED
+
+    def step(ev=None):
+        def mark(i):
+            if ev is not None:
+                ev[i].record()
+        mark(0); B.mxfp8_quantize(X, B.BOTH, P, E, *qX, S)
+        mark(1); B.mxfp8_quantize(W, B.BOTH, P, E, *qW, S)
+        mark(2); B.mxfp8_quantize(dY, B.BOTH, P, E, *qdY, S)
+        mark(3); B.mxfp8_gemm(qX[0], qX[1], qW[0], qW[1], T, F, H, B.K_MAJOR, B.K_MAJOR, E, E, Y)
+        mark(4); B.mxfp8_gemm(qdY[0], qdY[1], qW[2], qW[3], T, H, F, B.K_MAJOR, B.MN_MAJOR, E, E, dX)
+        mark(5); B.mxfp8_gemm(qdY[2], qdY[3], qX[2], qX[3], F, H, T, B.MN_MAJOR, B.MN_MAJOR, E, E, dW)
+        mark(6)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    if B.mxfp8_device_status() != 0:
+        raise SystemExit("device status word reports a timeout during warm-up")
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- timed region 1: K whole steps, device time, max over ranks
+    launches0 = B.mxfp8_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = B.mxfp8_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+
+    # ---- timed region 2: the same steps with an event before every launch -> per-kernel durations
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
+    for k in range(args.steps):
+        step(evs[k])
+    torch.cuda.synchronize()
+    dur = [[evs[k][i].elapsed_time(evs[k][i + 1]) for i in range(6)] for k in range(args.steps)]
+    mean = [statistics.mean(d[i] for d in dur) for i in range(6)]
+    cast_ms = sum(mean[0:3])
+    gemm_ms = dict(zip(("fprop", "dgrad", "wgrad"), mean[3:6]))
+    status = B.mxfp8_device_status()
+
+    # ---- end to end through the host-buffer C-ABI call (pinned host memory, copies inside)
+    e2e = None
+    if not args.no_e2e:
+        hx, hw, hdy = (t.cpu().pin_memory() for t in (X, W, dY))
+        hy = torch.empty((T, F), dtype=torch.bfloat16).pin_memory()
+        hdx = torch.empty((T, H), dtype=torch.bfloat16).pin_memory()
+        hdw = torch.empty((F, H), dtype=torch.bfloat16).pin_memory()
+        ws = torch.empty(B.mxfp8_linear_host_ws_bytes(T, H, F), dtype=torch.uint8, device=dev)
+        B.mxfp8_linear_host(hx, hw, hdy, P, hy, hdx, hdw, ws)
+        n_e2e = max(1, min(args.steps, 5))
+        barrier()
+        t0 = time.perf_counter()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(n_e2e):
+            B.mxfp8_linear_host(hx, hw, hdy, P, hy, hdx, hdw, ws)
+        g1.record()
+        barrier()
+        e2e_ms = g0.elapsed_time(g1) / n_e2e
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        assert torch.equal(hy.cuda(), Y), "host-buffer path and device path disagree"
+        e2e = {"value": world * STEP_FLOP / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": (T * H + F * H + T * F) * 2, "d2h_bytes_per_step": (T * F + T * H + F * H) * 2,
+               "steps": n_e2e}
+        del ws
+
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    fp8_peak = 2.0 * peaks["bf16_tflops"]                      # FP8 = 2x the BF16 tensor rate (Table 1)
+    gemm_tflops = {k: 2.0 * m * n * kk / (gemm_ms[k] * 1e-3) / 1e12 for k, (m, n, kk) in GEMM_SHAPES.items()}
+    gemm_all = STEP_FLOP / (sum(gemm_ms.values()) * 1e-3) / 1e12
+    cast_gbs = CAST_BYTES / (cast_ms * 1e-3) / 1e9
+    dom = max(gemm_ms, key=gemm_ms.get)                         # dominant kernel = slowest GEMM launch
+    value = world * STEP_FLOP / (ms_step * 1e-3) / 1e12
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        s, f, desc, threads = oracle_sample_seconds(8192)
+        cpu = {"value": STEP_FLOP / f / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+               "sample": desc, "sample_seconds": s}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8_e4m3 x fp8_e4m3 -> f32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: 192 MB of BF16 sources and 590 MB of outputs per step",
+                   "parallelism": "dp%d (independent batches, no collective)" % world},
+        "cast": {"value": cast_gbs, "unit": "GB/s", "ms": cast_ms, "bytes": CAST_BYTES,
+                 "frac_of_measured_copy": cast_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": cast_gbs / NOMINAL_HBM_GBS},
+        "gemm": {"value": gemm_all, "unit": "TFLOP/s", "ms": gemm_ms, "tflops": gemm_tflops,
+                 "frac_of_2x_measured_bf16": gemm_all / fp8_peak, "frac_of_nominal_4.5PF": gemm_all / NOMINAL_FP8_TFLOPS},
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel<256> (%s)" % dom, "achieved": gemm_tflops[dom],
+                     "peak": fp8_peak, "unit": "TFLOP/s", "frac": gemm_tflops[dom] / fp8_peak,
+                     "peak_source": "2 x %s bf16 burst TFLOP/s (Table 1: MXFP8 = 2x BF16)" % peaks["source"],
+                     "traffic": None},
+        "roofline_cast": {"bound": "hbm", "kernel": "quantize_kernel<bf16,e4m3,both>", "achieved": cast_gbs,
+                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cast_gbs / peaks["hbm_gbs"],
+                          "peak_source": peaks["source"], "traffic": None},
+        "e2e": e2e, "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_case(args):
+    """One kernel on one small case, a few launches, nothing else: the target of ncu captures.
+    quantize: BF16 8192x8192 in both orientations; gemm: the 8192x8192x2048 fprop product;
+    dequantize: 8192x8192 row-blocked bytes to BF16."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from paper_2506_08027_b200 import synth
+    torch.cuda.set_device(0)
+    n = 8192
+    P, E, S = B.RULE_PAPER, B.E4M3, B.SF_SWIZZLED
+    x = synth.device_tensor("activation", (n, n), 1)
+    q = B.alloc_quantize_outputs(n, n, B.BOTH, S)
+    reps = max(1, args.steps)
+    if args.case == "quantize":
+        for _ in range(reps):
+            B.mxfp8_quantize(x, B.BOTH, P, E, *q, S)
+    elif args.case == "dequantize":
+        B.mxfp8_quantize(x, B.BOTH, P, E, *q, S)
+        dst = torch.empty_like(x)
+        for _ in range(reps):
+            B.mxfp8_dequantize(q[0], q[1], B.ROW, E, S, dst)
+    else:
+        a = synth.device_tensor("activation", (T, H), 2)
+        w = synth.device_tensor("weight", (F, H), 3)
+        qa = B.alloc_quantize_outputs(T, H, B.ROW, S)
+        qw = B.alloc_quantize_outputs(F, H, B.ROW, S)
+        B.mxfp8_quantize(a, B.ROW, P, E, *qa, S)
+        B.mxfp8_quantize(w, B.ROW, P, E, *qw, S)
+        y = torch.empty((T, F), dtype=torch.bfloat16, device="cuda")
+        for _ in range(reps):
+            B.mxfp8_gemm(qa[0], qa[1], qw[0], qw[1], T, F, H, B.K_MAJOR, B.K_MAJOR, E, E, y)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": args.case, "launches": int(B.mxfp8_launch_count()), "device_status": B.mxfp8_device_status()}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "gemm"],
+                    help="run one kernel on one small case and exit (for profiler captures)")
+    args = ap.parse_args()
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -173,6 +173,26 @@ int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64
                         void* q_row_host, void* s_row_host, void* q_col_host, void* s_col_host,
                         int sf_layout, void* dev_ws, size_t dev_ws_bytes, void* stream);
 
+
+/*
+ * mxfp8_linear_host -- one training step of a linear layer Y = X * W^T through the MXFP8 path
+ * (Sec. 3.2, the FPROP / DGRAD / WGRAD workflow), with HOST inputs and outputs:
+ *   X [T, H], W [F, H], dY [T, F] in BF16 (host) are copied to the device, each is converted
+ *   once to MXFP8-E4M3 in BOTH orientations under `scale_rule`, then
+ *     FPROP  Y  [T, F] = X  * W^T   (row-blocked X,  row-blocked W)
+ *     DGRAD  dX [T, H] = dY * W     (row-blocked dY, column-blocked W)
+ *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
+ *   run as block-scaled GEMMs with BF16 output, and Y, dX, dW are copied back to the host.
+ * T, H, F must be multiples of 128.  dev_ws: device scratch of mxfp8_linear_host_ws_bytes(),
+ * 256-byte aligned.  Waits for `stream` before returning.  (The composition is the paper's
+ * workflow; the host-buffer packaging has no counterpart in the paper.)
+ */
+size_t mxfp8_linear_host_ws_bytes(int64_t T, int64_t H, int64_t F);
+int mxfp8_linear_host(const void* x_host, const void* w_host, const void* dy_host,
+                      int64_t T, int64_t H, int64_t F, int scale_rule,
+                      void* y_host, void* dx_host, void* dw_host,
+                      void* dev_ws, size_t dev_ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

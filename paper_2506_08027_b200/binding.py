@@ -24,6 +24,7 @@ EXPORTS = (
     "mxfp8_quantize", "mxfp8_dequantize", "mxfp8_gemm", "mxfp8_scale_bytes", "mxfp8_sf_offset",
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
+    "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host",
 )
 
 
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host_ws_bytes.argtypes = [i, i64, i64, i]
         L.mxfp8_quantize_host.restype = i
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
+        L.mxfp8_linear_host_ws_bytes.restype = sz
+        L.mxfp8_linear_host_ws_bytes.argtypes = [i64, i64, i64]
+        L.mxfp8_linear_host.restype = i
+        L.mxfp8_linear_host.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
         _lib = L
     return _lib
 
@@ -187,3 +192,17 @@ def mxfp8_quantize_host(src_host: torch.Tensor, orientation: int, scale_rule: in
                                      _ptr(q_col_host), _ptr(s_col_host), sf_layout, _ptr(dev_ws),
                                      dev_ws.numel() * dev_ws.element_size(), _stream(stream)),
            "mxfp8_quantize_host")
+
+
+def mxfp8_linear_host_ws_bytes(T: int, H: int, F: int) -> int:
+    return int(lib().mxfp8_linear_host_ws_bytes(T, H, F))
+
+
+def mxfp8_linear_host(x_host, w_host, dy_host, scale_rule: int, y_host, dx_host, dw_host,
+                      dev_ws: torch.Tensor, stream=None) -> None:
+    T, H = x_host.shape
+    F = w_host.shape[0]
+    _check(lib().mxfp8_linear_host(_ptr(x_host), _ptr(w_host), _ptr(dy_host), T, H, F, scale_rule,
+                                   _ptr(y_host), _ptr(dx_host), _ptr(dw_host), _ptr(dev_ws),
+                                   dev_ws.numel() * dev_ws.element_size(), _stream(stream)),
+           "mxfp8_linear_host")

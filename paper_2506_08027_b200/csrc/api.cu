@@ -96,3 +96,78 @@ extern "C" int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t 
         }
     return cudaStreamSynchronize(st) == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
+
+namespace {
+struct LinearWs {
+    char* src[3];      // X, W, dY (bf16)
+    char* q[3][2];     // row / col quantized copies
+    char* s[3][2];     // row / col scales (swizzled)
+    char* out[3];      // Y, dX, dW (bf16)
+    size_t total;
+};
+
+LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F)
+{
+    const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
+    const int64_t outs[3][2] = {{T, F}, {T, H}, {F, H}};
+    LinearWs w{};
+    size_t off = 0;
+    auto take = [&](size_t n) { char* p = base ? base + off : nullptr; off += up256(n); return p; };
+    for (int t = 0; t < 3; ++t) {
+        w.src[t] = take((size_t)shp[t][0] * shp[t][1] * 2);
+        for (int o = 0; o < 2; ++o) {
+            w.q[t][o] = take((size_t)shp[t][0] * shp[t][1]);
+            w.s[t][o] = take(mxfp8_scale_bytes(shp[t][0], shp[t][1], o + 1, MXFP8_SF_SWIZZLED));
+        }
+    }
+    for (int t = 0; t < 3; ++t) w.out[t] = take((size_t)outs[t][0] * outs[t][1] * 2);
+    w.total = off;
+    return w;
+}
+}  // namespace
+
+extern "C" size_t mxfp8_linear_host_ws_bytes(int64_t T, int64_t H, int64_t F)
+{
+    if (T <= 0 || H <= 0 || F <= 0) return 0;
+    return plan_linear(nullptr, T, H, F).total;
+}
+
+extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const void* dy_host,
+                                 int64_t T, int64_t H, int64_t F, int scale_rule,
+                                 void* y_host, void* dx_host, void* dw_host,
+                                 void* dev_ws, size_t dev_ws_bytes, void* stream)
+{
+    if (!x_host || !w_host || !dy_host || !y_host || !dx_host || !dw_host || !dev_ws) return MXFP8_ERR_NULL;
+    if (T <= 0 || H <= 0 || F <= 0) return MXFP8_ERR_SHAPE;
+    if ((T % 128) || (H % 128) || (F % 128)) return MXFP8_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(dev_ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
+    if (dev_ws_bytes < mxfp8_linear_host_ws_bytes(T, H, F)) return MXFP8_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F);
+    const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
+    const void* hsrc[3] = {x_host, w_host, dy_host};
+    for (int t = 0; t < 3; ++t) {
+        if (cudaMemcpyAsync(w.src[t], hsrc[t], (size_t)shp[t][0] * shp[t][1] * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return MXFP8_ERR_CUDA;
+        const int rc = mxfp8_quantize(w.src[t], MXFP8_BF16, shp[t][0], shp[t][1], MXFP8_BOTH, scale_rule, MXFP8_E4M3,
+                                      w.q[t][0], w.s[t][0], w.q[t][1], w.s[t][1], MXFP8_SF_SWIZZLED, stream);
+        if (rc != MXFP8_OK) return rc;
+    }
+    enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
+    int rc = mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR,
+                        MXFP8_E4M3, MXFP8_E4M3, w.out[0], MXFP8_BF16, nullptr, nullptr, 0, stream);
+    if (rc != MXFP8_OK) return rc;
+    rc = mxfp8_gemm(w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR,
+                    MXFP8_E4M3, MXFP8_E4M3, w.out[1], MXFP8_BF16, nullptr, nullptr, 0, stream);
+    if (rc != MXFP8_OK) return rc;
+    rc = mxfp8_gemm(w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR,
+                    MXFP8_E4M3, MXFP8_E4M3, w.out[2], MXFP8_BF16, nullptr, nullptr, 0, stream);
+    if (rc != MXFP8_OK) return rc;
+    void* hout[3] = {y_host, dx_host, dw_host};
+    const int64_t outs[3][2] = {{T, F}, {T, H}, {F, H}};
+    for (int t = 0; t < 3; ++t)
+        if (cudaMemcpyAsync(hout[t], w.out[t], (size_t)outs[t][0] * outs[t][1] * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return MXFP8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MXFP8_ERR_CUDA;
+    return mxfp8_device_status(stream);
+}
