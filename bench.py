@@ -325,7 +325,8 @@ def run_ours(args):
 
 def run_case(args):
     """One kernel on one small case, a few launches, nothing else: the target of ncu captures.
-    quantize: BF16 8192x8192 in both orientations; gemm: the 8192x8192x2048 fprop product;
+    quantize: BF16 8192x8192 in both orientations; gemm: the 8192x8192x2048 fprop product
+    (gemm8k: 8192^3);
     dequantize: 8192x8192 row-blocked bytes to BF16."""
     import torch
     from paper_2506_08027_b200 import binding as B
@@ -345,15 +346,16 @@ def run_case(args):
         for _ in range(reps):
             B.mxfp8_dequantize(q[0], q[1], B.ROW, E, S, dst)
     else:
-        a = synth.device_tensor("activation", (T, H), 2)
-        w = synth.device_tensor("weight", (F, H), 3)
-        qa = B.alloc_quantize_outputs(T, H, B.ROW, S)
-        qw = B.alloc_quantize_outputs(F, H, B.ROW, S)
+        m_, n_, k_ = (T, F, H) if args.case == "gemm" else (8192, 8192, 8192)
+        a = synth.device_tensor("activation", (m_, k_), 2)
+        w = synth.device_tensor("weight", (n_, k_), 3)
+        qa = B.alloc_quantize_outputs(m_, k_, B.ROW, S)
+        qw = B.alloc_quantize_outputs(n_, k_, B.ROW, S)
         B.mxfp8_quantize(a, B.ROW, P, E, *qa, S)
         B.mxfp8_quantize(w, B.ROW, P, E, *qw, S)
-        y = torch.empty((T, F), dtype=torch.bfloat16, device="cuda")
+        y = torch.empty((m_, n_), dtype=torch.bfloat16, device="cuda")
         for _ in range(reps):
-            B.mxfp8_gemm(qa[0], qa[1], qw[0], qw[1], T, F, H, B.K_MAJOR, B.K_MAJOR, E, E, y)
+            B.mxfp8_gemm(qa[0], qa[1], qw[0], qw[1], m_, n_, k_, B.K_MAJOR, B.K_MAJOR, E, E, y)
     torch.cuda.synchronize()
     print(json.dumps({"case": args.case, "launches": int(B.mxfp8_launch_count()), "device_status": B.mxfp8_device_status()}))
 
@@ -366,7 +368,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "gemm"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "gemm", "gemm8k"],
                     help="run one kernel on one small case and exit (for profiler captures)")
     args = ap.parse_args()
     if args.case:

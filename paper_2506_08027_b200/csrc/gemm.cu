@@ -2,16 +2,28 @@
 // (Sec. 2 and App. A.3: per 32-element block dot product of the FP8 elements, scaled by the
 // two blocks' UE8M0 scales, accumulated in FP32).
 //
-// Structure (one persistent CTA per SM, 192 threads, warp-specialised):
+// Structure (one persistent CTA per SM, 320 threads, warp-specialised):
 //   warp 0      TMA producer: A/B tiles (128-byte swizzle) and 512-byte scale atoms -> smem ring
 //   warp 1      MMA issuer (one thread): tcgen05.cp scales smem->TMEM, then
 //               tcgen05.mma.kind::mxf8f6f4.block_scale over the K loop; owns TMEM alloc/dealloc
-//   warps 2..5  epilogue: tcgen05.ld the FP32 accumulator from TMEM, convert, store D
+//   Two variants of one kernel template:
+//     PAIR = true : clusters of two CTAs work on one 256 x 256 tile with cta_group::2 MMAs.  Each
+//                   CTA loads its own 128 rows of A and its own 128-row half of B (no multicast),
+//                   all loads complete on the leader CTA's mbarrier, the leader issues the MMAs
+//                   for both, and each CTA drains its own 128 x 256 accumulator.  The tensor
+//                   core then reads only 8 KB of shared memory per CTA per MMA.
+//     PAIR = false: one CTA per 128 x BN tile (BN = 256 or 128) with cta_group::1, used when
+//                   M is not a multiple of 256.
+//   warps 2..9  epilogue: each warp drains its 32 lanes x BN/2 columns of the FP32 accumulator
+//               into registers (tcgen05.ld), releases the accumulator at once so the next
+//               tile's MMAs can start, then converts and writes D through a private 2 KB
+//               64-byte-swizzled staging buffer with TMA stores
 //   A CTA tile is 128 x BN (BN = 256 or 128) with K step 128 (= 4 MMAs of K = 32, one scale
 //   byte per row per MMA = one 4-byte TMEM column entry per K step).
 //   Every mbarrier wait is bounded: on expiry the kernel records MXFP8_ERR_DEVICE_TIMEOUT in
 //   the device status word, raises an abort flag that all roles poll, drains and exits.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "mxfp8_device.cuh"
 #include "mxfp8_host.h"
@@ -31,11 +43,13 @@ int read_and_clear_device_status(cudaStream_t stream)
 
 namespace {
 
-constexpr int BM = 128;            // tile rows (TMEM lanes)
+constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 128;            // K bytes per pipeline stage = one 128-byte swizzle row
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;
+constexpr int EPI_WARPS = 8;
+constexpr int EPI_BUF_BYTES = 2048;   // 32 rows x 64 bytes per epilogue warp
 constexpr int TMEM_COLS = 512;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // bounded waits give up after 2 s
+constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;  // bounded waits give up after 1 s
 
 struct GemmParams {
     int64_t M, N, K;
@@ -43,26 +57,33 @@ struct GemmParams {
     int a_elem, b_elem;
     int out_dtype;
     int tiles_m, tiles_n, num_tiles, num_kb;
+    int group_m;          // tile rasterisation: M-tiles per group (L2 reuse)
 };
 
-template <int BN> struct Cfg {
+// BN = accumulator columns per CTA = N extent of one tile.  In PAIR mode a tile has 2*BM rows.
+template <int BN, bool PAIR> struct Cfg {
     static constexpr int ACC_STAGES = (BN == 256) ? 1 : 2;
-    static constexpr int STAGES = (BN == 256) ? 4 : 6;
+    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // B rows this CTA loads
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
+    static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int SFB_ATOMS = BN / 128;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 512 + 512 * SFB_ATOMS;
+    static constexpr int STAGES = (206 * 1024) / STAGE_BYTES > 8 ? 8 : (206 * 1024) / STAGE_BYTES;
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;          // TMEM columns of scales per stage
     static constexpr int SF_COL0 = ACC_STAGES * BN;            // first scale column
-    static constexpr uint32_t STAGE_TX = A_BYTES + B_BYTES + 512 + 512 * SFB_ATOMS;
+    static constexpr uint32_t STAGE_TX = (PAIR ? 2u : 1u) * STAGE_BYTES;   // bytes landing per stage on the leader's barrier
     static constexpr int SMEM_A = 0;
     static constexpr int SMEM_B = SMEM_A + STAGES * A_BYTES;
     static constexpr int SMEM_SFA = SMEM_B + STAGES * B_BYTES;
     static constexpr int SMEM_SFB = SMEM_SFA + STAGES * 512;
-    static constexpr int SMEM_BAR = SMEM_SFB + STAGES * 512 * SFB_ATOMS;
+    static constexpr int SMEM_EPI = SMEM_SFB + STAGES * 512 * SFB_ATOMS;      // 8 x 2 KB, 512-aligned
     static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES + 1;
+    static constexpr int SMEM_BAR = SMEM_EPI + EPI_WARPS * EPI_BUF_BYTES;
     static constexpr int SMEM_MISC = SMEM_BAR + NUM_BARS * 8;  // tmem pointer, abort flag
     static constexpr int SMEM_TOTAL = SMEM_MISC + 16 + 1024;   // + slack to align the base to 1024
     static_assert(SF_COL0 + STAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
+    static_assert(SMEM_TOTAL <= 227 * 1024, "shared memory budget");
+    static_assert(SMEM_EPI % 512 == 0, "staging buffers need 512-byte alignment for the 64-byte swizzle");
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -80,6 +101,28 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// arrive on a barrier addressed in the cluster's shared window (possibly the peer CTA's)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// cluster-window address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -90,6 +133,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
+// One lane of a converged warp, chosen by the hardware.  Code around it stays warp-uniform, so
+// addresses and descriptors are computed once in the uniform datapath instead of per lane.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ uint64_t global_timer()
 {
     uint64_t t;
@@ -97,7 +152,7 @@ __device__ __forceinline__ uint64_t global_timer()
     return t;
 }
 // Bounded wait: false when the abort flag is up or the time limit passed (the latter also
-// records the timeout and raises the flag for the other roles).
+// records the timeout and raises the flag for the other roles of this CTA).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     uint32_t spins = 0;
@@ -116,37 +171,68 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
+// TMA tile loads.  In PAIR mode the copy lands in this CTA's shared memory while the
+// transaction bytes complete on the mbarrier address given (the leader CTA's barrier).
+template <bool PAIR>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1)
 {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+    if (PAIR)
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+template <bool PAIR>
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
 {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+    if (PAIR)
+        asm volatile(
+            "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// arrive on `bar` (same offset in every CTA of the pair when PAIR) once all MMAs issued so far retire
+template <bool PAIR>
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (PAIR)
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t desc)
 {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+    if (PAIR) asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+    else asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                        uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-        : "memory");
+    if (PAIR)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+            : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
 {
@@ -171,19 +257,31 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 // Block-scaled instruction descriptor: element formats, majorness, N>>3, UE8M0 scales, M>>4.
-__device__ __forceinline__ uint32_t make_idesc(int a_elem, int b_elem, int a_mn, int b_mn, int n)
+__device__ __forceinline__ uint32_t make_idesc(int a_elem, int b_elem, int a_mn, int b_mn, int m, int n)
 {
     return ((uint32_t)a_elem << 7) | ((uint32_t)b_elem << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-           ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24);
 }
 
-template <int BN>
+// Tile rasterisation: tiles are numbered group by group; a group is `group_m` M-tiles tall and
+// spans all N-tiles, M fastest inside it, so the tiles in flight at one time share few distinct
+// A row-blocks and B row-blocks and hit in L2.
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& tm, int& tn)
+{
+    const int per_group = p.group_m * p.tiles_n;
+    const int g = tile / per_group, r = tile - g * per_group;
+    const int gm = min(p.group_m, p.tiles_m - g * p.group_m);
+    tn = r / gm;
+    tm = g * p.group_m + (r - tn * gm);
+}
+
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-            const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb, void* __restrict__ D,
-            const GemmParams p)
+            const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
+            const __grid_constant__ CUtensorMap tmap_d, const GemmParams p)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, PAIR>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;   // 128-byte swizzle needs 1024-byte alignment
@@ -200,56 +298,77 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;   // 0 = leader (issues the MMAs)
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < C::ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < C::ACC_STAGES; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * EPI_WARPS);
+        }
         mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();      // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int64_t atoms_k = p.K >> 7;   // scale atoms along K (4 K-blocks each)
-
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;
+        // The whole warp walks the loop; one elected lane issues the copies.
+        {
+            int s = 0;
+            uint32_t ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-                const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-                const int m0 = tm * BM, n0 = tn * BN;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
-                    const int s = it % C::STAGES;
-                    const uint32_t ph = (it / C::STAGES) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t fb = full_bar(s);
-                    mbar_expect_tx(fb, C::STAGE_TX);
+            const int a_mn = p.a_mn, b_mn = p.b_mn, num_kb = p.num_kb;
+            for (int tile = worker; tile < p.num_tiles && ok; tile += workers) {
+                int tm, tn;
+                tile_coords(p, tile, tm, tn);
+                const int m_atom = tm * (PAIR ? 2 : 1) + (int)cta_rank;      // 128-row block of A / D
+                const int m0 = m_atom * BM;
+                const int n0 = tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);   // first B row this CTA loads
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ph ^ 1u, abort_flag));
+                    if (!ok) break;
+                    // all bytes of the pair are counted on the leader's barrier
+                    const uint32_t fb = PAIR ? map_to_cta(full_bar(s), 0) : full_bar(s);
                     const uint32_t sa = base + C::SMEM_A + s * C::A_BYTES;
                     const uint32_t sb = base + C::SMEM_B + s * C::B_BYTES;
                     const int k0 = kb * BK;
-                    if (!p.a_mn) tma_load_2d(sa, &tmap_a, fb, k0, m0);
-                    else tma_load_2d(sa, &tmap_a, fb, m0, k0);
-                    if (!p.b_mn) {
-                        tma_load_2d(sb, &tmap_b, fb, k0, n0);
-                    } else {
+                    if (elect_one()) {
+                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), C::STAGE_TX);
+                        if (!a_mn) tma_load_2d<PAIR>(sa, &tmap_a, fb, k0, m0);
+                        else tma_load_2d<PAIR>(sa, &tmap_a, fb, m0, k0);
+                        if (!b_mn) {
+                            tma_load_2d<PAIR>(sb, &tmap_b, fb, k0, n0);
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < C::SFB_ATOMS; ++j) tma_load_2d(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0);
+                            for (int j = 0; j < C::B_ROWS / 128; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0);
+                        }
+                        tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, &tmap_sfa, fb, 0, kb, m_atom);
+#pragma unroll
+                        for (int j = 0; j < C::SFB_ATOMS; ++j)      // every CTA needs the scales of all BN columns
+                            tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, &tmap_sfb, fb, 0, kb,
+                                              tn * C::SFB_ATOMS + j);
                     }
-                    bulk_load(base + C::SMEM_SFA + s * 512, sfa + ((int64_t)tm * atoms_k + kb) * 512, 512, fb);
-#pragma unroll
-                    for (int j = 0; j < C::SFB_ATOMS; ++j)
-                        bulk_load(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512,
-                                  sfb + ((int64_t)(tn * C::SFB_ATOMS + j) * atoms_k + kb) * 512, 512, fb);
+                    __syncwarp();
+                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
@@ -258,107 +377,163 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc0 = make_idesc(p.a_elem, p.b_elem, p.a_mn, p.b_mn, BN);
-            uint32_t it = 0, acc_it = 0;
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        // The whole warp walks the loop so that descriptors stay in uniform registers; one
+        // elected lane issues the tcgen05 instructions.
+        if (cta_rank == 0) {
+            const uint32_t idesc0 = make_idesc(p.a_elem, p.b_elem, p.a_mn, p.b_mn, PAIR ? 2 * BM : BM, BN);
+            // Descriptors differ between stages and K steps only in the 14-bit start-address
+            // field (16-byte units): keep the constant upper word and step the lower one.
+            //   K-major : next K step = 32 bytes along the swizzled row (2 units); 8-row groups 1024 B apart.
+            //   MN-major: next K step = 32 K-rows = 4096 bytes (256 units); 8-K-row groups 1024 B apart,
+            //             128-wide MN slabs 16384 B apart.
+            const uint32_t op_hi = (uint32_t)(smem_desc(0, 0, 1024, 2) >> 32);
+            const uint32_t a_lo0 = ((base + C::SMEM_A) >> 4) | (p.a_mn ? (16384u >> 4) << 16 : 0u);
+            const uint32_t b_lo0 = ((base + C::SMEM_B) >> 4) | (p.b_mn ? (16384u >> 4) << 16 : 0u);
+            const uint32_t a_kstep = p.a_mn ? 256u : 2u, b_kstep = p.b_mn ? 256u : 2u;
+            const uint32_t sf_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);   // scales: 32 rows x 16 B, 8-row groups 128 B apart
+            const uint32_t sfa_lo0 = (base + C::SMEM_SFA) >> 4, sfb_lo0 = (base + C::SMEM_SFB) >> 4;
+            auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
+            const int num_kb = p.num_kb;
+            int s = 0;
+            uint32_t ph = 0, acc_it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++acc_it) {
+            for (int tile = worker; tile < p.num_tiles && ok; tile += workers, ++acc_it) {
                 const int as = acc_it % C::ACC_STAGES;
                 const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-                if (!mbar_wait(tempty_bar(as), aph ^ 1u, abort_flag)) { ok = false; break; }
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(tempty_bar(as), aph ^ 1u, abort_flag));
+                if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * BN;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
-                    const int s = it % C::STAGES;
-                    const uint32_t ph = (it / C::STAGES) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), ph, abort_flag));
+                    if (!ok) break;
                     tc_fence_after();
                     const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS;
                     const uint32_t sfb_t = sfa_t + 4;
-                    // scales: 32 rows x 16 bytes per atom, no swizzle, 8-row groups 128 bytes apart
-                    tc_cp_sf(sfa_t, smem_desc(base + C::SMEM_SFA + s * 512, 0, 128, 0));
+                    const uint32_t a_lo = a_lo0 + s * (C::A_BYTES >> 4);
+                    const uint32_t b_lo = b_lo0 + s * (C::B_BYTES >> 4);
+                    if (elect_one()) {
+                        tc_cp_sf<PAIR>(sfa_t, desc64(sfa_lo0 + s * (512 >> 4), sf_hi));
 #pragma unroll
-                    for (int j = 0; j < C::SFB_ATOMS; ++j)
-                        tc_cp_sf(sfb_t + 4 * j, smem_desc(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, 0, 128, 0));
-                    const uint32_t sa = base + C::SMEM_A + s * C::A_BYTES;
-                    const uint32_t sb = base + C::SMEM_B + s * C::B_BYTES;
+                        for (int j = 0; j < C::SFB_ATOMS; ++j)
+                            tc_cp_sf<PAIR>(sfb_t + 4 * j, desc64(sfb_lo0 + (s * C::SFB_ATOMS + j) * (512 >> 4), sf_hi));
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        // K-major: 32 bytes further along the swizzled row; 8-row groups 1024 B apart.
-                        // MN-major: 32 K-rows (4096 B) further; 8-K-row groups 1024 B apart, 128-wide
-                        // MN slabs 16384 B apart.
-                        const uint64_t ad = p.a_mn ? smem_desc(sa + k * 4096, 16384, 1024, 2) : smem_desc(sa + k * 32, 0, 1024, 2);
-                        const uint64_t bd = p.b_mn ? smem_desc(sb + k * 4096, 16384, 1024, 2) : smem_desc(sb + k * 32, 0, 1024, 2);
-                        const uint32_t idesc = idesc0 | ((uint32_t)k << 29) | ((uint32_t)k << 4);
-                        tc_mma(d_tmem, ad, bd, idesc, sfa_t, sfb_t, (uint32_t)((kb | k) != 0));
+                        for (int k = 0; k < 4; ++k) {
+                            const uint32_t idesc = idesc0 | ((uint32_t)k << 29) | ((uint32_t)k << 4);   // scale byte k of the column entry
+                            tc_mma<PAIR>(d_tmem, desc64(a_lo + k * a_kstep, op_hi), desc64(b_lo + k * b_kstep, op_hi), idesc,
+                                         sfa_t, sfb_t, (uint32_t)((kb | k) != 0));
+                        }
+                        tc_commit<PAIR>(empty_bar(s));   // frees the smem stage (in both CTAs) once these MMAs have read it
+                        if (kb == num_kb - 1) tc_commit<PAIR>(tfull_bar(as));
                     }
-                    tc_commit(empty_bar(s));   // frees the smem stage once these MMAs have read it
+                    __syncwarp();
+                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (ok) tc_commit(tfull_bar(as));
             }
             if (!ok) {
                 // let MMAs already issued retire before TMEM is released
-                tc_commit(drain_bar);
+                if (elect_one()) tc_commit<PAIR>(drain_bar);
+                __syncwarp();
                 uint64_t t0 = global_timer();
                 while (!mbar_try_wait(drain_bar, 0) && global_timer() - t0 < WAIT_LIMIT_NS) {}
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        const int q = warp & 3;                 // TMEM lane quadrant this warp may read
-        const int row_in_tile = q * 32 + lane;
+        constexpr int CW = BN / 2;               // accumulator columns per epilogue warp
+        const int q = warp & 3;                  // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;        // which half of the tile's columns
+        const uint32_t buf = base + C::SMEM_EPI + (warp - 2) * EPI_BUF_BYTES;
+        // 64-byte swizzle of the staging buffer: 16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)
+        const uint32_t row_off = buf + lane * 64;
+        const uint32_t sw = (uint32_t)((lane >> 1) & 3);
         uint32_t acc_it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++acc_it) {
-            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+        for (int tile = worker; tile < p.num_tiles && ok; tile += workers, ++acc_it) {
+            int tm, tn;
+            tile_coords(p, tile, tm, tn);
             const int as = acc_it % C::ACC_STAGES;
             const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-            ok = mbar_wait(tfull_bar(as), aph, abort_flag);
-            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (lane == 0) ok = mbar_wait(tfull_bar(as), aph, abort_flag);   // one poller per warp
+            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
             if (!ok) break;
             tc_fence_after();
-            const int64_t row = (int64_t)tm * BM + row_in_tile;
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tc_ld32(t_row + c * 32, v);
-                tc_wait_ld();
-                const int64_t col = (int64_t)tn * BN + c * 32;
-                if (p.out_dtype == MXFP8_FP32) {
-                    float4* d = reinterpret_cast<float4*>(static_cast<float*>(D) + row * p.N + col);
+            uint32_t v[CW];
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN + half * CW;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        d[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                           __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                } else {
-                    uint4* d = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(D) + row * p.N + col);
+            for (int c = 0; c < CW / 32; ++c) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+            tc_wait_ld();
+            // the accumulator now lives in registers: hand TMEM back to the MMA warp of the leader
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
+                else mbar_arrive(tempty_bar(as));
+            }
+
+            const int row0 = (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
+            const int col0 = tn * BN + half * CW;
+            if (p.out_dtype == MXFP8_BF16) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                for (int ch = 0; ch < CW / 32; ++ch) {          // 32 columns = 64 bytes per row
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
                         uint32_t pk[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * j]),
-                                                                           __uint_as_float(v[8 * i + 2 * j + 1]));
-                            pk[j] = *reinterpret_cast<const uint32_t*>(&h);
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[ch * 32 + j * 8 + 2 * e]),
+                                                                            __uint_as_float(v[ch * 32 + j * 8 + 2 * e + 1]));
+                            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
                         }
-                        d[i] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(row_off + (((uint32_t)j ^ sw) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&tmap_d), "r"(col0 + ch * 32), "r"(row0), "r"(buf) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int ch = 0; ch < CW / 16; ++ch) {          // 16 columns = 64 bytes per row
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(row_off + (((uint32_t)j ^ sw) << 4)), "r"(v[ch * 16 + j * 4]), "r"(v[ch * 16 + j * 4 + 1]),
+                                       "r"(v[ch * 16 + j * 4 + 2]), "r"(v[ch * 16 + j * 4 + 3]) : "memory");
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&tmap_d), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(as));
         }
+        // all of this warp's stores must have left shared memory and reached global memory
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __syncwarp();
     }
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();      // nobody leaves while the peer may still signal this CTA's barriers
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
@@ -394,6 +569,35 @@ bool make_tmap(CUtensorMap* map, const void* base, uint64_t inner, uint64_t oute
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Scale buffer in the 128x4 atom layout seen as [mn_atoms][k_atoms][128 x u32]; one box = one atom.
+bool make_tmap_sf(CUtensorMap* map, const void* base, uint64_t mn_atoms, uint64_t k_atoms)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {128, k_atoms, mn_atoms};
+    const cuuint64_t strides[2] = {512, 512 * k_atoms};
+    const cuuint32_t box[3] = {128, 1, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Output matrix D [M, N] row-major: boxes of 32 rows x 64 bytes, 64-byte swizzle (store side).
+bool make_tmap_d(CUtensorMap* map, void* base, uint64_t M, uint64_t N, int out_dtype)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const bool f32 = out_dtype == MXFP8_FP32;
+    const cuuint64_t dims[2] = {N, M};
+    const cuuint64_t strides[1] = {N * (f32 ? 4u : 2u)};
+    const cuuint32_t box[2] = {f32 ? 16u : 32u, 32u};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides,
+              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count()
 {
     static int n = [] {
@@ -405,23 +609,39 @@ int sm_count()
     return n;
 }
 
-template <int BN>
-int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const uint8_t* sfa, const uint8_t* sfb, void* D,
-                GemmParams p, cudaStream_t stream)
+struct GemmMaps { CUtensorMap a, b, sfa, sfb, d; };
+
+template <int BN, bool PAIR>
+int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
 {
-    using C = Cfg<BN>;
-    if (cudaFuncSetAttribute(gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
+    using C = Cfg<BN, PAIR>;
+    auto kernel = gemm_kernel<BN, PAIR>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
         return MXFP8_ERR_CUDA;
-    p.tiles_m = (int)(p.M / BM);
+    p.tiles_m = (int)(p.M / (PAIR ? 2 * BM : BM));
     p.tiles_n = (int)(p.N / BN);
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.num_kb = (int)(p.K / BK);
+    { const char* e = getenv("MXFP8_GROUP_M"); p.group_m = e ? atoi(e) : 8; if (p.group_m < 1) p.group_m = 1; }
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
-    const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-    gemm_kernel<BN><<<grid, GEMM_THREADS, C::SMEM_TOTAL, stream>>>(ta, tb, sfa, sfb, D, p);
+    const int max_workers = PAIR ? sms / 2 : sms;
+    const int workers = p.num_tiles < max_workers ? p.num_tiles : max_workers;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * workers : workers));
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_TOTAL;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, p);
     count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+    return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
 }  // namespace
@@ -443,7 +663,7 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     if (b_elem != MXFP8_E4M3 && b_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs) return MXFP8_ERR_NULL;
-    if (!D && !epi) return MXFP8_ERR_NULL;
+    if (!D) return epi ? MXFP8_ERR_UNSUPPORTED : MXFP8_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || (K % 32)) return MXFP8_ERR_SHAPE;
     if ((M % 128) || (N % 128) || (K % 128)) return MXFP8_ERR_UNSUPPORTED;
     if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
@@ -454,15 +674,18 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     p.M = M; p.N = N; p.K = K;
     p.a_mn = a_major; p.b_mn = b_major; p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
     const bool wide = (N % 256) == 0;
-    const uint32_t bn = wide ? 256 : 128;
-    CUtensorMap ta, tb;
-    const bool oka = a_major == MXFP8_K_MAJOR ? make_tmap(&ta, Aq, (uint64_t)K, (uint64_t)M, 128, 128)
-                                              : make_tmap(&ta, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
-    const bool okb = b_major == MXFP8_K_MAJOR ? make_tmap(&tb, Bq, (uint64_t)K, (uint64_t)N, 128, bn)
-                                              : make_tmap(&tb, Bq, (uint64_t)N, (uint64_t)K, 128, 128);
-    if (!oka || !okb) return MXFP8_ERR_CUDA;
+    const bool pair = wide && (M % 256) == 0;
+    // rows of B one CTA loads per TMA box (K-major B): half a tile in pair mode
+    const uint32_t b_box_rows = pair ? 128u : (wide ? 256u : 128u);
+    GemmMaps m;
+    const bool oka = a_major == MXFP8_K_MAJOR ? make_tmap(&m.a, Aq, (uint64_t)K, (uint64_t)M, 128, 128)
+                                              : make_tmap(&m.a, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
+    const bool okb = b_major == MXFP8_K_MAJOR ? make_tmap(&m.b, Bq, (uint64_t)K, (uint64_t)N, 128, b_box_rows)
+                                              : make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)K, 128, 128);
+    const bool oks = make_tmap_sf(&m.sfa, As, (uint64_t)(M / 128), (uint64_t)(K / 128)) &&
+                     make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(K / 128));
+    if (!oka || !okb || !oks || !make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype)) return MXFP8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const uint8_t* sa = static_cast<const uint8_t*>(As);
-    const uint8_t* sb = static_cast<const uint8_t*>(Bs);
-    return wide ? launch_gemm<256>(ta, tb, sa, sb, D, p, st) : launch_gemm<128>(ta, tb, sa, sb, D, p, st);
+    if (pair) return launch_gemm<256, true>(m, p, st);
+    return wide ? launch_gemm<256, false>(m, p, st) : launch_gemm<128, false>(m, p, st);
 }
