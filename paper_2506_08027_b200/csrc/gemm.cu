@@ -24,6 +24,7 @@
 //   the device status word, raises an abort flag that all roles poll, drains and exits.
 #include <cuda.h>
 #include <cstdlib>
+#include <cstring>
 
 #include "mxfp8_device.cuh"
 #include "mxfp8_host.h"
@@ -58,20 +59,26 @@ struct GemmParams {
     int out_dtype;
     int tiles_m, tiles_n, num_tiles, num_kb;
     int group_m;          // tile rasterisation: M-tiles per group (L2 reuse)
+    uint32_t stage_tx;    // bytes that land per pipeline stage on the (leader's) full barrier
 };
 
-// BN = accumulator columns per CTA = N extent of one tile.  In PAIR mode a tile has 2*BM rows.
+// BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
+// tile has 2*BM rows.  BN = 256 leaves room for one accumulator only (2 x 256 columns would fill
+// TMEM and the scales need columns too); BN = 192 and 128 double-buffer it, so the epilogue of
+// one tile runs under the MMAs of the next.
 template <int BN, bool PAIR> struct Cfg {
     static constexpr int ACC_STAGES = (BN == 256) ? 1 : 2;
-    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // B rows this CTA loads
+    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // B rows (N indices) this CTA loads
+    static constexpr int B_SLABS = (B_ROWS + 127) / 128;       // 128-wide slabs when B is MN-major
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = B_ROWS * BK;
-    static constexpr int SFB_ATOMS = BN / 128;
+    static constexpr int B_BYTES_K = B_ROWS * BK;              // bytes landing per stage, K-major B
+    static constexpr int B_BYTES_MN = B_SLABS * 128 * BK;      // bytes landing per stage, MN-major B
+    static constexpr int B_BYTES = B_BYTES_MN;                 // reservation (>= both)
+    static constexpr int SFB_ATOMS = (BN + 127) / 128;         // a BN-wide tile starting at a multiple of 64 spans this many atoms
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 512 + 512 * SFB_ATOMS;
     static constexpr int STAGES = (206 * 1024) / STAGE_BYTES > 8 ? 8 : (206 * 1024) / STAGE_BYTES;
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;          // TMEM columns of scales per stage
     static constexpr int SF_COL0 = ACC_STAGES * BN;            // first scale column
-    static constexpr uint32_t STAGE_TX = (PAIR ? 2u : 1u) * STAGE_BYTES;   // bytes landing per stage on the leader's barrier
     static constexpr int SMEM_A = 0;
     static constexpr int SMEM_B = SMEM_A + STAGES * A_BYTES;
     static constexpr int SMEM_SFA = SMEM_B + STAGES * B_BYTES;
@@ -84,6 +91,7 @@ template <int BN, bool PAIR> struct Cfg {
     static_assert(SF_COL0 + STAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
     static_assert(SMEM_TOTAL <= 227 * 1024, "shared memory budget");
     static_assert(SMEM_EPI % 512 == 0, "staging buffers need 512-byte alignment for the 64-byte swizzle");
+    static_assert((BN / 2) % 32 == 0, "each epilogue warp owns whole 32-column chunks");
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -170,6 +178,39 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
     return true;
+}
+// Whole-warp wait of the two latency-critical roles (TMA producer, MMA issuer): all lanes spin
+// on the non-blocking test so the warp reacts within a few cycles of the phase flip; the
+// suspending try_wait costs a wake-up latency that the smem ring cannot hide.
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    uint32_t spins = 0;
+    uint64_t t0 = 0;
+    bool ok = true;
+    while (!mbar_test_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) { ok = false; break; }
+            const uint64_t now = global_timer();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
+                ok = false;
+                break;
+            }
+        }
+    }
+    return __all_sync(0xFFFFFFFFu, ok);
 }
 // TMA tile loads.  In PAIR mode the copy lands in this CTA's shared memory while the
 // transaction bytes complete on the mbarrier address given (the leader CTA's barrier).
@@ -331,20 +372,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        // The whole warp walks the loop; one elected lane issues the copies.
+        // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
+        // ring-depth-unrolled loop as the MMA warp.
         {
-            int s = 0;
+            const int a_mn = p.a_mn, b_mn = p.b_mn, num_kb = p.num_kb;
+            const int my_tiles = (p.num_tiles - worker + workers - 1) / workers;
+            const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_kb;
+            int kb = 0, tile = worker;
+            int m_atom = 0, m0 = 0, n0 = 0, sfb_atom0 = 0;
             uint32_t ph = 0;
             bool ok = true;
-            const int a_mn = p.a_mn, b_mn = p.b_mn, num_kb = p.num_kb;
-            for (int tile = worker; tile < p.num_tiles && ok; tile += workers) {
-                int tm, tn;
-                tile_coords(p, tile, tm, tn);
-                const int m_atom = tm * (PAIR ? 2 : 1) + (int)cta_rank;      // 128-row block of A / D
-                const int m0 = m_atom * BM;
-                const int n0 = tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);   // first B row this CTA loads
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ph ^ 1u, abort_flag));
+            for (uint32_t g0 = 0; g0 < total && ok; g0 += C::STAGES) {
+#pragma unroll
+                for (int s = 0; s < C::STAGES; ++s) {
+                    if (g0 + s >= total) break;
+                    if (kb == 0) {
+                        int tm, tn;
+                        tile_coords(p, tile, tm, tn);
+                        m_atom = tm * (PAIR ? 2 : 1) + (int)cta_rank;             // 128-row block of A / D
+                        m0 = m_atom * BM;
+                        n0 = tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);    // first B row this CTA loads
+                        sfb_atom0 = (tn * BN) >> 7;                               // scale atom holding the tile's first column
+                    }
+                    ok = warp_wait(empty_bar(s), ph ^ 1u, abort_flag);
                     if (!ok) break;
                     // all bytes of the pair are counted on the leader's barrier
                     const uint32_t fb = PAIR ? map_to_cta(full_bar(s), 0) : full_bar(s);
@@ -352,24 +402,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     const uint32_t sb = base + C::SMEM_B + s * C::B_BYTES;
                     const int k0 = kb * BK;
                     if (elect_one()) {
-                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), C::STAGE_TX);
+                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), p.stage_tx);
                         if (!a_mn) tma_load_2d<PAIR>(sa, &tmap_a, fb, k0, m0);
                         else tma_load_2d<PAIR>(sa, &tmap_a, fb, m0, k0);
                         if (!b_mn) {
                             tma_load_2d<PAIR>(sb, &tmap_b, fb, k0, n0);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < C::B_ROWS / 128; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0);
+                            for (int j = 0; j < C::B_SLABS; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0);
                         }
                         tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, &tmap_sfa, fb, 0, kb, m_atom);
 #pragma unroll
                         for (int j = 0; j < C::SFB_ATOMS; ++j)      // every CTA needs the scales of all BN columns
                             tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, &tmap_sfb, fb, 0, kb,
-                                              tn * C::SFB_ATOMS + j);
+                                              sfb_atom0 + j);
                     }
                     __syncwarp();
-                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+                    if (++kb == num_kb) { kb = 0; tile += workers; }
                 }
+                ph ^= 1u;
             }
             if (!ok) {
                 // give copies already in flight time to land before the CTA's smem is released
@@ -379,7 +430,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         // The whole warp walks the loop so that descriptors stay in uniform registers; one
-        // elected lane issues the tcgen05 instructions.
+        // elected lane issues the tcgen05 instructions.  The loop runs over all K blocks of all
+        // tiles of this worker and is unrolled by the ring depth, so the stage index is a
+        // compile-time constant and every descriptor is "loop-invariant base + immediate".
         if (cta_rank == 0) {
             const uint32_t idesc0 = make_idesc(p.a_elem, p.b_elem, p.a_mn, p.b_mn, PAIR ? 2 * BM : BM, BN);
             // Descriptors differ between stages and K steps only in the 14-bit start-address
@@ -395,24 +448,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t sfa_lo0 = (base + C::SMEM_SFA) >> 4, sfb_lo0 = (base + C::SMEM_SFB) >> 4;
             auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
             const int num_kb = p.num_kb;
-            int s = 0;
-            uint32_t ph = 0, acc_it = 0;
+            const int my_tiles = (p.num_tiles - worker + workers - 1) / workers;
+            const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_kb;
+            int kb = 0, tile = worker;
+            uint32_t ph = 0, acc_it = 0, d_tmem = tmem_base, sfb_skip = 0;
+            int as = 0;
             bool ok = true;
-            for (int tile = worker; tile < p.num_tiles && ok; tile += workers, ++acc_it) {
-                const int as = acc_it % C::ACC_STAGES;
-                const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(tempty_bar(as), aph ^ 1u, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + as * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), ph, abort_flag));
+            for (uint32_t g0 = 0; g0 < total && ok; g0 += C::STAGES) {
+#pragma unroll
+                for (int s = 0; s < C::STAGES; ++s) {
+                    if (g0 + s >= total) break;
+                    if (kb == 0) {   // first K block of a tile: the accumulator must have been drained
+                        as = acc_it % C::ACC_STAGES;
+                        const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
+                        ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag);
+                        if (!ok) break;
+                        d_tmem = tmem_base + as * BN;
+                        int tm, tn;
+                        tile_coords(p, tile, tm, tn);
+                        // a tile that starts in the middle of a 128-wide scale atom reads its B scales from
+                        // the matching TMEM column of the copied atoms (32 columns of B per TMEM column)
+                        sfb_skip = (uint32_t)(((tn * BN) & 127) >> 5);
+                    }
+                    ok = warp_wait(full_bar(s), ph, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS;
                     const uint32_t sfb_t = sfa_t + 4;
-                    const uint32_t a_lo = a_lo0 + s * (C::A_BYTES >> 4);
-                    const uint32_t b_lo = b_lo0 + s * (C::B_BYTES >> 4);
                     if (elect_one()) {
                         tc_cp_sf<PAIR>(sfa_t, desc64(sfa_lo0 + s * (512 >> 4), sf_hi));
 #pragma unroll
@@ -421,15 +483,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             const uint32_t idesc = idesc0 | ((uint32_t)k << 29) | ((uint32_t)k << 4);   // scale byte k of the column entry
-                            tc_mma<PAIR>(d_tmem, desc64(a_lo + k * a_kstep, op_hi), desc64(b_lo + k * b_kstep, op_hi), idesc,
-                                         sfa_t, sfb_t, (uint32_t)((kb | k) != 0));
+                            tc_mma<PAIR>(d_tmem, desc64(a_lo0 + s * (C::A_BYTES >> 4) + k * a_kstep, op_hi),
+                                         desc64(b_lo0 + s * (C::B_BYTES >> 4) + k * b_kstep, op_hi), idesc,
+                                         sfa_t, sfb_t + sfb_skip, (uint32_t)((kb | k) != 0));
                         }
                         tc_commit<PAIR>(empty_bar(s));   // frees the smem stage (in both CTAs) once these MMAs have read it
                         if (kb == num_kb - 1) tc_commit<PAIR>(tfull_bar(as));
                     }
                     __syncwarp();
-                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+                    if (++kb == num_kb) { kb = 0; tile += workers; ++acc_it; }
                 }
+                ph ^= 1u;
             }
             if (!ok) {
                 // let MMAs already issued retire before TMEM is released
@@ -450,12 +514,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         const uint32_t sw = (uint32_t)((lane >> 1) & 3);
         uint32_t acc_it = 0;
         bool ok = true;
+        const int n_total = (int)p.N;
         for (int tile = worker; tile < p.num_tiles && ok; tile += workers, ++acc_it) {
             int tm, tn;
             tile_coords(p, tile, tm, tn);
             const int as = acc_it % C::ACC_STAGES;
             const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-            if (lane == 0) ok = mbar_wait(tfull_bar(as), aph, abort_flag);   // one poller per warp
+            if (lane == 0) ok = mbar_wait(tfull_bar(as), aph, abort_flag);   // one suspending poller per warp
             ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
             if (!ok) break;
             tc_fence_after();
@@ -477,6 +542,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (p.out_dtype == MXFP8_BF16) {
 #pragma unroll
                 for (int ch = 0; ch < CW / 32; ++ch) {          // 32 columns = 64 bytes per row
+                    if (col0 + ch * 32 >= n_total) break;       // ragged last tile: nothing to store
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
 #pragma unroll
@@ -502,6 +568,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             } else {
 #pragma unroll
                 for (int ch = 0; ch < CW / 16; ++ch) {          // 16 columns = 64 bytes per row
+                    if (col0 + ch * 16 >= n_total) break;
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
 #pragma unroll
@@ -619,10 +686,11 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
         return MXFP8_ERR_CUDA;
     p.tiles_m = (int)(p.M / (PAIR ? 2 * BM : BM));
-    p.tiles_n = (int)(p.N / BN);
+    p.tiles_n = (int)((p.N + BN - 1) / BN);
+    p.stage_tx = (PAIR ? 2u : 1u) * (uint32_t)(C::A_BYTES + (p.b_mn ? C::B_BYTES_MN : C::B_BYTES_K) + 512 + 512 * C::SFB_ATOMS);
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.num_kb = (int)(p.K / BK);
-    { const char* e = getenv("MXFP8_GROUP_M"); p.group_m = e ? atoi(e) : 8; if (p.group_m < 1) p.group_m = 1; }
+    p.group_m = 16;
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
     const int max_workers = PAIR ? sms / 2 : sms;
@@ -673,10 +741,35 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     GemmParams p{};
     p.M = M; p.N = N; p.K = K;
     p.a_mn = a_major; p.b_mn = b_major; p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
-    const bool wide = (N % 256) == 0;
-    const bool pair = wide && (M % 256) == 0;
-    // rows of B one CTA loads per TMA box (K-major B): half a tile in pair mode
-    const uint32_t b_box_rows = pair ? 128u : (wide ? 256u : 128u);
+    // tile shape: estimated cycles = waves x (MMA cycles per tile + what the epilogue adds when it
+    // cannot run under the next tile's MMAs)
+    const int sms = sm_count();
+    if (sms <= 0) return MXFP8_ERR_CUDA;
+    int best_bn = 128;
+    bool best_pair = false;
+    double best_cost = 1e300;
+    // testing aid: MXFP8_GEMM_TILE = "256p" | "192p" | "256" | "192" | "128" forces a shape ("p" = CTA pair)
+    const char* force = getenv("MXFP8_GEMM_TILE");
+    for (int pass = force ? 0 : 1; pass < 2 && best_cost >= 1e300; ++pass)
+    for (int bn : {256, 192, 128}) {
+        for (int pr = 1; pr >= 0; --pr) {
+            if (pr && ((M % 256) || bn == 128)) continue;
+            if (pass == 0) {   // forced shape, when it applies to this problem
+                if (atoi(force) != bn || (strchr(force, 'p') != nullptr) != (pr != 0)) continue;
+            }
+            const int64_t tiles = (M / (pr ? 256 : 128)) * ((N + bn - 1) / bn);
+            const int64_t workers = pr ? sms / 2 : sms;
+            const int64_t waves = (tiles + workers - 1) / workers;
+            // cycles per 128-deep K block measured on B200 for each shape (TMA feed and MMA issue
+            // included), plus the part of the epilogue that cannot run under the next tile's MMAs
+            const double kblock = pr ? (bn == 256 ? 624.0 : 747.0) : (bn == 256 ? 759.0 : (bn == 192 ? 770.0 : 450.0));
+            const double per_tile = (double)(K / 128) * kblock + (bn == 256 ? 1600.0 : 300.0);
+            const double cost = (double)waves * per_tile;
+            if (cost < best_cost) { best_cost = cost; best_bn = bn; best_pair = pr != 0; }
+        }
+    }
+    if (best_cost >= 1e300) return MXFP8_ERR_UNSUPPORTED;
+    const uint32_t b_box_rows = (uint32_t)(best_pair ? best_bn / 2 : best_bn);   // K-major B rows per TMA box
     GemmMaps m;
     const bool oka = a_major == MXFP8_K_MAJOR ? make_tmap(&m.a, Aq, (uint64_t)K, (uint64_t)M, 128, 128)
                                               : make_tmap(&m.a, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
@@ -686,6 +779,7 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
                      make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(K / 128));
     if (!oka || !okb || !oks || !make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype)) return MXFP8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (pair) return launch_gemm<256, true>(m, p, st);
-    return wide ? launch_gemm<256, false>(m, p, st) : launch_gemm<128, false>(m, p, st);
+    if (best_pair) return best_bn == 256 ? launch_gemm<256, true>(m, p, st) : launch_gemm<192, true>(m, p, st);
+    if (best_bn == 256) return launch_gemm<256, false>(m, p, st);
+    return best_bn == 192 ? launch_gemm<192, false>(m, p, st) : launch_gemm<128, false>(m, p, st);
 }
