@@ -39,7 +39,9 @@ int read_and_clear_device_status(cudaStream_t stream)
     int h = 0, z = 0;
     if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return MXFP8_ERR_CUDA;
     if (h != 0 && cudaMemcpyToSymbol(g_device_status, &z, sizeof(int)) != cudaSuccess) return MXFP8_ERR_CUDA;
-    return h == 0 ? MXFP8_OK : MXFP8_ERR_DEVICE_TIMEOUT;
+    const int q = quantize_read_and_clear_status();
+    if (q == MXFP8_ERR_CUDA) return q;
+    return (h == 0 && q == MXFP8_OK) ? MXFP8_OK : MXFP8_ERR_DEVICE_TIMEOUT;
 }
 
 namespace {

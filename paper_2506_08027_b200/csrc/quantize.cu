@@ -304,6 +304,9 @@ extern "C" int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int6
     if (!aligned16(src)) return MXFP8_ERR_ALIGN;
     if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
     if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    if (quantize_tma_eligible(src_dtype, rows, cols))
+        return quantize_tma_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
+                                   q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
     return quantize_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
                            q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
 }

@@ -1,0 +1,470 @@
+// Fast path of mxfp8_quantize: TMA in, math, TMA out (Sec. 3.2 / 3.3, Algorithm 1, App. A.1-A.2).
+//
+// The generic kernel in quantize.cu spends most of its issue slots on global address
+// arithmetic, predicates and per-row shuffles.  Here a CTA owns a tile of 128 rows x 256 bytes
+// (128 BF16 or 64 FP32 columns) that one TMA tensor load brings into shared memory (ragged edges
+// are zero-filled by the hardware), all arithmetic reads and writes shared memory at compile-time
+// offsets, and the FP8 bytes of both orientations leave as two TMA tensor stores (clipped at the
+// tensor edge by the hardware).  Only the scale bytes (1/32 of the output) use plain stores.
+//
+//   warp w owns rows 32w .. 32w+31 of the tile; lane l owns 8 bytes (4 BF16 / 2 FP32) of every row
+//   pass A (column blocks): amax down the 32 rows inside the lane, packed bf16x2 max for BF16
+//   pass B (row blocks)   : amax across the lanes of a 32-column block by xor-shuffles; BF16 rows
+//                           go through the shuffles two at a time (one in each half of a register)
+//   scale: integer form of Algorithm 1 / App. A.1 on the amax bit pattern (see mxfp8_device.cuh)
+//   cast : x * 2^-e in FP32 (exact), cvt.rn.satfinite to e4m3x2 / e5m2x2
+#include <cuda.h>
+
+#include "mxfp8_device.cuh"
+#include "mxfp8_host.h"
+
+namespace mxfp8 {
+
+__device__ int g_quantize_status = 0;   // bounded TMA wait expired (read through mxfp8_device_status)
+
+int quantize_read_and_clear_status()
+{
+    int h = 0, z = 0;
+    if (cudaMemcpyFromSymbol(&h, g_quantize_status, sizeof(int)) != cudaSuccess) return MXFP8_ERR_CUDA;
+    if (h != 0 && cudaMemcpyToSymbol(g_quantize_status, &z, sizeof(int)) != cudaSuccess) return MXFP8_ERR_CUDA;
+    return h == 0 ? MXFP8_OK : MXFP8_ERR_DEVICE_TIMEOUT;
+}
+
+namespace {
+
+constexpr int T_ROWS = 128;
+constexpr int T_BYTES = 256;                 // source bytes per tile row
+constexpr int IN_BYTES = T_ROWS * T_BYTES;   // 32 KB
+constexpr int Q_MAX_BYTES = T_ROWS * 128;    // 16 KB per orientation (BF16 tile; FP32 tile uses half)
+constexpr int QT_THREADS = 128;
+constexpr uint64_t QT_WAIT_LIMIT_NS = 1000000000ull;
+
+struct QParams {
+    int64_t rows, cols;
+    int rule, sf_layout;
+    int tiles_x, tiles_y;
+    uint8_t* s_row;
+    uint8_t* s_col;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 2^(127 - b) and b for a block with this (finite, non-negative) amax bit pattern.
+//   rule_offset = 0x1FFFFF (paper: a mantissa above 1.75 carries into the exponent = round up)
+//               = 0        (ocp: floor)
+//   e' = biased exponent after the carry; b = max(e' - emax, 0); 1/X has exponent field 254 - b.
+template <int ELEM>
+__device__ __forceinline__ uint32_t inv_exp_field(uint32_t amax_bits, uint32_t rule_offset)
+{
+    const int e = (int)((amax_bits + rule_offset) >> 23);
+    return (uint32_t)min(254 + ElemTraits<ELEM>::emax - e, 254);
+}
+
+__device__ __forceinline__ uint32_t hmax2_abs(uint32_t a, uint32_t b)
+{
+    const __nv_bfloat162 x = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&a));
+    const __nv_bfloat162 y = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+    const __nv_bfloat162 m = __hmax2(x, y);   // NaN operands are ignored (maxNum)
+    return *reinterpret_cast<const uint32_t*>(&m);
+}
+__device__ __forceinline__ uint32_t hmax2(uint32_t a, uint32_t b)
+{
+    const __nv_bfloat162 m = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&m);
+}
+// |bf16| halves that are +Inf or NaN become 0 (finite-only maximum, rare path)
+__device__ __forceinline__ uint32_t finite_abs2(uint32_t w)
+{
+    uint32_t a = w & 0x7FFF7FFFu;
+    if ((a & 0x0000FFFFu) >= 0x00007F80u) a &= 0xFFFF0000u;
+    if ((a & 0xFFFF0000u) >= 0x7F800000u) a &= 0x0000FFFFu;
+    return a;
+}
+
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+__global__ void __launch_bounds__(QT_THREADS)
+quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const __grid_constant__ CUtensorMap tmap_qrow,
+                    const __grid_constant__ CUtensorMap tmap_qcol, const QParams p)
+{
+    constexpr bool BF = (DTYPE == MXFP8_BF16);
+    constexpr int VEC = BF ? 4 : 2;                 // elements per lane per row
+    constexpr int T_COLS = T_BYTES / (BF ? 2 : 4);  // 128 or 64
+    constexpr int NKB = T_COLS / 32;                // row blocks per tile row: 4 or 2
+    constexpr int LPB = 32 / VEC;                   // lanes per row block: 8 or 16
+
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint8_t* in_tile = smem;                               // [128][256]
+    uint8_t* qrow_tile = smem + IN_BYTES;                  // [128][T_COLS]
+    uint8_t* qcol_tile = qrow_tile + Q_MAX_BYTES;          // [128][T_COLS]
+    uint8_t* sm_row = qcol_tile + Q_MAX_BYTES;             // [128][4]
+    uint8_t* sm_col = sm_row + 512;                        // [T_COLS][4]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sm_col + 512);
+    const uint32_t bar_a = smem_addr(bar);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rule_offset = (p.rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
+
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int num_tiles = p.tiles_x * p.tiles_y;
+    int tile = blockIdx.x;
+    uint32_t phase = 0;
+    if (tid == 0 && tile < num_tiles) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"((uint32_t)IN_BYTES) : "memory");
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                     ::"r"(smem_addr(in_tile)), "l"(&tmap_src), "r"(bar_a), "r"((tile % p.tiles_x) * T_COLS), "r"((tile / p.tiles_x) * T_ROWS)
+                     : "memory");
+    }
+
+    for (; tile < num_tiles; tile += gridDim.x) {
+        const int tile_x = tile % p.tiles_x, tile_y = tile / p.tiles_x;
+        const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
+
+        // wait for the tile (bounded: on expiry report through the status word and leave)
+        {
+            uint32_t ok = 0, spins = 0;
+            uint64_t t0 = 0;
+            while (true) {
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(bar_a), "r"(phase) : "memory");
+                if (ok) break;
+                if ((++spins & 0xFFu) == 0) {
+                    uint64_t now;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > QT_WAIT_LIMIT_NS) break;
+                }
+            }
+            if (!__syncthreads_and((int)ok)) {
+                if (tid == 0) atomicExch(&g_quantize_status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
+                return;
+            }
+        }
+        phase ^= 1u;
+
+        const uint8_t* my_in = in_tile + warp * 32 * T_BYTES + lane * 8;
+
+        // ---- pass A: column blocks, amax down this warp's 32 rows inside the lane ----------
+        float col_inv[VEC];
+        if (DO_COL) {
+            uint32_t cbits[VEC];
+            if constexpr (BF) {
+                uint32_t m0 = 0u, m1 = 0u;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+                    m0 = hmax2_abs(m0, w.x);
+                    m1 = hmax2_abs(m1, w.y);
+                }
+                if ((((m0 + 0x00800080u) | (m1 + 0x00800080u)) & 0x80008000u) != 0u) {   // an Inf got in: finite-only redo
+                    m0 = m1 = 0u;
+#pragma unroll 4
+                    for (int j = 0; j < 32; ++j) {
+                        const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+                        m0 = hmax2(m0, finite_abs2(w.x));
+                        m1 = hmax2(m1, finite_abs2(w.y));
+                    }
+                }
+                cbits[0] = m0 << 16; cbits[1] = m0 & 0xFFFF0000u;
+                cbits[2] = m1 << 16; cbits[3] = m1 & 0xFFFF0000u;
+            } else {
+                float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+                    a0 = fmaxf(a0, fabsf(w.x));
+                    a1 = fmaxf(a1, fabsf(w.y));
+                }
+                if (a0 == INFINITY || a1 == INFINITY) {
+                    a0 = a1 = 0.f;
+#pragma unroll 4
+                    for (int j = 0; j < 32; ++j) {
+                        const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+                        if (fabsf(w.x) < INFINITY) a0 = fmaxf(a0, fabsf(w.x));
+                        if (fabsf(w.y) < INFINITY) a1 = fmaxf(a1, fabsf(w.y));
+                    }
+                }
+                cbits[0] = __float_as_uint(a0);
+                cbits[1] = __float_as_uint(a1);
+            }
+            uint32_t packed_b = 0u;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
+                col_inv[i] = __uint_as_float(ie << 23);
+                packed_b |= (254u - ie) << (8 * i);
+            }
+            // sm_col[c][w]: column c of the tile, row block w
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) sm_col[(lane * VEC + i) * 4 + warp] = (uint8_t)(packed_b >> (8 * i));
+        }
+
+        // ---- pass B: rows; BF16 rows go through the shuffle reduction in pairs ------------------
+        uint8_t* my_qrow = qrow_tile + warp * 32 * T_COLS + lane * VEC;
+        uint8_t* my_qcol = qcol_tile + warp * 32 * T_COLS + lane * VEC;
+#pragma unroll 4
+        for (int j = 0; j < 32; j += 2) {
+            float x0[VEC], x1[VEC];
+            float inv0 = 1.f, inv1 = 1.f;
+            if constexpr (BF) {
+                const uint2 w0 = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+                const uint2 w1 = *reinterpret_cast<const uint2*>(my_in + (j + 1) * T_BYTES);
+                x0[0] = __uint_as_float(w0.x << 16); x0[1] = __uint_as_float(w0.x & 0xFFFF0000u);
+                x0[2] = __uint_as_float(w0.y << 16); x0[3] = __uint_as_float(w0.y & 0xFFFF0000u);
+                x1[0] = __uint_as_float(w1.x << 16); x1[1] = __uint_as_float(w1.x & 0xFFFF0000u);
+                x1[2] = __uint_as_float(w1.y << 16); x1[3] = __uint_as_float(w1.y & 0xFFFF0000u);
+                if (DO_ROW) {
+                    const uint32_t m0 = hmax2_abs(w0.x, w0.y);               // row j  : (max |e0|,|e2| ; max |e1|,|e3|)
+                    const uint32_t m1 = hmax2_abs(w1.x, w1.y);               // row j+1
+                    uint32_t z = hmax2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));   // (amax_j, amax_j+1) of this lane
+#pragma unroll
+                    for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
+                    if (__any_sync(0xFFFFFFFFu, ((z + 0x00800080u) & 0x80008000u) != 0u)) {   // rare: an Inf got in
+                        const uint32_t f0 = hmax2(finite_abs2(w0.x), finite_abs2(w0.y));
+                        const uint32_t f1 = hmax2(finite_abs2(w1.x), finite_abs2(w1.y));
+                        z = hmax2(__byte_perm(f0, f1, 0x5410), __byte_perm(f0, f1, 0x7632));
+#pragma unroll
+                        for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
+                    }
+                    const uint32_t ie0 = inv_exp_field<ELEM>(z << 16, rule_offset);
+                    const uint32_t ie1 = inv_exp_field<ELEM>(z & 0xFFFF0000u, rule_offset);
+                    inv0 = __uint_as_float(ie0 << 23);
+                    inv1 = __uint_as_float(ie1 << 23);
+                    if ((lane & (LPB - 1)) == 0) {
+                        sm_row[(warp * 32 + j) * 4 + lane / LPB] = (uint8_t)(254u - ie0);
+                        sm_row[(warp * 32 + j + 1) * 4 + lane / LPB] = (uint8_t)(254u - ie1);
+                    }
+                }
+            } else {
+                const float2 w0 = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+                const float2 w1 = *reinterpret_cast<const float2*>(my_in + (j + 1) * T_BYTES);
+                x0[0] = w0.x; x0[1] = w0.y;
+                x1[0] = w1.x; x1[1] = w1.y;
+                if (DO_ROW) {
+                    float a0 = fmaxf(fabsf(w0.x), fabsf(w0.y)), a1 = fmaxf(fabsf(w1.x), fabsf(w1.y));
+                    a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f);                 // two NaNs -> 0
+#pragma unroll
+                    for (int off = 1; off < LPB; off <<= 1) {
+                        a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
+                        a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
+                    }
+                    if (__any_sync(0xFFFFFFFFu, a0 == INFINITY || a1 == INFINITY)) {
+                        a0 = 0.f; a1 = 0.f;
+                        if (fabsf(w0.x) < INFINITY) a0 = fabsf(w0.x);
+                        if (fabsf(w0.y) < INFINITY) a0 = fmaxf(a0, fabsf(w0.y));
+                        if (fabsf(w1.x) < INFINITY) a1 = fabsf(w1.x);
+                        if (fabsf(w1.y) < INFINITY) a1 = fmaxf(a1, fabsf(w1.y));
+#pragma unroll
+                        for (int off = 1; off < LPB; off <<= 1) {
+                            a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
+                            a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
+                        }
+                    }
+                    const uint32_t ie0 = inv_exp_field<ELEM>(__float_as_uint(a0), rule_offset);
+                    const uint32_t ie1 = inv_exp_field<ELEM>(__float_as_uint(a1), rule_offset);
+                    inv0 = __uint_as_float(ie0 << 23);
+                    inv1 = __uint_as_float(ie1 << 23);
+                    if ((lane & (LPB - 1)) == 0) {
+                        sm_row[(warp * 32 + j) * 4 + lane / LPB] = (uint8_t)(254u - ie0);
+                        sm_row[(warp * 32 + j + 1) * 4 + lane / LPB] = (uint8_t)(254u - ie1);
+                    }
+                }
+            }
+            if (DO_ROW) {
+                if constexpr (VEC == 4) {
+                    *reinterpret_cast<uint32_t*>(my_qrow + j * T_COLS) = cvt_fp8x4<ELEM>(x0[0] * inv0, x0[1] * inv0, x0[2] * inv0, x0[3] * inv0);
+                    *reinterpret_cast<uint32_t*>(my_qrow + (j + 1) * T_COLS) = cvt_fp8x4<ELEM>(x1[0] * inv1, x1[1] * inv1, x1[2] * inv1, x1[3] * inv1);
+                } else {
+                    *reinterpret_cast<uint16_t*>(my_qrow + j * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * inv0, x0[1] * inv0);
+                    *reinterpret_cast<uint16_t*>(my_qrow + (j + 1) * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * inv1, x1[1] * inv1);
+                }
+            }
+            if (DO_COL) {
+                if constexpr (VEC == 4) {
+                    *reinterpret_cast<uint32_t*>(my_qcol + j * T_COLS) =
+                        cvt_fp8x4<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1], x0[2] * col_inv[2], x0[3] * col_inv[3]);
+                    *reinterpret_cast<uint32_t*>(my_qcol + (j + 1) * T_COLS) =
+                        cvt_fp8x4<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1], x1[2] * col_inv[2], x1[3] * col_inv[3]);
+                } else {
+                    *reinterpret_cast<uint16_t*>(my_qcol + j * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1]);
+                    *reinterpret_cast<uint16_t*>(my_qcol + (j + 1) * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1]);
+                }
+            }
+        }
+
+        // shared-memory writes -> visible to the TMA engine; the input tile is free to be refilled
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+
+        if (tid == 0) {
+            if (DO_ROW)
+                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                             ::"l"(&tmap_qrow), "r"((int)gcol0), "r"((int)grow0), "r"(smem_addr(qrow_tile)) : "memory");
+            if (DO_COL)
+                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                             ::"l"(&tmap_qcol), "r"((int)gcol0), "r"((int)grow0), "r"(smem_addr(qcol_tile)) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            const int next = tile + gridDim.x;
+            if (next < num_tiles) {   // prefetch the next tile under the stores
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"((uint32_t)IN_BYTES) : "memory");
+                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                             ::"r"(smem_addr(in_tile)), "l"(&tmap_src), "r"(bar_a), "r"((next % p.tiles_x) * T_COLS), "r"((next / p.tiles_x) * T_ROWS)
+                             : "memory");
+            }
+        }
+
+        // ---- scale bytes (1/32 of the output): plain stores from the staging arrays ----------
+        if (DO_ROW) {
+            const int64_t r = grow0 + tid, ncb = p.cols >> 5, kb0 = (int64_t)tile_x * NKB;
+            const int nkb = (int)min((int64_t)NKB, ncb - kb0);
+            if (p.sf_layout == MXFP8_SF_SWIZZLED) {
+                // every row of a started 128-row atom is written (pad rows / pad K-blocks get 0)
+                uint8_t* d = p.s_row + ((int64_t)tile_y * ((ncb + 3) >> 2) + (kb0 >> 2)) * 512 + (tid & 31) * 16 + (tid >> 5) * 4 + (kb0 & 3);
+                uint32_t v = 0u;
+                if (r < p.rows)
+                    for (int kb = 0; kb < nkb; ++kb) v |= (uint32_t)sm_row[tid * 4 + kb] << (8 * kb);
+                // a 64-column FP32 tile owns half of the atom's 4 K-blocks; the left half also zeroes
+                // the right half when no tile exists there (pad K-blocks)
+                if (NKB == 4 || ((kb0 & 3) == 0 && kb0 + NKB >= ncb)) *reinterpret_cast<uint32_t*>(d) = v;
+                else *reinterpret_cast<uint16_t*>(d) = (uint16_t)v;
+            } else if (r < p.rows) {
+                uint8_t* d = p.s_row + r * ncb + kb0;
+                for (int kb = 0; kb < nkb; ++kb) d[kb] = sm_row[tid * 4 + kb];
+            }
+        }
+        if (DO_COL && tid < T_COLS) {
+            const int64_t c = gcol0 + tid, nrb = p.rows >> 5, rb0 = (int64_t)tile_y * 4;
+            const int nrb_here = (int)min((int64_t)4, nrb - rb0);
+            if (p.sf_layout == MXFP8_SF_SWIZZLED) {
+                const int64_t padded_cols = ((p.cols + 127) >> 7) << 7;
+                if (c < padded_cols) {
+                    uint8_t* d = p.s_col + ((c >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + (c & 31) * 16 + ((c >> 5) & 3) * 4;
+                    uint32_t v = 0u;
+                    if (c < p.cols)
+                        for (int w = 0; w < nrb_here; ++w) v |= (uint32_t)sm_col[tid * 4 + w] << (8 * w);
+                    *reinterpret_cast<uint32_t*>(d) = v;
+                    // pad columns no tile covers (FP32 tiles are 64 wide, atoms 128 wide)
+                    if (T_COLS == 64 && tile_x == p.tiles_x - 1 && c + 64 >= (int64_t)p.tiles_x * 64 && c + 64 < padded_cols)
+                        *reinterpret_cast<uint32_t*>(p.s_col + (((c + 64) >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + ((c + 64) & 31) * 16 + (((c + 64) >> 5) & 3) * 4) = 0u;
+                }
+            } else if (c < p.cols) {
+                for (int w = 0; w < nrb_here; ++w) p.s_col[(rb0 + w) * p.cols + c] = sm_col[tid * 4 + w];
+            }
+        }
+
+        // the staging tiles may be overwritten once the stores have read them
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncthreads();
+    }
+    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn qt_encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t esz, void* base, uint64_t cols, uint64_t rows,
+                 uint32_t box_cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = qt_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * esz};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int qt_sm_count()
+{
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        return v;
+    }();
+    return n;
+}
+
+template <int DTYPE, int ELEM, bool R, bool C>
+cudaError_t launch(const CUtensorMap& ms, const CUtensorMap& mr, const CUtensorMap& mc, const QParams& p, cudaStream_t stream)
+{
+    constexpr int SMEM = IN_BYTES + 2 * Q_MAX_BYTES + 1024 + 16;
+    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    if (err != cudaSuccess) return err;
+    const int tiles = p.tiles_x * p.tiles_y;
+    const int max_ctas = qt_sm_count() * 3;
+    const int grid = tiles < max_ctas ? tiles : max_ctas;
+    kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, mr, mc, p);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+template <int DTYPE, int ELEM>
+cudaError_t launch_o(int orientation, const CUtensorMap& ms, const CUtensorMap& mr, const CUtensorMap& mc, const QParams& p, cudaStream_t st)
+{
+    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false>(ms, mr, mc, p, st);
+    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true>(ms, mr, mc, p, st);
+    return launch<DTYPE, ELEM, true, true>(ms, mr, mc, p, st);
+}
+
+}  // namespace
+
+bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
+{
+    // TMA needs 16-byte row pitches for the source and for the byte outputs; tile counts must fit an int
+    if (cols % 16) return false;
+    const int64_t t_cols = (src_dtype == MXFP8_BF16) ? 128 : 64;
+    const int64_t tiles = ((cols + t_cols - 1) / t_cols) * ((rows + T_ROWS - 1) / T_ROWS);
+    return tiles < 0x7FFFFFFFLL && rows < 0x7FFFFFFFLL && cols < 0x7FFFFFFFLL && qt_encode_fn() != nullptr;
+}
+
+int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
+                        int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
+                        int sf_layout, cudaStream_t stream)
+{
+    const bool bf = src_dtype == MXFP8_BF16;
+    const uint32_t t_cols = bf ? 128 : 64;
+    CUtensorMap ms, mr, mc;
+    if (!make_map_2d(&ms, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
+                     const_cast<void*>(src), (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS))
+        return MXFP8_ERR_CUDA;
+    void* qr = (orientation & MXFP8_ROW) ? q_row : q_col;   // an unused map still has to be valid
+    void* qc = (orientation & MXFP8_COL) ? q_col : q_row;
+    if (!make_map_2d(&mr, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qr, (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS) ||
+        !make_map_2d(&mc, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qc, (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS))
+        return MXFP8_ERR_CUDA;
+    QParams p{};
+    p.rows = rows; p.cols = cols; p.rule = scale_rule; p.sf_layout = sf_layout;
+    p.tiles_x = (int)((cols + t_cols - 1) / t_cols);
+    p.tiles_y = (int)((rows + T_ROWS - 1) / T_ROWS);
+    p.s_row = static_cast<uint8_t*>(s_row);
+    p.s_col = static_cast<uint8_t*>(s_col);
+    cudaError_t err;
+    if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3>(orientation, ms, mr, mc, p, stream)
+                                     : launch_o<MXFP8_BF16, MXFP8_E5M2>(orientation, ms, mr, mc, p, stream);
+    else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3>(orientation, ms, mr, mc, p, stream)
+                                  : launch_o<MXFP8_FP32, MXFP8_E5M2>(orientation, ms, mr, mc, p, stream);
+    return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}
+
+}  // namespace mxfp8
