@@ -1,11 +1,12 @@
-// Fast path of mxfp8_quantize: TMA in, math, TMA out (Sec. 3.2 / 3.3, Algorithm 1, App. A.1-A.2).
+// Fast path of mxfp8_quantize: TMA in, math, coalesced stores out (Sec. 3.2 / 3.3, Algorithm 1,
+// App. A.1-A.2).
 //
 // The generic kernel in quantize.cu spends most of its issue slots on global address
-// arithmetic, predicates and per-row shuffles.  Here a CTA owns a tile of 128 rows x 256 bytes
-// (128 BF16 or 64 FP32 columns) that one TMA tensor load brings into shared memory (ragged edges
-// are zero-filled by the hardware), all arithmetic reads and writes shared memory at compile-time
-// offsets, and the FP8 bytes of both orientations leave as two TMA tensor stores (clipped at the
-// tensor edge by the hardware).  Only the scale bytes (1/32 of the output) use plain stores.
+// arithmetic and predicates.  Here a CTA owns tiles of 128 rows x 256 bytes (128 BF16 or 64 FP32
+// columns).  TMA tensor loads bring them into a two-deep shared-memory ring (ragged edges are
+// zero-filled by the hardware, the next tile is in flight while the current one is processed),
+// the arithmetic reads shared memory at compile-time offsets, and the FP8 bytes go straight to
+// global memory: every warp store covers 128 (BF16) or 64 (FP32) contiguous bytes of one row.
 //
 //   warp w owns rows 32w .. 32w+31 of the tile; lane l owns 8 bytes (4 BF16 / 2 FP32) of every row
 //   pass A (column blocks): amax down the 32 rows inside the lane, packed bf16x2 max for BF16
@@ -35,7 +36,6 @@ namespace {
 constexpr int T_ROWS = 128;
 constexpr int T_BYTES = 256;                 // source bytes per tile row
 constexpr int IN_BYTES = T_ROWS * T_BYTES;   // 32 KB
-constexpr int Q_MAX_BYTES = T_ROWS * 128;    // 16 KB per orientation (BF16 tile; FP32 tile uses half)
 constexpr int QT_THREADS = 128;
 constexpr uint64_t QT_WAIT_LIMIT_NS = 1000000000ull;
 
@@ -43,6 +43,8 @@ struct QParams {
     int64_t rows, cols;
     int rule, sf_layout;
     int tiles_x, tiles_y;
+    uint8_t* q_row;
+    uint8_t* q_col;
     uint8_t* s_row;
     uint8_t* s_col;
 };
@@ -81,10 +83,206 @@ __device__ __forceinline__ uint32_t finite_abs2(uint32_t w)
     return a;
 }
 
+// flags a packed pair of bf16 magnitudes if either half is Inf or NaN
+__device__ __forceinline__ uint32_t nonfinite2(uint32_t z) { return (z + 0x00800080u) & 0x80008000u; }
+
+// One 32-row slab, fast path: every element finite (checked at the end; the caller reruns the
+// slab through slab_careful otherwise), all rows and columns inside the tensor.  Returns
+// whether any lane of the warp met an Inf / NaN.
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+__device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
+                                          uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
+                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset)
+{
+    constexpr bool BF = (DTYPE == MXFP8_BF16);
+    constexpr int VEC = BF ? 4 : 2;
+    constexpr int LPB = 32 / VEC;
+    uint32_t bad = 0u;
+    float col_inv[VEC];
+    if (DO_COL) {
+        uint32_t cbits[VEC];
+        if constexpr (BF) {
+            uint32_t m0 = 0u, m1 = 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+                m0 = hmax2_abs(m0, w.x);
+                m1 = hmax2_abs(m1, w.y);
+            }
+            bad |= nonfinite2(m0) | nonfinite2(m1);
+            cbits[0] = m0 << 16; cbits[1] = m0 & 0xFFFF0000u;
+            cbits[2] = m1 << 16; cbits[3] = m1 & 0xFFFF0000u;
+        } else {
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+                a0 = fmaxf(a0, fabsf(w.x));
+                a1 = fmaxf(a1, fabsf(w.y));
+            }
+            bad |= (uint32_t)(a0 == INFINITY) | (uint32_t)(a1 == INFINITY);
+            cbits[0] = __float_as_uint(a0);
+            cbits[1] = __float_as_uint(a1);
+        }
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
+            col_inv[i] = __uint_as_float(ie << 23);
+            my_sm_col[i * 4] = (uint8_t)(254u - ie);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) {
+        float x0[VEC], x1[VEC];
+        float inv0 = 1.f, inv1 = 1.f;
+        if constexpr (BF) {
+            const uint2 w0 = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+            const uint2 w1 = *reinterpret_cast<const uint2*>(my_in + (j + 1) * T_BYTES);
+            x0[0] = __uint_as_float(w0.x << 16); x0[1] = __uint_as_float(w0.x & 0xFFFF0000u);
+            x0[2] = __uint_as_float(w0.y << 16); x0[3] = __uint_as_float(w0.y & 0xFFFF0000u);
+            x1[0] = __uint_as_float(w1.x << 16); x1[1] = __uint_as_float(w1.x & 0xFFFF0000u);
+            x1[2] = __uint_as_float(w1.y << 16); x1[3] = __uint_as_float(w1.y & 0xFFFF0000u);
+            if (DO_ROW) {
+                const uint32_t m0 = hmax2_abs(w0.x, w0.y);               // row j  : (max |e0|,|e2| ; max |e1|,|e3|)
+                const uint32_t m1 = hmax2_abs(w1.x, w1.y);               // row j+1
+                uint32_t z = hmax2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));   // (amax_j, amax_j+1) of this lane
+#pragma unroll
+                for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
+                bad |= nonfinite2(z);
+                const uint32_t ie0 = inv_exp_field<ELEM>(z << 16, rule_offset);
+                const uint32_t ie1 = inv_exp_field<ELEM>(z & 0xFFFF0000u, rule_offset);
+                inv0 = __uint_as_float(ie0 << 23);
+                inv1 = __uint_as_float(ie1 << 23);
+                if ((lane & (LPB - 1)) == 0) {
+                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
+                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
+                }
+            }
+        } else {
+            const float2 w0 = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+            const float2 w1 = *reinterpret_cast<const float2*>(my_in + (j + 1) * T_BYTES);
+            x0[0] = w0.x; x0[1] = w0.y;
+            x1[0] = w1.x; x1[1] = w1.y;
+            if (DO_ROW) {
+                float a0 = fmaxf(fmaxf(fabsf(w0.x), fabsf(w0.y)), 0.f), a1 = fmaxf(fmaxf(fabsf(w1.x), fabsf(w1.y)), 0.f);
+#pragma unroll
+                for (int off = 1; off < LPB; off <<= 1) {
+                    a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
+                    a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
+                }
+                bad |= (uint32_t)(a0 == INFINITY) | (uint32_t)(a1 == INFINITY);
+                const uint32_t ie0 = inv_exp_field<ELEM>(__float_as_uint(a0), rule_offset);
+                const uint32_t ie1 = inv_exp_field<ELEM>(__float_as_uint(a1), rule_offset);
+                inv0 = __uint_as_float(ie0 << 23);
+                inv1 = __uint_as_float(ie1 << 23);
+                if ((lane & (LPB - 1)) == 0) {
+                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
+                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
+                }
+            }
+        }
+        uint8_t* r0 = my_qrow + (uint64_t)j * pitch;
+        uint8_t* c0 = my_qcol + (uint64_t)j * pitch;
+        if constexpr (VEC == 4) {
+            if (DO_ROW) {
+                *reinterpret_cast<uint32_t*>(r0) = cvt_fp8x4<ELEM>(x0[0] * inv0, x0[1] * inv0, x0[2] * inv0, x0[3] * inv0);
+                *reinterpret_cast<uint32_t*>(r0 + pitch) = cvt_fp8x4<ELEM>(x1[0] * inv1, x1[1] * inv1, x1[2] * inv1, x1[3] * inv1);
+            }
+            if (DO_COL) {
+                *reinterpret_cast<uint32_t*>(c0) = cvt_fp8x4<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1], x0[2] * col_inv[2], x0[3] * col_inv[3]);
+                *reinterpret_cast<uint32_t*>(c0 + pitch) = cvt_fp8x4<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1], x1[2] * col_inv[2], x1[3] * col_inv[3]);
+            }
+        } else {
+            if (DO_ROW) {
+                *reinterpret_cast<uint16_t*>(r0) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * inv0, x0[1] * inv0);
+                *reinterpret_cast<uint16_t*>(r0 + pitch) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * inv1, x1[1] * inv1);
+            }
+            if (DO_COL) {
+                *reinterpret_cast<uint16_t*>(c0) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1]);
+                *reinterpret_cast<uint16_t*>(c0 + pitch) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1]);
+            }
+        }
+    }
+    return __any_sync(0xFFFFFFFFu, bad != 0u);
+}
+
+// The same slab with everything the fast path leaves out: Inf and NaN elements stay out of
+// amax (App. / Sec. 3.3 leaves their handling open; see mxfp8.h), rows and columns outside the
+// tensor are not stored.  Rare, so compact rather than fast.
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+__device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
+                                          uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
+                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset, int rows_here, bool col_ok)
+{
+    constexpr bool BF = (DTYPE == MXFP8_BF16);
+    constexpr int VEC = BF ? 4 : 2;
+    constexpr int LPB = 32 / VEC;
+    auto load = [&](int j, float (&x)[VEC]) {
+        if constexpr (BF) {
+            const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
+            x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xFFFF0000u);
+            x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xFFFF0000u);
+        } else {
+            const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
+            x[0] = w.x; x[1] = w.y;
+        }
+    };
+    float col_inv[VEC];
+    if (DO_COL) {
+        float cmax[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) cmax[i] = 0.f;
+#pragma unroll 1
+        for (int j = 0; j < 32; ++j) {
+            float x[VEC];
+            load(j, x);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float a = fabsf(x[i]);
+                if (a < INFINITY) cmax[i] = fmaxf(cmax[i], a);   // false for NaN as well
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(cmax[i]), rule_offset);
+            col_inv[i] = __uint_as_float(ie << 23);
+            my_sm_col[i * 4] = (uint8_t)(254u - ie);
+        }
+    }
+#pragma unroll 1
+    for (int j = 0; j < 32; ++j) {
+        float x[VEC];
+        load(j, x);
+        const bool live = col_ok && j < rows_here;
+        if (DO_ROW) {
+            float m = 0.f;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float a = fabsf(x[i]);
+                if (a < INFINITY) m = fmaxf(m, a);
+            }
+#pragma unroll
+            for (int off = 1; off < LPB; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+            const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(m), rule_offset);
+            const float inv = __uint_as_float(ie << 23);
+            if ((lane & (LPB - 1)) == 0) my_sm_row[j * 4] = (uint8_t)(254u - ie);
+            if (live) {
+                if constexpr (VEC == 4) *reinterpret_cast<uint32_t*>(my_qrow + (uint64_t)j * pitch) = cvt_fp8x4<ELEM>(x[0] * inv, x[1] * inv, x[2] * inv, x[3] * inv);
+                else *reinterpret_cast<uint16_t*>(my_qrow + (uint64_t)j * pitch) = (uint16_t)cvt_fp8x2<ELEM>(x[0] * inv, x[1] * inv);
+            }
+        }
+        if (DO_COL && live) {
+            if constexpr (VEC == 4)
+                *reinterpret_cast<uint32_t*>(my_qcol + (uint64_t)j * pitch) = cvt_fp8x4<ELEM>(x[0] * col_inv[0], x[1] * col_inv[1], x[2] * col_inv[2], x[3] * col_inv[3]);
+            else
+                *reinterpret_cast<uint16_t*>(my_qcol + (uint64_t)j * pitch) = (uint16_t)cvt_fp8x2<ELEM>(x[0] * col_inv[0], x[1] * col_inv[1]);
+        }
+    }
+}
+
 template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
 __global__ void __launch_bounds__(QT_THREADS)
-quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const __grid_constant__ CUtensorMap tmap_qrow,
-                    const __grid_constant__ CUtensorMap tmap_qcol, const QParams p)
+quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams p)
 {
     constexpr bool BF = (DTYPE == MXFP8_BF16);
     constexpr int VEC = BF ? 4 : 2;                 // elements per lane per row
@@ -93,34 +291,41 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const __grid_c
     constexpr int LPB = 32 / VEC;                   // lanes per row block: 8 or 16
 
     extern __shared__ __align__(128) uint8_t smem[];
-    uint8_t* in_tile = smem;                               // [128][256]
-    uint8_t* qrow_tile = smem + IN_BYTES;                  // [128][T_COLS]
-    uint8_t* qcol_tile = qrow_tile + Q_MAX_BYTES;          // [128][T_COLS]
-    uint8_t* sm_row = qcol_tile + Q_MAX_BYTES;             // [128][4]
-    uint8_t* sm_col = sm_row + 512;                        // [T_COLS][4]
-    uint64_t* bar = reinterpret_cast<uint64_t*>(sm_col + 512);
-    const uint32_t bar_a = smem_addr(bar);
+    uint8_t* in_ring = smem;                               // 2 x [128][256]
+    uint8_t* sm_scales = smem + 2 * IN_BYTES;              // 2 x ([128][4] row scales + [T_COLS][4] column scales)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;   // warp = 32-row slab of the tile
     const uint32_t rule_offset = (p.rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
 
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
     const int num_tiles = p.tiles_x * p.tiles_y;
-    int tile = blockIdx.x;
-    uint32_t phase = 0;
-    if (tid == 0 && tile < num_tiles) {
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"((uint32_t)IN_BYTES) : "memory");
+    auto issue_load = [&](int t, int buf) {   // one thread: tile t -> ring slot buf
+        const uint32_t b = smem_addr(&bars[buf]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(in_tile)), "l"(&tmap_src), "r"(bar_a), "r"((tile % p.tiles_x) * T_COLS), "r"((tile / p.tiles_x) * T_ROWS)
+                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&tmap_src), "r"(b), "r"((t % p.tiles_x) * T_COLS), "r"((t / p.tiles_x) * T_ROWS)
                      : "memory");
+    };
+    int tile = blockIdx.x;
+    if (tid == 0) {
+        if (tile < num_tiles) issue_load(tile, 0);
+        if (tile + (int)gridDim.x < num_tiles) issue_load(tile + gridDim.x, 1);
     }
 
-    for (; tile < num_tiles; tile += gridDim.x) {
+    for (int it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t phase = (uint32_t)(it >> 1) & 1u;
+        const uint32_t bar_a = smem_addr(&bars[buf]);
+        uint8_t* in_tile = in_ring + buf * IN_BYTES;
+        uint8_t* sm_row = sm_scales + buf * 1024;          // [128][4]
+        uint8_t* sm_col = sm_row + 512;                    // [T_COLS][4]
         const int tile_x = tile % p.tiles_x, tile_y = tile / p.tiles_x;
         const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
 
@@ -144,181 +349,34 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const __grid_c
                 return;
             }
         }
-        phase ^= 1u;
-
+        // this warp's slab: 32 rows; first the fully unrolled fast path (no special values, whole
+        // slab inside the tensor), and if it saw an Inf / NaN or the slab is ragged, the careful path
         const uint8_t* my_in = in_tile + warp * 32 * T_BYTES + lane * 8;
+        const int64_t my_col = gcol0 + lane * VEC;
+        const int rows_here = (int)min((int64_t)32, p.rows - (grow0 + warp * 32));   // rows of this slab inside the tensor
+        const bool col_ok = my_col < p.cols;                                         // cols % 16 == 0: a lane's bytes are all in or all out
+        uint8_t* my_qrow = p.q_row + (grow0 + warp * 32) * p.cols + my_col;
+        uint8_t* my_qcol = p.q_col + (grow0 + warp * 32) * p.cols + my_col;
+        const uint32_t pitch = (uint32_t)p.cols;
+        uint8_t* my_sm_row = sm_row + warp * 128 + lane / LPB;
+        uint8_t* my_sm_col = sm_col + lane * VEC * 4 + warp;
+        const bool whole = __all_sync(0xFFFFFFFFu, col_ok) && rows_here == 32;
+        bool special = !whole;
+        if (whole)
+            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset);
+        if (special && rows_here > 0)
+            slab_careful<DTYPE, ELEM, DO_ROW, DO_COL>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
+                                                       rows_here, col_ok);
 
-        // ---- pass A: column blocks, amax down this warp's 32 rows inside the lane ----------
-        float col_inv[VEC];
-        if (DO_COL) {
-            uint32_t cbits[VEC];
-            if constexpr (BF) {
-                uint32_t m0 = 0u, m1 = 0u;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-                    m0 = hmax2_abs(m0, w.x);
-                    m1 = hmax2_abs(m1, w.y);
-                }
-                if ((((m0 + 0x00800080u) | (m1 + 0x00800080u)) & 0x80008000u) != 0u) {   // an Inf got in: finite-only redo
-                    m0 = m1 = 0u;
-#pragma unroll 4
-                    for (int j = 0; j < 32; ++j) {
-                        const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-                        m0 = hmax2(m0, finite_abs2(w.x));
-                        m1 = hmax2(m1, finite_abs2(w.y));
-                    }
-                }
-                cbits[0] = m0 << 16; cbits[1] = m0 & 0xFFFF0000u;
-                cbits[2] = m1 << 16; cbits[3] = m1 & 0xFFFF0000u;
-            } else {
-                float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-                    a0 = fmaxf(a0, fabsf(w.x));
-                    a1 = fmaxf(a1, fabsf(w.y));
-                }
-                if (a0 == INFINITY || a1 == INFINITY) {
-                    a0 = a1 = 0.f;
-#pragma unroll 4
-                    for (int j = 0; j < 32; ++j) {
-                        const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-                        if (fabsf(w.x) < INFINITY) a0 = fmaxf(a0, fabsf(w.x));
-                        if (fabsf(w.y) < INFINITY) a1 = fmaxf(a1, fabsf(w.y));
-                    }
-                }
-                cbits[0] = __float_as_uint(a0);
-                cbits[1] = __float_as_uint(a1);
-            }
-            uint32_t packed_b = 0u;
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
-                col_inv[i] = __uint_as_float(ie << 23);
-                packed_b |= (254u - ie) << (8 * i);
-            }
-            // sm_col[c][w]: column c of the tile, row block w
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) sm_col[(lane * VEC + i) * 4 + warp] = (uint8_t)(packed_b >> (8 * i));
-        }
-
-        // ---- pass B: rows; BF16 rows go through the shuffle reduction in pairs ------------------
-        uint8_t* my_qrow = qrow_tile + warp * 32 * T_COLS + lane * VEC;
-        uint8_t* my_qcol = qcol_tile + warp * 32 * T_COLS + lane * VEC;
-#pragma unroll 4
-        for (int j = 0; j < 32; j += 2) {
-            float x0[VEC], x1[VEC];
-            float inv0 = 1.f, inv1 = 1.f;
-            if constexpr (BF) {
-                const uint2 w0 = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-                const uint2 w1 = *reinterpret_cast<const uint2*>(my_in + (j + 1) * T_BYTES);
-                x0[0] = __uint_as_float(w0.x << 16); x0[1] = __uint_as_float(w0.x & 0xFFFF0000u);
-                x0[2] = __uint_as_float(w0.y << 16); x0[3] = __uint_as_float(w0.y & 0xFFFF0000u);
-                x1[0] = __uint_as_float(w1.x << 16); x1[1] = __uint_as_float(w1.x & 0xFFFF0000u);
-                x1[2] = __uint_as_float(w1.y << 16); x1[3] = __uint_as_float(w1.y & 0xFFFF0000u);
-                if (DO_ROW) {
-                    const uint32_t m0 = hmax2_abs(w0.x, w0.y);               // row j  : (max |e0|,|e2| ; max |e1|,|e3|)
-                    const uint32_t m1 = hmax2_abs(w1.x, w1.y);               // row j+1
-                    uint32_t z = hmax2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));   // (amax_j, amax_j+1) of this lane
-#pragma unroll
-                    for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
-                    if (__any_sync(0xFFFFFFFFu, ((z + 0x00800080u) & 0x80008000u) != 0u)) {   // rare: an Inf got in
-                        const uint32_t f0 = hmax2(finite_abs2(w0.x), finite_abs2(w0.y));
-                        const uint32_t f1 = hmax2(finite_abs2(w1.x), finite_abs2(w1.y));
-                        z = hmax2(__byte_perm(f0, f1, 0x5410), __byte_perm(f0, f1, 0x7632));
-#pragma unroll
-                        for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
-                    }
-                    const uint32_t ie0 = inv_exp_field<ELEM>(z << 16, rule_offset);
-                    const uint32_t ie1 = inv_exp_field<ELEM>(z & 0xFFFF0000u, rule_offset);
-                    inv0 = __uint_as_float(ie0 << 23);
-                    inv1 = __uint_as_float(ie1 << 23);
-                    if ((lane & (LPB - 1)) == 0) {
-                        sm_row[(warp * 32 + j) * 4 + lane / LPB] = (uint8_t)(254u - ie0);
-                        sm_row[(warp * 32 + j + 1) * 4 + lane / LPB] = (uint8_t)(254u - ie1);
-                    }
-                }
-            } else {
-                const float2 w0 = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-                const float2 w1 = *reinterpret_cast<const float2*>(my_in + (j + 1) * T_BYTES);
-                x0[0] = w0.x; x0[1] = w0.y;
-                x1[0] = w1.x; x1[1] = w1.y;
-                if (DO_ROW) {
-                    float a0 = fmaxf(fabsf(w0.x), fabsf(w0.y)), a1 = fmaxf(fabsf(w1.x), fabsf(w1.y));
-                    a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f);                 // two NaNs -> 0
-#pragma unroll
-                    for (int off = 1; off < LPB; off <<= 1) {
-                        a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
-                        a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
-                    }
-                    if (__any_sync(0xFFFFFFFFu, a0 == INFINITY || a1 == INFINITY)) {
-                        a0 = 0.f; a1 = 0.f;
-                        if (fabsf(w0.x) < INFINITY) a0 = fabsf(w0.x);
-                        if (fabsf(w0.y) < INFINITY) a0 = fmaxf(a0, fabsf(w0.y));
-                        if (fabsf(w1.x) < INFINITY) a1 = fabsf(w1.x);
-                        if (fabsf(w1.y) < INFINITY) a1 = fmaxf(a1, fabsf(w1.y));
-#pragma unroll
-                        for (int off = 1; off < LPB; off <<= 1) {
-                            a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
-                            a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
-                        }
-                    }
-                    const uint32_t ie0 = inv_exp_field<ELEM>(__float_as_uint(a0), rule_offset);
-                    const uint32_t ie1 = inv_exp_field<ELEM>(__float_as_uint(a1), rule_offset);
-                    inv0 = __uint_as_float(ie0 << 23);
-                    inv1 = __uint_as_float(ie1 << 23);
-                    if ((lane & (LPB - 1)) == 0) {
-                        sm_row[(warp * 32 + j) * 4 + lane / LPB] = (uint8_t)(254u - ie0);
-                        sm_row[(warp * 32 + j + 1) * 4 + lane / LPB] = (uint8_t)(254u - ie1);
-                    }
-                }
-            }
-            if (DO_ROW) {
-                if constexpr (VEC == 4) {
-                    *reinterpret_cast<uint32_t*>(my_qrow + j * T_COLS) = cvt_fp8x4<ELEM>(x0[0] * inv0, x0[1] * inv0, x0[2] * inv0, x0[3] * inv0);
-                    *reinterpret_cast<uint32_t*>(my_qrow + (j + 1) * T_COLS) = cvt_fp8x4<ELEM>(x1[0] * inv1, x1[1] * inv1, x1[2] * inv1, x1[3] * inv1);
-                } else {
-                    *reinterpret_cast<uint16_t*>(my_qrow + j * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * inv0, x0[1] * inv0);
-                    *reinterpret_cast<uint16_t*>(my_qrow + (j + 1) * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * inv1, x1[1] * inv1);
-                }
-            }
-            if (DO_COL) {
-                if constexpr (VEC == 4) {
-                    *reinterpret_cast<uint32_t*>(my_qcol + j * T_COLS) =
-                        cvt_fp8x4<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1], x0[2] * col_inv[2], x0[3] * col_inv[3]);
-                    *reinterpret_cast<uint32_t*>(my_qcol + (j + 1) * T_COLS) =
-                        cvt_fp8x4<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1], x1[2] * col_inv[2], x1[3] * col_inv[3]);
-                } else {
-                    *reinterpret_cast<uint16_t*>(my_qcol + j * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1]);
-                    *reinterpret_cast<uint16_t*>(my_qcol + (j + 1) * T_COLS) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1]);
-                }
-            }
-        }
-
-        // shared-memory writes -> visible to the TMA engine; the input tile is free to be refilled
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // every warp is done with this ring slot: refill it with the tile after next
         __syncthreads();
-
         if (tid == 0) {
-            if (DO_ROW)
-                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                             ::"l"(&tmap_qrow), "r"((int)gcol0), "r"((int)grow0), "r"(smem_addr(qrow_tile)) : "memory");
-            if (DO_COL)
-                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                             ::"l"(&tmap_qcol), "r"((int)gcol0), "r"((int)grow0), "r"(smem_addr(qcol_tile)) : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            const int next = tile + gridDim.x;
-            if (next < num_tiles) {   // prefetch the next tile under the stores
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"((uint32_t)IN_BYTES) : "memory");
-                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                             ::"r"(smem_addr(in_tile)), "l"(&tmap_src), "r"(bar_a), "r"((next % p.tiles_x) * T_COLS), "r"((next / p.tiles_x) * T_ROWS)
-                             : "memory");
-            }
+            const int next = tile + 2 * (int)gridDim.x;
+            if (next < num_tiles) issue_load(next, buf);
         }
 
         // ---- scale bytes (1/32 of the output): plain stores from the staging arrays ----------
-        if (DO_ROW) {
+        if (DO_ROW && tid < T_ROWS) {
             const int64_t r = grow0 + tid, ncb = p.cols >> 5, kb0 = (int64_t)tile_x * NKB;
             const int nkb = (int)min((int64_t)NKB, ncb - kb0);
             if (p.sf_layout == MXFP8_SF_SWIZZLED) {
@@ -355,12 +413,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const __grid_c
                 for (int w = 0; w < nrb_here; ++w) p.s_col[(rb0 + w) * p.cols + c] = sm_col[tid * 4 + w];
             }
         }
-
-        // the staging tiles may be overwritten once the stores have read them
-        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        __syncthreads();
     }
-    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -405,26 +458,26 @@ int qt_sm_count()
 }
 
 template <int DTYPE, int ELEM, bool R, bool C>
-cudaError_t launch(const CUtensorMap& ms, const CUtensorMap& mr, const CUtensorMap& mc, const QParams& p, cudaStream_t stream)
+cudaError_t launch(const CUtensorMap& ms, const QParams& p, cudaStream_t stream)
 {
-    constexpr int SMEM = IN_BYTES + 2 * Q_MAX_BYTES + 1024 + 16;
+    constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
     auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C>;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (err != cudaSuccess) return err;
     const int tiles = p.tiles_x * p.tiles_y;
     const int max_ctas = qt_sm_count() * 3;
     const int grid = tiles < max_ctas ? tiles : max_ctas;
-    kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, mr, mc, p);
+    kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, p);
     count_launch(1);
     return cudaGetLastError();
 }
 
 template <int DTYPE, int ELEM>
-cudaError_t launch_o(int orientation, const CUtensorMap& ms, const CUtensorMap& mr, const CUtensorMap& mc, const QParams& p, cudaStream_t st)
+cudaError_t launch_o(int orientation, const CUtensorMap& ms, const QParams& p, cudaStream_t st)
 {
-    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false>(ms, mr, mc, p, st);
-    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true>(ms, mr, mc, p, st);
-    return launch<DTYPE, ELEM, true, true>(ms, mr, mc, p, st);
+    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false>(ms, p, st);
+    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true>(ms, p, st);
+    return launch<DTYPE, ELEM, true, true>(ms, p, st);
 }
 
 }  // namespace
@@ -444,26 +497,23 @@ int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t co
 {
     const bool bf = src_dtype == MXFP8_BF16;
     const uint32_t t_cols = bf ? 128 : 64;
-    CUtensorMap ms, mr, mc;
+    CUtensorMap ms;
     if (!make_map_2d(&ms, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
                      const_cast<void*>(src), (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS))
-        return MXFP8_ERR_CUDA;
-    void* qr = (orientation & MXFP8_ROW) ? q_row : q_col;   // an unused map still has to be valid
-    void* qc = (orientation & MXFP8_COL) ? q_col : q_row;
-    if (!make_map_2d(&mr, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qr, (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS) ||
-        !make_map_2d(&mc, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qc, (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS))
         return MXFP8_ERR_CUDA;
     QParams p{};
     p.rows = rows; p.cols = cols; p.rule = scale_rule; p.sf_layout = sf_layout;
     p.tiles_x = (int)((cols + t_cols - 1) / t_cols);
     p.tiles_y = (int)((rows + T_ROWS - 1) / T_ROWS);
+    p.q_row = static_cast<uint8_t*>(q_row);
+    p.q_col = static_cast<uint8_t*>(q_col);
     p.s_row = static_cast<uint8_t*>(s_row);
     p.s_col = static_cast<uint8_t*>(s_col);
     cudaError_t err;
-    if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3>(orientation, ms, mr, mc, p, stream)
-                                     : launch_o<MXFP8_BF16, MXFP8_E5M2>(orientation, ms, mr, mc, p, stream);
-    else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3>(orientation, ms, mr, mc, p, stream)
-                                  : launch_o<MXFP8_FP32, MXFP8_E5M2>(orientation, ms, mr, mc, p, stream);
+    if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3>(orientation, ms, p, stream)
+                                     : launch_o<MXFP8_BF16, MXFP8_E5M2>(orientation, ms, p, stream);
+    else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3>(orientation, ms, p, stream)
+                                  : launch_o<MXFP8_FP32, MXFP8_E5M2>(orientation, ms, p, stream);
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
