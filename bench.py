@@ -123,13 +123,23 @@ def oracle_sample_seconds(sample_rows: int = 256):
         q[name, "c"] = orc.quantize_threads(t, orc.COL, orc.RULE_PAPER, orc.E4M3, threads)
     t_cast = time.perf_counter() - t0
     cast_full = t_cast * (T * H + F * H + T * F) / float(r * H + r * H + r * F)
-    # GEMM sample: r x r outputs of fprop over the full K = H (decoded FP64 operands, two products)
     t0 = time.perf_counter()
-    d, s = orc.gemm_f64(q["x", "r"][0], q["x", "r"][1], q["w", "r"][0], q["w", "r"][1])
-    t_gemm = time.perf_counter() - t0
-    gemm_full = t_gemm * STEP_FLOP / (2.0 * r * r * H)
-    desc = ("%d rows of X, W, dY quantized in both orientations on %d threads; %dx%dx%d FP64 product "
-            "(+|A||B| bound product) via numpy; scaled linearly to the full step" % (r, threads, r, r, H))
+    if r == T:
+        # the whole step: all three products in FP64 over the decoded operands (+ the |A||B| bound products)
+        orc.gemm_f64(q["x", "r"][0], q["x", "r"][1], q["w", "r"][0], q["w", "r"][1], "k", "k")            # fprop
+        orc.gemm_f64(q["dy", "r"][0], q["dy", "r"][1], q["w", "c"][0], q["w", "c"][1], "k", "mn")         # dgrad
+        orc.gemm_f64(q["dy", "c"][0], q["dy", "c"][1], q["x", "c"][0], q["x", "c"][1], "mn", "mn")        # wgrad
+        t_gemm = time.perf_counter() - t0
+        gemm_full = t_gemm
+        desc = ("the whole step on the host: X, W, dY quantized in both orientations on %d threads (row slabs), then "
+                "fprop, dgrad, wgrad as FP64 products of the decoded operands (+ the |A||B| bound products) via numpy" % threads)
+    else:
+        # GEMM sample: r x r outputs of fprop over the full K = H (decoded FP64 operands, two products)
+        orc.gemm_f64(q["x", "r"][0], q["x", "r"][1], q["w", "r"][0], q["w", "r"][1])
+        t_gemm = time.perf_counter() - t0
+        gemm_full = t_gemm * STEP_FLOP / (2.0 * r * r * H)
+        desc = ("%d rows of X, W, dY quantized in both orientations on %d threads; %dx%dx%d FP64 product "
+                "(+|A||B| bound product) via numpy; scaled linearly to the full step" % (r, threads, r, r, H))
     return t_cast + t_gemm, cast_full + gemm_full, desc, threads
 
 
