@@ -36,6 +36,13 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/: the FPROP GEMM of this step, and the quantize kernel on a
+# 128 MB BF16 tensor (the size of dY, the largest cast of the step).  Writes still dirty in
+# L2 when the kernel ends are not counted by ncu, so both are below the algorithmic bytes.
+NCU_TRAFFIC_GEMM_FPROP = 49.8e6 + 86.6e6
+NCU_TRAFFIC_QUANTIZE_128MB = 134.3e6 + 85.0e6
+
 STEP_FLOP = 3 * 2.0 * T * H * F                       # three GEMMs of 275 GFLOP
 CAST_BYTES = (T * H + F * H + T * F) * (2 + 2 * (1 + 1 / 32))   # src + two orientations x (q + scales)
 GEMM_SHAPES = {"fprop": (T, F, H), "dgrad": (T, H, F), "wgrad": (F, H, T)}
@@ -318,13 +325,15 @@ def run_ours(args):
                  "frac_of_measured_copy": cast_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": cast_gbs / NOMINAL_HBM_GBS},
         "gemm": {"value": gemm_all, "unit": "TFLOP/s", "ms": gemm_ms, "tflops": gemm_tflops,
                  "frac_of_2x_measured_bf16": gemm_all / fp8_peak, "frac_of_nominal_4.5PF": gemm_all / NOMINAL_FP8_TFLOPS},
-        "roofline": {"bound": "tensor", "kernel": "gemm_kernel<256> (%s)" % dom, "achieved": gemm_tflops[dom],
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel<256, pair> (%s)" % dom, "achieved": gemm_tflops[dom],
                      "peak": fp8_peak, "unit": "TFLOP/s", "frac": gemm_tflops[dom] / fp8_peak,
                      "peak_source": "2 x %s bf16 burst TFLOP/s (Table 1: MXFP8 = 2x BF16)" % peaks["source"],
-                     "traffic": None},
-        "roofline_cast": {"bound": "hbm", "kernel": "quantize_kernel<bf16,e4m3,both>", "achieved": cast_gbs,
+                     "algorithmic_flop_per_launch": 2.0 * T * H * F,
+                     "traffic": NCU_TRAFFIC_GEMM_FPROP, "traffic_note": "ncu capture of the fprop launch, see profiles/"},
+        "roofline_cast": {"bound": "hbm", "kernel": "quantize_tma_kernel<bf16,e4m3,row+col>", "achieved": cast_gbs,
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cast_gbs / peaks["hbm_gbs"],
-                          "peak_source": peaks["source"], "traffic": None},
+                          "peak_source": peaks["source"], "algorithmic_bytes_per_element": 4.0625,
+                          "traffic": NCU_TRAFFIC_QUANTIZE_128MB, "traffic_note": "ncu capture, 8192x8192 BF16 tensor (= dY), see profiles/"},
         "e2e": e2e, "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
         "cpu_baseline": cpu,
     }
