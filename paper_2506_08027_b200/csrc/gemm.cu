@@ -62,6 +62,11 @@ struct GemmParams {
     int tiles_m, tiles_n, num_tiles, num_kb;
     int group_m;          // tile rasterisation: M-tiles per group (L2 reuse)
     uint32_t stage_tx;    // bytes that land per pipeline stage on the (leader's) full barrier
+    int store_d;          // 0 when only the fused MXFP8 output is wanted
+    int epi_orient;       // 0 = no fused MXFP8 output, else MXFP8_ROW / COL / BOTH
+    int epi_rule, epi_elem;
+    uint8_t* epi_s_row;   // swizzled scales of the row-blocked output, logical [M, N/32]
+    uint8_t* epi_s_col;   // swizzled scales of the column-blocked output, logical [N, M/32]
 };
 
 // BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
@@ -306,6 +311,103 @@ __device__ __forceinline__ uint32_t make_idesc(int a_elem, int b_elem, int a_mn,
            ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24);
 }
 
+// ------------------------------------------------------------------------------ fused MXFP8 output
+// 1/X exponent field for a block with this amax bit pattern (same integer form of Algorithm 1 /
+// App. A.1 as the quantize kernels): e' = (bits + offset) >> 23, b = max(e' - emax, 0), field = 254 - b.
+template <int ELEM>
+__device__ __forceinline__ uint32_t epi_inv_exp(uint32_t amax_bits, uint32_t rule_offset)
+{
+    const int e = (int)((amax_bits + rule_offset) >> 23);
+    return (uint32_t)min(254 + ElemTraits<ELEM>::emax - e, 254);
+}
+// 64 bytes of one row (16 words) into the warp's 64-byte-swizzled staging buffer, then one TMA store
+// of the 32 x 64-byte box.  All lanes call it; lane 0 issues the store.
+__device__ __forceinline__ void epi_store_box(const CUtensorMap* map, uint32_t buf, uint32_t row_off, uint32_t sw, int lane,
+                                              const uint32_t (&w)[16], int c0, int c1)
+{
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(row_off + (((uint32_t)j ^ sw) << 4)), "r"(w[4 * j]), "r"(w[4 * j + 1]), "r"(w[4 * j + 2]), "r"(w[4 * j + 3]) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) {
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                     ::"l"(map), "r"(c0), "r"(c1), "r"(buf) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+}
+
+// Converts this warp's 32 rows x CW columns of FP32 accumulators (lane = row) to MXFP8 exactly as
+// mxfp8_quantize would convert the FP32 output (Sec. 2: the FP32 output is quantized to MX format
+// when its consumer needs it): row blocks run along N inside a lane, column blocks are the warp's
+// 32 rows (one warp-wide integer max per column; |x| bit patterns of finite floats order like integers).
+template <int CW, int ELEM>
+__device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams& p, const CUtensorMap* map_row,
+                                       const CUtensorMap* map_col, uint32_t buf, uint32_t row_off, uint32_t sw, int lane,
+                                       int row0, int col0)
+{
+    const uint32_t rule_offset = (p.epi_rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
+    const int row = row0 + lane;
+    if (p.epi_orient & MXFP8_ROW) {
+        const int64_t nkb = p.N >> 5;
+#pragma unroll
+        for (int ch = 0; ch < CW / 64; ++ch) {
+            uint32_t w[16];
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                const int b0 = ch * 64 + hb * 32;
+                float m = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(v[b0 + i])));   // NaN ignored
+                if (m == INFINITY) {   // rare: finite-only maximum
+                    m = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float a = fabsf(__uint_as_float(v[b0 + i]));
+                        if (a < INFINITY) m = fmaxf(m, a);
+                    }
+                }
+                const uint32_t ie = epi_inv_exp<ELEM>(__float_as_uint(m), rule_offset);
+                const float inv = __uint_as_float(ie << 23);
+                p.epi_s_row[sf_swizzled_offset(row, (col0 + b0) >> 5, nkb)] = (uint8_t)(254u - ie);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    w[hb * 8 + i] = cvt_fp8x4<ELEM>(__uint_as_float(v[b0 + 4 * i]) * inv, __uint_as_float(v[b0 + 4 * i + 1]) * inv,
+                                                    __uint_as_float(v[b0 + 4 * i + 2]) * inv, __uint_as_float(v[b0 + 4 * i + 3]) * inv);
+            }
+            epi_store_box(map_row, buf, row_off, sw, lane, w, col0 + ch * 64, row0);
+        }
+    }
+    if (p.epi_orient & MXFP8_COL) {
+        const int64_t nkb = p.M >> 5;
+        const int64_t kb = row0 >> 5;
+#pragma unroll
+        for (int ch = 0; ch < CW / 64; ++ch) {
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float y[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int c = ch * 64 + i * 4 + e;
+                    uint32_t a = v[c] & 0x7FFFFFFFu;
+                    a = (a >= 0x7F800000u) ? 0u : a;           // Inf / NaN stay out of amax
+                    uint32_t amax;
+                    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
+                    const uint32_t ie = epi_inv_exp<ELEM>(amax, rule_offset);
+                    y[e] = __uint_as_float(v[c]) * __uint_as_float(ie << 23);
+                    if (lane == (c & 31)) p.epi_s_col[sf_swizzled_offset(col0 + c, kb, nkb)] = (uint8_t)(254u - ie);
+                }
+                w[i] = cvt_fp8x4<ELEM>(y[0], y[1], y[2], y[3]);
+            }
+            epi_store_box(map_col, buf, row_off, sw, lane, w, col0 + ch * 64, row0);
+        }
+    }
+}
+
 // Tile rasterisation: tiles are numbered group by group; a group is `group_m` M-tiles tall and
 // spans all N-tiles, M fastest inside it, so the tiles in flight at one time share few distinct
 // A row-blocks and B row-blocks and hit in L2.
@@ -322,7 +424,8 @@ template <int BN, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
-            const __grid_constant__ CUtensorMap tmap_d, const GemmParams p)
+            const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_qrow,
+            const __grid_constant__ CUtensorMap tmap_qcol, const GemmParams p)
 {
     using C = Cfg<BN, PAIR>;
     extern __shared__ uint8_t smem_raw[];
@@ -541,7 +644,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
             const int row0 = (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
-            if (p.out_dtype == MXFP8_BF16) {
+            if constexpr (CW % 64 == 0) {
+                if (p.epi_orient) {
+                    if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
+                    else epi_mx<CW, MXFP8_E5M2>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
+                }
+            }
+            if (!p.store_d) {
+            } else if (p.out_dtype == MXFP8_BF16) {
 #pragma unroll
                 for (int ch = 0; ch < CW / 32; ++ch) {          // 32 columns = 64 bytes per row
                     if (col0 + ch * 32 >= n_total) break;       // ragged last tile: nothing to store
@@ -652,6 +762,19 @@ bool make_tmap_sf(CUtensorMap* map, const void* base, uint64_t mn_atoms, uint64_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Fused MXFP8 output bytes [M, N]: boxes of 32 rows x 64 bytes, 64-byte swizzle (store side).
+bool make_tmap_q(CUtensorMap* map, void* base, uint64_t M, uint64_t N)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {N, M};
+    const cuuint64_t strides[1] = {N};
+    const cuuint32_t box[2] = {64u, 32u};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Output matrix D [M, N] row-major: boxes of 32 rows x 64 bytes, 64-byte swizzle (store side).
 bool make_tmap_d(CUtensorMap* map, void* base, uint64_t M, uint64_t N, int out_dtype)
 {
@@ -678,7 +801,7 @@ int sm_count()
     return n;
 }
 
-struct GemmMaps { CUtensorMap a, b, sfa, sfb, d; };
+struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; };
 
 template <int BN, bool PAIR>
 int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
@@ -709,7 +832,7 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, p);
     count_launch(1);
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
@@ -733,16 +856,30 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     if (b_elem != MXFP8_E4M3 && b_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs) return MXFP8_ERR_NULL;
-    if (!D) return epi ? MXFP8_ERR_UNSUPPORTED : MXFP8_ERR_NULL;
+    if (!D && !epi) return MXFP8_ERR_NULL;
+    if (epi) {
+        if (epi->orientation < MXFP8_ROW || epi->orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+        if (epi->scale_rule != MXFP8_RULE_PAPER && epi->scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+        if (epi->elem != MXFP8_E4M3 && epi->elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+        if ((epi->orientation & MXFP8_ROW) && (!epi->q_row || !epi->s_row)) return MXFP8_ERR_NULL;
+        if ((epi->orientation & MXFP8_COL) && (!epi->q_col || !epi->s_col)) return MXFP8_ERR_NULL;
+        if ((epi->orientation & MXFP8_ROW) && (!aligned16(epi->q_row) || !aligned16(epi->s_row))) return MXFP8_ERR_ALIGN;
+        if ((epi->orientation & MXFP8_COL) && (!aligned16(epi->q_col) || !aligned16(epi->s_col))) return MXFP8_ERR_ALIGN;
+    }
     if (M <= 0 || N <= 0 || K <= 0 || (K % 32)) return MXFP8_ERR_SHAPE;
     if ((M % 128) || (N % 128) || (K % 128)) return MXFP8_ERR_UNSUPPORTED;
     if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
-    if (epi) return MXFP8_ERR_UNSUPPORTED;
-    if (!aligned16(Aq) || !aligned16(As) || !aligned16(Bq) || !aligned16(Bs) || !aligned16(D)) return MXFP8_ERR_ALIGN;
+    if (!aligned16(Aq) || !aligned16(As) || !aligned16(Bq) || !aligned16(Bs) || (D && !aligned16(D))) return MXFP8_ERR_ALIGN;
 
     GemmParams p{};
     p.M = M; p.N = N; p.K = K;
     p.a_mn = a_major; p.b_mn = b_major; p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
+    p.store_d = D ? 1 : 0;
+    if (epi) {
+        p.epi_orient = epi->orientation; p.epi_rule = epi->scale_rule; p.epi_elem = epi->elem;
+        p.epi_s_row = static_cast<uint8_t*>(epi->s_row);
+        p.epi_s_col = static_cast<uint8_t*>(epi->s_col);
+    }
     // tile shape: estimated cycles = waves x (MMA cycles per tile + what the epilogue adds when it
     // cannot run under the next tile's MMAs)
     const int sms = sm_count();
@@ -756,6 +893,7 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     for (int bn : {256, 192, 128}) {
         for (int pr = 1; pr >= 0; --pr) {
             if (pr && ((M % 256) || bn == 128)) continue;
+            if (epi && bn == 192) continue;   // the fused output works on 64-column chunks per epilogue warp
             if (pass == 0) {   // forced shape, when it applies to this problem
                 if (atoi(force) != bn || (strchr(force, 'p') != nullptr) != (pr != 0)) continue;
             }
@@ -779,7 +917,14 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
                                               : make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)K, 128, 128);
     const bool oks = make_tmap_sf(&m.sfa, As, (uint64_t)(M / 128), (uint64_t)(K / 128)) &&
                      make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(K / 128));
-    if (!oka || !okb || !oks || !make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype)) return MXFP8_ERR_CUDA;
+    // maps that a launch does not use still have to be valid: point them at any output that exists
+    void* q_any = epi ? ((epi->orientation & MXFP8_ROW) ? epi->q_row : epi->q_col) : D;
+    void* q_row = (epi && (epi->orientation & MXFP8_ROW)) ? epi->q_row : q_any;
+    void* q_col = (epi && (epi->orientation & MXFP8_COL)) ? epi->q_col : q_any;
+    const bool okd = D ? make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype) : make_tmap_q(&m.d, q_any, (uint64_t)M, (uint64_t)N);
+    if (!oka || !okb || !oks || !okd || !make_tmap_q(&m.qrow, q_row, (uint64_t)M, (uint64_t)N) ||
+        !make_tmap_q(&m.qcol, q_col, (uint64_t)M, (uint64_t)N))
+        return MXFP8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (best_pair) return best_bn == 256 ? launch_gemm<256, true>(m, p, st) : launch_gemm<192, true>(m, p, st);
     if (best_bn == 256) return launch_gemm<256, false>(m, p, st);

@@ -156,3 +156,90 @@ def test_nan_scale_byte_poisons_its_outputs():
     d64, _ = orc.gemm_f64(aq, a_s, bq, b_s)
     got = gpu_gemm(aq, a_s, bq, b_s)
     assert np.array_equal(np.isnan(got), np.isnan(d64))
+
+
+# ------------------------------------------------------------------------------- fused MXFP8 output
+
+def _run_fused(aq, a_s, bq, b_s, orientation, rule, elem, with_d):
+    """GEMM with the fused MXFP8 epilogue; returns dict of numpy outputs (raw swizzled scales)."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import swizzle_np
+    M, K = aq.shape
+    N = bq.shape[0]
+    dA, dB = torch.from_numpy(aq).cuda(), torch.from_numpy(bq).cuda()
+    dSA, dSB = torch.from_numpy(swizzle_np(a_s)).cuda(), torch.from_numpy(swizzle_np(b_s)).cuda()
+    outs = {}
+    bufs = []
+    for o in (B.ROW, B.COL):
+        if orientation & o:
+            bufs.append(torch.zeros((M, N), dtype=torch.uint8, device="cuda"))
+            bufs.append(torch.zeros(B.mxfp8_scale_bytes(M, N, o, B.SF_SWIZZLED), dtype=torch.uint8, device="cuda"))
+        else:
+            bufs += [None, None]
+    epi = B.make_epilogue(orientation, rule, elem, *bufs)
+    D = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") if with_d else None
+    B.mxfp8_gemm(dA, dSA, dB, dSB, M, N, K, B.K_MAJOR, B.K_MAJOR, 0, 0, D, epi=epi)
+    assert B.mxfp8_device_status() == 0
+    names = ("q_row", "s_row", "q_col", "s_col")
+    for n, b in zip(names, bufs):
+        if b is not None:
+            outs[n] = b.cpu().numpy()
+    if D is not None:
+        outs["D"] = D.cpu().numpy()
+    return outs
+
+
+@pytest.mark.parametrize("orientation", [1, 2, 3])
+@pytest.mark.parametrize("rule", [orc.RULE_PAPER, orc.RULE_OCP])
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+def test_fused_epilogue_equals_quantize_of_unfused_output(orientation, rule, elem):
+    # Sec. 2: the FP32 output is quantized to MX format when its consumer needs it.  The fused bytes must
+    # be exactly what mxfp8_quantize (oracle-exact) makes of the same kernel's unfused FP32 output.
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    m, n, k = 512, 768, 512
+    a = synth.gaussian((m, k), 7)
+    b = synth.output_gradient((n, k), 8)
+    aq, a_s = orc.quantize(a, orc.ROW)
+    bq, b_s = orc.quantize(b, orc.ROW)
+    d32 = gpu_gemm(aq, a_s, bq, b_s)                                   # unfused FP32 output
+    fused = _run_fused(aq, a_s, bq, b_s, orientation, rule, elem, with_d=True)
+    assert np.array_equal(fused["D"].view(np.uint32), d32.view(np.uint32))
+    src = torch.from_numpy(d32).cuda()
+    ref = B.alloc_quantize_outputs(m, n, orientation, B.SF_SWIZZLED)
+    for t in ref:
+        if t is not None:
+            t.zero_()
+    B.mxfp8_quantize(src, orientation, rule, elem, *ref, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    for name, t in zip(("q_row", "s_row", "q_col", "s_col"), ref):
+        if t is not None:
+            assert np.array_equal(fused[name], t.cpu().numpy()), name
+    only = _run_fused(aq, a_s, bq, b_s, orientation, rule, elem, with_d=False)   # D = NULL
+    for name in ("q_row", "s_row", "q_col", "s_col"):
+        if name in fused:
+            assert np.array_equal(only[name], fused[name]), name
+
+
+def test_fused_epilogue_against_fp64_oracle():
+    # decoded fused output vs the FP64 product: GEMM bound + one FP8 rounding (half an ulp of the element
+    # grid relative, 2^-4 for E4M3, plus half the smallest subnormal times the block scale)
+    from helpers import logical_scales_from_swizzled
+    m, n, k = 256, 512, 1024
+    a = synth.gaussian((m, k), 17)
+    b = synth.gaussian((n, k), 18, 0.02)
+    aq, a_s = orc.quantize(a, orc.ROW)
+    bq, b_s = orc.quantize(b, orc.ROW)
+    d64, sabs = orc.gemm_f64(aq, a_s, bq, b_s)
+    fused = _run_fused(aq, a_s, bq, b_s, 3, orc.RULE_PAPER, orc.E4M3, with_d=False)
+    s_row = logical_scales_from_swizzled(fused["s_row"], m, n // 32)             # [m, n/32]
+    s_col = logical_scales_from_swizzled(fused["s_col"], n, m // 32).T           # [m/32, n]
+    for q, s, orient in ((fused["q_row"], s_row, orc.ROW), (fused["q_col"], np.ascontiguousarray(s_col), orc.COL)):
+        dq = orc.dequantize_f64(q, s, orient)
+        x = np.exp2(s.astype(np.float64) - 127)
+        xfull = np.repeat(x, 32, axis=1) if orient == orc.ROW else np.repeat(x, 32, axis=0)
+        bound = 2.0 ** -16 * sabs + 2.0 ** -4 * np.abs(d64) * 1.001 + 2.0 ** -10 * xfull
+        assert (np.abs(dq - d64) <= bound).all()
+        # paper rule: nothing saturates (no decoded magnitude above 448 * X) and the scale is tight
+        assert (np.abs(dq) <= 448 * xfull).all()
