@@ -178,6 +178,22 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------------ GPU arm
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Device time of the slowest rank (the job finishes when the last rank does)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, ms_step: float) -> float:
+    """TFLOP/s of the whole job: every rank runs the same step on its own batch (weak scaling)."""
+    return world * STEP_FLOP / (ms_step * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -246,11 +262,7 @@ def run_ours(args):
     e1.record()
     barrier()
     launches = B.mxfp8_launch_count() - launches0
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     ms_step = ms_total / args.steps
 
     # ---- timed region 2: the same steps with an event before every launch -> per-kernel durations
@@ -282,13 +294,9 @@ def run_ours(args):
             B.mxfp8_linear_host(hx, hw, hdy, P, hy, hdx, hdw, ws)
         g1.record()
         barrier()
-        e2e_ms = g0.elapsed_time(g1) / n_e2e
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(g0.elapsed_time(g1) / n_e2e, world, dev)
         assert torch.equal(hy.cuda(), Y), "host-buffer path and device path disagree"
-        e2e = {"value": world * STEP_FLOP / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        e2e = {"value": whole_job_value(world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": (T * H + F * H + T * F) * 2, "d2h_bytes_per_step": (T * F + T * H + F * H) * 2,
                "steps": n_e2e}
         del ws
@@ -307,7 +315,7 @@ def run_ours(args):
     gemm_all = STEP_FLOP / (sum(gemm_ms.values()) * 1e-3) / 1e12
     cast_gbs = CAST_BYTES / (cast_ms * 1e-3) / 1e9
     dom = max(gemm_ms, key=gemm_ms.get)                         # dominant kernel = slowest GEMM launch
-    value = world * STEP_FLOP / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(world, ms_step)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

@@ -243,3 +243,52 @@ def test_fused_epilogue_against_fp64_oracle():
         assert (np.abs(dq - d64) <= bound).all()
         # paper rule: nothing saturates (no decoded magnitude above 448 * X) and the scale is tight
         assert (np.abs(dq) <= 448 * xfull).all()
+
+
+# ------------------------------------------------------------------------------- benchmark sizes
+
+def test_bench_step_shapes_sampled_rows():
+    """The three GEMMs of the benchmark step at full size (tokens 8192, hidden 2048, FFN 8192), in the
+    launch configuration bench.py times.  Operands are quantized by the oracle on the host; 48 sampled
+    output rows of each product (first, last, tile edges, random) are checked element by element against
+    the FP64 oracle; the BF16 output must be the RNE rounding of the FP32 output."""
+    import os
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import swizzle_np
+    T, H, F = 8192, 2048, 8192
+    thr = os.cpu_count() or 1
+    x = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.gaussian((T, H), synth.seed_for(2, 0))))
+    w = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.gaussian((F, H), synth.seed_for(2, 1), 0.02)))
+    dy = synth.bf16_bits_as_f32(synth.f32_to_bf16_bits(synth.output_gradient((T, F), synth.seed_for(2, 2))))
+    q = {}
+    for name, t in (("x", x), ("w", w), ("dy", dy)):
+        q[name, "r"] = orc.quantize_threads(t, orc.ROW, orc.RULE_PAPER, orc.E4M3, thr)
+        q[name, "c"] = orc.quantize_threads(t, orc.COL, orc.RULE_PAPER, orc.E4M3, thr)
+    dev = {}
+    for key, (qq, ss) in q.items():
+        s_log = ss if key[1] == "r" else np.ascontiguousarray(ss.T)
+        dev[key] = (torch.from_numpy(qq).cuda(), torch.from_numpy(swizzle_np(s_log)).cuda())
+    rng = np.random.default_rng(5)
+    cases = (("fprop", ("x", "r"), ("w", "r"), "k", "k", T, F, H),
+             ("dgrad", ("dy", "r"), ("w", "c"), "k", "mn", T, H, F),
+             ("wgrad", ("dy", "c"), ("x", "c"), "mn", "mn", F, H, T))
+    for name, ka, kb, am, bm, M, N, K in cases:
+        rows = np.unique(np.concatenate([[0, 1, 127, 128, 255, 256, M - 257, M - 256, M - 129, M - 128, M - 1],
+                                         rng.integers(0, M, 37)]))
+        d32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        dbf = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        args = (dev[ka][0], dev[ka][1], dev[kb][0], dev[kb][1], M, N, K,
+                B.MN_MAJOR if am == "mn" else B.K_MAJOR, B.MN_MAJOR if bm == "mn" else B.K_MAJOR, 0, 0)
+        B.mxfp8_gemm(*args, d32)
+        B.mxfp8_gemm(*args, dbf)
+        assert B.mxfp8_device_status() == 0
+        assert torch.equal(d32.to(torch.bfloat16), dbf), name
+        aq, a_s = q[ka]
+        if am == "k":
+            a_sub, as_sub = aq[rows], a_s[rows]
+        else:
+            a_sub, as_sub = np.ascontiguousarray(aq[:, rows]), np.ascontiguousarray(a_s[:, rows])
+        d64, sabs = orc.gemm_f64(a_sub, as_sub, q[kb][0], q[kb][1], am, bm)
+        got = d32[torch.from_numpy(rows).cuda()].cpu().numpy()
+        check_gemm_tolerance(got, d64, sabs, name)
