@@ -86,10 +86,74 @@ dequantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, 
     }
 }
 
+// Fast path (cols % 128 == 0): a warp step covers 128 consecutive elements of one row; lane l owns
+// elements 4l..4l+3, so the loads (4 bytes per lane) and the stores (16 bytes FP32 / 8 bytes BF16
+// per lane) of a warp are contiguous.  Each warp takes UNROLL consecutive steps with all its loads
+// issued before the first use.
+template <int ELEM, int DST, int ORIENT>
+__global__ void __launch_bounds__(256)
+dequantize_vec_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, int64_t rows, int64_t cols,
+                      int sf_layout, void* __restrict__ dst_v, int64_t groups)
+{
+    constexpr int UNROLL = 8;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t g0 = warp * UNROLL;
+    if (g0 >= groups) return;
+    const int64_t groups_per_row = cols >> 7;
+    uint32_t w[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u)
+        w[u] = (g0 + u < groups) ? __ldcs(reinterpret_cast<const uint32_t*>(q) + (g0 + u) * 32 + lane) : 0u;
+    int64_t r = g0 / groups_per_row;                       // one division per warp, then step
+    int64_t cg = g0 - r * groups_per_row;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u, ++cg) {
+        if (g0 + u >= groups) break;
+        if (cg == groups_per_row) { cg = 0; ++r; }
+        const int64_t c = cg * 128 + lane * 4;
+        float sc[4];
+        if (ORIENT == MXFP8_ROW) {
+            const int64_t ncb = cols >> 5, kb = c >> 5;
+            const float v = scale_value(s[(sf_layout == MXFP8_SF_SWIZZLED) ? sf_swizzled_offset(r, kb, ncb) : r * ncb + kb]);
+            sc[0] = sc[1] = sc[2] = sc[3] = v;
+        } else {
+            const int64_t nrb = rows >> 5, kb = r >> 5;
+            if (sf_layout == MXFP8_SF_SWIZZLED) {
+                const uint8_t* base = s + sf_swizzled_offset(c, kb, nrb);   // columns c..c+3 share the atom: 16 bytes apart
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sc[i] = scale_value(base[i * 16]);
+            } else {
+                const uint32_t four = *reinterpret_cast<const uint32_t*>(s + kb * cols + c);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sc[i] = scale_value((four >> (8 * i)) & 0xFFu);
+            }
+        }
+        const float2 lo = fp8x2_to_float2<ELEM>(w[u] & 0xFFFFu), hi = fp8x2_to_float2<ELEM>(w[u] >> 16);
+        const float o0 = lo.x * sc[0], o1 = lo.y * sc[1], o2 = hi.x * sc[2], o3 = hi.y * sc[3];
+        if (DST == MXFP8_FP32) {
+            __stcs(reinterpret_cast<float4*>(static_cast<float*>(dst_v) + r * cols + c), make_float4(o0, o1, o2, o3));
+        } else {
+            const __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b2 = __floats2bfloat162_rn(o2, o3);
+            __stcs(reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(dst_v) + r * cols + c),
+                   make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b2)));
+        }
+    }
+}
+
 template <int ELEM, int DST, int ORIENT>
 cudaError_t launch(const uint8_t* q, const uint8_t* s, int64_t rows, int64_t cols, int sf_layout,
                    void* dst, cudaStream_t stream)
 {
+    if ((cols & 127) == 0) {
+        const int64_t groups = rows * (cols / 128);            // warp steps of 128 elements
+        const int64_t warps = (groups + 7) / 8;
+        const int64_t blocks = (warps + 7) / 8;                // 8 warps per block
+        if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+        dequantize_vec_kernel<ELEM, DST, ORIENT><<<(unsigned)blocks, 256, 0, stream>>>(q, s, rows, cols, sf_layout, dst, groups);
+        count_launch(1);
+        return cudaGetLastError();
+    }
     const int64_t chunks = (cols + 15) / 16;
     const int64_t blocks = (rows * chunks + 255) / 256;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;

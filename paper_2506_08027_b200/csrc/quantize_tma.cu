@@ -74,15 +74,6 @@ __device__ __forceinline__ uint32_t hmax2(uint32_t a, uint32_t b)
     const __nv_bfloat162 m = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
     return *reinterpret_cast<const uint32_t*>(&m);
 }
-// |bf16| halves that are +Inf or NaN become 0 (finite-only maximum, rare path)
-__device__ __forceinline__ uint32_t finite_abs2(uint32_t w)
-{
-    uint32_t a = w & 0x7FFF7FFFu;
-    if ((a & 0x0000FFFFu) >= 0x00007F80u) a &= 0xFFFF0000u;
-    if ((a & 0xFFFF0000u) >= 0x7F800000u) a &= 0x0000FFFFu;
-    return a;
-}
-
 // flags a packed pair of bf16 magnitudes if either half is Inf or NaN
 __device__ __forceinline__ uint32_t nonfinite2(uint32_t z) { return (z + 0x00800080u) & 0x80008000u; }
 
