@@ -116,10 +116,12 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// arrive on a barrier addressed in the cluster's shared window (possibly the peer CTA's)
+// arrive on a barrier addressed in the cluster's shared window (possibly the peer CTA's).  Default
+// semantics (release at CTA scope): a cluster-scope release costs a memory fence of about a
+// microsecond per tile, and nothing but the tcgen05-fenced TMEM hand-off is ordered by this barrier.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // cluster-window address of the same shared-memory offset in CTA `rank` of this cluster
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
