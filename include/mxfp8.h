@@ -126,8 +126,11 @@ typedef struct {
  *   epi                NULL, or the fused MXFP8 output described above.
  *   workspace          device scratch of at least mxfp8_gemm_workspace_bytes(); may be NULL
  *                      when that is 0.  Contents are undefined afterwards.
- * Requirements: K % 128 == 0, M % 128 == 0, N % 128 == 0 (else ERR_UNSUPPORTED); K % 32 != 0
- * is ERR_SHAPE; all pointers 16-byte aligned (operands 128-byte aligned when MN-major).
+ * Requirements: K % 32 == 0 (else ERR_SHAPE).  Ragged M, N and K (not multiples of the tile) are
+ * handled by the hardware's out-of-bounds fill and clipping; what remains are the 16-byte row
+ * pitches TMA needs: M % 16 == 0 for an MN-major A, N % 16 == 0 for an MN-major B, N % 8 == 0 for
+ * BF16 output, N % 4 == 0 for FP32 output; with `epi`, M % 128 == 0 and N % 128 == 0
+ * (ERR_UNSUPPORTED otherwise).  All pointers 16-byte aligned.
  * A bounded wait that expires inside the kernel sets the device status word; read it with
  * mxfp8_device_status().  The result is deterministic (same inputs, same bytes).
  */

@@ -23,6 +23,7 @@
 //   Every mbarrier wait is bounded: on expiry the kernel records MXFP8_ERR_DEVICE_TIMEOUT in
 //   the device status word, raises an abort flag that all roles poll, drains and exits.
 #include <cuda.h>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -646,13 +647,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
             const int row0 = (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
+            const bool rows_inside = row0 < (int)p.M;        // ragged last M tile: a 32-row box entirely outside stores nothing
             if constexpr (CW % 64 == 0) {
-                if (p.epi_orient) {
+                if (p.epi_orient && rows_inside) {
                     if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
                     else epi_mx<CW, MXFP8_E5M2>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
                 }
             }
-            if (!p.store_d) {
+            if (!p.store_d || !rows_inside) {
             } else if (p.out_dtype == MXFP8_BF16) {
 #pragma unroll
                 for (int ch = 0; ch < CW / 32; ++ch) {          // 32 columns = 64 bytes per row
@@ -812,11 +814,11 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     auto kernel = gemm_kernel<BN, PAIR>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
         return MXFP8_ERR_CUDA;
-    p.tiles_m = (int)(p.M / (PAIR ? 2 * BM : BM));
+    p.tiles_m = (int)((p.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM));
     p.tiles_n = (int)((p.N + BN - 1) / BN);
     p.stage_tx = (PAIR ? 2u : 1u) * (uint32_t)(C::A_BYTES + (p.b_mn ? C::B_BYTES_MN : C::B_BYTES_K) + 512 + 512 * C::SFB_ATOMS);
     p.num_tiles = p.tiles_m * p.tiles_n;
-    p.num_kb = (int)(p.K / BK);
+    p.num_kb = (int)((p.K + BK - 1) / BK);   // a ragged K tail is zero-filled by TMA (operands) and by the scale pads
     p.group_m = 16;
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
@@ -835,6 +837,9 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, p);
+    if (getenv("MXFP8_LOG"))
+        fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d -> %s\n", cfg.gridDim.x, GEMM_THREADS,
+                C::SMEM_TOTAL, p.tiles_m, p.tiles_n, p.num_kb, cudaGetErrorString(err));
     count_launch(1);
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
@@ -869,7 +874,11 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
         if ((epi->orientation & MXFP8_COL) && (!aligned16(epi->q_col) || !aligned16(epi->s_col))) return MXFP8_ERR_ALIGN;
     }
     if (M <= 0 || N <= 0 || K <= 0 || (K % 32)) return MXFP8_ERR_SHAPE;
-    if ((M % 128) || (N % 128) || (K % 128)) return MXFP8_ERR_UNSUPPORTED;
+    // TMA needs 16-byte row pitches: MN-major operands and the output constrain M and N
+    if (a_major == MXFP8_MN_MAJOR && (M % 16)) return MXFP8_ERR_UNSUPPORTED;
+    if (b_major == MXFP8_MN_MAJOR && (N % 16)) return MXFP8_ERR_UNSUPPORTED;
+    if (D && (N % (out_dtype == MXFP8_FP32 ? 4 : 8))) return MXFP8_ERR_UNSUPPORTED;
+    if (epi && ((M % 128) || (N % 128))) return MXFP8_ERR_UNSUPPORTED;   // the fused output writes whole scale atoms
     if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
     if (!aligned16(Aq) || !aligned16(As) || !aligned16(Bq) || !aligned16(Bs) || (D && !aligned16(D))) return MXFP8_ERR_ALIGN;
 
@@ -894,12 +903,12 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     for (int pass = force ? 0 : 1; pass < 2 && best_cost >= 1e300; ++pass)
     for (int bn : {256, 192, 128}) {
         for (int pr = 1; pr >= 0; --pr) {
-            if (pr && ((M % 256) || bn == 128)) continue;
+            if (pr && (M <= 128 || bn == 128)) continue;
             if (epi && bn == 192) continue;   // the fused output works on 64-column chunks per epilogue warp
             if (pass == 0) {   // forced shape, when it applies to this problem
                 if (atoi(force) != bn || (strchr(force, 'p') != nullptr) != (pr != 0)) continue;
             }
-            const int64_t tiles = (M / (pr ? 256 : 128)) * ((N + bn - 1) / bn);
+            const int64_t tiles = ((M + (pr ? 255 : 127)) / (pr ? 256 : 128)) * ((N + bn - 1) / bn);
             const int64_t workers = pr ? sms / 2 : sms;
             const int64_t waves = (tiles + workers - 1) / workers;
             // cycles per 128-deep K block measured on B200 for each shape (TMA feed and MMA issue
@@ -917,16 +926,20 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
                                               : make_tmap(&m.a, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
     const bool okb = b_major == MXFP8_K_MAJOR ? make_tmap(&m.b, Bq, (uint64_t)K, (uint64_t)N, 128, b_box_rows)
                                               : make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)K, 128, 128);
-    const bool oks = make_tmap_sf(&m.sfa, As, (uint64_t)(M / 128), (uint64_t)(K / 128)) &&
-                     make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(K / 128));
+    const bool oks = make_tmap_sf(&m.sfa, As, (uint64_t)((M + 127) / 128), (uint64_t)((K + 127) / 128)) &&
+                     make_tmap_sf(&m.sfb, Bs, (uint64_t)((N + 127) / 128), (uint64_t)((K + 127) / 128));
     // maps that a launch does not use still have to be valid: point them at any output that exists
     void* q_any = epi ? ((epi->orientation & MXFP8_ROW) ? epi->q_row : epi->q_col) : D;
     void* q_row = (epi && (epi->orientation & MXFP8_ROW)) ? epi->q_row : q_any;
     void* q_col = (epi && (epi->orientation & MXFP8_COL)) ? epi->q_col : q_any;
     const bool okd = D ? make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype) : make_tmap_q(&m.d, q_any, (uint64_t)M, (uint64_t)N);
-    if (!oka || !okb || !oks || !okd || !make_tmap_q(&m.qrow, q_row, (uint64_t)M, (uint64_t)N) ||
-        !make_tmap_q(&m.qcol, q_col, (uint64_t)M, (uint64_t)N))
-        return MXFP8_ERR_CUDA;
+    bool okq = true;
+    if (epi) okq = make_tmap_q(&m.qrow, q_row, (uint64_t)M, (uint64_t)N) && make_tmap_q(&m.qcol, q_col, (uint64_t)M, (uint64_t)N);
+    else if (okd) { m.qrow = m.d; m.qcol = m.d; }   // never dereferenced without an epilogue, but must be valid maps
+    if (getenv("MXFP8_LOG"))
+        fprintf(stderr, "mxfp8_gemm M=%lld N=%lld K=%lld tile=%d%s maps: a=%d b=%d sf=%d d=%d q=%d\n", (long long)M, (long long)N,
+                (long long)K, best_bn, best_pair ? "p" : "", (int)oka, (int)okb, (int)oks, (int)okd, (int)okq);
+    if (!oka || !okb || !oks || !okd || !okq) return MXFP8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (best_pair) return best_bn == 256 ? launch_gemm<256, true>(m, p, st) : launch_gemm<192, true>(m, p, st);
     if (best_bn == 256) return launch_gemm<256, false>(m, p, st);

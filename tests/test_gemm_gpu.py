@@ -292,3 +292,38 @@ def test_bench_step_shapes_sampled_rows():
         d64, sabs = orc.gemm_f64(a_sub, as_sub, q[kb][0], q[kb][1], am, bm)
         got = d32[torch.from_numpy(rows).cuda()].cpu().numpy()
         check_gemm_tolerance(got, d64, sabs, name)
+
+
+@pytest.mark.parametrize("shape", [(200, 136, 160), (72, 264, 96), (1, 8, 32), (257, 520, 416), (384, 200, 2080), (130, 256, 128)])
+@pytest.mark.parametrize("majors", [("k", "k"), ("k", "mn"), ("mn", "mn")])
+def test_ragged_shapes(shape, majors):
+    # M, N, K that are not multiples of the tile: out-of-range rows / columns / K are zero-filled on load
+    # and clipped on store; the scale buffers are padded to whole atoms (pad bytes 0) as mxfp8_quantize writes them
+    m, n, k = shape
+    if majors[0] == "mn" and m % 16:
+        pytest.skip("MN-major A needs M % 16 == 0")
+    if majors[1] == "mn" and n % 16:
+        pytest.skip("MN-major B needs N % 16 == 0")
+    rng = np.random.default_rng(m * 7 + n * 3 + k)
+    ai, aq = int_operand(rng, m, k)
+    bi, bq = int_operand(rng, n, k)
+    # unit scales: integer products, exact in FP32 for any accumulation order
+    a_s = np.full((m, k // 32), 127, np.uint8)
+    b_s = np.full((n, k // 32), 127, np.uint8)
+    A, SA = stored(aq, a_s, majors[0])
+    B_, SB = stored(bq, b_s, majors[1])
+    got = gpu_gemm(A, SA, B_, SB, majors[0], majors[1])
+    want = (ai @ bi.T).astype(np.float64)
+    assert np.array_equal(got.astype(np.float64), want), "max |diff| = %g" % np.abs(got - want).max()
+    # random scales: tolerance against the FP64 oracle
+    a_s = rng.integers(110, 140, (m, k // 32)).astype(np.uint8)
+    b_s = rng.integers(110, 140, (n, k // 32)).astype(np.uint8)
+    A, SA = stored(aq, a_s, majors[0])
+    B_, SB = stored(bq, b_s, majors[1])
+    d64, sabs = orc.gemm_f64(A, SA, B_, SB, majors[0], majors[1])
+    got = gpu_gemm(A, SA, B_, SB, majors[0], majors[1])
+    check_gemm_tolerance(got, d64, sabs, str(shape))
+    if n % 8 == 0:
+        gotb = gpu_gemm(A, SA, B_, SB, majors[0], majors[1], out="bf16")
+        import torch
+        assert np.array_equal(gotb, torch.from_numpy(got).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))

@@ -67,5 +67,6 @@ def test_argument_validation_happens_on_the_host():
     assert g(None, p, p, p, 128, 128, 128, 0, 0, 0, 0, p, 0, None, None, 0, None) == -1
     assert g(p, p, p, p, 128, 128, 100, 0, 0, 0, 0, p, 0, None, None, 0, None) == -3
     assert g(p, p, p, p, 128, 128, 128, 3, 0, 0, 0, p, 0, None, None, 0, None) == -2
-    assert g(p, p, p, p, 100, 128, 128, 0, 0, 0, 0, p, 0, None, None, 0, None) == -5
+    assert g(p, p, p, p, 100, 128, 128, 1, 0, 0, 0, p, 0, None, None, 0, None) == -5   # MN-major A needs M % 16 == 0
+    assert g(p, p, p, p, 128, 130, 128, 0, 0, 0, 0, p, 1, None, None, 0, None) == -5   # BF16 output needs N % 8 == 0
     assert "timeout" in B.status_string(-7) or "wait" in B.status_string(-7)
