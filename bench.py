@@ -387,6 +387,106 @@ def run_case(args):
     print(json.dumps({"case": args.case, "launches": int(B.mxfp8_launch_count()), "device_status": B.mxfp8_device_status()}))
 
 
+def _time_calls(fn, n_bufs, min_iters=10, min_ms=30.0):
+    """Average device time of fn(i) in ms (CUDA events), i cycling through n_bufs rotated buffers."""
+    import torch
+    for i in range(3):
+        fn(i % n_bufs)
+    torch.cuda.synchronize()
+    iters = min_iters
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i % n_bufs)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if ms >= min_ms or iters >= 2000:
+            return ms / iters
+        iters *= 4
+
+
+def run_sweep(args):
+    """Tables for the cast sweep (sizes x shapes x dtypes x orientations) and the GEMM shape sweep
+    (square sizes, the skinny wgrad, the 8B decoder-block GEMMs, with and without the fused MXFP8
+    output).  Prints markdown; not part of the one-line contract."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from paper_2506_08027_b200 import synth
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    P, S = B.RULE_PAPER, B.SF_SWIZZLED
+    if args.sweep == "cast":
+        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy |")
+        print("|---|---|---|---|---|---|---|---|---|")
+        for dtype, esz in (("bf16", 2), ("fp32", 4)):
+            for nbytes in (1 << 20, 16 << 20, 256 << 20, 1 << 30, 4 << 30):
+                for cols in (4096, 14336, 8288):
+                    if nbytes >= (1 << 30) and cols != 4096 and dtype == "fp32":
+                        continue
+                    rows = max(32, (nbytes // (cols * esz)) // 32 * 32)
+                    kind = "gradient_like" if cols == 14336 else ("student_t" if cols == 8288 else "gaussian")
+                    n_bufs = max(1, min(4, int((768 << 20) // (rows * cols * esz)) + 1)) if nbytes < (1 << 30) else 1
+                    srcs = [synth.device_tensor(kind, (rows, cols), 7 + i, dtype) for i in range(n_bufs)]
+                    for orient, oname in ((B.ROW, "row"), (B.COL, "col"), (B.BOTH, "both")):
+                        for elem in ((B.E4M3, B.E5M2) if (orient == B.BOTH and cols == 4096) else (B.E4M3,)):
+                            outs = B.alloc_quantize_outputs(rows, cols, orient, S)
+                            ms = _time_calls(lambda i: B.mxfp8_quantize(srcs[i], orient, P, elem, *outs, S), n_bufs)
+                            by = rows * cols * (esz + (2 if orient == B.BOTH else 1) * (1 + 1 / 32))
+                            gbs = by / ms / 1e6
+                            print("| %s | %d MB | %d x %d | %s | %s | %s | %.1f | %.0f | %.2f |" % (
+                                dtype, nbytes >> 20, rows, cols, kind, oname, "e4m3" if elem == B.E4M3 else "e5m2",
+                                ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+                            del outs
+                    del srcs
+                    torch.cuda.empty_cache()
+        return
+    shapes = [("square", n, n, n, 0, 0) for n in (1024, 2048, 4096, 8192, 16384)]
+    shapes.append(("skinny wgrad", 4096, 4096, 65536, 1, 1))
+    Tk = 16384
+    for name, fin, fout in (("qkv", 4096, 6144), ("o", 4096, 4096), ("ffn_up", 4096, 28672), ("ffn_down", 14336, 4096)):
+        shapes.append((name + " fprop", Tk, fout, fin, 0, 0))
+        shapes.append((name + " dgrad", Tk, fin, fout, 0, 1))
+        shapes.append((name + " wgrad", fout, fin, Tk, 1, 1))
+    print("| case | M | N | K | majors | out | fused MX out | us | TFLOP/s | of 2x measured BF16 |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
+    fp8_peak = 2.0 * peaks["bf16_tflops"]
+    for name, M, N, K, am, bm in shapes:
+        def operand(mn, k, major, seed):
+            if major == 0:
+                x = synth.device_tensor("gaussian", (mn, k), seed)
+                o = B.alloc_quantize_outputs(mn, k, B.ROW, S)
+                B.mxfp8_quantize(x, B.ROW, P, B.E4M3, *o, S)
+                return o[0], o[1]
+            x = synth.device_tensor("gaussian", (k, mn), seed)
+            o = B.alloc_quantize_outputs(k, mn, B.COL, S)
+            B.mxfp8_quantize(x, B.COL, P, B.E4M3, *o, S)
+            return o[2], o[3]
+        Aq, As = operand(M, K, am, 11)
+        Bq, Bs = operand(N, K, bm, 12)
+        for out_dt, oname in ((torch.bfloat16, "bf16"), (torch.float32, "fp32")):
+            for epi_o in (0, B.ROW, B.BOTH):
+                if epi_o and out_dt == torch.float32:
+                    continue
+                if epi_o == B.BOTH and name == "square" and M not in (4096, 8192):
+                    continue
+                D = torch.empty((M, N), dtype=out_dt, device="cuda")
+                epi, keep = None, None
+                if epi_o:
+                    keep = B.alloc_quantize_outputs(M, N, epi_o, S)
+                    epi = B.make_epilogue(epi_o, P, B.E4M3, *keep)
+                ms = _time_calls(lambda i: B.mxfp8_gemm(Aq, As, Bq, Bs, M, N, K, am, bm, B.E4M3, B.E4M3, D, epi=epi), 1, 10, 20.0)
+                tf = 2.0 * M * N * K / ms / 1e9
+                print("| %s | %d | %d | %d | %s%s | %s | %s | %.1f | %.0f | %.2f |" % (
+                    name, M, N, K, "kn"[0] if am == 0 else "m", "k" if bm == 0 else "n", oname,
+                    {0: "-", B.ROW: "row", B.BOTH: "row+col"}[epi_o], ms * 1e3, tf, tf / fp8_peak), flush=True)
+                del D, keep, epi
+        del Aq, As, Bq, Bs
+        torch.cuda.empty_cache()
+    assert B.mxfp8_device_status() == 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -397,8 +497,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "gemm", "gemm8k"],
                     help="run one kernel on one small case and exit (for profiler captures)")
+    ap.add_argument("--sweep", default=None, choices=["cast", "gemm"],
+                    help="print the cast-bandwidth or GEMM-shape sweep as a markdown table and exit")
     args = ap.parse_args()
-    if args.case:
+    if args.sweep:
+        run_sweep(args)
+    elif args.case:
         run_case(args)
     elif args.impl == "reference":
         run_reference(args)
