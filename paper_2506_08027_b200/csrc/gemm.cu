@@ -387,6 +387,42 @@ __device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams
     if (p.epi_orient & MXFP8_COL) {
         const int64_t nkb = p.M >> 5;
         const int64_t kb = row0 >> 5;
+        // Column c of this warp's CW columns is "owned" by lane c % 32 (slot c / 32): one warp-wide integer
+        // max per column (|x| bit patterns of finite floats order like integers), the owner keeps the
+        // result, computes scale and 1/X for its CW/32 columns, stores their scale bytes, and hands 1/X
+        // out again by shuffle when the column is cast.
+        uint32_t own[CW / 32];
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+            uint32_t amax;
+            asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(v[c] & 0x7FFFFFFFu));
+            if ((c & 31) == 0) own[c >> 5] = amax;                 // every lane takes it, then the owner's survives
+            else if (lane == (c & 31)) own[c >> 5] = amax;
+        }
+        bool special = false;
+#pragma unroll
+        for (int j = 0; j < CW / 32; ++j) special |= own[j] >= 0x7F800000u;     // an Inf or NaN reached an amax
+        if (__any_sync(0xFFFFFFFFu, special)) {
+            // rare: redo the maxima without the non-finite elements
+#pragma unroll 1
+            for (int c = 0; c < CW; ++c) {
+                uint32_t a = v[c] & 0x7FFFFFFFu, amax;
+                a = (a >= 0x7F800000u) ? 0u : a;
+                asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
+                if (lane == (c & 31)) {
+#pragma unroll
+                    for (int j = 0; j < CW / 32; ++j)
+                        if (j == (c >> 5)) own[j] = amax;
+                }
+            }
+        }
+        float own_inv[CW / 32];
+#pragma unroll
+        for (int j = 0; j < CW / 32; ++j) {
+            const uint32_t ie = epi_inv_exp<ELEM>(own[j], rule_offset);
+            own_inv[j] = __uint_as_float(ie << 23);
+            p.epi_s_col[sf_swizzled_offset(col0 + j * 32 + lane, kb, nkb)] = (uint8_t)(254u - ie);
+        }
 #pragma unroll
         for (int ch = 0; ch < CW / 64; ++ch) {
             uint32_t w[16];
@@ -396,13 +432,7 @@ __device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int c = ch * 64 + i * 4 + e;
-                    uint32_t a = v[c] & 0x7FFFFFFFu;
-                    a = (a >= 0x7F800000u) ? 0u : a;           // Inf / NaN stay out of amax
-                    uint32_t amax;
-                    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
-                    const uint32_t ie = epi_inv_exp<ELEM>(amax, rule_offset);
-                    y[e] = __uint_as_float(v[c]) * __uint_as_float(ie << 23);
-                    if (lane == (c & 31)) p.epi_s_col[sf_swizzled_offset(col0 + c, kb, nkb)] = (uint8_t)(254u - ie);
+                    y[e] = __uint_as_float(v[c]) * __shfl_sync(0xFFFFFFFFu, own_inv[c >> 5], c & 31);
                 }
                 w[i] = cvt_fp8x4<ELEM>(y[0], y[1], y[2], y[3]);
             }
