@@ -354,7 +354,8 @@ def run_case(args):
     """One kernel on one small case, a few launches, nothing else: the target of ncu captures.
     quantize: BF16 8192x8192 in both orientations; gemm: the 8192x8192x2048 fprop product
     (gemm8k: 8192^3);
-    dequantize: 8192x8192 row-blocked bytes to BF16."""
+    dequantize: 8192x8192 row-blocked bytes to BF16; fake_quantize: the BF16 8192x8192 round trip,
+    row blocks."""
     import torch
     from paper_2506_08027_b200 import binding as B
     from paper_2506_08027_b200 import synth
@@ -367,6 +368,10 @@ def run_case(args):
     if args.case == "quantize":
         for _ in range(reps):
             B.mxfp8_quantize(x, B.BOTH, P, E, *q, S)
+    elif args.case == "fake_quantize":
+        dst = torch.empty_like(x)
+        for _ in range(reps):
+            B.mxfp8_fake_quantize(x, B.ROW, P, E, dst, None)
     elif args.case == "dequantize":
         B.mxfp8_quantize(x, B.BOTH, P, E, *q, S)
         dst = torch.empty_like(x)
@@ -442,6 +447,22 @@ def run_sweep(args):
                     del srcs
                     torch.cuda.empty_cache()
         return
+    if args.sweep == "emu":
+        # the MXFP8 round trip (Sec. 3.1): reads the source once, writes one same-dtype tensor per orientation
+        print("| dtype | rows x cols | orient | us | GB/s | of measured copy |")
+        print("|---|---|---|---|---|---|")
+        for dtype, esz in (("bf16", 2), ("fp32", 4)):
+            for rows, cols in ((2048, 4096), (8192, 8192), (16384, 14336)):
+                src = synth.device_tensor("gaussian", (rows, cols), 11, dtype)
+                dr, dc = torch.empty_like(src), torch.empty_like(src)
+                for orient, oname in ((B.ROW, "row"), (B.COL, "col"), (B.BOTH, "both")):
+                    ms = _time_calls(lambda i: B.mxfp8_fake_quantize(src, orient, P, B.E4M3, dr if orient & B.ROW else None,
+                                                                       dc if orient & B.COL else None), 1)
+                    gbs = rows * cols * esz * (3 if orient == B.BOTH else 2) / ms / 1e6
+                    print("| %s | %d x %d | %s | %.1f | %.0f | %.2f |" % (dtype, rows, cols, oname, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+                del src, dr, dc
+                torch.cuda.empty_cache()
+        return
     shapes = [("square", n, n, n, 0, 0) for n in (1024, 2048, 4096, 8192, 16384)]
     shapes.append(("skinny wgrad", 4096, 4096, 65536, 1, 1))
     Tk = 16384
@@ -495,10 +516,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "gemm", "gemm8k"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k"],
                     help="run one kernel on one small case and exit (for profiler captures)")
-    ap.add_argument("--sweep", default=None, choices=["cast", "gemm"],
-                    help="print the cast-bandwidth or GEMM-shape sweep as a markdown table and exit")
+    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu"],
+                    help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)

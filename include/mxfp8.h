@@ -96,6 +96,18 @@ int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int64_t cols,
                      void* dst, int dst_dtype, void* stream);
 
 /*
+ * mxfp8_fake_quantize -- the MXFP8 round trip in one pass: dst = decode(quantize(src)) in the source's
+ * own dtype (BF16 -> MXFP8 -> BF16 is how the paper's accuracy runs emulated MX arithmetic ahead of
+ * BF16 GEMMs, Sec. 3.1).  Same block / scale / cast rules and the same special-value handling as
+ * mxfp8_quantize; the result equals mxfp8_dequantize(mxfp8_quantize(src)) bit for bit.
+ *   dst_row / dst_col  [rows, cols] of src_dtype, one per requested orientation, 16-byte aligned.
+ *   Needs cols % 16 == 0 (ERR_UNSUPPORTED otherwise) besides the rules of mxfp8_quantize.
+ */
+int mxfp8_fake_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                        int orientation, int scale_rule, int elem,
+                        void* dst_row, void* dst_col, void* stream);
+
+/*
  * Optional fused epilogue of mxfp8_gemm: the FP32 accumulator tile is converted to MXFP8
  * exactly as mxfp8_quantize would convert the FP32 output D[M, N] (Sec. 2: the FP32 output is
  * quantized to MX format when its consumer needs it).  ROW blocks run along N, COL blocks
@@ -176,6 +188,23 @@ int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64
                         void* q_row_host, void* s_row_host, void* q_col_host, void* s_col_host,
                         int sf_layout, void* dev_ws, size_t dev_ws_bytes, void* stream);
 
+
+/*
+ * mxfp8_linear -- one training step of a linear layer Y = X * W^T through the MXFP8 path on
+ * DEVICE buffers (Sec. 3.2, the FPROP / DGRAD / WGRAD workflow): X [T, H], W [F, H], dY [T, F]
+ * in BF16 are each converted once to MXFP8-E4M3 in BOTH orientations under `scale_rule`, then
+ *     FPROP  Y  [T, F] = X  * W^T   (row-blocked X,  row-blocked W)
+ *     DGRAD  dX [T, H] = dY * W     (row-blocked dY, column-blocked W)
+ *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
+ * run as block-scaled GEMMs with BF16 output: six kernel launches on `stream`, no wait.
+ * T, H, F must be multiples of 128 (ERR_UNSUPPORTED).  ws: device scratch for the quantized
+ * copies, mxfp8_linear_ws_bytes() bytes, 256-byte aligned, owned by the caller.  All tensors
+ * 16-byte aligned, row-major, dense.
+ */
+size_t mxfp8_linear_ws_bytes(int64_t T, int64_t H, int64_t F);
+int mxfp8_linear(const void* x, const void* w, const void* dy,
+                 int64_t T, int64_t H, int64_t F, int scale_rule,
+                 void* y, void* dx, void* dw, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * mxfp8_linear_host -- one training step of a linear layer Y = X * W^T through the MXFP8 path

@@ -24,7 +24,7 @@ EXPORTS = (
     "mxfp8_quantize", "mxfp8_dequantize", "mxfp8_gemm", "mxfp8_scale_bytes", "mxfp8_sf_offset",
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
-    "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host",
+    "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes", "mxfp8_linear",
 )
 
 
@@ -76,6 +76,12 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host_ws_bytes.argtypes = [i, i64, i64, i]
         L.mxfp8_quantize_host.restype = i
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
+        L.mxfp8_fake_quantize.restype = i
+        L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_linear_ws_bytes.restype = sz
+        L.mxfp8_linear_ws_bytes.argtypes = [i64, i64, i64]
+        L.mxfp8_linear.restype = i
+        L.mxfp8_linear.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
         L.mxfp8_linear_host_ws_bytes.restype = sz
         L.mxfp8_linear_host_ws_bytes.argtypes = [i64, i64, i64]
         L.mxfp8_linear_host.restype = i
@@ -206,3 +212,21 @@ def mxfp8_linear_host(x_host, w_host, dy_host, scale_rule: int, y_host, dx_host,
                                    _ptr(y_host), _ptr(dx_host), _ptr(dw_host), _ptr(dev_ws),
                                    dev_ws.numel() * dev_ws.element_size(), _stream(stream)),
            "mxfp8_linear_host")
+
+
+def mxfp8_fake_quantize(src: torch.Tensor, orientation: int, scale_rule: int, elem: int,
+                        dst_row, dst_col, stream=None) -> None:
+    rows, cols = src.shape
+    _check(lib().mxfp8_fake_quantize(_ptr(src), _dtype_code(src), rows, cols, orientation, scale_rule, elem,
+                                     _ptr(dst_row), _ptr(dst_col), _stream(stream)), "mxfp8_fake_quantize")
+
+
+def mxfp8_linear_ws_bytes(T: int, H: int, F: int) -> int:
+    return int(lib().mxfp8_linear_ws_bytes(T, H, F))
+
+
+def mxfp8_linear(x, w, dy, scale_rule: int, y, dx, dw, ws, stream=None) -> None:
+    T, H = x.shape
+    F = w.shape[0]
+    _check(lib().mxfp8_linear(_ptr(x), _ptr(w), _ptr(dy), T, H, F, scale_rule, _ptr(y), _ptr(dx), _ptr(dw),
+                              _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "mxfp8_linear")

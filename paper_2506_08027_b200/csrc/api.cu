@@ -99,14 +99,16 @@ extern "C" int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t 
 
 namespace {
 struct LinearWs {
-    char* src[3];      // X, W, dY (bf16)
+    char* src[3];      // X, W, dY (bf16); host variant only
     char* q[3][2];     // row / col quantized copies
     char* s[3][2];     // row / col scales (swizzled)
-    char* out[3];      // Y, dX, dW (bf16)
+    char* out[3];      // Y, dX, dW (bf16); host variant only
     size_t total;
 };
 
-LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F)
+// Carves the scratch of one linear-layer step out of `base` (null: sizes only).  `staging` adds
+// device copies of the three inputs and the three outputs for the host-buffer variant.
+LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F, bool staging)
 {
     const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
     const int64_t outs[3][2] = {{T, F}, {T, H}, {F, H}};
@@ -114,22 +116,71 @@ LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F)
     size_t off = 0;
     auto take = [&](size_t n) { char* p = base ? base + off : nullptr; off += up256(n); return p; };
     for (int t = 0; t < 3; ++t) {
-        w.src[t] = take((size_t)shp[t][0] * shp[t][1] * 2);
+        if (staging) w.src[t] = take((size_t)shp[t][0] * shp[t][1] * 2);
         for (int o = 0; o < 2; ++o) {
             w.q[t][o] = take((size_t)shp[t][0] * shp[t][1]);
             w.s[t][o] = take(mxfp8_scale_bytes(shp[t][0], shp[t][1], o + 1, MXFP8_SF_SWIZZLED));
         }
     }
-    for (int t = 0; t < 3; ++t) w.out[t] = take((size_t)outs[t][0] * outs[t][1] * 2);
+    if (staging)
+        for (int t = 0; t < 3; ++t) w.out[t] = take((size_t)outs[t][0] * outs[t][1] * 2);
     w.total = off;
     return w;
 }
+
+// The six launches of one step on device buffers: three BOTH-orientation conversions, then
+// FPROP, DGRAD and WGRAD (Sec. 3.2).
+int linear_device(const LinearWs& w, const void* x, const void* wt, const void* dy, int64_t T, int64_t H, int64_t F,
+                  int scale_rule, void* y, void* dx, void* dw, void* stream)
+{
+    const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
+    const void* src[3] = {x, wt, dy};
+    for (int t = 0; t < 3; ++t) {
+        const int rc = mxfp8_quantize(src[t], MXFP8_BF16, shp[t][0], shp[t][1], MXFP8_BOTH, scale_rule, MXFP8_E4M3,
+                                      w.q[t][0], w.s[t][0], w.q[t][1], w.s[t][1], MXFP8_SF_SWIZZLED, stream);
+        if (rc != MXFP8_OK) return rc;
+    }
+    enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
+    int rc = mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR,
+                        MXFP8_E4M3, MXFP8_E4M3, y, MXFP8_BF16, nullptr, nullptr, 0, stream);
+    if (rc != MXFP8_OK) return rc;
+    rc = mxfp8_gemm(w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR,
+                    MXFP8_E4M3, MXFP8_E4M3, dx, MXFP8_BF16, nullptr, nullptr, 0, stream);
+    if (rc != MXFP8_OK) return rc;
+    return mxfp8_gemm(w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR,
+                      MXFP8_E4M3, MXFP8_E4M3, dw, MXFP8_BF16, nullptr, nullptr, 0, stream);
+}
+
+int linear_check(int64_t T, int64_t H, int64_t F, int scale_rule)
+{
+    if (T <= 0 || H <= 0 || F <= 0) return MXFP8_ERR_SHAPE;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if ((T % 128) || (H % 128) || (F % 128)) return MXFP8_ERR_UNSUPPORTED;
+    return MXFP8_OK;
+}
 }  // namespace
+
+extern "C" size_t mxfp8_linear_ws_bytes(int64_t T, int64_t H, int64_t F)
+{
+    if (T <= 0 || H <= 0 || F <= 0) return 0;
+    return plan_linear(nullptr, T, H, F, false).total;
+}
+
+extern "C" int mxfp8_linear(const void* x, const void* w, const void* dy,
+                            int64_t T, int64_t H, int64_t F, int scale_rule,
+                            void* y, void* dx, void* dw, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!x || !w || !dy || !y || !dx || !dw || !ws) return MXFP8_ERR_NULL;
+    if (const int rc = linear_check(T, H, F, scale_rule)) return rc;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
+    if (ws_bytes < mxfp8_linear_ws_bytes(T, H, F)) return MXFP8_ERR_WORKSPACE;
+    return linear_device(plan_linear(static_cast<char*>(ws), T, H, F, false), x, w, dy, T, H, F, scale_rule, y, dx, dw, stream);
+}
 
 extern "C" size_t mxfp8_linear_host_ws_bytes(int64_t T, int64_t H, int64_t F)
 {
     if (T <= 0 || H <= 0 || F <= 0) return 0;
-    return plan_linear(nullptr, T, H, F).total;
+    return plan_linear(nullptr, T, H, F, true).total;
 }
 
 extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const void* dy_host,
@@ -138,30 +189,17 @@ extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const v
                                  void* dev_ws, size_t dev_ws_bytes, void* stream)
 {
     if (!x_host || !w_host || !dy_host || !y_host || !dx_host || !dw_host || !dev_ws) return MXFP8_ERR_NULL;
-    if (T <= 0 || H <= 0 || F <= 0) return MXFP8_ERR_SHAPE;
-    if ((T % 128) || (H % 128) || (F % 128)) return MXFP8_ERR_UNSUPPORTED;
+    if (const int rc = linear_check(T, H, F, scale_rule)) return rc;
     if ((reinterpret_cast<uintptr_t>(dev_ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
     if (dev_ws_bytes < mxfp8_linear_host_ws_bytes(T, H, F)) return MXFP8_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F);
+    const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F, true);
     const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
     const void* hsrc[3] = {x_host, w_host, dy_host};
-    for (int t = 0; t < 3; ++t) {
+    for (int t = 0; t < 3; ++t)
         if (cudaMemcpyAsync(w.src[t], hsrc[t], (size_t)shp[t][0] * shp[t][1] * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return MXFP8_ERR_CUDA;
-        const int rc = mxfp8_quantize(w.src[t], MXFP8_BF16, shp[t][0], shp[t][1], MXFP8_BOTH, scale_rule, MXFP8_E4M3,
-                                      w.q[t][0], w.s[t][0], w.q[t][1], w.s[t][1], MXFP8_SF_SWIZZLED, stream);
-        if (rc != MXFP8_OK) return rc;
-    }
-    enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
-    int rc = mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR,
-                        MXFP8_E4M3, MXFP8_E4M3, w.out[0], MXFP8_BF16, nullptr, nullptr, 0, stream);
-    if (rc != MXFP8_OK) return rc;
-    rc = mxfp8_gemm(w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR,
-                    MXFP8_E4M3, MXFP8_E4M3, w.out[1], MXFP8_BF16, nullptr, nullptr, 0, stream);
-    if (rc != MXFP8_OK) return rc;
-    rc = mxfp8_gemm(w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR,
-                    MXFP8_E4M3, MXFP8_E4M3, w.out[2], MXFP8_BF16, nullptr, nullptr, 0, stream);
+    const int rc = linear_device(w, w.src[0], w.src[1], w.src[2], T, H, F, scale_rule, w.out[0], w.out[1], w.out[2], stream);
     if (rc != MXFP8_OK) return rc;
     void* hout[3] = {y_host, dx_host, dw_host};
     const int64_t outs[3][2] = {{T, F}, {T, H}, {F, H}};

@@ -24,7 +24,7 @@ int quantize_device(const void* src, int src_dtype, int64_t rows, int64_t cols, 
 bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols);
 int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
                         int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
-                        int sf_layout, cudaStream_t stream);
+                        int sf_layout, cudaStream_t stream, bool emulate = false);
 int quantize_read_and_clear_status();
 
 // Device status word (bounded waits report here); defined in gemm.cu.

@@ -310,3 +310,25 @@ extern "C" int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int6
     return quantize_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
                            q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
 }
+
+extern "C" int mxfp8_fake_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                   int orientation, int scale_rule, int elem,
+                                   void* dst_row, void* dst_col, void* stream)
+{
+    using namespace mxfp8;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!src) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && !dst_row) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && !dst_col) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(src) || ((orientation & MXFP8_ROW) && !aligned16(dst_row)) || ((orientation & MXFP8_COL) && !aligned16(dst_col)))
+        return MXFP8_ERR_ALIGN;
+    if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
+    return quantize_tma_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, dst_row, nullptr, dst_col, nullptr,
+                               MXFP8_SF_SWIZZLED, static_cast<cudaStream_t>(stream), true);
+}

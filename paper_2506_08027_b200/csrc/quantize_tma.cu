@@ -77,10 +77,44 @@ __device__ __forceinline__ uint32_t hmax2(uint32_t a, uint32_t b)
 // flags a packed pair of bf16 magnitudes if either half is Inf or NaN
 __device__ __forceinline__ uint32_t nonfinite2(uint32_t z) { return (z + 0x00800080u) & 0x80008000u; }
 
+// X = 2^(b-127) as FP32 from the exponent field of 1/X (b = 254 - field; b = 0 is the subnormal 2^-127)
+__device__ __forceinline__ float scale_from_inv(float inv)
+{
+    const uint32_t b = 254u - (__float_as_uint(inv) >> 23);
+    return __uint_as_float(b ? (b << 23) : 0x00400000u);
+}
+
+// One lane's VEC elements of one row: cast x * inv to FP8 and store the codes (EMU = false), or store
+// the decoded values code * X in the source's own dtype (EMU = true: the MXFP8 round trip the paper's
+// Hopper runs used, Sec. 3.1).  The decoded product is exact in FP32; BF16 output is one RNE of it.
+template <int ELEM, int VEC, bool EMU>
+__device__ __forceinline__ void emit(uint8_t* dst, const float (&x)[VEC], const float (&inv)[VEC], const float (&xs)[VEC])
+{
+    if constexpr (VEC == 4) {
+        const uint32_t c = cvt_fp8x4<ELEM>(x[0] * inv[0], x[1] * inv[1], x[2] * inv[2], x[3] * inv[3]);
+        if constexpr (!EMU) {
+            *reinterpret_cast<uint32_t*>(dst) = c;
+        } else {
+            const float2 lo = fp8x2_to_float2<ELEM>(c & 0xFFFFu), hi = fp8x2_to_float2<ELEM>(c >> 16);
+            const __nv_bfloat162 a = __floats2bfloat162_rn(lo.x * xs[0], lo.y * xs[1]);
+            const __nv_bfloat162 b = __floats2bfloat162_rn(hi.x * xs[2], hi.y * xs[3]);
+            *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+        }
+    } else {
+        const uint32_t c = cvt_fp8x2<ELEM>(x[0] * inv[0], x[1] * inv[1]);
+        if constexpr (!EMU) {
+            *reinterpret_cast<uint16_t*>(dst) = (uint16_t)c;
+        } else {
+            const float2 f = fp8x2_to_float2<ELEM>(c);
+            *reinterpret_cast<float2*>(dst) = make_float2(f.x * xs[0], f.y * xs[1]);
+        }
+    }
+}
+
 // One 32-row slab, fast path: every element finite (checked at the end; the caller reruns the
 // slab through slab_careful otherwise), all rows and columns inside the tensor.  Returns
 // whether any lane of the warp met an Inf / NaN.
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
 __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
                                           uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
                                           uint8_t* my_sm_col, int lane, uint32_t rule_offset)
@@ -89,7 +123,9 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
     constexpr int VEC = BF ? 4 : 2;
     constexpr int LPB = 32 / VEC;
     uint32_t bad = 0u;
-    float col_inv[VEC];
+    float col_inv[VEC], col_xs[VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) { col_inv[i] = 1.f; col_xs[i] = 1.f; }
     if (DO_COL) {
         uint32_t cbits[VEC];
         if constexpr (BF) {
@@ -119,6 +155,7 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
         for (int i = 0; i < VEC; ++i) {
             const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
             col_inv[i] = __uint_as_float(ie << 23);
+            col_xs[i] = scale_from_inv(col_inv[i]);
             my_sm_col[i * 4] = (uint8_t)(254u - ie);
         }
     }
@@ -174,24 +211,17 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
         }
         uint8_t* r0 = my_qrow + (uint64_t)j * pitch;
         uint8_t* c0 = my_qcol + (uint64_t)j * pitch;
-        if constexpr (VEC == 4) {
-            if (DO_ROW) {
-                *reinterpret_cast<uint32_t*>(r0) = cvt_fp8x4<ELEM>(x0[0] * inv0, x0[1] * inv0, x0[2] * inv0, x0[3] * inv0);
-                *reinterpret_cast<uint32_t*>(r0 + pitch) = cvt_fp8x4<ELEM>(x1[0] * inv1, x1[1] * inv1, x1[2] * inv1, x1[3] * inv1);
-            }
-            if (DO_COL) {
-                *reinterpret_cast<uint32_t*>(c0) = cvt_fp8x4<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1], x0[2] * col_inv[2], x0[3] * col_inv[3]);
-                *reinterpret_cast<uint32_t*>(c0 + pitch) = cvt_fp8x4<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1], x1[2] * col_inv[2], x1[3] * col_inv[3]);
-            }
-        } else {
-            if (DO_ROW) {
-                *reinterpret_cast<uint16_t*>(r0) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * inv0, x0[1] * inv0);
-                *reinterpret_cast<uint16_t*>(r0 + pitch) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * inv1, x1[1] * inv1);
-            }
-            if (DO_COL) {
-                *reinterpret_cast<uint16_t*>(c0) = (uint16_t)cvt_fp8x2<ELEM>(x0[0] * col_inv[0], x0[1] * col_inv[1]);
-                *reinterpret_cast<uint16_t*>(c0 + pitch) = (uint16_t)cvt_fp8x2<ELEM>(x1[0] * col_inv[0], x1[1] * col_inv[1]);
-            }
+        if (DO_ROW) {
+            float i0[VEC], i1[VEC], s0[VEC], s1[VEC];
+            const float xs0 = EMU ? scale_from_inv(inv0) : 0.f, xs1 = EMU ? scale_from_inv(inv1) : 0.f;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) { i0[i] = inv0; i1[i] = inv1; s0[i] = xs0; s1[i] = xs1; }
+            emit<ELEM, VEC, EMU>(r0, x0, i0, s0);
+            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1);
+        }
+        if (DO_COL) {
+            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs);
+            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs);
         }
     }
     return __any_sync(0xFFFFFFFFu, bad != 0u);
@@ -200,7 +230,7 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
 // The same slab with everything the fast path leaves out: Inf and NaN elements stay out of
 // amax (App. / Sec. 3.3 leaves their handling open; see mxfp8.h), rows and columns outside the
 // tensor are not stored.  Rare, so compact rather than fast.
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
 __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
                                           uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
                                           uint8_t* my_sm_col, int lane, uint32_t rule_offset, int rows_here, bool col_ok)
@@ -218,7 +248,9 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
             x[0] = w.x; x[1] = w.y;
         }
     };
-    float col_inv[VEC];
+    float col_inv[VEC], col_xs[VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) { col_inv[i] = 1.f; col_xs[i] = 1.f; }
     if (DO_COL) {
         float cmax[VEC];
 #pragma unroll
@@ -237,6 +269,7 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
         for (int i = 0; i < VEC; ++i) {
             const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(cmax[i]), rule_offset);
             col_inv[i] = __uint_as_float(ie << 23);
+            col_xs[i] = scale_from_inv(col_inv[i]);
             my_sm_col[i * 4] = (uint8_t)(254u - ie);
         }
     }
@@ -258,20 +291,17 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
             const float inv = __uint_as_float(ie << 23);
             if ((lane & (LPB - 1)) == 0) my_sm_row[j * 4] = (uint8_t)(254u - ie);
             if (live) {
-                if constexpr (VEC == 4) *reinterpret_cast<uint32_t*>(my_qrow + (uint64_t)j * pitch) = cvt_fp8x4<ELEM>(x[0] * inv, x[1] * inv, x[2] * inv, x[3] * inv);
-                else *reinterpret_cast<uint16_t*>(my_qrow + (uint64_t)j * pitch) = (uint16_t)cvt_fp8x2<ELEM>(x[0] * inv, x[1] * inv);
+                float iv[VEC], sv[VEC];
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) { iv[i] = inv; sv[i] = scale_from_inv(inv); }
+                emit<ELEM, VEC, EMU>(my_qrow + (uint64_t)j * pitch, x, iv, sv);
             }
         }
-        if (DO_COL && live) {
-            if constexpr (VEC == 4)
-                *reinterpret_cast<uint32_t*>(my_qcol + (uint64_t)j * pitch) = cvt_fp8x4<ELEM>(x[0] * col_inv[0], x[1] * col_inv[1], x[2] * col_inv[2], x[3] * col_inv[3]);
-            else
-                *reinterpret_cast<uint16_t*>(my_qcol + (uint64_t)j * pitch) = (uint16_t)cvt_fp8x2<ELEM>(x[0] * col_inv[0], x[1] * col_inv[1]);
-        }
+        if (DO_COL && live) emit<ELEM, VEC, EMU>(my_qcol + (uint64_t)j * pitch, x, col_inv, col_xs);
     }
 }
 
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL>
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
 __global__ void __launch_bounds__(QT_THREADS)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams p)
 {
@@ -346,17 +376,19 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
         const int64_t my_col = gcol0 + lane * VEC;
         const int rows_here = (int)min((int64_t)32, p.rows - (grow0 + warp * 32));   // rows of this slab inside the tensor
         const bool col_ok = my_col < p.cols;                                         // cols % 16 == 0: a lane's bytes are all in or all out
-        uint8_t* my_qrow = p.q_row + (grow0 + warp * 32) * p.cols + my_col;
-        uint8_t* my_qcol = p.q_col + (grow0 + warp * 32) * p.cols + my_col;
-        const uint32_t pitch = (uint32_t)p.cols;
+        // bytes per stored element: 1 (FP8 code), or the source's size when the decoded value is stored
+        constexpr int OUT_ESZ = EMU ? (BF ? 2 : 4) : 1;
+        uint8_t* my_qrow = p.q_row + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
+        uint8_t* my_qcol = p.q_col + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
+        const uint32_t pitch = (uint32_t)p.cols * OUT_ESZ;
         uint8_t* my_sm_row = sm_row + warp * 128 + lane / LPB;
         uint8_t* my_sm_col = sm_col + lane * VEC * 4 + warp;
         const bool whole = __all_sync(0xFFFFFFFFu, col_ok) && rows_here == 32;
         bool special = !whole;
         if (whole)
-            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset);
+            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset);
         if (special && rows_here > 0)
-            slab_careful<DTYPE, ELEM, DO_ROW, DO_COL>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
+            slab_careful<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
                                                        rows_here, col_ok);
 
         // every warp is done with this ring slot: refill it with the tile after next
@@ -367,7 +399,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
         }
 
         // ---- scale bytes (1/32 of the output): plain stores from the staging arrays ----------
-        if (DO_ROW && tid < T_ROWS) {
+        if (DO_ROW && !EMU && tid < T_ROWS) {
             const int64_t r = grow0 + tid, ncb = p.cols >> 5, kb0 = (int64_t)tile_x * NKB;
             const int nkb = (int)min((int64_t)NKB, ncb - kb0);
             if (p.sf_layout == MXFP8_SF_SWIZZLED) {
@@ -385,7 +417,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
                 for (int kb = 0; kb < nkb; ++kb) d[kb] = sm_row[tid * 4 + kb];
             }
         }
-        if (DO_COL && tid < T_COLS) {
+        if (DO_COL && !EMU && tid < T_COLS) {
             const int64_t c = gcol0 + tid, nrb = p.rows >> 5, rb0 = (int64_t)tile_y * 4;
             const int nrb_here = (int)min((int64_t)4, nrb - rb0);
             if (p.sf_layout == MXFP8_SF_SWIZZLED) {
@@ -448,11 +480,11 @@ int qt_sm_count()
     return n;
 }
 
-template <int DTYPE, int ELEM, bool R, bool C>
+template <int DTYPE, int ELEM, bool R, bool C, bool EMU>
 cudaError_t launch(const CUtensorMap& ms, const QParams& p, cudaStream_t stream)
 {
     constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
-    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C>;
+    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU>;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (err != cudaSuccess) return err;
     const int tiles = p.tiles_x * p.tiles_y;
@@ -463,12 +495,12 @@ cudaError_t launch(const CUtensorMap& ms, const QParams& p, cudaStream_t stream)
     return cudaGetLastError();
 }
 
-template <int DTYPE, int ELEM>
+template <int DTYPE, int ELEM, bool EMU>
 cudaError_t launch_o(int orientation, const CUtensorMap& ms, const QParams& p, cudaStream_t st)
 {
-    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false>(ms, p, st);
-    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true>(ms, p, st);
-    return launch<DTYPE, ELEM, true, true>(ms, p, st);
+    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU>(ms, p, st);
+    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU>(ms, p, st);
+    return launch<DTYPE, ELEM, true, true, EMU>(ms, p, st);
 }
 
 }  // namespace
@@ -484,7 +516,7 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
 
 int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
                         int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
-                        int sf_layout, cudaStream_t stream)
+                        int sf_layout, cudaStream_t stream, bool emulate)
 {
     const bool bf = src_dtype == MXFP8_BF16;
     const uint32_t t_cols = bf ? 128 : 64;
@@ -501,10 +533,17 @@ int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t co
     p.s_row = static_cast<uint8_t*>(s_row);
     p.s_col = static_cast<uint8_t*>(s_col);
     cudaError_t err;
-    if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3>(orientation, ms, p, stream)
-                                     : launch_o<MXFP8_BF16, MXFP8_E5M2>(orientation, ms, p, stream);
-    else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3>(orientation, ms, p, stream)
-                                  : launch_o<MXFP8_FP32, MXFP8_E5M2>(orientation, ms, p, stream);
+    if (emulate) {
+        if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3, true>(orientation, ms, p, stream)
+                                         : launch_o<MXFP8_BF16, MXFP8_E5M2, true>(orientation, ms, p, stream);
+        else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3, true>(orientation, ms, p, stream)
+                                      : launch_o<MXFP8_FP32, MXFP8_E5M2, true>(orientation, ms, p, stream);
+    } else {
+        if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3, false>(orientation, ms, p, stream)
+                                         : launch_o<MXFP8_BF16, MXFP8_E5M2, false>(orientation, ms, p, stream);
+        else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3, false>(orientation, ms, p, stream)
+                                      : launch_o<MXFP8_FP32, MXFP8_E5M2, false>(orientation, ms, p, stream);
+    }
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
