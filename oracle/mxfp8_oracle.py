@@ -200,3 +200,56 @@ def gemm_f64(aq, a_s, bq, b_s, a_major: str = "k", b_major: str = "k",
         d = a @ b.T
         sabs = np.abs(a) @ np.abs(b).T
     return d, sabs
+
+
+def grouped_gemm_f64(aq, a_s, bq, b_s, offsets, mode: str = "m", b_major: str = "k",
+                     a_elem: int = E4M3, b_elem: int = E4M3):
+    """Per-expert block-scaled products of a mixture-of-experts layer (App. A.4 trains one with the
+    same recipe: every expert's GEMMs are the products of Sec. 2 on that expert's tokens).
+
+    `offsets` (length G+1, non-decreasing, multiples of 32) splits the token axis into G groups;
+    group g owns tokens offsets[g] .. offsets[g+1]-1.
+
+    mode "m" (fprop / dgrad): A stored [T, K] with ROW blocks; B holds the G expert matrices stacked:
+        b_major "k":  stored [G*N, K], ROW blocks, expert g = rows g*N .. (g+1)*N-1
+        b_major "mn": stored [G*K, N], COL blocks, expert g = rows g*K .. (g+1)*K-1
+      D [T, N]: D[t, :] = A[t, :] . B_g^T for t in group g.
+    mode "k" (wgrad): A stored [T, M] and B stored [T, N], both with COL blocks (blocks run down the
+      token axis); D [G*M, N]: D_g = A_g^T . B_g summed over the tokens of group g (zeros for an
+      empty group).
+    Returns (D, S), S the matching sums of |a*b|.
+    """
+    offsets = [int(o) for o in offsets]
+    G = len(offsets) - 1
+    if mode == "m":
+        a = dequantize_f64(aq, a_s, ROW, a_elem)
+        T, K = a.shape
+        if b_major == "k":
+            b = dequantize_f64(bq, b_s, ROW, b_elem)
+            N = b.shape[0] // G
+            experts = [b[g * N:(g + 1) * N, :] for g in range(G)]
+        else:
+            b = dequantize_f64(bq, b_s, COL, b_elem)
+            N = b.shape[1]
+            experts = [b[g * K:(g + 1) * K, :].T for g in range(G)]
+        d = np.zeros((T, N))
+        sabs = np.zeros((T, N))
+        with np.errstate(invalid="ignore", over="ignore"):
+            for g in range(G):
+                lo, hi = offsets[g], offsets[g + 1]
+                d[lo:hi] = a[lo:hi] @ experts[g].T
+                sabs[lo:hi] = np.abs(a[lo:hi]) @ np.abs(experts[g]).T
+        return d, sabs
+    if mode != "k":
+        raise ValueError(mode)
+    a = dequantize_f64(aq, a_s, COL, a_elem)
+    b = dequantize_f64(bq, b_s, COL, b_elem)
+    M, N = a.shape[1], b.shape[1]
+    d = np.zeros((G * M, N))
+    sabs = np.zeros((G * M, N))
+    with np.errstate(invalid="ignore", over="ignore"):
+        for g in range(G):
+            lo, hi = offsets[g], offsets[g + 1]
+            d[g * M:(g + 1) * M] = a[lo:hi].T @ b[lo:hi]
+            sabs[g * M:(g + 1) * M] = np.abs(a[lo:hi]).T @ np.abs(b[lo:hi])
+    return d, sabs

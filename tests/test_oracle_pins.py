@@ -526,3 +526,62 @@ def test_gemm_oracle_exact_integers_and_scales():
     b_s3[4, 0] = 0xFF
     d4, _ = orc.gemm_f64(aq, a_s, bq, b_s3)
     assert np.all(np.isnan(d4[:, 4])) and not np.isnan(d4[:, :4]).any()
+
+
+def _small_int_operand(rng, shape):
+    ints = np.array([-4, -3, -2, -1, 0, 1, 2, 3, 4])
+    vals = rng.choice(ints, shape)
+    enc = {int(v): orc.fp8_encode(float(v)) for v in ints}
+    return vals, np.vectorize(enc.get)(vals).astype(np.uint8)
+
+
+def test_grouped_gemm_oracle_against_integer_loops_and_dense_special_cases():
+    # Every expert's product written out with Python integers (unit scales, small integer elements),
+    # an empty expert included; then the reductions to the dense oracle: one group is the dense
+    # product, and zeroing the other experts' tokens turns the dense product into one group's.
+    rng = np.random.default_rng(11)
+    offsets = [0, 32, 32, 96, 128]               # expert 1 is empty
+    G, T, K, N = 4, 128, 64, 6
+    ai, aq = _small_int_operand(rng, (T, K))
+    a_s = np.full((T, K // 32), 127, np.uint8)
+    # mode "m", K-major stacked B [G*N, K]
+    bi, bq = _small_int_operand(rng, (G * N, K))
+    b_s = np.full((G * N, K // 32), 127, np.uint8)
+    b_s[7, 1] = 129                               # one block of expert 1 (row 7 = expert 1, n = 1) scaled by 4
+    d, sabs = orc.grouped_gemm_f64(aq, a_s, bq, b_s, offsets, "m", "k")
+    for t in (0, 31, 32, 95, 96, 127):
+        g = max(i for i in range(G) if offsets[i] <= t and offsets[i + 1] > t)
+        for n in range(N):
+            row = g * N + n
+            want = sum(int(ai[t, k]) * int(bi[row, k]) * (4 if (row == 7 and k >= 32) else 1) for k in range(K))
+            assert d[t, n] == want
+            assert sabs[t, n] == sum(abs(int(ai[t, k]) * int(bi[row, k])) * (4 if (row == 7 and k >= 32) else 1) for k in range(K))
+    # mode "m", MN-major stacked B [G*K, N]: the same experts stored transposed give the same result
+    bq_t = np.concatenate([np.ascontiguousarray(bq[g * N:(g + 1) * N].T) for g in range(G)], axis=0)
+    bs_t = np.concatenate([np.ascontiguousarray(b_s[g * N:(g + 1) * N].T) for g in range(G)], axis=0)
+    d_t, sabs_t = orc.grouped_gemm_f64(aq, a_s, bq_t, bs_t, offsets, "m", "mn")
+    assert np.array_equal(d_t, d) and np.array_equal(sabs_t, sabs)
+    # one group == the dense oracle
+    d1, s1 = orc.grouped_gemm_f64(aq, a_s, bq[:N], b_s[:N], [0, T], "m", "k")
+    dd, sd = orc.gemm_f64(aq, a_s, bq[:N], b_s[:N])
+    assert np.array_equal(d1, dd) and np.array_equal(s1, sd)
+    # mode "k": D_g = A_g^T B_g; integer loops, then dense oracle on operands whose other tokens are zeroed
+    M = 5
+    xi, xq = _small_int_operand(rng, (T, M))
+    yi, yq = _small_int_operand(rng, (T, N))
+    x_s = np.full((T // 32, M), 127, np.uint8)
+    y_s = np.full((T // 32, N), 127, np.uint8)
+    y_s[2, 3] = 126                               # tokens 64..95 of column 3 scaled by 1/2 (expert 2)
+    dk, sk = orc.grouped_gemm_f64(xq, x_s, yq, y_s, offsets, "k")
+    assert dk.shape == (G * M, N)
+    assert not dk[M:2 * M].any() and not sk[M:2 * M].any()      # empty expert: zeros
+    for g in range(G):
+        for m in range(M):
+            for n in range(N):
+                want = sum(int(xi[t, m]) * int(yi[t, n]) * (0.5 if (n == 3 and 64 <= t < 96) else 1)
+                           for t in range(offsets[g], offsets[g + 1]))
+                assert dk[g * M + m, n] == want
+        xz = np.zeros_like(xq)
+        xz[offsets[g]:offsets[g + 1]] = xq[offsets[g]:offsets[g + 1]]
+        dz, sz = orc.gemm_f64(xz, x_s, yq, y_s, "mn", "mn")
+        assert np.array_equal(dk[g * M:(g + 1) * M], dz) and np.array_equal(sk[g * M:(g + 1) * M], sz)
