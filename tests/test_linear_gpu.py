@@ -33,9 +33,9 @@ def oracle_linear(x, w, dy, rule):
 
 
 def check_bf16_result(got_f32, d64, sabs, what):
-    # FP32 accumulation bound of the GEMM plus one BF16 rounding (half an ulp: 2^-9 relative)
+    # FP32 accumulation bound of the GEMM plus one BF16 rounding (8-bit significand: half an ulp <= 2^-8 relative)
     err = np.abs(got_f32.astype(np.float64) - d64)
-    bound = 2.0 ** -16 * sabs + 2.0 ** -9 * np.abs(d64) + 2.0 ** -126
+    bound = 2.0 ** -16 * sabs + 2.0 ** -8 * np.abs(d64) + 2.0 ** -126
     worst = float((err / bound).max())
     assert worst <= 1.0, "%s: worst err/bound %.3g" % (what, worst)
 
