@@ -388,34 +388,23 @@ __device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams
         const int64_t nkb = p.M >> 5;
         const int64_t kb = row0 >> 5;
         // Column c of this warp's CW columns is "owned" by lane c % 32 (slot c / 32): one warp-wide integer
-        // max per column (|x| bit patterns of finite floats order like integers), the owner keeps the
-        // result, computes scale and 1/X for its CW/32 columns, stores their scale bytes, and hands 1/X
-        // out again by shuffle when the column is cast.
-        uint32_t own[CW / 32];
+        // max per column, the owner keeps the result, computes scale and 1/X for its CW/32 columns, stores
+        // their scale bytes, and hands 1/X out again by shuffle when the column is cast.
+        // |x| bit patterns of finite floats order like integers; adding one exponent step makes the
+        // patterns of Inf and NaN wrap to negative numbers, so a SIGNED max leaves them out of the
+        // maximum without a second pass (all reductions issue back to back, nothing branches on them).
+        int own_biased[CW / 32];
 #pragma unroll
         for (int c = 0; c < CW; ++c) {
-            uint32_t amax;
-            asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(v[c] & 0x7FFFFFFFu));
-            if ((c & 31) == 0) own[c >> 5] = amax;                 // every lane takes it, then the owner's survives
-            else if (lane == (c & 31)) own[c >> 5] = amax;
+            const int a = (int)((v[c] & 0x7FFFFFFFu) + 0x00800000u);
+            int amax;
+            asm volatile("redux.sync.max.s32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
+            if ((c & 31) == 0) own_biased[c >> 5] = amax;          // every lane takes it, then the owner's survives
+            else if (lane == (c & 31)) own_biased[c >> 5] = amax;
         }
-        bool special = false;
+        uint32_t own[CW / 32];
 #pragma unroll
-        for (int j = 0; j < CW / 32; ++j) special |= own[j] >= 0x7F800000u;     // an Inf or NaN reached an amax
-        if (__any_sync(0xFFFFFFFFu, special)) {
-            // rare: redo the maxima without the non-finite elements
-#pragma unroll 1
-            for (int c = 0; c < CW; ++c) {
-                uint32_t a = v[c] & 0x7FFFFFFFu, amax;
-                a = (a >= 0x7F800000u) ? 0u : a;
-                asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
-                if (lane == (c & 31)) {
-#pragma unroll
-                    for (int j = 0; j < CW / 32; ++j)
-                        if (j == (c >> 5)) own[j] = amax;
-                }
-            }
-        }
+        for (int j = 0; j < CW / 32; ++j) own[j] = (uint32_t)(max(own_biased[j], 0x00800000) - 0x00800000);   // no finite element: 0
         float own_inv[CW / 32];
 #pragma unroll
         for (int j = 0; j < CW / 32; ++j) {
