@@ -48,7 +48,8 @@ typedef enum {
     MXFP8_ERR_UNSUPPORTED = -5,    /* valid request this build does not implement         */
     MXFP8_ERR_CUDA = -6,           /* a CUDA runtime/driver call or a launch failed       */
     MXFP8_ERR_DEVICE_TIMEOUT = -7, /* a bounded wait inside a kernel ran out              */
-    MXFP8_ERR_WORKSPACE = -8       /* workspace missing or too small                      */
+    MXFP8_ERR_WORKSPACE = -8,      /* workspace missing or too small                      */
+    MXFP8_ERR_DEVICE_ARGS = -9     /* a kernel found invalid values in a device-side argument array */
 } mxfp8_status;
 
 enum { MXFP8_FP32 = 0, MXFP8_BF16 = 1 };                 /* source / destination dtype   */
@@ -165,7 +166,7 @@ int64_t mxfp8_sf_offset(int64_t mn, int64_t kblock, int64_t n_kblocks, int sf_la
 size_t mxfp8_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int out_dtype, int has_epilogue);
 
 /* Waits for `stream`, then returns and clears the device status word of the current device:
- * MXFP8_OK, MXFP8_ERR_DEVICE_TIMEOUT, or MXFP8_ERR_CUDA if the wait itself failed.
+ * MXFP8_OK, MXFP8_ERR_DEVICE_TIMEOUT, MXFP8_ERR_DEVICE_ARGS, or MXFP8_ERR_CUDA if the wait itself failed.
  * This is the only device-pointer call that synchronises. */
 int mxfp8_device_status(void* stream);
 

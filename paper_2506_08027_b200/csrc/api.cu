@@ -33,6 +33,7 @@ extern "C" const char* mxfp8_status_string(int status)
         case MXFP8_ERR_CUDA: return "CUDA error";
         case MXFP8_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
         case MXFP8_ERR_WORKSPACE: return "workspace missing or too small";
+        case MXFP8_ERR_DEVICE_ARGS: return "invalid values in a device-side argument array";
         default: return "unknown status";
     }
 }

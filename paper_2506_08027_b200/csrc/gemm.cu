@@ -42,6 +42,7 @@ int read_and_clear_device_status(cudaStream_t stream)
     if (h != 0 && cudaMemcpyToSymbol(g_device_status, &z, sizeof(int)) != cudaSuccess) return MXFP8_ERR_CUDA;
     const int q = quantize_read_and_clear_status();
     if (q == MXFP8_ERR_CUDA) return q;
+    if (h == MXFP8_ERR_DEVICE_ARGS) return h;
     return (h == 0 && q == MXFP8_OK) ? MXFP8_OK : MXFP8_ERR_DEVICE_TIMEOUT;
 }
 
@@ -68,7 +69,17 @@ struct GemmParams {
     int epi_rule, epi_elem;
     uint8_t* epi_s_row;   // swizzled scales of the row-blocked output, logical [M, N/32]
     uint8_t* epi_s_col;   // swizzled scales of the column-blocked output, logical [N, M/32]
+    // grouped (per-expert) products: device array of num_groups + 1 token offsets, multiples of 128
+    const int32_t* group_offsets;
+    int num_groups;
+    int token_limit;      // offsets may not pass this (tokens in the grouped tensor)
 };
+
+constexpr int MAX_GROUPS = 256;
+// MODE of the kernel: one dense product, or one product per expert of a mixture-of-experts layer
+//   GROUP_M: the rows of A (tokens) are grouped, B holds one matrix per expert   (fprop, dgrad)
+//   GROUP_K: the reduction axis (tokens) is grouped, D holds one matrix per expert (wgrad)
+enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2 };
 
 // BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
 // tile has 2*BM rows.  BN = 256 leaves room for one accumulator only (2 x 256 columns would fill
@@ -94,8 +105,9 @@ template <int BN, bool PAIR> struct Cfg {
     static constexpr int SMEM_EPI = SMEM_SFB + STAGES * 512 * SFB_ATOMS;      // 8 x 2 KB, 512-aligned
     static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES + 1;
     static constexpr int SMEM_BAR = SMEM_EPI + EPI_WARPS * EPI_BUF_BYTES;
-    static constexpr int SMEM_MISC = SMEM_BAR + NUM_BARS * 8;  // tmem pointer, abort flag
-    static constexpr int SMEM_TOTAL = SMEM_MISC + 16 + 1024;   // + slack to align the base to 1024
+    static constexpr int SMEM_MISC = SMEM_BAR + NUM_BARS * 8;  // tmem pointer, abort flag, bad-offsets flag
+    static constexpr int SMEM_GROUPS = SMEM_MISC + 16;         // group offsets and first-tile indices, (MAX_GROUPS + 1) ints each
+    static constexpr int SMEM_TOTAL = SMEM_GROUPS + 2 * (MAX_GROUPS + 1) * 4 + 4 + 1024;   // + slack to align the base to 1024
     static_assert(SF_COL0 + STAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
     static_assert(SMEM_TOTAL <= 227 * 1024, "shared memory budget");
     static_assert(SMEM_EPI % 512 == 0, "staging buffers need 512-byte alignment for the 64-byte swizzle");
@@ -433,16 +445,77 @@ __device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams
 // Tile rasterisation: tiles are numbered group by group; a group is `group_m` M-tiles tall and
 // spans all N-tiles, M fastest inside it, so the tiles in flight at one time share few distinct
 // A row-blocks and B row-blocks and hit in L2.
-__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& tm, int& tn)
+__device__ __forceinline__ void tile_coords(int group_m, int tiles_m, int tiles_n, int tile, int& tm, int& tn)
 {
-    const int per_group = p.group_m * p.tiles_n;
+    const int per_group = group_m * tiles_n;
     const int g = tile / per_group, r = tile - g * per_group;
-    const int gm = min(p.group_m, p.tiles_m - g * p.group_m);
+    const int gm = min(group_m, tiles_m - g * group_m);
     tn = r / gm;
-    tm = g * p.group_m + (r - tn * gm);
+    tm = g * group_m + (r - tn * gm);
 }
 
-template <int BN, bool PAIR>
+// Where one tile sits.  For a dense product everything but (tm, tn) is a constant; the grouped
+// modes shift the operand coordinates to the tile's expert:
+//   GROUP_M: A / SFA / D rows start at the expert's first token; B is the expert's matrix inside the
+//            stack (K-major B [G*N, K]: N-coordinate + g*N; MN-major B [G*K, N]: K-coordinate + g*K)
+//   GROUP_K: the K loop runs over the expert's tokens only; D rows start at g*M
+struct TileCtx {
+    int tm, tn;         // tile position inside its expert's output (rows in units of the tile height)
+    int row0;           // added to A's MN coordinate (GROUP_M: the expert's first token)
+    int d_row_extra;    // added on top of that for the D row (GROUP_K: g * M)
+    int rows_end;       // D rows at or beyond this one are not stored
+    int ka0, kb0;       // K-block offsets of A (and its scales) and of B (and its scales)
+    int bn_off;         // added to B's MN coordinate
+    int sfb_atom_off;   // added to the MN atom index of B's scales
+    int nkb;            // K blocks of this tile
+};
+
+template <int MODE, int TM>
+__device__ __forceinline__ TileCtx decode_tile(const GemmParams& p, const int* goff, const int* tstart, int tile, int& g)
+{
+    TileCtx t;
+    if constexpr (MODE == DENSE) {
+        tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile, t.tm, t.tn);
+        t.row0 = 0; t.d_row_extra = 0; t.rows_end = (int)p.M; t.ka0 = 0; t.kb0 = 0; t.bn_off = 0; t.sfb_atom_off = 0;
+        t.nkb = p.num_kb;
+    } else if constexpr (MODE == GROUP_M) {
+        while (tile >= tstart[g + 1]) ++g;          // tiles only move forward: g is a cursor
+        const int lo = goff[g], hi = goff[g + 1];
+        tile_coords(p.group_m, (hi - lo + TM - 1) / TM, p.tiles_n, tile - tstart[g], t.tm, t.tn);
+        t.row0 = lo; t.d_row_extra = 0; t.rows_end = hi; t.ka0 = 0; t.nkb = p.num_kb;
+        if (p.b_mn) { t.kb0 = g * p.num_kb; t.bn_off = 0; t.sfb_atom_off = 0; }
+        else { t.kb0 = 0; t.bn_off = g * (int)p.N; t.sfb_atom_off = (g * (int)p.N) >> 7; }
+    } else {
+        const int per_expert = p.tiles_m * p.tiles_n;
+        g = tile / per_expert;
+        tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile - g * per_expert, t.tm, t.tn);
+        const int lo = goff[g], hi = goff[g + 1];
+        t.row0 = 0; t.d_row_extra = g * (int)p.M; t.rows_end = (g + 1) * (int)p.M;
+        t.ka0 = lo >> 7; t.kb0 = lo >> 7; t.bn_off = 0; t.sfb_atom_off = 0;
+        t.nkb = (hi - lo) >> 7;
+    }
+    return t;
+}
+
+// K blocks this worker will run through: the flat loops of the producer and the MMA issuer count them.
+template <int MODE>
+__device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const int* goff, int num_tiles, int worker, int workers)
+{
+    if (num_tiles <= worker) return 0u;
+    if constexpr (MODE != GROUP_K) {
+        return (uint32_t)((num_tiles - worker + workers - 1) / workers) * (uint32_t)p.num_kb;
+    } else {
+        const int per_expert = p.tiles_m * p.tiles_n;
+        uint32_t total = 0;
+        for (int tile = worker; tile < num_tiles; tile += workers) {
+            const int g = tile / per_expert;
+            total += (uint32_t)((goff[g + 1] - goff[g]) >> 7);
+        }
+        return total;
+    }
+}
+
+template <int BN, bool PAIR, int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
@@ -463,6 +536,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const uint32_t drain_bar = bar0 + 8u * (2 * C::STAGES + 2 * C::ACC_STAGES);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + C::SMEM_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::SMEM_MISC + 4);
+    volatile int* bad_groups = reinterpret_cast<volatile int*>(base_ptr + C::SMEM_MISC + 8);
+    int* goff = reinterpret_cast<int*>(base_ptr + C::SMEM_GROUPS);      // group offsets (tokens)
+    int* tstart = goff + (MAX_GROUPS + 1);                              // GROUP_M: first tile of each group
+    constexpr int TM = PAIR ? 2 * BM : BM;                              // tile height
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -478,7 +555,41 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
         mbar_init(drain_bar, 1);
         *abort_flag = 0;
+        *bad_groups = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if constexpr (MODE != DENSE) {
+        // every CTA reads the offsets, checks them (non-negative, non-decreasing, multiples of 128,
+        // inside the tensor) and, for GROUP_M, turns them into the first tile index of each group
+        const int G = p.num_groups;
+        for (int i = threadIdx.x; i <= G; i += GEMM_THREADS) goff[i] = p.group_offsets[i];
+        __syncthreads();
+        if (warp == 2) {
+            bool bad = false;
+            int run = 0;
+            for (int i0 = 0; i0 < G; i0 += 32) {
+                const int i = i0 + lane;
+                int cnt = 0;
+                if (i < G) {
+                    const int lo = goff[i], hi = goff[i + 1];
+                    if (lo < 0 || hi < lo || ((lo | hi) & 127) || hi > p.token_limit) bad = true;
+                    else if (MODE == GROUP_M) cnt = ((hi - lo + TM - 1) / TM) * p.tiles_n;
+                }
+                int x = cnt;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
+                    if (lane >= d) x += y;
+                }
+                if (i < G) tstart[i + 1] = run + x;
+                run += __shfl_sync(0xFFFFFFFFu, x, 31);
+            }
+            bad = __any_sync(0xFFFFFFFFu, bad);
+            if (lane == 0) {
+                tstart[0] = 0;
+                if (bad) { *bad_groups = 1; atomicExch(&g_device_status, (int)MXFP8_ERR_DEVICE_ARGS); }
+            }
+        }
     }
     if (warp == 1) {
         if (PAIR) {
@@ -496,17 +607,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     if (PAIR) cluster_sync_all();      // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // tiles of the whole launch (none when the offsets were rejected)
+    const int num_tiles = MODE == DENSE ? p.num_tiles
+                        : (*bad_groups ? 0 : (MODE == GROUP_M ? tstart[p.num_groups] : p.num_groups * p.tiles_m * p.tiles_n));
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
         // ring-depth-unrolled loop as the MMA warp.
         {
-            const int a_mn = p.a_mn, b_mn = p.b_mn, num_kb = p.num_kb;
-            const int my_tiles = (p.num_tiles - worker + workers - 1) / workers;
-            const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_kb;
-            int kb = 0, tile = worker;
-            int m_atom = 0, m0 = 0, n0 = 0, sfb_atom0 = 0;
+            const int a_mn = p.a_mn, b_mn = p.b_mn;
+            const uint32_t total = worker_k_blocks<MODE>(p, goff, num_tiles, worker, workers);
+            int kb = 0, tile = worker, gcur = 0;
+            int m_atom = 0, m0 = 0, n0 = 0, sfb_atom0 = 0, ka0 = 0, kb0 = 0, nkb = p.num_kb;
             uint32_t ph = 0;
             bool ok = true;
             for (uint32_t g0 = 0; g0 < total && ok; g0 += C::STAGES) {
@@ -514,12 +627,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 for (int s = 0; s < C::STAGES; ++s) {
                     if (g0 + s >= total) break;
                     if (kb == 0) {
-                        int tm, tn;
-                        tile_coords(p, tile, tm, tn);
-                        m_atom = tm * (PAIR ? 2 : 1) + (int)cta_rank;             // 128-row block of A / D
-                        m0 = m_atom * BM;
-                        n0 = tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);    // first B row this CTA loads
-                        sfb_atom0 = (tn * BN) >> 7;                               // scale atom holding the tile's first column
+                        TileCtx t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur);
+                        if constexpr (MODE == GROUP_K) {
+                            while (t.nkb == 0) { tile += workers; t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur); }   // expert without tokens
+                        }
+                        m0 = t.row0 + (t.tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM;   // first row of A this CTA loads
+                        m_atom = m0 >> 7;                                             // its scale atom
+                        n0 = t.bn_off + t.tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);    // first B row this CTA loads
+                        sfb_atom0 = t.sfb_atom_off + ((t.tn * BN) >> 7);              // scale atom holding the tile's first column
+                        ka0 = t.ka0; kb0 = t.kb0; nkb = t.nkb;
                     }
                     ok = warp_wait(empty_bar(s), ph ^ 1u, abort_flag);
                     if (!ok) break;
@@ -527,25 +643,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     const uint32_t fb = PAIR ? map_to_cta(full_bar(s), 0) : full_bar(s);
                     const uint32_t sa = base + C::SMEM_A + s * C::A_BYTES;
                     const uint32_t sb = base + C::SMEM_B + s * C::B_BYTES;
-                    const int k0 = kb * BK;
+                    const int k0a = (ka0 + kb) * BK, k0b = (kb0 + kb) * BK;
                     if (elect_one()) {
                         if (cta_rank == 0) mbar_expect_tx(full_bar(s), p.stage_tx);
-                        if (!a_mn) tma_load_2d<PAIR>(sa, &tmap_a, fb, k0, m0);
-                        else tma_load_2d<PAIR>(sa, &tmap_a, fb, m0, k0);
+                        if (!a_mn) tma_load_2d<PAIR>(sa, &tmap_a, fb, k0a, m0);
+                        else tma_load_2d<PAIR>(sa, &tmap_a, fb, m0, k0a);
                         if (!b_mn) {
-                            tma_load_2d<PAIR>(sb, &tmap_b, fb, k0, n0);
+                            tma_load_2d<PAIR>(sb, &tmap_b, fb, k0b, n0);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < C::B_SLABS; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0);
+                            for (int j = 0; j < C::B_SLABS; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0b);
                         }
-                        tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, &tmap_sfa, fb, 0, kb, m_atom);
+                        tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, &tmap_sfa, fb, 0, ka0 + kb, m_atom);
 #pragma unroll
                         for (int j = 0; j < C::SFB_ATOMS; ++j)      // every CTA needs the scales of all BN columns
-                            tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, &tmap_sfb, fb, 0, kb,
+                            tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, &tmap_sfb, fb, 0, kb0 + kb,
                                               sfb_atom0 + j);
                     }
                     __syncwarp();
-                    if (++kb == num_kb) { kb = 0; tile += workers; }
+                    if (++kb == nkb) { kb = 0; tile += workers; }
                 }
                 ph ^= 1u;
             }
@@ -574,10 +690,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t sf_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);   // scales: 32 rows x 16 B, 8-row groups 128 B apart
             const uint32_t sfa_lo0 = (base + C::SMEM_SFA) >> 4, sfb_lo0 = (base + C::SMEM_SFB) >> 4;
             auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
-            const int num_kb = p.num_kb;
-            const int my_tiles = (p.num_tiles - worker + workers - 1) / workers;
-            const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_kb;
-            int kb = 0, tile = worker;
+            const uint32_t total = worker_k_blocks<MODE>(p, goff, num_tiles, worker, workers);
+            int kb = 0, tile = worker, gcur = 0, num_kb = p.num_kb;
             uint32_t ph = 0, acc_it = 0, d_tmem = tmem_base, sfb_skip = 0;
             int as = 0;
             bool ok = true;
@@ -591,11 +705,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                         ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag);
                         if (!ok) break;
                         d_tmem = tmem_base + as * BN;
-                        int tm, tn;
-                        tile_coords(p, tile, tm, tn);
+                        TileCtx t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur);
+                        if constexpr (MODE == GROUP_K) {
+                            while (t.nkb == 0) { tile += workers; t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur); }   // expert without tokens
+                        }
+                        num_kb = t.nkb;
                         // a tile that starts in the middle of a 128-wide scale atom reads its B scales from
                         // the matching TMEM column of the copied atoms (32 columns of B per TMEM column)
-                        sfb_skip = (uint32_t)(((tn * BN) & 127) >> 5);
+                        sfb_skip = (uint32_t)(((t.tn * BN) & 127) >> 5);
                     }
                     ok = warp_wait(full_bar(s), ph, abort_flag);
                     if (!ok) break;
@@ -642,31 +759,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         uint32_t acc_it = 0;
         bool ok = true;
         const int n_total = (int)p.N;
-        for (int tile = worker; tile < p.num_tiles && ok; tile += workers, ++acc_it) {
-            int tm, tn;
-            tile_coords(p, tile, tm, tn);
-            const int as = acc_it % C::ACC_STAGES;
-            const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-            if (lane == 0) ok = mbar_wait(tfull_bar(as), aph, abort_flag);   // one suspending poller per warp
-            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-            if (!ok) break;
-            tc_fence_after();
+        int gcur = 0;
+        for (int tile = worker; tile < num_tiles && ok; tile += workers) {
+            const TileCtx t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur);
+            const int tm = t.tm, tn = t.tn;
             uint32_t v[CW];
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN + half * CW;
+            if (MODE == GROUP_K && t.nkb == 0) {
+                // an expert without tokens: its product is all zeros and no MMA ran for this tile
 #pragma unroll
-            for (int c = 0; c < CW / 32; ++c) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
-            tc_wait_ld();
-            // the accumulator now lives in registers: hand TMEM back to the MMA warp of the leader
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
-                else mbar_arrive(tempty_bar(as));
+                for (int c = 0; c < CW; ++c) v[c] = 0u;
+            } else {
+                const int as = acc_it % C::ACC_STAGES;
+                const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
+                ++acc_it;
+                if (lane == 0) ok = mbar_wait(tfull_bar(as), aph, abort_flag);   // one suspending poller per warp
+                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN + half * CW;
+#pragma unroll
+                for (int c = 0; c < CW / 32; ++c) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+                tc_wait_ld();
+                // the accumulator now lives in registers: hand TMEM back to the MMA warp of the leader
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
+                    else mbar_arrive(tempty_bar(as));
+                }
             }
 
-            const int row0 = (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
+            const int row0 = t.row0 + t.d_row_extra + (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
-            const bool rows_inside = row0 < (int)p.M;        // ragged last M tile: a 32-row box entirely outside stores nothing
+            const bool rows_inside = row0 < t.rows_end;      // ragged last M tile / rows of the next expert: a 32-row box entirely outside stores nothing
             if constexpr (CW % 64 == 0) {
                 if (p.epi_orient && rows_inside) {
                     if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
