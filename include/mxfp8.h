@@ -162,6 +162,38 @@ size_t mxfp8_scale_bytes(int64_t rows, int64_t cols, int orientation, int sf_lay
  * SWIZZLED: the 128x4 atom formula in the header comment.  Host helper, no device work. */
 int64_t mxfp8_sf_offset(int64_t mn, int64_t kblock, int64_t n_kblocks, int sf_layout);
 
+/*
+ * mxfp8_grouped_gemm -- the per-expert products of a mixture-of-experts layer in one launch (App. A.4
+ * trains a mixture-of-experts model with the same recipe; each expert's FPROP / DGRAD / WGRAD is the
+ * block-scaled product of Sec. 2 restricted to the tokens routed to that expert).
+ *
+ * Tokens are sorted by expert; group_offsets (DEVICE pointer, num_groups + 1 int32 values, 4-byte
+ * aligned) gives the first token of every expert and the end of the last: non-negative,
+ * non-decreasing, multiples of 128, at most the token count.  The kernel reads and checks them
+ * on the device (no host synchronisation); a violation makes the launch store nothing and leaves
+ * MXFP8_ERR_DEVICE_ARGS in the device status word.  Rows before group_offsets[0] and from
+ * group_offsets[num_groups] on belong to no expert and are left untouched (GROUP_M) / unused (GROUP_K).
+ *
+ * mode MXFP8_GROUP_M (FPROP, DGRAD): M = tokens.
+ *     Aq [M, K] K-major with ROW blocks, As its swizzled scales (logical [M, K/32]).
+ *     B = the experts' matrices stacked, quantized as ONE tensor by mxfp8_quantize:
+ *         b_major K:  Bq [G*N, K], ROW blocks, scales logical [G*N, K/32]   (expert g = rows g*N ..)
+ *         b_major MN: Bq [G*K, N], COL blocks, scales logical [N, G*K/32]   (expert g = rows g*K ..)
+ *     D [M, N]: row t = A[t, :] . B_g^T for the expert g that owns token t.
+ * mode MXFP8_GROUP_K (WGRAD): K = tokens; b_major must be MN.
+ *     Aq [K, M] and Bq [K, N], both with COL blocks (blocks run down the token axis), scales
+ *     logical [M, K/32] and [N, K/32].
+ *     D [G*M, N]: rows g*M .. = A_g^T . B_g summed over expert g's tokens; zeros for an expert
+ *     without tokens.
+ * M, N, K multiples of 128; num_groups <= 256; element formats and output dtype as mxfp8_gemm;
+ * FP32 accumulation; all pointers device, 16-byte aligned; nothing is allocated.
+ */
+enum { MXFP8_GROUP_M = 1, MXFP8_GROUP_K = 2 };
+int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq, const void* Bs,
+                       const int32_t* group_offsets, int num_groups, int mode,
+                       int64_t M, int64_t N, int64_t K, int b_major, int a_elem, int b_elem,
+                       void* D, int out_dtype, void* stream);
+
 /* Scratch bytes mxfp8_gemm needs for this problem (0 when none). */
 size_t mxfp8_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int out_dtype, int has_epilogue);
 

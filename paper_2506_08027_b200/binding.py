@@ -19,12 +19,14 @@ RULE_PAPER, RULE_OCP = 0, 1
 E4M3, E5M2 = 0, 1
 SF_LINEAR, SF_SWIZZLED = 0, 1
 K_MAJOR, MN_MAJOR = 0, 1
+ERR_DEVICE_TIMEOUT, ERR_DEVICE_ARGS = -7, -9
 
 EXPORTS = (
     "mxfp8_quantize", "mxfp8_dequantize", "mxfp8_gemm", "mxfp8_scale_bytes", "mxfp8_sf_offset",
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
-    "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes", "mxfp8_linear",
+    "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
+    "mxfp8_linear", "mxfp8_grouped_gemm",
 )
 
 
@@ -78,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
         L.mxfp8_fake_quantize.restype = i
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_grouped_gemm.restype = i
+        L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
         L.mxfp8_linear_ws_bytes.restype = sz
         L.mxfp8_linear_ws_bytes.argtypes = [i64, i64, i64]
         L.mxfp8_linear.restype = i
@@ -230,3 +234,14 @@ def mxfp8_linear(x, w, dy, scale_rule: int, y, dx, dw, ws, stream=None) -> None:
     F = w.shape[0]
     _check(lib().mxfp8_linear(_ptr(x), _ptr(w), _ptr(dy), T, H, F, scale_rule, _ptr(y), _ptr(dx), _ptr(dw),
                               _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "mxfp8_linear")
+
+
+GROUP_M, GROUP_K = 1, 2
+
+
+def mxfp8_grouped_gemm(aq, a_s, bq, b_s, group_offsets: torch.Tensor, mode: int, M: int, N: int, K: int,
+                       b_major: int, a_elem: int, b_elem: int, D: torch.Tensor, stream=None) -> None:
+    assert group_offsets.dtype == torch.int32 and group_offsets.is_cuda
+    _check(lib().mxfp8_grouped_gemm(_ptr(aq), _ptr(a_s), _ptr(bq), _ptr(b_s), _ptr(group_offsets),
+                                    group_offsets.numel() - 1, mode, M, N, K, b_major, a_elem, b_elem,
+                                    _ptr(D), _dtype_code(D), _stream(stream)), "mxfp8_grouped_gemm")

@@ -951,11 +951,11 @@ int sm_count()
 
 struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; };
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, int MODE = DENSE>
 int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
 {
     using C = Cfg<BN, PAIR>;
-    auto kernel = gemm_kernel<BN, PAIR>;
+    auto kernel = gemm_kernel<BN, PAIR, MODE>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
         return MXFP8_ERR_CUDA;
     p.tiles_m = (int)((p.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM));
@@ -967,7 +967,12 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
     const int max_workers = PAIR ? sms / 2 : sms;
-    const int workers = p.num_tiles < max_workers ? p.num_tiles : max_workers;
+    // tiles known to the host: all of them (dense), an upper bound (GROUP_M: every group may end in a
+    // partly filled tile; the kernel counts the real ones), tiles of all experts (GROUP_K)
+    int64_t host_tiles = p.num_tiles;
+    if (MODE == GROUP_M) host_tiles = ((int64_t)p.tiles_m + p.num_groups) * p.tiles_n;
+    if (MODE == GROUP_K) host_tiles = (int64_t)p.num_tiles * p.num_groups;
+    const int workers = host_tiles < max_workers ? (int)host_tiles : max_workers;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * workers : workers));
     cfg.blockDim = dim3(GEMM_THREADS);
@@ -1088,4 +1093,78 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     if (best_pair) return best_bn == 256 ? launch_gemm<256, true>(m, p, st) : launch_gemm<192, true>(m, p, st);
     if (best_bn == 256) return launch_gemm<256, false>(m, p, st);
     return best_bn == 192 ? launch_gemm<192, false>(m, p, st) : launch_gemm<128, false>(m, p, st);
+}
+
+extern "C" int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq, const void* Bs,
+                                  const int32_t* group_offsets, int num_groups, int mode,
+                                  int64_t M, int64_t N, int64_t K, int b_major, int a_elem, int b_elem,
+                                  void* D, int out_dtype, void* stream)
+{
+    using namespace mxfp8;
+    if (mode != MXFP8_GROUP_M && mode != MXFP8_GROUP_K) return MXFP8_ERR_ENUM;
+    if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
+    if (a_elem != MXFP8_E4M3 && a_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (b_elem != MXFP8_E4M3 && b_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (!Aq || !As || !Bq || !Bs || !group_offsets || !D) return MXFP8_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || num_groups <= 0) return MXFP8_ERR_SHAPE;
+    if (num_groups > MAX_GROUPS) return MXFP8_ERR_UNSUPPORTED;
+    if (mode == MXFP8_GROUP_K && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_UNSUPPORTED;   // both operands are token-major
+    // whole scale atoms per expert on every axis that is stacked or split
+    if ((M % 128) || (N % 128) || (K % 128)) return MXFP8_ERR_UNSUPPORTED;
+    const int64_t G = num_groups;
+    const int64_t d_rows = mode == MXFP8_GROUP_M ? M : G * M;
+    const int64_t b_stack = mode == MXFP8_GROUP_M ? (b_major == MXFP8_K_MAJOR ? G * N : G * K) : 0;
+    if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF || d_rows > 0x3FFFFFFF || b_stack > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
+    if (!aligned16(Aq) || !aligned16(As) || !aligned16(Bq) || !aligned16(Bs) || !aligned16(D) ||
+        (reinterpret_cast<uintptr_t>(group_offsets) & 3u))
+        return MXFP8_ERR_ALIGN;
+
+    GemmParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
+    p.store_d = 1;
+    p.group_offsets = group_offsets;
+    p.num_groups = num_groups;
+    const int sms = sm_count();
+    if (sms <= 0) return MXFP8_ERR_CUDA;
+    GemmMaps m;
+    bool ok;
+    bool pair;
+    if (mode == MXFP8_GROUP_M) {
+        // A [M tokens, K] K-major; B stacked per expert; D [M, N].  CTA pairs (256-row tiles) pay
+        // off once an average expert fills a few of them; the host only knows the average.
+        p.a_mn = 0; p.b_mn = b_major;
+        p.token_limit = (int)M;
+        pair = (M / G) >= 512;
+        const char* force = getenv("MXFP8_GEMM_TILE");
+        if (force) pair = strchr(force, 'p') != nullptr;
+        ok = make_tmap(&m.a, Aq, (uint64_t)K, (uint64_t)M, 128, 128);
+        ok = ok && (b_major == MXFP8_K_MAJOR ? make_tmap(&m.b, Bq, (uint64_t)K, (uint64_t)(G * N), 128, pair ? 128 : 256)
+                                             : make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)(G * K), 128, 128));
+        ok = ok && make_tmap_sf(&m.sfa, As, (uint64_t)(M / 128), (uint64_t)(K / 128));
+        ok = ok && (b_major == MXFP8_K_MAJOR ? make_tmap_sf(&m.sfb, Bs, (uint64_t)(G * N / 128), (uint64_t)(K / 128))
+                                             : make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(G * K / 128)));
+        ok = ok && make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype);
+    } else {
+        // A [K tokens, M] and B [K tokens, N], both MN-major with blocks down the token axis; D [G*M, N]
+        p.a_mn = 1; p.b_mn = 1;
+        p.token_limit = (int)K;
+        pair = (M % 256) == 0;
+        const char* force = getenv("MXFP8_GEMM_TILE");
+        if (force) pair = strchr(force, 'p') != nullptr;
+        ok = make_tmap(&m.a, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
+        ok = ok && make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)K, 128, 128);
+        ok = ok && make_tmap_sf(&m.sfa, As, (uint64_t)(M / 128), (uint64_t)(K / 128));
+        ok = ok && make_tmap_sf(&m.sfb, Bs, (uint64_t)(N / 128), (uint64_t)(K / 128));
+        ok = ok && make_tmap_d(&m.d, D, (uint64_t)(G * M), (uint64_t)N, out_dtype);
+    }
+    if (getenv("MXFP8_LOG"))
+        fprintf(stderr, "mxfp8_grouped_gemm mode=%d G=%d M=%lld N=%lld K=%lld tile=256%s maps=%d\n", mode, num_groups, (long long)M,
+                (long long)N, (long long)K, pair ? "p" : "", (int)ok);
+    if (!ok) return MXFP8_ERR_CUDA;
+    m.qrow = m.d; m.qcol = m.d;   // no fused MXFP8 output in the grouped modes; the maps only have to be valid
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (mode == MXFP8_GROUP_M) return pair ? launch_gemm<256, true, GROUP_M>(m, p, st) : launch_gemm<256, false, GROUP_M>(m, p, st);
+    return pair ? launch_gemm<256, true, GROUP_K>(m, p, st) : launch_gemm<256, false, GROUP_K>(m, p, st);
 }
