@@ -447,6 +447,49 @@ def run_sweep(args):
                     del srcs
                     torch.cuda.empty_cache()
         return
+    if args.sweep == "moe":
+        # per-expert GEMMs of a mixture-of-experts FFN (App. A.4 trains a 16B-total / 2.5B-active model; the layer here
+        # has that class's shape: hidden 2048, expert FFN 1408, 64 experts, 6 experts per token, 8192 tokens per batch).
+        # Token counts per expert are multinomial, each expert's segment padded to a multiple of 128 rows.
+        import numpy as np
+        Hd, Fe, G, topk, tokens = 2048, 1408, 64, 6, 8192
+        print("| case | experts | routed tokens (padded) | N | K | us | TFLOP/s | of 2x measured BF16 | dense GEMM of the same size: us |")
+        print("|---|---|---|---|---|---|---|---|---|")
+        for skew, label in ((0.0, "uniform routing"), (1.0, "skewed routing")):
+            rng = np.random.default_rng(2506)
+            w = np.exp(skew * rng.standard_normal(G))
+            counts = rng.multinomial(tokens * topk, w / w.sum())
+            padded = (counts + 127) // 128 * 128
+            offs = np.concatenate([[0], np.cumsum(padded)]).astype(np.int32)
+            Tt = int(offs[-1])
+            off_d = torch.from_numpy(offs).cuda()
+            x = synth.device_tensor("activation", (Tt, Hd), 21)
+            dy = synth.device_tensor("output_gradient", (Tt, Fe), 22)
+            wst = synth.device_tensor("weight", (G * Fe, Hd), 23)
+            qx = B.alloc_quantize_outputs(Tt, Hd, B.BOTH, S); B.mxfp8_quantize(x, B.BOTH, P, B.E4M3, *qx, S)
+            qdy = B.alloc_quantize_outputs(Tt, Fe, B.BOTH, S); B.mxfp8_quantize(dy, B.BOTH, P, B.E4M3, *qdy, S)
+            qw = B.alloc_quantize_outputs(G * Fe, Hd, B.BOTH, S); B.mxfp8_quantize(wst, B.BOTH, P, B.E4M3, *qw, S)
+            y = torch.empty((Tt, Fe), dtype=torch.bfloat16, device="cuda")
+            dx = torch.empty((Tt, Hd), dtype=torch.bfloat16, device="cuda")
+            dw = torch.empty((G * Fe, Hd), dtype=torch.bfloat16, device="cuda")
+            cases = (
+                ("fprop", lambda i: B.mxfp8_grouped_gemm(qx[0], qx[1], qw[0], qw[1], off_d, B.GROUP_M, Tt, Fe, Hd, B.K_MAJOR, B.E4M3, B.E4M3, y),
+                 Fe, Hd, lambda i: B.mxfp8_gemm(qx[0], qx[1], qw[0], qw[1], Tt, Fe, Hd, B.K_MAJOR, B.K_MAJOR, B.E4M3, B.E4M3, y)),
+                ("dgrad", lambda i: B.mxfp8_grouped_gemm(qdy[0], qdy[1], qw[2], qw[3], off_d, B.GROUP_M, Tt, Hd, Fe, B.MN_MAJOR, B.E4M3, B.E4M3, dx),
+                 Hd, Fe, lambda i: B.mxfp8_gemm(qdy[0], qdy[1], qw[2], qw[3], Tt, Hd, Fe, B.K_MAJOR, B.MN_MAJOR, B.E4M3, B.E4M3, dx)),
+                ("wgrad", lambda i: B.mxfp8_grouped_gemm(qdy[2], qdy[3], qx[2], qx[3], off_d, B.GROUP_K, Fe, Hd, Tt, B.MN_MAJOR, B.E4M3, B.E4M3, dw),
+                 Hd, None, lambda i: B.mxfp8_gemm(qdy[2], qdy[3], qx[2], qx[3], Fe, Hd, Tt, B.MN_MAJOR, B.MN_MAJOR, B.E4M3, B.E4M3, dw[:Fe])),
+            )
+            for name, fn, n_, k_, dense in cases:
+                ms = _time_calls(fn, 1)
+                ms_dense = _time_calls(dense, 1)
+                flop = 2.0 * Tt * Fe * Hd
+                tf = flop / ms / 1e9
+                print("| %s, %s | %d | %d (%d) | %d | %s | %.1f | %.0f | %.2f | %.1f |" % (
+                    name, label, G, int(counts.sum()), Tt, n_, k_ if k_ else "tokens of the expert", ms * 1e3, tf,
+                    tf / (2 * peaks["bf16_tflops"]), ms_dense * 1e3), flush=True)
+            assert B.mxfp8_device_status() == 0
+        return
     if args.sweep == "emu":
         # the MXFP8 round trip (Sec. 3.1): reads the source once, writes one same-dtype tensor per orientation
         print("| dtype | rows x cols | orient | us | GB/s | of measured copy |")
@@ -518,7 +561,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k"],
                     help="run one kernel on one small case and exit (for profiler captures)")
-    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu"],
+    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
     args = ap.parse_args()
     if args.sweep:

@@ -699,12 +699,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
                 for (int s = 0; s < C::STAGES; ++s) {
                     if (g0 + s >= total) break;
-                    if (kb == 0) {   // first K block of a tile: the accumulator must have been drained
-                        as = acc_it % C::ACC_STAGES;
-                        const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
-                        ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag);
-                        if (!ok) break;
-                        d_tmem = tmem_base + as * BN;
+                    if (kb == 0) {   // first K block of a tile
+                        // where the tile sits: worked out before the wait, so it runs under the epilogue's drain
                         TileCtx t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur);
                         if constexpr (MODE == GROUP_K) {
                             while (t.nkb == 0) { tile += workers; t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur); }   // expert without tokens
@@ -713,6 +709,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                         // a tile that starts in the middle of a 128-wide scale atom reads its B scales from
                         // the matching TMEM column of the copied atoms (32 columns of B per TMEM column)
                         sfb_skip = (uint32_t)(((t.tn * BN) & 127) >> 5);
+                        // the accumulator must have been drained
+                        as = acc_it % C::ACC_STAGES;
+                        const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
+                        ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag);
+                        if (!ok) break;
+                        d_tmem = tmem_base + as * BN;
                     }
                     ok = warp_wait(full_bar(s), ph, abort_flag);
                     if (!ok) break;
