@@ -97,6 +97,30 @@ int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int64_t cols,
                      void* dst, int dst_dtype, void* stream);
 
 /*
+ * mxfp8_quantize_multi -- mxfp8_quantize of up to MXFP8_QUANTIZE_MULTI_MAX tensors in ONE launch.
+ * A training step casts several tensors at the same point (Sec. 3.2: activations, weights and
+ * gradients each need their MXFP8 copies before the GEMMs that read them); small tensors do not fill
+ * the machine alone, and one launch shares the ramp-up and the tail between them.  The results are
+ * those of separate mxfp8_quantize calls, bit for bit.  (The batching itself has no counterpart in
+ * the paper.)
+ *   items   HOST array of `count` entries: source, shape and the outputs the orientation needs
+ *           (same meaning, layout and alignment as in mxfp8_quantize; device pointers).
+ *   All tensors share src_dtype, orientation, scale_rule, elem and sf_layout.
+ *   Every tensor needs cols % 16 == 0 (ERR_UNSUPPORTED otherwise).
+ */
+#define MXFP8_QUANTIZE_MULTI_MAX 8
+typedef struct mxfp8_quantize_item {
+    const void* src;
+    int64_t rows, cols;
+    void* q_row;
+    void* s_row;
+    void* q_col;
+    void* s_col;
+} mxfp8_quantize_item;
+int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count, int src_dtype,
+                         int orientation, int scale_rule, int elem, int sf_layout, void* stream);
+
+/*
  * mxfp8_fake_quantize -- the MXFP8 round trip in one pass: dst = decode(quantize(src)) in the source's
  * own dtype (BF16 -> MXFP8 -> BF16 is how the paper's accuracy runs emulated MX arithmetic ahead of
  * BF16 GEMMs, Sec. 3.1).  Same block / scale / cast rules and the same special-value handling as
@@ -229,7 +253,8 @@ int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64
  *     FPROP  Y  [T, F] = X  * W^T   (row-blocked X,  row-blocked W)
  *     DGRAD  dX [T, H] = dY * W     (row-blocked dY, column-blocked W)
  *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
- * run as block-scaled GEMMs with BF16 output: six kernel launches on `stream`, no wait.
+ * run as block-scaled GEMMs with BF16 output: four kernel launches on `stream` (the three casts
+ * share one), no wait.
  * T, H, F must be multiples of 128 (ERR_UNSUPPORTED).  ws: device scratch for the quantized
  * copies, mxfp8_linear_ws_bytes() bytes, 256-byte aligned, owned by the caller.  All tensors
  * 16-byte aligned, row-major, dense.

@@ -26,7 +26,7 @@ EXPORTS = (
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
-    "mxfp8_linear", "mxfp8_grouped_gemm",
+    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi",
 )
 
 
@@ -34,6 +34,12 @@ class Mxfp8Error(RuntimeError):
     def __init__(self, status: int, what: str):
         super().__init__("%s failed: %d (%s)" % (what, status, status_string(status)))
         self.status = status
+
+
+class _QuantizeItem(ctypes.Structure):
+    _fields_ = [("src", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("q_row", ctypes.c_void_p), ("s_row", ctypes.c_void_p),
+                ("q_col", ctypes.c_void_p), ("s_col", ctypes.c_void_p)]
 
 
 class _Epilogue(ctypes.Structure):
@@ -80,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
         L.mxfp8_fake_quantize.restype = i
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_quantize_multi.restype = i
+        L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
         L.mxfp8_grouped_gemm.restype = i
         L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
         L.mxfp8_linear_ws_bytes.restype = sz
@@ -245,3 +253,21 @@ def mxfp8_grouped_gemm(aq, a_s, bq, b_s, group_offsets: torch.Tensor, mode: int,
     _check(lib().mxfp8_grouped_gemm(_ptr(aq), _ptr(a_s), _ptr(bq), _ptr(b_s), _ptr(group_offsets),
                                     group_offsets.numel() - 1, mode, M, N, K, b_major, a_elem, b_elem,
                                     _ptr(D), _dtype_code(D), _stream(stream)), "mxfp8_grouped_gemm")
+
+
+def make_quantize_items(entries):
+    """entries: sequence of (src, q_row, s_row, q_col, s_col) tensors (None where unused).  Returns the
+    ctypes array mxfp8_quantize_multi takes; build it once and reuse it while the tensors live."""
+    arr = (_QuantizeItem * len(entries))()
+    for k, (src, q_row, s_row, q_col, s_col) in enumerate(entries):
+        assert src.is_contiguous()
+        arr[k].src = src.data_ptr()
+        arr[k].rows, arr[k].cols = src.shape
+        arr[k].q_row, arr[k].s_row, arr[k].q_col, arr[k].s_col = _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col)
+    return arr
+
+
+def mxfp8_quantize_multi(items, src_dtype: int, orientation: int, scale_rule: int, elem: int, sf_layout: int,
+                         stream=None) -> None:
+    _check(lib().mxfp8_quantize_multi(items, len(items), src_dtype, orientation, scale_rule, elem, sf_layout,
+                                      _stream(stream)), "mxfp8_quantize_multi")

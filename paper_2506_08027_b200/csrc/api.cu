@@ -129,16 +129,17 @@ LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F, bool staging)
     return w;
 }
 
-// The six launches of one step on device buffers: three BOTH-orientation conversions, then
+// The four launches of one step on device buffers: the three BOTH-orientation conversions in one, then
 // FPROP, DGRAD and WGRAD (Sec. 3.2).
 int linear_device(const LinearWs& w, const void* x, const void* wt, const void* dy, int64_t T, int64_t H, int64_t F,
                   int scale_rule, void* y, void* dx, void* dw, void* stream)
 {
     const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
     const void* src[3] = {x, wt, dy};
-    for (int t = 0; t < 3; ++t) {
-        const int rc = mxfp8_quantize(src[t], MXFP8_BF16, shp[t][0], shp[t][1], MXFP8_BOTH, scale_rule, MXFP8_E4M3,
-                                      w.q[t][0], w.s[t][0], w.q[t][1], w.s[t][1], MXFP8_SF_SWIZZLED, stream);
+    mxfp8_quantize_item items[3];
+    for (int t = 0; t < 3; ++t) items[t] = mxfp8_quantize_item{src[t], shp[t][0], shp[t][1], w.q[t][0], w.s[t][0], w.q[t][1], w.s[t][1]};
+    {   // the three casts share one launch
+        const int rc = mxfp8_quantize_multi(items, 3, MXFP8_BF16, MXFP8_BOTH, scale_rule, MXFP8_E4M3, MXFP8_SF_SWIZZLED, stream);
         if (rc != MXFP8_OK) return rc;
     }
     enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };

@@ -25,6 +25,14 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols);
 int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
                         int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
                         int sf_layout, cudaStream_t stream, bool emulate = false);
+// Several tensors of one dtype in one launch (same orientation, rule, element format, scale layout).
+struct QuantizeItem {
+    const void* src;
+    int64_t rows, cols;
+    void *q_row, *s_row, *q_col, *s_col;
+};
+int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
+                       int sf_layout, cudaStream_t stream, bool emulate = false);
 int quantize_read_and_clear_status();
 
 // Device status word (bounded waits report here); defined in gemm.cu.

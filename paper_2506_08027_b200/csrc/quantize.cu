@@ -332,3 +332,33 @@ extern "C" int mxfp8_fake_quantize(const void* src, int src_dtype, int64_t rows,
     return quantize_tma_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, dst_row, nullptr, dst_col, nullptr,
                                MXFP8_SF_SWIZZLED, static_cast<cudaStream_t>(stream), true);
 }
+
+extern "C" int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count, int src_dtype,
+                                    int orientation, int scale_rule, int elem, int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!items) return MXFP8_ERR_NULL;
+    if (count < 1) return MXFP8_ERR_SHAPE;
+    if (count > MXFP8_QUANTIZE_MULTI_MAX) return MXFP8_ERR_UNSUPPORTED;
+    QuantizeItem batch[MXFP8_QUANTIZE_MULTI_MAX];
+    for (int i = 0; i < count; ++i) {
+        const mxfp8_quantize_item& it = items[i];
+        if (!it.src) return MXFP8_ERR_NULL;
+        if ((orientation & MXFP8_ROW) && (!it.q_row || !it.s_row)) return MXFP8_ERR_NULL;
+        if ((orientation & MXFP8_COL) && (!it.q_col || !it.s_col)) return MXFP8_ERR_NULL;
+        if (it.rows <= 0 || it.cols <= 0) return MXFP8_ERR_SHAPE;
+        if ((orientation & MXFP8_ROW) && (it.cols % 32)) return MXFP8_ERR_SHAPE;
+        if ((orientation & MXFP8_COL) && (it.rows % 32)) return MXFP8_ERR_SHAPE;
+        if (!aligned16(it.src)) return MXFP8_ERR_ALIGN;
+        if ((orientation & MXFP8_ROW) && (!aligned16(it.q_row) || !aligned16(it.s_row))) return MXFP8_ERR_ALIGN;
+        if ((orientation & MXFP8_COL) && (!aligned16(it.q_col) || !aligned16(it.s_col))) return MXFP8_ERR_ALIGN;
+        if (!quantize_tma_eligible(src_dtype, it.rows, it.cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
+        batch[i] = QuantizeItem{it.src, it.rows, it.cols, it.q_row, it.s_row, it.q_col, it.s_col};
+    }
+    return quantize_tma_batch(batch, count, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream));
+}

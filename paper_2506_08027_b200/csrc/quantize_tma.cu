@@ -49,6 +49,17 @@ struct QParams {
     uint8_t* s_col;
 };
 
+// One launch converts up to QT_MAX_TENSORS tensors: their tiles are numbered one tensor after the
+// other and dealt out to the CTAs as one pool, so small tensors share one ramp-up and one tail and
+// the per-CTA tile counts even out.
+constexpr int QT_MAX_TENSORS = 8;
+struct QBatch {
+    int count;
+    int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
+    QParams t[QT_MAX_TENSORS];
+};
+struct QMaps { CUtensorMap m[QT_MAX_TENSORS]; };
+
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // 2^(127 - b) and b for a block with this (finite, non-negative) amax bit pattern.
@@ -302,8 +313,8 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
 }
 
 template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
-__global__ void __launch_bounds__(QT_THREADS)
-quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams p)
+__global__ void __launch_bounds__(QT_THREADS, 3)
+quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QBatch batch)
 {
     constexpr bool BF = (DTYPE == MXFP8_BF16);
     constexpr int VEC = BF ? 4 : 2;                 // elements per lane per row
@@ -317,7 +328,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;   // warp = 32-row slab of the tile
-    const uint32_t rule_offset = (p.rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
+    const uint32_t rule_offset = (batch.t[0].rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
 
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
@@ -326,15 +337,18 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
     }
     __syncthreads();
 
-    const int num_tiles = p.tiles_x * p.tiles_y;
+    const int num_tiles = batch.tile_start[batch.count];
+    int load_ti = 0;                          // tensor of the tile being loaded (tiles only move forward)
     auto issue_load = [&](int t, int buf) {   // one thread: tile t -> ring slot buf
+        while (t >= batch.tile_start[load_ti + 1]) ++load_ti;
+        const int lt = t - batch.tile_start[load_ti], tx = batch.t[load_ti].tiles_x;
         const uint32_t b = smem_addr(&bars[buf]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&tmap_src), "r"(b), "r"((t % p.tiles_x) * T_COLS), "r"((t / p.tiles_x) * T_ROWS)
+                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&maps.m[load_ti]), "r"(b), "r"((lt % tx) * T_COLS), "r"((lt / tx) * T_ROWS)
                      : "memory");
     };
-    int tile = blockIdx.x;
+    int tile = blockIdx.x, ti = 0;
     if (tid == 0) {
         if (tile < num_tiles) issue_load(tile, 0);
         if (tile + (int)gridDim.x < num_tiles) issue_load(tile + gridDim.x, 1);
@@ -347,7 +361,10 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap_src, const QParams 
         uint8_t* in_tile = in_ring + buf * IN_BYTES;
         uint8_t* sm_row = sm_scales + buf * 1024;          // [128][4]
         uint8_t* sm_col = sm_row + 512;                    // [T_COLS][4]
-        const int tile_x = tile % p.tiles_x, tile_y = tile / p.tiles_x;
+        while (tile >= batch.tile_start[ti + 1]) ++ti;
+        const QParams& p = batch.t[ti];
+        const int ltile = tile - batch.tile_start[ti];
+        const int tile_x = ltile % p.tiles_x, tile_y = ltile / p.tiles_x;
         const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
 
         // wait for the tile (bounded: on expiry report through the status word and leave)
@@ -481,13 +498,13 @@ int qt_sm_count()
 }
 
 template <int DTYPE, int ELEM, bool R, bool C, bool EMU>
-cudaError_t launch(const CUtensorMap& ms, const QParams& p, cudaStream_t stream)
+cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
 {
     constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
     auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU>;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (err != cudaSuccess) return err;
-    const int tiles = p.tiles_x * p.tiles_y;
+    const int tiles = p.tile_start[p.count];
     const int max_ctas = qt_sm_count() * 3;
     const int grid = tiles < max_ctas ? tiles : max_ctas;
     kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, p);
@@ -496,7 +513,7 @@ cudaError_t launch(const CUtensorMap& ms, const QParams& p, cudaStream_t stream)
 }
 
 template <int DTYPE, int ELEM, bool EMU>
-cudaError_t launch_o(int orientation, const CUtensorMap& ms, const QParams& p, cudaStream_t st)
+cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
     if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU>(ms, p, st);
     if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU>(ms, p, st);
@@ -514,24 +531,35 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
     return tiles < 0x7FFFFFFFLL && rows < 0x7FFFFFFFLL && cols < 0x7FFFFFFFLL && qt_encode_fn() != nullptr;
 }
 
-int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
-                        int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
-                        int sf_layout, cudaStream_t stream, bool emulate)
+int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
+                       int sf_layout, cudaStream_t stream, bool emulate)
 {
+    if (count < 1 || count > QT_MAX_TENSORS) return MXFP8_ERR_UNSUPPORTED;
     const bool bf = src_dtype == MXFP8_BF16;
     const uint32_t t_cols = bf ? 128 : 64;
-    CUtensorMap ms;
-    if (!make_map_2d(&ms, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
-                     const_cast<void*>(src), (uint64_t)cols, (uint64_t)rows, t_cols, T_ROWS))
-        return MXFP8_ERR_CUDA;
-    QParams p{};
-    p.rows = rows; p.cols = cols; p.rule = scale_rule; p.sf_layout = sf_layout;
-    p.tiles_x = (int)((cols + t_cols - 1) / t_cols);
-    p.tiles_y = (int)((rows + T_ROWS - 1) / T_ROWS);
-    p.q_row = static_cast<uint8_t*>(q_row);
-    p.q_col = static_cast<uint8_t*>(q_col);
-    p.s_row = static_cast<uint8_t*>(s_row);
-    p.s_col = static_cast<uint8_t*>(s_col);
+    QMaps ms;
+    QBatch p{};
+    p.count = count;
+    int64_t tiles = 0;
+    for (int i = 0; i < QT_MAX_TENSORS; ++i) {
+        const QuantizeItem& it = items[i < count ? i : 0];   // unused slots repeat the first tensor: every map stays valid
+        if (!make_map_2d(&ms.m[i], bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
+                         const_cast<void*>(it.src), (uint64_t)it.cols, (uint64_t)it.rows, t_cols, T_ROWS))
+            return MXFP8_ERR_CUDA;
+        if (i >= count) continue;
+        QParams& q = p.t[i];
+        q.rows = it.rows; q.cols = it.cols; q.rule = scale_rule; q.sf_layout = sf_layout;
+        q.tiles_x = (int)((it.cols + t_cols - 1) / t_cols);
+        q.tiles_y = (int)((it.rows + T_ROWS - 1) / T_ROWS);
+        q.q_row = static_cast<uint8_t*>(it.q_row);
+        q.q_col = static_cast<uint8_t*>(it.q_col);
+        q.s_row = static_cast<uint8_t*>(it.s_row);
+        q.s_col = static_cast<uint8_t*>(it.s_col);
+        p.tile_start[i] = (int)tiles;
+        tiles += (int64_t)q.tiles_x * q.tiles_y;
+        if (tiles >= 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
+    }
+    for (int i = count; i <= QT_MAX_TENSORS; ++i) p.tile_start[i] = (int)tiles;
     cudaError_t err;
     if (emulate) {
         if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3, true>(orientation, ms, p, stream)
@@ -547,4 +575,14 @@ int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t co
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
+}  // namespace mxfp8
+
+namespace mxfp8 {
+int quantize_tma_device(const void* src, int src_dtype, int64_t rows, int64_t cols, int orientation,
+                        int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col,
+                        int sf_layout, cudaStream_t stream, bool emulate)
+{
+    const QuantizeItem one{src, rows, cols, q_row, s_row, q_col, s_col};
+    return quantize_tma_batch(&one, 1, src_dtype, orientation, scale_rule, elem, sf_layout, stream, emulate);
+}
 }  // namespace mxfp8

@@ -213,3 +213,58 @@ def test_quantize_host_variant():
     assert np.array_equal(host[0].numpy().reshape(rows, cols), wq) and np.array_equal(host[1].numpy().reshape(rows, -1), wsr)
     wq, wsc = orc.quantize(xf, orc.COL)
     assert np.array_equal(host[2].numpy().reshape(rows, cols), wq) and np.array_equal(host[3].numpy().reshape(-1, cols), wsc)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("orientation", [ROW, COL, BOTH])
+def test_quantize_multi_equals_oracle_per_tensor(dtype, orientation):
+    # several tensors of different shapes (ragged tiles, a single-tile tensor) in one launch
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import Guarded, logical_scales_from_swizzled
+    shapes = [(160, 352), (32, 32), (384, 1056), (128, 128), (96, 4096 + 128)]
+    hosts = [as_dtype(synth.draw(synth.DISTRIBUTIONS[i % 4], s, 900 + i), dtype) for i, s in enumerate(shapes)]
+    srcs = [torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(h).cuda()
+            for h in hosts]
+    outs, entries = [], []
+    for (rows, cols), src in zip(shapes, srcs):
+        g = {}
+        for o, name in ((ROW, "row"), (COL, "col")):
+            if orientation & o:
+                g["q_" + name] = Guarded(rows * cols)
+                g["s_" + name] = Guarded(B.mxfp8_scale_bytes(rows, cols, o, SWIZZLED))
+        outs.append(g)
+        v = lambda k: g[k].view if k in g else None
+        entries.append((src, v("q_row"), v("s_row"), v("q_col"), v("s_col")))
+    items = B.make_quantize_items(entries)
+    before = B.mxfp8_launch_count()
+    B.mxfp8_quantize_multi(items, B.BF16 if dtype == "bf16" else B.FP32, orientation, B.RULE_PAPER, B.E4M3, SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_launch_count() - before == 1
+    assert B.mxfp8_device_status() == 0
+    for (rows, cols), h, g in zip(shapes, hosts, outs):
+        x = orc.bf16_bits_to_f32(h) if dtype == "bf16" else h
+        for o, name in ((orc.ROW, "row"), (orc.COL, "col")):
+            if ("q_" + name) not in g:
+                continue
+            g["q_" + name].check(); g["s_" + name].check()
+            wq, ws = orc.quantize(x, o, orc.RULE_PAPER, orc.E4M3)
+            assert_q_equal(g["q_" + name].numpy().reshape(rows, cols), wq, orc.E4M3, "%s %s" % ((rows, cols), name))
+            mn, nkb = (rows, cols // 32) if name == "row" else (cols, rows // 32)
+            logical = logical_scales_from_swizzled(g["s_" + name].numpy(), mn, nkb)
+            assert np.array_equal(logical if name == "row" else logical.T, ws), "scales %s %s" % ((rows, cols), name)
+
+
+def test_quantize_multi_argument_errors():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    x = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    q, s, _, _ = B.alloc_quantize_outputs(64, 64, B.ROW, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):                      # more tensors than one launch takes
+        B.mxfp8_quantize_multi(B.make_quantize_items([(x, q, s, None, None)] * 9), B.BF16, B.ROW, B.RULE_PAPER, B.E4M3, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):                      # missing output
+        B.mxfp8_quantize_multi(B.make_quantize_items([(x, q, None, None, None)]), B.BF16, B.ROW, B.RULE_PAPER, B.E4M3, B.SF_LINEAR)
+    y = torch.zeros(64, 40, dtype=torch.bfloat16, device="cuda")
+    _, _, qc, sc = B.alloc_quantize_outputs(64, 40, B.COL, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):                      # cols % 16 != 0 has no batched path
+        B.mxfp8_quantize_multi(B.make_quantize_items([(y, None, None, qc, sc)]), B.BF16, B.COL, B.RULE_PAPER, B.E4M3, B.SF_LINEAR)
