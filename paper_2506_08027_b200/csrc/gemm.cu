@@ -958,8 +958,8 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
 {
     using C = Cfg<BN, PAIR>;
     auto kernel = gemm_kernel<BN, PAIR, MODE>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_TOTAL) != cudaSuccess)
-        return MXFP8_ERR_CUDA;
+    static unsigned long long smem_set = 0;
+    if (ensure_dynamic_smem(kernel, C::SMEM_TOTAL, smem_set) != cudaSuccess) return MXFP8_ERR_CUDA;
     p.tiles_m = (int)((p.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM));
     p.tiles_n = (int)((p.N + BN - 1) / BN);
     p.stage_tx = (PAIR ? 2u : 1u) * (uint32_t)(C::A_BYTES + (p.b_mn ? C::B_BYTES_MN : C::B_BYTES_K) + 512 + 512 * C::SFB_ATOMS);

@@ -11,6 +11,22 @@ namespace mxfp8 {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Raises a kernel's dynamic shared-memory limit once per (kernel instantiation, device): the call
+// costs several microseconds of host time and its effect lasts for the life of the context.
+// `done` is a bit mask of devices, one static per call site.
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long long& done)
+{
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (__atomic_load_n(&done, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (err == cudaSuccess) __atomic_fetch_or(&done, bit, __ATOMIC_RELEASE);
+    return err;
+}
+
 // Launch accounting (mxfp8_launch_count).
 int64_t launches();
 void count_launch(int n);

@@ -502,7 +502,8 @@ cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
 {
     constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
     auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU>;
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    static unsigned long long smem_set = 0;
+    cudaError_t err = ensure_dynamic_smem(kernel, SMEM, smem_set);
     if (err != cudaSuccess) return err;
     const int tiles = p.tile_start[p.count];
     const int max_ctas = qt_sm_count() * 3;
