@@ -39,8 +39,19 @@
 
 /* Element formats (Table 1 and Sec. 2): E4M3 is 1-4-3 with one NaN pattern and
  * no infinity, max 1.75*2^8, min subnormal 2^-9; E5M2 is 1-5-2 with IEEE
- * specials, max 1.75*2^15, min subnormal 2^-16. */
+ * specials, max 1.75*2^15, min subnormal 2^-16.
+ * The 6- and 4-bit element formats of Table 1 (MXFP6: E2M3, E3M2; MXFP4: E2M1)
+ * have a sign bit, no infinity and no NaN: E2M3 (bias 1) max 1.875*2^2, min
+ * subnormal 2^-3; E3M2 (bias 3) max 1.75*2^4, min subnormal 2^-4 (Table 1
+ * prints 2^-3 there, which no 1-3-2 format with that maximum has; the bias-3
+ * format of the OCP MX specification the paper builds on is taken); E2M1
+ * (bias 1) max 1.5*2^2, min subnormal 2^-1.  A code sits in the low bits of
+ * its byte. */
+#define ORC_E2M3 3
+#define ORC_E3M2 4
+#define ORC_E2M1 5
 typedef struct {
+    int ebits;       /* exponent bits                                  */
     int mbits;       /* mantissa bits                                  */
     int bias;        /* exponent bias                                  */
     int emin;        /* exponent of the smallest normal                */
@@ -54,10 +65,19 @@ static orc_fmt orc_format(int elem)
 {
     orc_fmt f;
     if (elem == ORC_E5M2) {
-        f.mbits = 2; f.bias = 15; f.emin = -14; f.emax = 15;
+        f.ebits = 5; f.mbits = 2; f.bias = 15; f.emin = -14; f.emax = 15;
         f.destmax = 57344.0; f.max_code = 0x7B; f.nan_code = 0x7F;
+    } else if (elem == ORC_E2M3) {
+        f.ebits = 2; f.mbits = 3; f.bias = 1; f.emin = 0; f.emax = 2;
+        f.destmax = 7.5; f.max_code = 0x1F; f.nan_code = 0x1F;     /* no NaN: see orc_fp8_encode */
+    } else if (elem == ORC_E3M2) {
+        f.ebits = 3; f.mbits = 2; f.bias = 3; f.emin = -2; f.emax = 4;
+        f.destmax = 28.0; f.max_code = 0x1F; f.nan_code = 0x1F;
+    } else if (elem == ORC_E2M1) {
+        f.ebits = 2; f.mbits = 1; f.bias = 1; f.emin = 0; f.emax = 2;
+        f.destmax = 6.0; f.max_code = 0x07; f.nan_code = 0x07;
     } else {
-        f.mbits = 3; f.bias = 7; f.emin = -6; f.emax = 8;
+        f.ebits = 4; f.mbits = 3; f.bias = 7; f.emin = -6; f.emax = 8;
         f.destmax = 448.0; f.max_code = 0x7E; f.nan_code = 0x7F;
     }
     return f;
@@ -67,15 +87,17 @@ static orc_fmt orc_format(int elem)
 double orc_fp8_decode(int code, int elem)
 {
     orc_fmt f = orc_format(elem);
-    int sign = (code >> 7) & 1;
-    int efield = (code & 0x7F) >> f.mbits;
-    int mfield = code & ((1 << f.mbits) - 1);
+    int sbit = f.ebits + f.mbits;                         /* position of the sign bit */
+    int sign = (code >> sbit) & 1;
+    int mag = code & ((1 << sbit) - 1);                   /* bits above the sign are ignored */
+    int efield = mag >> f.mbits;
+    int mfield = mag & ((1 << f.mbits) - 1);
     double v;
     if (elem == ORC_E4M3) {
-        if ((code & 0x7F) == 0x7F) return NAN;           /* the single NaN pattern */
-    } else {
+        if (mag == 0x7F) return NAN;                      /* the single NaN pattern */
+    } else if (elem == ORC_E5M2) {
         if (efield == 31) return mfield ? NAN : (sign ? -INFINITY : INFINITY);
-    }
+    }                                                     /* the 6- and 4-bit formats have no specials */
     if (efield == 0)
         v = ldexp((double)mfield, f.emin - f.mbits);      /* subnormal: 0.m * 2^emin */
     else
@@ -85,15 +107,18 @@ double orc_fp8_decode(int code, int elem)
 
 /* Quantize_to_fp8 (Sec. 3.3, App. A.2): round-to-nearest-ties-to-even onto the
  * element grid, subnormals included, then saturate: magnitudes above destmax
- * (infinity too) become +-destmax.  NaN stays NaN.  The sign of zero and of
- * values that round to zero is kept. */
+ * (infinity too) become +-destmax.  NaN stays NaN where the format has one; the
+ * 6- and 4-bit formats have none and the paper does not say what a NaN element
+ * becomes there: this oracle emits +destmax (the saturating hardware convert's
+ * choice), parity unpinned for that case.  The sign of zero and of values that
+ * round to zero is kept. */
 int orc_fp8_encode(double x, int elem)
 {
     orc_fmt f = orc_format(elem);
     int sign, code, ex;
     double a, k;
     if (isnan(x)) return f.nan_code;
-    sign = signbit(x) ? 0x80 : 0;
+    sign = signbit(x) ? (1 << (f.ebits + f.mbits)) : 0;
     a = fabs(x);
     if (a >= f.destmax) return sign | f.max_code;
     if (a < ldexp(1.0, f.emin)) {
@@ -178,7 +203,7 @@ int orc_quantize(const float *src, int64_t rows, int64_t cols, int orientation,
                     double x = (double)v[i];
                     int code;
                     if (isnan(x)) code = f.nan_code;
-                    else if (isinf(x)) code = (x < 0 ? 0x80 : 0) | f.max_code;
+                    else if (isinf(x)) code = (x < 0 ? (1 << (f.ebits + f.mbits)) : 0) | f.max_code;
                     else code = orc_fp8_encode(ldexp(x, -(b - 127)), elem);   /* V_i / X */
                     q[r * cols + cb * 32 + i] = (uint8_t)code;
                 }
@@ -194,7 +219,7 @@ int orc_quantize(const float *src, int64_t rows, int64_t cols, int orientation,
                     double x = (double)v[(int64_t)i * cols];
                     int code;
                     if (isnan(x)) code = f.nan_code;
-                    else if (isinf(x)) code = (x < 0 ? 0x80 : 0) | f.max_code;
+                    else if (isinf(x)) code = (x < 0 ? (1 << (f.ebits + f.mbits)) : 0) | f.max_code;
                     else code = orc_fp8_encode(ldexp(x, -(b - 127)), elem);
                     q[(rb * 32 + i) * cols + c] = (uint8_t)code;
                 }

@@ -15,6 +15,7 @@ import threading
 import numpy as np
 
 E4M3, E5M2 = 0, 1
+E2M3, E3M2, E2M1 = 3, 4, 5      # the 6- and 4-bit element formats of Table 1
 RULE_PAPER, RULE_OCP = 0, 1
 ROW, COL = 1, 2
 

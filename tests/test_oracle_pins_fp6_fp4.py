@@ -1,0 +1,162 @@
+"""Pins of the oracle's 6- and 4-bit element formats (Table 1: MXFP6 E2M3 / E3M2, MXFP4 E2M1):
+the printed constants, a library's decode tables and casts, exact-rational nearest search, ties,
+saturation, and the two scale rules against their exact definitions."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle as orc
+
+FMT = {
+    orc.E2M3: dict(bits=6, destmax=7.5, min_sub=2.0 ** -3, emax=2, name="float6_e2m3fn"),
+    orc.E3M2: dict(bits=6, destmax=28.0, min_sub=2.0 ** -4, emax=4, name="float6_e3m2fn"),
+    orc.E2M1: dict(bits=4, destmax=6.0, min_sub=2.0 ** -1, emax=2, name="float4_e2m1fn"),
+}
+ELEMS = list(FMT)
+
+
+def codes(elem, signed=True):
+    n = 1 << FMT[elem]["bits"]
+    return range(n if signed else n // 2)
+
+
+def test_table1_constants():
+    # Table 1: maximum normal 1.875*2^2, 1.75*2^4, 1.5*2^2; minimum subnormal 2^-3 (E2M3), 2^-1 (E2M1).
+    # E3M2: the table prints 2^-3; the bias-3 format with that maximum has 2^-4 (reading stated in the oracle).
+    assert FMT[orc.E2M3]["destmax"] == 1.875 * 2 ** 2 and FMT[orc.E3M2]["destmax"] == 1.75 * 2 ** 4
+    assert FMT[orc.E2M1]["destmax"] == 1.5 * 2 ** 2
+    for elem, f in FMT.items():
+        vals = [orc.fp8_decode(c, elem) for c in codes(elem, signed=False)]
+        assert all(math.isfinite(v) for v in vals)                # no Inf, no NaN
+        assert max(vals) == f["destmax"]
+        assert min(v for v in vals if v > 0) == f["min_sub"]
+        assert vals == sorted(vals) and len(set(vals)) == len(vals)
+        half = 1 << (f["bits"] - 1)
+        for c in codes(elem, signed=False):                        # sign bit mirrors the value
+            assert orc.fp8_decode(c | half, elem) == -vals[c] or (vals[c] == 0 and math.copysign(1, orc.fp8_decode(c | half, elem)) == -1)
+    # dynamic range in binades as Table 1 lists them: log2(max / min subnormal)
+    assert round(math.log2(7.5 / 2 ** -3), 1) == 5.9
+    assert round(math.log2(6.0 / 2 ** -1), 1) == 3.6
+    assert round(math.log2(28.0 / 2 ** -4), 1) == 8.8     # 8.8 binades fit 2^-4, not the printed 2^-3 (that gives 7.8)
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_decode_matches_library_tables(elem):
+    import ml_dtypes
+    dt = getattr(ml_dtypes, FMT[elem]["name"])
+    n = 1 << FMT[elem]["bits"]
+    lib = np.arange(n, dtype=np.uint8).view(dt).astype(np.float64)
+    mine = np.array([orc.fp8_decode(c, elem) for c in range(n)])
+    assert np.array_equal(lib, mine)
+    assert np.array_equal(np.signbit(lib), np.signbit(mine))
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_encode_roundtrip_and_ties(elem):
+    half = 1 << (FMT[elem]["bits"] - 1)
+    pos = list(codes(elem, signed=False))
+    for c in codes(elem):
+        assert orc.fp8_encode(orc.fp8_decode(c, elem), elem) == c
+    for lo, hi in zip(pos[:-1], pos[1:]):
+        a, b = orc.fp8_decode(lo, elem), orc.fp8_decode(hi, elem)
+        mid = (a + b) / 2
+        even = lo if lo % 2 == 0 else hi
+        assert orc.fp8_encode(mid, elem) == even
+        assert orc.fp8_encode(-mid, elem) == (even | half)
+        assert orc.fp8_encode(math.nextafter(mid, 0.0), elem) == lo
+        assert orc.fp8_encode(math.nextafter(mid, math.inf), elem) == hi
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_encode_is_nearest_by_exact_search_and_saturates(elem):
+    rng = np.random.default_rng(5)
+    f = FMT[elem]
+    half = 1 << (f["bits"] - 1)
+    finite = [(c, Fraction(orc.fp8_decode(c, elem))) for c in codes(elem, signed=False)]
+    xs = np.concatenate([rng.standard_normal(400) * s for s in (0.05, 1.0, f["destmax"] / 2, f["destmax"] * 2)])
+    for x in xs.astype(np.float32):
+        fx = abs(Fraction(float(x)))
+        got = orc.fp8_encode(float(x), elem)
+        assert (got >> (f["bits"] - 1)) == int(np.signbit(x))
+        if fx >= Fraction(f["destmax"]):
+            assert (got & (half - 1)) == half - 1                  # saturates to the largest magnitude
+        else:
+            best = min(abs(fx - v) for _, v in finite)
+            assert abs(fx - Fraction(orc.fp8_decode(got & (half - 1), elem))) == best
+    for x in (f["destmax"], f["destmax"] * 1.01, 1e30, math.inf):
+        assert orc.fp8_encode(x, elem) == half - 1 and orc.fp8_encode(-x, elem) == (2 * half - 1)
+    assert orc.fp8_encode(0.0, elem) == 0 and orc.fp8_encode(-0.0, elem) == half
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_encode_matches_library_cast_in_range(elem):
+    import ml_dtypes
+    dt = getattr(ml_dtypes, FMT[elem]["name"])
+    top = FMT[elem]["destmax"]
+    rng = np.random.default_rng(13)
+    x = np.concatenate([rng.uniform(-top, top, 5000), rng.standard_normal(3000) * 0.3]).astype(np.float32)
+    x = x[np.abs(x) <= top]
+    mine = np.array([orc.fp8_encode(float(v), elem) for v in x], dtype=np.uint8)
+    lib = x.astype(dt).view(np.uint8)
+    assert np.array_equal(mine, lib)
+
+
+def paper_byte_exact(amax: Fraction, destmax: Fraction) -> int:
+    # smallest n in [-127, 127] with amax <= destmax * 2^n  (Algorithm 1, order of App. A.1)
+    for n in range(-127, 128):
+        if amax <= destmax * Fraction(2) ** n:
+            return n + 127
+    return 254
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_scale_rules_match_exact_definition_and_never_overflow(elem):
+    rng = np.random.default_rng(3)
+    f = FMT[elem]
+    top = Fraction(f["destmax"])
+    amaxes = np.concatenate([
+        np.exp2(rng.uniform(-140, 127, 1500)),
+        np.float32(f["destmax"]) * np.exp2(rng.integers(-100, 100, 300)).astype(np.float32),     # exactly destmax * 2^k
+        np.nextafter(np.float32(f["destmax"]) * np.exp2(rng.integers(-100, 100, 300)).astype(np.float32), np.float32(np.inf)),
+        [0.0, 2.0 ** -149, 2.0 ** -126, 3.0e38],
+    ]).astype(np.float32)
+    for a in amaxes:
+        fa = Fraction(float(a))
+        b = orc.scale_byte(a, elem, orc.RULE_PAPER)
+        assert b == paper_byte_exact(fa, top)
+        assert fa / Fraction(2) ** (b - 127) <= top                       # the block maximum fits the element range
+        bo = orc.scale_byte(a, elem, orc.RULE_OCP)
+        want = -127 if a == 0 else max(-127, min(127, math.floor(math.log2(fa)) - f["emax"]))
+        if a != 0 and Fraction(2) ** math.floor(math.log2(fa)) > fa:      # float log2 rounded up across a power of two
+            want -= 1
+        assert bo == want + 127
+        assert b in (bo, bo + 1)                                          # rounding up adds at most one step
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_quantize_dequantize_blocks_bruteforce(elem):
+    # every output of the tensor routine equals the scalar pieces applied block by block
+    rng = np.random.default_rng(23)
+    x = (rng.standard_normal((64, 96)) * np.exp2(rng.integers(-12, 12, (64, 1)))).astype(np.float32)
+    x[3, 0:32] = 0.0
+    for o in (orc.ROW, orc.COL):
+        q, s = orc.quantize(x, o, orc.RULE_PAPER, elem)
+        assert q.max() < (1 << FMT[elem]["bits"])                         # code in the low bits of its byte
+        d = orc.dequantize_f64(q, s, o, elem)
+        for r, c in ((0, 0), (3, 5), (17, 40), (63, 95), (32, 64)):
+            blk = x[r, (c // 32) * 32:(c // 32 + 1) * 32] if o == orc.ROW else x[(r // 32) * 32:(r // 32 + 1) * 32, c]
+            b = orc.scale_byte(np.abs(blk).max(), elem, orc.RULE_PAPER)
+            sb = s[r, c // 32] if o == orc.ROW else s[r // 32, c]
+            assert sb == b
+            code = orc.fp8_encode(math.ldexp(float(x[r, c]), -(b - 127)), elem)
+            assert q[r, c] == code
+            assert d[r, c] == math.ldexp(orc.fp8_decode(code, elem), b - 127)
+        # the block maximum survives within half a unit in the last place of the format
+        rel = np.abs(d - x) / np.maximum(np.abs(x), 1e-30)
+        amax_pos = np.abs(x) == (np.abs(x).reshape(64, 3, 32).max(axis=2, keepdims=True).repeat(32, axis=2).reshape(64, 96)
+                                 if o == orc.ROW else
+                                 np.abs(x).reshape(2, 32, 96).max(axis=1, keepdims=True).repeat(32, axis=1).reshape(64, 96))
+        mbits = {orc.E2M3: 3, orc.E3M2: 2, orc.E2M1: 1}[elem]
+        assert (rel[amax_pos & (x != 0)] <= 2.0 ** -(mbits + 1)).all()
