@@ -17,6 +17,7 @@ FP32, BF16 = 0, 1
 ROW, COL, BOTH = 1, 2, 3
 RULE_PAPER, RULE_OCP = 0, 1
 E4M3, E5M2 = 0, 1
+E2M3, E3M2, E2M1 = 3, 4, 5          # MXFP6 / MXFP4 elements: conversion kernels only
 SF_LINEAR, SF_SWIZZLED = 0, 1
 K_MAJOR, MN_MAJOR = 0, 1
 ERR_DEVICE_TIMEOUT, ERR_DEVICE_ARGS = -7, -9

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxfp8.so")
-SOURCES = ["quantize.cu", "quantize_tma.cu", "dequantize.cu", "gemm.cu", "api.cu"]
+SOURCES = ["quantize.cu", "quantize_tma.cu", "quantize_tma_fp6_fp4.cu", "dequantize.cu", "gemm.cu", "api.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC",
@@ -25,15 +25,31 @@ def _stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile with nvcc if the library is missing or older than its sources."""
+    """Compile with nvcc if the library is missing or older than its sources: one object file
+    per source (in parallel), then one link."""
     if not (force or _stale()):
         return LIB
+    from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".%d.tmp" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
+    objdir = os.path.join(HERE, ".obj.%d" % os.getpid())
+    os.makedirs(objdir, exist_ok=True)
+    compile_flags = [f for f in NVCC_FLAGS if f != "-shared"] + (["-Xptxas", "-v"] if verbose else [])
+
+    def compile_one(src):
+        obj = os.path.join(objdir, src + ".o")
+        subprocess.check_call([nvcc] + compile_flags + ["-c", os.path.join(CSRC, src), "-o", obj])
+        return obj
+
+    try:
+        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+            objs = list(pool.map(compile_one, SOURCES))
+        tmp = LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs)
+        os.replace(tmp, LIB)
+    finally:
+        for f in os.listdir(objdir):
+            os.remove(os.path.join(objdir, f))
+        os.rmdir(objdir)
     return LIB
 
 

@@ -179,7 +179,7 @@ extern "C" int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int6
 {
     using namespace mxfp8;
     if (orientation != MXFP8_ROW && orientation != MXFP8_COL) return MXFP8_ERR_ENUM;
-    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
     if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
     if (dst_dtype != MXFP8_FP32 && dst_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!q || !s || !dst) return MXFP8_ERR_NULL;
@@ -190,11 +190,19 @@ extern "C" int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int6
     const uint8_t* ss = static_cast<const uint8_t*>(s);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t err;
-    if (elem == MXFP8_E4M3)
-        err = dst_dtype == MXFP8_FP32 ? launch_o<MXFP8_E4M3, MXFP8_FP32>(orientation, qq, ss, rows, cols, sf_layout, dst, st)
-                                      : launch_o<MXFP8_E4M3, MXFP8_BF16>(orientation, qq, ss, rows, cols, sf_layout, dst, st);
-    else
-        err = dst_dtype == MXFP8_FP32 ? launch_o<MXFP8_E5M2, MXFP8_FP32>(orientation, qq, ss, rows, cols, sf_layout, dst, st)
-                                      : launch_o<MXFP8_E5M2, MXFP8_BF16>(orientation, qq, ss, rows, cols, sf_layout, dst, st);
+#define MXFP8_ELEM_CASE(E)                                                                                               \
+    case E:                                                                                                               \
+        err = dst_dtype == MXFP8_FP32 ? launch_o<E, MXFP8_FP32>(orientation, qq, ss, rows, cols, sf_layout, dst, st)     \
+                                      : launch_o<E, MXFP8_BF16>(orientation, qq, ss, rows, cols, sf_layout, dst, st);    \
+        break;
+    switch (elem) {
+        MXFP8_ELEM_CASE(MXFP8_E4M3)
+        MXFP8_ELEM_CASE(MXFP8_E5M2)
+        MXFP8_ELEM_CASE(MXFP8_E2M3)
+        MXFP8_ELEM_CASE(MXFP8_E3M2)
+        MXFP8_ELEM_CASE(MXFP8_E2M1)
+        default: err = cudaErrorInvalidValue;
+    }
+#undef MXFP8_ELEM_CASE
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }

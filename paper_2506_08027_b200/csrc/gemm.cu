@@ -364,7 +364,7 @@ __device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams
                                        const CUtensorMap* map_col, uint32_t buf, uint32_t row_off, uint32_t sw, int lane,
                                        int row0, int col0)
 {
-    const uint32_t rule_offset = (p.epi_rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
+    const uint32_t rule_offset = (p.epi_rule == MXFP8_RULE_PAPER) ? paper_offset<ELEM>() : 0u;
     const int row = row0 + lane;
     if (p.epi_orient & MXFP8_ROW) {
         const int64_t nkb = p.N >> 5;
@@ -1010,15 +1010,16 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     (void)workspace; (void)workspace_bytes;
     if (a_major != MXFP8_K_MAJOR && a_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
     if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
-    if (a_elem != MXFP8_E4M3 && a_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
-    if (b_elem != MXFP8_E4M3 && b_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(a_elem) || !valid_elem(b_elem)) return MXFP8_ERR_ENUM;
+    if (!fp8_elem(a_elem) || !fp8_elem(b_elem)) return MXFP8_ERR_UNSUPPORTED;   // 6- and 4-bit operands need the packed tensor-core layout
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs) return MXFP8_ERR_NULL;
     if (!D && !epi) return MXFP8_ERR_NULL;
     if (epi) {
         if (epi->orientation < MXFP8_ROW || epi->orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
         if (epi->scale_rule != MXFP8_RULE_PAPER && epi->scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
-        if (epi->elem != MXFP8_E4M3 && epi->elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+        if (!valid_elem(epi->elem)) return MXFP8_ERR_ENUM;
+        if (!fp8_elem(epi->elem)) return MXFP8_ERR_UNSUPPORTED;
         if ((epi->orientation & MXFP8_ROW) && (!epi->q_row || !epi->s_row)) return MXFP8_ERR_NULL;
         if ((epi->orientation & MXFP8_COL) && (!epi->q_col || !epi->s_col)) return MXFP8_ERR_NULL;
         if ((epi->orientation & MXFP8_ROW) && (!aligned16(epi->q_row) || !aligned16(epi->s_row))) return MXFP8_ERR_ALIGN;
@@ -1105,8 +1106,8 @@ extern "C" int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq
     using namespace mxfp8;
     if (mode != MXFP8_GROUP_M && mode != MXFP8_GROUP_K) return MXFP8_ERR_ENUM;
     if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
-    if (a_elem != MXFP8_E4M3 && a_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
-    if (b_elem != MXFP8_E4M3 && b_elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(a_elem) || !valid_elem(b_elem)) return MXFP8_ERR_ENUM;
+    if (!fp8_elem(a_elem) || !fp8_elem(b_elem)) return MXFP8_ERR_UNSUPPORTED;   // 6- and 4-bit operands need the packed tensor-core layout
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs || !group_offsets || !D) return MXFP8_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || num_groups <= 0) return MXFP8_ERR_SHAPE;

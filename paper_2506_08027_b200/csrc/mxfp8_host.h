@@ -10,6 +10,9 @@
 namespace mxfp8 {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// element types of the conversion kernels (Table 1) / of the tensor-core path of this library
+inline bool valid_elem(int e) { return e == MXFP8_E4M3 || e == MXFP8_E5M2 || e == MXFP8_E2M3 || e == MXFP8_E3M2 || e == MXFP8_E2M1; }
+inline bool fp8_elem(int e) { return e == MXFP8_E4M3 || e == MXFP8_E5M2; }
 
 // Raises a kernel's dynamic shared-memory limit once per (kernel instantiation, device): the call
 // costs several microseconds of host time and its effect lasts for the life of the context.

@@ -270,15 +270,21 @@ int quantize_device(const void* src, int src_dtype, int64_t rows, int64_t cols, 
     cudaError_t err;
     uint8_t *qr = static_cast<uint8_t*>(q_row), *sr = static_cast<uint8_t*>(s_row);
     uint8_t *qc = static_cast<uint8_t*>(q_col), *sc = static_cast<uint8_t*>(s_col);
-    if (src_dtype == MXFP8_BF16) {
-        err = (elem == MXFP8_E4M3)
-                  ? launch_quantize<MXFP8_BF16, MXFP8_E4M3>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream)
-                  : launch_quantize<MXFP8_BF16, MXFP8_E5M2>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream);
-    } else {
-        err = (elem == MXFP8_E4M3)
-                  ? launch_quantize<MXFP8_FP32, MXFP8_E4M3>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream)
-                  : launch_quantize<MXFP8_FP32, MXFP8_E5M2>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream);
+#define MXFP8_ELEM_CASE(E)                                                                                                        \
+    case E:                                                                                                                        \
+        err = src_dtype == MXFP8_BF16                                                                                              \
+                  ? launch_quantize<MXFP8_BF16, E>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream)   \
+                  : launch_quantize<MXFP8_FP32, E>(src, rows, cols, orientation, scale_rule, sf_layout, qr, sr, qc, sc, stream);  \
+        break;
+    switch (elem) {
+        MXFP8_ELEM_CASE(MXFP8_E4M3)
+        MXFP8_ELEM_CASE(MXFP8_E5M2)
+        MXFP8_ELEM_CASE(MXFP8_E2M3)
+        MXFP8_ELEM_CASE(MXFP8_E3M2)
+        MXFP8_ELEM_CASE(MXFP8_E2M1)
+        default: err = cudaErrorInvalidValue;
     }
+#undef MXFP8_ELEM_CASE
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
@@ -293,7 +299,7 @@ extern "C" int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int6
     if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
     if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
-    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
     if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
     if (!src) return MXFP8_ERR_NULL;
     if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
@@ -319,7 +325,7 @@ extern "C" int mxfp8_fake_quantize(const void* src, int src_dtype, int64_t rows,
     if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
     if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
-    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
     if (!src) return MXFP8_ERR_NULL;
     if ((orientation & MXFP8_ROW) && !dst_row) return MXFP8_ERR_NULL;
     if ((orientation & MXFP8_COL) && !dst_col) return MXFP8_ERR_NULL;
@@ -340,7 +346,7 @@ extern "C" int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count,
     if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
     if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
-    if (elem != MXFP8_E4M3 && elem != MXFP8_E5M2) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
     if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
     if (!items) return MXFP8_ERR_NULL;
     if (count < 1) return MXFP8_ERR_SHAPE;

@@ -1,23 +1,6 @@
-// Fast path of mxfp8_quantize: TMA in, math, coalesced stores out (Sec. 3.2 / 3.3, Algorithm 1,
-// App. A.1-A.2).
-//
-// The generic kernel in quantize.cu spends most of its issue slots on global address
-// arithmetic and predicates.  Here a CTA owns tiles of 128 rows x 256 bytes (128 BF16 or 64 FP32
-// columns).  TMA tensor loads bring them into a two-deep shared-memory ring (ragged edges are
-// zero-filled by the hardware, the next tile is in flight while the current one is processed),
-// the arithmetic reads shared memory at compile-time offsets, and the FP8 bytes go straight to
-// global memory: every warp store covers 128 (BF16) or 64 (FP32) contiguous bytes of one row.
-//
-//   warp w owns rows 32w .. 32w+31 of the tile; lane l owns 8 bytes (4 BF16 / 2 FP32) of every row
-//   pass A (column blocks): amax down the 32 rows inside the lane, packed bf16x2 max for BF16
-//   pass B (row blocks)   : amax across the lanes of a 32-column block by xor-shuffles; BF16 rows
-//                           go through the shuffles two at a time (one in each half of a register)
-//   scale: integer form of Algorithm 1 / App. A.1 on the amax bit pattern (see mxfp8_device.cuh)
-//   cast : x * 2^-e in FP32 (exact), cvt.rn.satfinite to e4m3x2 / e5m2x2
-#include <cuda.h>
-
-#include "mxfp8_device.cuh"
-#include "mxfp8_host.h"
+// Host side of the TMA fast path of mxfp8_quantize (kernels: quantize_tma_kernel.cuh) and the
+// kernels of the two 8-bit element types; the 6- and 4-bit ones are compiled in quantize_tma_fp6_fp4.cu.
+#include "quantize_tma_kernel.cuh"
 
 namespace mxfp8 {
 
@@ -31,430 +14,11 @@ int quantize_read_and_clear_status()
     return h == 0 ? MXFP8_OK : MXFP8_ERR_DEVICE_TIMEOUT;
 }
 
+// defined in quantize_tma_fp6_fp4.cu (opaque pointers: the batch types live in an unnamed namespace)
+cudaError_t quantize_tma_launch_fp6_fp4(int elem, bool bf16_src, int orientation, bool emulate, const void* maps,
+                                        const void* batch, cudaStream_t st);
+
 namespace {
-
-constexpr int T_ROWS = 128;
-constexpr int T_BYTES = 256;                 // source bytes per tile row
-constexpr int IN_BYTES = T_ROWS * T_BYTES;   // 32 KB
-constexpr int QT_THREADS = 128;
-constexpr uint64_t QT_WAIT_LIMIT_NS = 1000000000ull;
-
-struct QParams {
-    int64_t rows, cols;
-    int rule, sf_layout;
-    int tiles_x, tiles_y;
-    uint8_t* q_row;
-    uint8_t* q_col;
-    uint8_t* s_row;
-    uint8_t* s_col;
-};
-
-// One launch converts up to QT_MAX_TENSORS tensors: their tiles are numbered one tensor after the
-// other and dealt out to the CTAs as one pool, so small tensors share one ramp-up and one tail and
-// the per-CTA tile counts even out.
-constexpr int QT_MAX_TENSORS = 8;
-struct QBatch {
-    int count;
-    int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
-    QParams t[QT_MAX_TENSORS];
-};
-struct QMaps { CUtensorMap m[QT_MAX_TENSORS]; };
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// 2^(127 - b) and b for a block with this (finite, non-negative) amax bit pattern.
-//   rule_offset = 0x1FFFFF (paper: a mantissa above 1.75 carries into the exponent = round up)
-//               = 0        (ocp: floor)
-//   e' = biased exponent after the carry; b = max(e' - emax, 0); 1/X has exponent field 254 - b.
-template <int ELEM>
-__device__ __forceinline__ uint32_t inv_exp_field(uint32_t amax_bits, uint32_t rule_offset)
-{
-    const int e = (int)((amax_bits + rule_offset) >> 23);
-    return (uint32_t)min(254 + ElemTraits<ELEM>::emax - e, 254);
-}
-
-__device__ __forceinline__ uint32_t hmax2_abs(uint32_t a, uint32_t b)
-{
-    const __nv_bfloat162 x = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&a));
-    const __nv_bfloat162 y = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&b));
-    const __nv_bfloat162 m = __hmax2(x, y);   // NaN operands are ignored (maxNum)
-    return *reinterpret_cast<const uint32_t*>(&m);
-}
-__device__ __forceinline__ uint32_t hmax2(uint32_t a, uint32_t b)
-{
-    const __nv_bfloat162 m = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
-    return *reinterpret_cast<const uint32_t*>(&m);
-}
-// flags a packed pair of bf16 magnitudes if either half is Inf or NaN
-__device__ __forceinline__ uint32_t nonfinite2(uint32_t z) { return (z + 0x00800080u) & 0x80008000u; }
-
-// X = 2^(b-127) as FP32 from the exponent field of 1/X (b = 254 - field; b = 0 is the subnormal 2^-127)
-__device__ __forceinline__ float scale_from_inv(float inv)
-{
-    const uint32_t b = 254u - (__float_as_uint(inv) >> 23);
-    return __uint_as_float(b ? (b << 23) : 0x00400000u);
-}
-
-// One lane's VEC elements of one row: cast x * inv to FP8 and store the codes (EMU = false), or store
-// the decoded values code * X in the source's own dtype (EMU = true: the MXFP8 round trip the paper's
-// Hopper runs used, Sec. 3.1).  The decoded product is exact in FP32; BF16 output is one RNE of it.
-template <int ELEM, int VEC, bool EMU>
-__device__ __forceinline__ void emit(uint8_t* dst, const float (&x)[VEC], const float (&inv)[VEC], const float (&xs)[VEC])
-{
-    if constexpr (VEC == 4) {
-        const uint32_t c = cvt_fp8x4<ELEM>(x[0] * inv[0], x[1] * inv[1], x[2] * inv[2], x[3] * inv[3]);
-        if constexpr (!EMU) {
-            *reinterpret_cast<uint32_t*>(dst) = c;
-        } else {
-            const float2 lo = fp8x2_to_float2<ELEM>(c & 0xFFFFu), hi = fp8x2_to_float2<ELEM>(c >> 16);
-            const __nv_bfloat162 a = __floats2bfloat162_rn(lo.x * xs[0], lo.y * xs[1]);
-            const __nv_bfloat162 b = __floats2bfloat162_rn(hi.x * xs[2], hi.y * xs[3]);
-            *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
-        }
-    } else {
-        const uint32_t c = cvt_fp8x2<ELEM>(x[0] * inv[0], x[1] * inv[1]);
-        if constexpr (!EMU) {
-            *reinterpret_cast<uint16_t*>(dst) = (uint16_t)c;
-        } else {
-            const float2 f = fp8x2_to_float2<ELEM>(c);
-            *reinterpret_cast<float2*>(dst) = make_float2(f.x * xs[0], f.y * xs[1]);
-        }
-    }
-}
-
-// One 32-row slab, fast path: every element finite (checked at the end; the caller reruns the
-// slab through slab_careful otherwise), all rows and columns inside the tensor.  Returns
-// whether any lane of the warp met an Inf / NaN.
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
-__device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
-                                          uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
-                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset)
-{
-    constexpr bool BF = (DTYPE == MXFP8_BF16);
-    constexpr int VEC = BF ? 4 : 2;
-    constexpr int LPB = 32 / VEC;
-    uint32_t bad = 0u;
-    float col_inv[VEC], col_xs[VEC];
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) { col_inv[i] = 1.f; col_xs[i] = 1.f; }
-    if (DO_COL) {
-        uint32_t cbits[VEC];
-        if constexpr (BF) {
-            uint32_t m0 = 0u, m1 = 0u;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-                m0 = hmax2_abs(m0, w.x);
-                m1 = hmax2_abs(m1, w.y);
-            }
-            bad |= nonfinite2(m0) | nonfinite2(m1);
-            cbits[0] = m0 << 16; cbits[1] = m0 & 0xFFFF0000u;
-            cbits[2] = m1 << 16; cbits[3] = m1 & 0xFFFF0000u;
-        } else {
-            float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-                a0 = fmaxf(a0, fabsf(w.x));
-                a1 = fmaxf(a1, fabsf(w.y));
-            }
-            bad |= (uint32_t)(a0 == INFINITY) | (uint32_t)(a1 == INFINITY);
-            cbits[0] = __float_as_uint(a0);
-            cbits[1] = __float_as_uint(a1);
-        }
-#pragma unroll
-        for (int i = 0; i < VEC; ++i) {
-            const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
-            col_inv[i] = __uint_as_float(ie << 23);
-            col_xs[i] = scale_from_inv(col_inv[i]);
-            my_sm_col[i * 4] = (uint8_t)(254u - ie);
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < 32; j += 2) {
-        float x0[VEC], x1[VEC];
-        float inv0 = 1.f, inv1 = 1.f;
-        if constexpr (BF) {
-            const uint2 w0 = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-            const uint2 w1 = *reinterpret_cast<const uint2*>(my_in + (j + 1) * T_BYTES);
-            x0[0] = __uint_as_float(w0.x << 16); x0[1] = __uint_as_float(w0.x & 0xFFFF0000u);
-            x0[2] = __uint_as_float(w0.y << 16); x0[3] = __uint_as_float(w0.y & 0xFFFF0000u);
-            x1[0] = __uint_as_float(w1.x << 16); x1[1] = __uint_as_float(w1.x & 0xFFFF0000u);
-            x1[2] = __uint_as_float(w1.y << 16); x1[3] = __uint_as_float(w1.y & 0xFFFF0000u);
-            if (DO_ROW) {
-                const uint32_t m0 = hmax2_abs(w0.x, w0.y);               // row j  : (max |e0|,|e2| ; max |e1|,|e3|)
-                const uint32_t m1 = hmax2_abs(w1.x, w1.y);               // row j+1
-                uint32_t z = hmax2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));   // (amax_j, amax_j+1) of this lane
-#pragma unroll
-                for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
-                bad |= nonfinite2(z);
-                const uint32_t ie0 = inv_exp_field<ELEM>(z << 16, rule_offset);
-                const uint32_t ie1 = inv_exp_field<ELEM>(z & 0xFFFF0000u, rule_offset);
-                inv0 = __uint_as_float(ie0 << 23);
-                inv1 = __uint_as_float(ie1 << 23);
-                if ((lane & (LPB - 1)) == 0) {
-                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
-                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
-                }
-            }
-        } else {
-            const float2 w0 = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-            const float2 w1 = *reinterpret_cast<const float2*>(my_in + (j + 1) * T_BYTES);
-            x0[0] = w0.x; x0[1] = w0.y;
-            x1[0] = w1.x; x1[1] = w1.y;
-            if (DO_ROW) {
-                float a0 = fmaxf(fmaxf(fabsf(w0.x), fabsf(w0.y)), 0.f), a1 = fmaxf(fmaxf(fabsf(w1.x), fabsf(w1.y)), 0.f);
-#pragma unroll
-                for (int off = 1; off < LPB; off <<= 1) {
-                    a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, off));
-                    a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, off));
-                }
-                bad |= (uint32_t)(a0 == INFINITY) | (uint32_t)(a1 == INFINITY);
-                const uint32_t ie0 = inv_exp_field<ELEM>(__float_as_uint(a0), rule_offset);
-                const uint32_t ie1 = inv_exp_field<ELEM>(__float_as_uint(a1), rule_offset);
-                inv0 = __uint_as_float(ie0 << 23);
-                inv1 = __uint_as_float(ie1 << 23);
-                if ((lane & (LPB - 1)) == 0) {
-                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
-                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
-                }
-            }
-        }
-        uint8_t* r0 = my_qrow + (uint64_t)j * pitch;
-        uint8_t* c0 = my_qcol + (uint64_t)j * pitch;
-        if (DO_ROW) {
-            float i0[VEC], i1[VEC], s0[VEC], s1[VEC];
-            const float xs0 = EMU ? scale_from_inv(inv0) : 0.f, xs1 = EMU ? scale_from_inv(inv1) : 0.f;
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) { i0[i] = inv0; i1[i] = inv1; s0[i] = xs0; s1[i] = xs1; }
-            emit<ELEM, VEC, EMU>(r0, x0, i0, s0);
-            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1);
-        }
-        if (DO_COL) {
-            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs);
-            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs);
-        }
-    }
-    return __any_sync(0xFFFFFFFFu, bad != 0u);
-}
-
-// The same slab with everything the fast path leaves out: Inf and NaN elements stay out of
-// amax (App. / Sec. 3.3 leaves their handling open; see mxfp8.h), rows and columns outside the
-// tensor are not stored.  Rare, so compact rather than fast.
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
-__device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
-                                          uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
-                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset, int rows_here, bool col_ok)
-{
-    constexpr bool BF = (DTYPE == MXFP8_BF16);
-    constexpr int VEC = BF ? 4 : 2;
-    constexpr int LPB = 32 / VEC;
-    auto load = [&](int j, float (&x)[VEC]) {
-        if constexpr (BF) {
-            const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-            x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xFFFF0000u);
-            x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xFFFF0000u);
-        } else {
-            const float2 w = *reinterpret_cast<const float2*>(my_in + j * T_BYTES);
-            x[0] = w.x; x[1] = w.y;
-        }
-    };
-    float col_inv[VEC], col_xs[VEC];
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) { col_inv[i] = 1.f; col_xs[i] = 1.f; }
-    if (DO_COL) {
-        float cmax[VEC];
-#pragma unroll
-        for (int i = 0; i < VEC; ++i) cmax[i] = 0.f;
-#pragma unroll 1
-        for (int j = 0; j < 32; ++j) {
-            float x[VEC];
-            load(j, x);
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                const float a = fabsf(x[i]);
-                if (a < INFINITY) cmax[i] = fmaxf(cmax[i], a);   // false for NaN as well
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < VEC; ++i) {
-            const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(cmax[i]), rule_offset);
-            col_inv[i] = __uint_as_float(ie << 23);
-            col_xs[i] = scale_from_inv(col_inv[i]);
-            my_sm_col[i * 4] = (uint8_t)(254u - ie);
-        }
-    }
-#pragma unroll 1
-    for (int j = 0; j < 32; ++j) {
-        float x[VEC];
-        load(j, x);
-        const bool live = col_ok && j < rows_here;
-        if (DO_ROW) {
-            float m = 0.f;
-#pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                const float a = fabsf(x[i]);
-                if (a < INFINITY) m = fmaxf(m, a);
-            }
-#pragma unroll
-            for (int off = 1; off < LPB; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
-            const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(m), rule_offset);
-            const float inv = __uint_as_float(ie << 23);
-            if ((lane & (LPB - 1)) == 0) my_sm_row[j * 4] = (uint8_t)(254u - ie);
-            if (live) {
-                float iv[VEC], sv[VEC];
-#pragma unroll
-                for (int i = 0; i < VEC; ++i) { iv[i] = inv; sv[i] = scale_from_inv(inv); }
-                emit<ELEM, VEC, EMU>(my_qrow + (uint64_t)j * pitch, x, iv, sv);
-            }
-        }
-        if (DO_COL && live) emit<ELEM, VEC, EMU>(my_qcol + (uint64_t)j * pitch, x, col_inv, col_xs);
-    }
-}
-
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
-__global__ void __launch_bounds__(QT_THREADS, 3)
-quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QBatch batch)
-{
-    constexpr bool BF = (DTYPE == MXFP8_BF16);
-    constexpr int VEC = BF ? 4 : 2;                 // elements per lane per row
-    constexpr int T_COLS = T_BYTES / (BF ? 2 : 4);  // 128 or 64
-    constexpr int NKB = T_COLS / 32;                // row blocks per tile row: 4 or 2
-    constexpr int LPB = 32 / VEC;                   // lanes per row block: 8 or 16
-
-    extern __shared__ __align__(128) uint8_t smem[];
-    uint8_t* in_ring = smem;                               // 2 x [128][256]
-    uint8_t* sm_scales = smem + 2 * IN_BYTES;              // 2 x ([128][4] row scales + [T_COLS][4] column scales)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;   // warp = 32-row slab of the tile
-    const uint32_t rule_offset = (batch.t[0].rule == MXFP8_RULE_PAPER) ? 0x1FFFFFu : 0u;
-
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const int num_tiles = batch.tile_start[batch.count];
-    int load_ti = 0;                          // tensor of the tile being loaded (tiles only move forward)
-    auto issue_load = [&](int t, int buf) {   // one thread: tile t -> ring slot buf
-        while (t >= batch.tile_start[load_ti + 1]) ++load_ti;
-        const int lt = t - batch.tile_start[load_ti], tx = batch.t[load_ti].tiles_x;
-        const uint32_t b = smem_addr(&bars[buf]);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
-        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&maps.m[load_ti]), "r"(b), "r"((lt % tx) * T_COLS), "r"((lt / tx) * T_ROWS)
-                     : "memory");
-    };
-    int tile = blockIdx.x, ti = 0;
-    if (tid == 0) {
-        if (tile < num_tiles) issue_load(tile, 0);
-        if (tile + (int)gridDim.x < num_tiles) issue_load(tile + gridDim.x, 1);
-    }
-
-    for (int it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
-        const int buf = it & 1;
-        const uint32_t phase = (uint32_t)(it >> 1) & 1u;
-        const uint32_t bar_a = smem_addr(&bars[buf]);
-        uint8_t* in_tile = in_ring + buf * IN_BYTES;
-        uint8_t* sm_row = sm_scales + buf * 1024;          // [128][4]
-        uint8_t* sm_col = sm_row + 512;                    // [T_COLS][4]
-        while (tile >= batch.tile_start[ti + 1]) ++ti;
-        const QParams& p = batch.t[ti];
-        const int ltile = tile - batch.tile_start[ti];
-        const int tile_x = ltile % p.tiles_x, tile_y = ltile / p.tiles_x;
-        const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
-
-        // wait for the tile (bounded: on expiry report through the status word and leave)
-        {
-            uint32_t ok = 0, spins = 0;
-            uint64_t t0 = 0;
-            while (true) {
-                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                             : "=r"(ok) : "r"(bar_a), "r"(phase) : "memory");
-                if (ok) break;
-                if ((++spins & 0xFFu) == 0) {
-                    uint64_t now;
-                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > QT_WAIT_LIMIT_NS) break;
-                }
-            }
-            if (!__syncthreads_and((int)ok)) {
-                if (tid == 0) atomicExch(&g_quantize_status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
-                return;
-            }
-        }
-        // this warp's slab: 32 rows; first the fully unrolled fast path (no special values, whole
-        // slab inside the tensor), and if it saw an Inf / NaN or the slab is ragged, the careful path
-        const uint8_t* my_in = in_tile + warp * 32 * T_BYTES + lane * 8;
-        const int64_t my_col = gcol0 + lane * VEC;
-        const int rows_here = (int)min((int64_t)32, p.rows - (grow0 + warp * 32));   // rows of this slab inside the tensor
-        const bool col_ok = my_col < p.cols;                                         // cols % 16 == 0: a lane's bytes are all in or all out
-        // bytes per stored element: 1 (FP8 code), or the source's size when the decoded value is stored
-        constexpr int OUT_ESZ = EMU ? (BF ? 2 : 4) : 1;
-        uint8_t* my_qrow = p.q_row + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
-        uint8_t* my_qcol = p.q_col + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
-        const uint32_t pitch = (uint32_t)p.cols * OUT_ESZ;
-        uint8_t* my_sm_row = sm_row + warp * 128 + lane / LPB;
-        uint8_t* my_sm_col = sm_col + lane * VEC * 4 + warp;
-        const bool whole = __all_sync(0xFFFFFFFFu, col_ok) && rows_here == 32;
-        bool special = !whole;
-        if (whole)
-            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset);
-        if (special && rows_here > 0)
-            slab_careful<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
-                                                       rows_here, col_ok);
-
-        // every warp is done with this ring slot: refill it with the tile after next
-        __syncthreads();
-        if (tid == 0) {
-            const int next = tile + 2 * (int)gridDim.x;
-            if (next < num_tiles) issue_load(next, buf);
-        }
-
-        // ---- scale bytes (1/32 of the output): plain stores from the staging arrays ----------
-        if (DO_ROW && !EMU && tid < T_ROWS) {
-            const int64_t r = grow0 + tid, ncb = p.cols >> 5, kb0 = (int64_t)tile_x * NKB;
-            const int nkb = (int)min((int64_t)NKB, ncb - kb0);
-            if (p.sf_layout == MXFP8_SF_SWIZZLED) {
-                // every row of a started 128-row atom is written (pad rows / pad K-blocks get 0)
-                uint8_t* d = p.s_row + ((int64_t)tile_y * ((ncb + 3) >> 2) + (kb0 >> 2)) * 512 + (tid & 31) * 16 + (tid >> 5) * 4 + (kb0 & 3);
-                uint32_t v = 0u;
-                if (r < p.rows)
-                    for (int kb = 0; kb < nkb; ++kb) v |= (uint32_t)sm_row[tid * 4 + kb] << (8 * kb);
-                // a 64-column FP32 tile owns half of the atom's 4 K-blocks; the left half also zeroes
-                // the right half when no tile exists there (pad K-blocks)
-                if (NKB == 4 || ((kb0 & 3) == 0 && kb0 + NKB >= ncb)) *reinterpret_cast<uint32_t*>(d) = v;
-                else *reinterpret_cast<uint16_t*>(d) = (uint16_t)v;
-            } else if (r < p.rows) {
-                uint8_t* d = p.s_row + r * ncb + kb0;
-                for (int kb = 0; kb < nkb; ++kb) d[kb] = sm_row[tid * 4 + kb];
-            }
-        }
-        if (DO_COL && !EMU && tid < T_COLS) {
-            const int64_t c = gcol0 + tid, nrb = p.rows >> 5, rb0 = (int64_t)tile_y * 4;
-            const int nrb_here = (int)min((int64_t)4, nrb - rb0);
-            if (p.sf_layout == MXFP8_SF_SWIZZLED) {
-                const int64_t padded_cols = ((p.cols + 127) >> 7) << 7;
-                if (c < padded_cols) {
-                    uint8_t* d = p.s_col + ((c >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + (c & 31) * 16 + ((c >> 5) & 3) * 4;
-                    uint32_t v = 0u;
-                    if (c < p.cols)
-                        for (int w = 0; w < nrb_here; ++w) v |= (uint32_t)sm_col[tid * 4 + w] << (8 * w);
-                    *reinterpret_cast<uint32_t*>(d) = v;
-                    // pad columns no tile covers (FP32 tiles are 64 wide, atoms 128 wide)
-                    if (T_COLS == 64 && tile_x == p.tiles_x - 1 && c + 64 >= (int64_t)p.tiles_x * 64 && c + 64 < padded_cols)
-                        *reinterpret_cast<uint32_t*>(p.s_col + (((c + 64) >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + ((c + 64) & 31) * 16 + (((c + 64) >> 5) & 3) * 4) = 0u;
-                }
-            } else if (c < p.cols) {
-                for (int w = 0; w < nrb_here; ++w) p.s_col[(rb0 + w) * p.cols + c] = sm_col[tid * 4 + w];
-            }
-        }
-    }
-}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -484,41 +48,6 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t esz, void* bas
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int qt_sm_count()
-{
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return v;
-    }();
-    return n;
-}
-
-template <int DTYPE, int ELEM, bool R, bool C, bool EMU>
-cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
-{
-    constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
-    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU>;
-    static unsigned long long smem_set = 0;
-    cudaError_t err = ensure_dynamic_smem(kernel, SMEM, smem_set);
-    if (err != cudaSuccess) return err;
-    const int tiles = p.tile_start[p.count];
-    const int max_ctas = qt_sm_count() * 3;
-    const int grid = tiles < max_ctas ? tiles : max_ctas;
-    kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, p);
-    count_launch(1);
-    return cudaGetLastError();
-}
-
-template <int DTYPE, int ELEM, bool EMU>
-cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStream_t st)
-{
-    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU>(ms, p, st);
-    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU>(ms, p, st);
-    return launch<DTYPE, ELEM, true, true, EMU>(ms, p, st);
 }
 
 }  // namespace
@@ -561,17 +90,17 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
         if (tiles >= 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
     }
     for (int i = count; i <= QT_MAX_TENSORS; ++i) p.tile_start[i] = (int)tiles;
+    static int* status_word = [] {
+        void* ptr = nullptr;
+        return cudaGetSymbolAddress(&ptr, g_quantize_status) == cudaSuccess ? static_cast<int*>(ptr) : nullptr;
+    }();
+    if (!status_word) return MXFP8_ERR_CUDA;
+    p.status = status_word;
     cudaError_t err;
-    if (emulate) {
-        if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3, true>(orientation, ms, p, stream)
-                                         : launch_o<MXFP8_BF16, MXFP8_E5M2, true>(orientation, ms, p, stream);
-        else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3, true>(orientation, ms, p, stream)
-                                      : launch_o<MXFP8_FP32, MXFP8_E5M2, true>(orientation, ms, p, stream);
-    } else {
-        if (bf) err = elem == MXFP8_E4M3 ? launch_o<MXFP8_BF16, MXFP8_E4M3, false>(orientation, ms, p, stream)
-                                         : launch_o<MXFP8_BF16, MXFP8_E5M2, false>(orientation, ms, p, stream);
-        else err = elem == MXFP8_E4M3 ? launch_o<MXFP8_FP32, MXFP8_E4M3, false>(orientation, ms, p, stream)
-                                      : launch_o<MXFP8_FP32, MXFP8_E5M2, false>(orientation, ms, p, stream);
+    switch (elem) {
+        case MXFP8_E4M3: err = quantize_tma_launch<MXFP8_E4M3>(bf, orientation, emulate, ms, p, stream); break;
+        case MXFP8_E5M2: err = quantize_tma_launch<MXFP8_E5M2>(bf, orientation, emulate, ms, p, stream); break;
+        default: err = quantize_tma_launch_fp6_fp4(elem, bf, orientation, emulate, &ms, &p, stream); break;
     }
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }

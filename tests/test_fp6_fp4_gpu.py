@@ -1,0 +1,115 @@
+"""The 6- and 4-bit element formats of Table 1 (MXFP6: E2M3, E3M2; MXFP4: E2M1) through
+mxfp8_quantize / mxfp8_quantize_multi / mxfp8_dequantize / mxfp8_fake_quantize: bit-exact
+against the oracle, same scale algorithm as MXFP8."""
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2506_08027_b200 import synth
+from helpers import check_against_oracle
+from test_fake_quant_gpu import check as check_round_trip
+
+pytestmark = pytest.mark.gpu
+
+ROW, COL, BOTH = 1, 2, 3
+LINEAR, SWIZZLED = 0, 1
+ELEMS = [orc.E2M3, orc.E3M2, orc.E2M1]
+
+
+def as_dtype(x32, dtype):
+    return synth.f32_to_bf16_bits(x32) if dtype == "bf16" else x32
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("rule", [orc.RULE_PAPER, orc.RULE_OCP])
+@pytest.mark.parametrize("elem", ELEMS)
+def test_pr1_reference_tensor(dtype, rule, elem):
+    x = as_dtype(synth.pr1_tensor(0), dtype)
+    for orientation in (ROW, COL, BOTH):
+        check_against_oracle(x, dtype, orientation, rule, elem, SWIZZLED, "pr1 o=%d" % orientation)
+    check_against_oracle(x, dtype, BOTH, rule, elem, LINEAR, "pr1 linear")
+
+
+@pytest.mark.parametrize("dist", synth.DISTRIBUTIONS)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("elem", ELEMS)
+def test_value_distributions(dist, dtype, elem):
+    # "nonfinite" includes NaN and +-Inf elements: these formats have no such codes (NaN -> +max, Inf -> +-max)
+    x = as_dtype(synth.draw(dist, (256, 1024), synth.seed_for(6, synth.DISTRIBUTIONS.index(dist))), dtype)
+    for rule in (orc.RULE_PAPER, orc.RULE_OCP):
+        check_against_oracle(x, dtype, BOTH, rule, elem, SWIZZLED, "%s rule=%d" % (dist, rule))
+
+
+@pytest.mark.parametrize("shape", [(32, 32), (7, 64), (160, 352), (384, 8288), (64, 100), (64, 33)])
+@pytest.mark.parametrize("elem", ELEMS)
+def test_ragged_shapes_and_generic_path(shape, elem):
+    rows, cols = shape
+    for dtype in ("fp32", "bf16"):
+        x = as_dtype(synth.student_t(shape, 77 + rows + cols), dtype)
+        orients = ([ROW] if cols % 32 == 0 else []) + ([COL] if rows % 32 == 0 else [])
+        if cols % 32 == 0 and rows % 32 == 0:
+            orients.append(BOTH)
+        for o in orients:
+            check_against_oracle(x, dtype, o, orc.RULE_PAPER, elem, SWIZZLED, "%s o=%d" % (shape, o))
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_scale_boundaries_at_the_largest_normal(elem):
+    # block maxima exactly at destmax * 2^k, one FP32 step above and below: the rule's rounding decides here
+    top = {orc.E2M3: 7.5, orc.E3M2: 28.0, orc.E2M1: 6.0}[elem]
+    x = np.zeros((96, 64), np.float32)
+    k = np.arange(96) - 40
+    x[:, 0] = np.float32(top) * np.exp2(k).astype(np.float32)
+    x[:, 32] = np.nextafter(x[:, 0], np.float32(np.inf))
+    x[:, 1] = np.float32(0.3) * x[:, 0]
+    x[:, 33] = -np.nextafter(x[:, 0], np.float32(0))
+    for rule in (orc.RULE_PAPER, orc.RULE_OCP):
+        check_against_oracle(x, "fp32", BOTH, rule, elem, LINEAR, "boundaries")
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+@pytest.mark.parametrize("dst", ["f32", "bf16"])
+def test_dequantize_exhaustive_codes_and_scales(elem, dst):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    bits = 4 if elem == orc.E2M1 else 6
+    codes = (np.arange(256) % (1 << bits)).astype(np.uint8)
+    q = np.tile(np.repeat(codes, 32)[None, :], (256, 1))            # [256, 8192]
+    s = np.repeat(np.arange(256, dtype=np.uint8)[:, None], 256, axis=1)
+    want = orc.dequantize(q, s, orc.ROW, elem, dst)
+    out = torch.empty(q.shape, dtype=torch.float32 if dst == "f32" else torch.bfloat16, device="cuda")
+    B.mxfp8_dequantize(torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda().view(-1), B.ROW, elem, B.SF_LINEAR, out)
+    torch.cuda.synchronize()
+    if dst == "f32":
+        got = out.cpu().numpy()
+        nan = np.isnan(want)
+        assert np.array_equal(np.isnan(got), nan)
+        assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+    else:
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        nan = (want & 0x7FFF) > 0x7F80
+        assert np.array_equal((got & 0x7FFF) > 0x7F80, nan)
+        assert np.array_equal(got[~nan], want[~nan])
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_fake_quantize_round_trip(elem, dtype):
+    for dist in ("gaussian", "gradient_like", "nonfinite"):
+        x = as_dtype(synth.draw(dist, (160, 416), 31), dtype)
+        for rule in (orc.RULE_PAPER, orc.RULE_OCP):
+            check_round_trip(x, dtype, BOTH, rule, elem, "%s rule=%d" % (dist, rule))
+
+
+def test_gemm_rejects_sub_byte_operands_as_unsupported():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    z = torch.zeros(128, 128, dtype=torch.uint8, device="cuda")
+    sc = torch.zeros(512, dtype=torch.uint8, device="cuda")
+    D = torch.empty(128, 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, B.E2M3, B.E4M3, D)
+    assert e.value.status == -5
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, 2, B.E4M3, D)     # 2 is no element code
+    assert e.value.status == -2
