@@ -40,8 +40,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # summarised under profiles/: the FPROP GEMM of this step, and the quantize kernel on a
 # 128 MB BF16 tensor (the size of dY, the largest cast of the step).  Writes still dirty in
 # L2 when the kernel ends are not counted by ncu, so both are below the algorithmic bytes.
-NCU_TRAFFIC_GEMM_FPROP = 49.8e6 + 86.6e6
-NCU_TRAFFIC_QUANTIZE_128MB = 134.3e6 + 85.0e6
+NCU_TRAFFIC_GEMM_FPROP = 49.8e6 + 85.3e6
+NCU_TRAFFIC_QUANTIZE_128MB = 134.3e6 + 84.2e6     # one 8192 x 8192 BF16 tensor, both orientations (272.6 MB algorithmic)
 
 STEP_FLOP = 3 * 2.0 * T * H * F                       # three GEMMs of 275 GFLOP
 CAST_BYTES = (T * H + F * H + T * F) * (2 + 2 * (1 + 1 / 32))   # src + two orientations x (q + scales)
@@ -342,7 +342,10 @@ def run_ours(args):
         "roofline_cast": {"bound": "hbm", "kernel": "quantize_tma_kernel<bf16,e4m3,row+col>", "achieved": cast_gbs,
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cast_gbs / peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "algorithmic_bytes_per_element": 4.0625,
-                          "traffic": NCU_TRAFFIC_QUANTIZE_128MB, "traffic_note": "ncu capture, 8192x8192 BF16 tensor (= dY), see profiles/"},
+                          "algorithmic_bytes_per_launch": CAST_BYTES,
+                          "traffic": NCU_TRAFFIC_QUANTIZE_128MB * CAST_BYTES / (T * F * 4.0625),
+                          "traffic_note": "ncu capture of one 8192x8192 BF16 tensor (= dY alone), scaled by bytes to the batched launch "
+                                          "over X, W and dY (traffic grows with the bytes converted); see profiles/"},
         "e2e": e2e, "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
         "cpu_baseline": cpu,
     }
