@@ -144,6 +144,36 @@ def test_large_tensor_sampled():
         assert_q_equal(qc[sl].cpu().numpy(), wq, orc.E4M3)
 
 
+def test_benchmark_step_cast_in_its_launch_configuration_sampled():
+    # the benchmark's cast: X [8192, 2048], W [8192, 2048], dY [8192, 8192] (BF16, drawn on the device) in ONE
+    # batched launch, both orientations, swizzled scales; the oracle checks sampled 128-row slabs of every tensor
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import logical_scales_from_swizzled
+    T, H, F = 8192, 2048, 8192
+    tensors = [synth.device_tensor("activation", (T, H), synth.seed_for(2, 0)),
+               synth.device_tensor("weight", (F, H), synth.seed_for(2, 1)),
+               synth.device_tensor("output_gradient", (T, F), synth.seed_for(2, 2))]
+    outs = [B.alloc_quantize_outputs(t.shape[0], t.shape[1], B.BOTH, B.SF_SWIZZLED) for t in tensors]
+    items = B.make_quantize_items([(t,) + o for t, o in zip(tensors, outs)])
+    B.mxfp8_quantize_multi(items, B.BF16, B.BOTH, B.RULE_PAPER, B.E4M3, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for src, (qr, sr, qc, sc) in zip(tensors, outs):
+        rows, cols = src.shape
+        s_row = logical_scales_from_swizzled(sr.cpu().numpy(), rows, cols // 32)            # [rows, cols/32]
+        s_col = logical_scales_from_swizzled(sc.cpu().numpy(), cols, rows // 32).T          # [rows/32, cols]
+        for r0 in (0, 2048 + 128, rows - 128):
+            sl = slice(r0, r0 + 128)
+            x = orc.bf16_bits_to_f32(src[sl].view(torch.int16).cpu().numpy().view(np.uint16))
+            wq, ws = orc.quantize(x, orc.ROW)
+            assert np.array_equal(s_row[sl], ws)
+            assert_q_equal(qr[sl].cpu().numpy(), wq, orc.E4M3)
+            wq, ws = orc.quantize(x, orc.COL)
+            assert np.array_equal(s_col[r0 // 32:r0 // 32 + 4], ws)
+            assert_q_equal(qc[sl].cpu().numpy(), wq, orc.E4M3)
+
+
 # ------------------------------------------------------------------------------- dequantize
 
 @pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
