@@ -55,12 +55,14 @@ typedef enum {
 enum { MXFP8_FP32 = 0, MXFP8_BF16 = 1 };                 /* source / destination dtype   */
 enum { MXFP8_ROW = 1, MXFP8_COL = 2, MXFP8_BOTH = 3 };   /* block orientation (bit mask) */
 enum { MXFP8_RULE_PAPER = 0, MXFP8_RULE_OCP = 1 };       /* scale rounding rule          */
-/* Element encodings (Table 1).  E4M3 / E5M2 are the MXFP8 elements.  E2M3 / E3M2 (MXFP6) and E2M1
- * (MXFP4) share the block size, the scale type and both scale rules; they have no Inf and no NaN
- * (a NaN input becomes +max, +-Inf becomes +-max), and their codes are stored one per byte in the
- * low 6 / 4 bits (upper bits zero).  mxfp8_quantize, mxfp8_quantize_multi, mxfp8_dequantize and
- * mxfp8_fake_quantize take all five; mxfp8_gemm and the fused GEMM output take the two 8-bit ones.
- * The values are the tensor cores' own format codes. */
+/* Element encodings (Table 1).  E4M3 / E5M2 are the MXFP8 elements, one code per byte.  E2M3 / E3M2
+ * (MXFP6) and E2M1 (MXFP4) share the block size, the scale type and both scale rules; they have no Inf
+ * and no NaN (a NaN input becomes +max, +-Inf becomes +-max).  Their codes are stored the way the tensor
+ * cores read them: every 16 consecutive codes of a row share one 16-byte slot, code i in bits
+ * [w*i, w*i + w) of the slot taken as a little-endian integer (w = 6 or 4), the other bytes zero.  A
+ * [rows, cols] code tensor therefore still has `cols` bytes per row and needs cols % 16 == 0
+ * (MXFP8_ERR_UNSUPPORTED otherwise).  Every entry point takes all five, except the fused GEMM output
+ * (8-bit elements only).  The values are the tensor cores' own format codes. */
 enum { MXFP8_E4M3 = 0, MXFP8_E5M2 = 1, MXFP8_E2M3 = 3, MXFP8_E3M2 = 4, MXFP8_E2M1 = 5 };
 enum { MXFP8_SF_LINEAR = 0, MXFP8_SF_SWIZZLED = 1 };     /* scale layout                 */
 enum { MXFP8_K_MAJOR = 0, MXFP8_MN_MAJOR = 1 };          /* GEMM operand storage         */

@@ -9,5 +9,5 @@ from .mxfp8_oracle import (  # noqa: F401
     E4M3, E5M2, E2M3, E3M2, E2M1, RULE_PAPER, RULE_OCP, ROW, COL,
     build_oracle, fp8_decode, fp8_encode, scale_byte, quantize, dequantize_f64,
     dequantize, bf16_bits_to_f32, sf_offset_swizzled,
-    swizzle_scales, gemm_f64, quantize_threads, grouped_gemm_f64,
+    swizzle_scales, gemm_f64, quantize_threads, grouped_gemm_f64, code_bits, pack_codes16, unpack_codes16,
 )

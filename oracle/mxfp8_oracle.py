@@ -254,3 +254,46 @@ def grouped_gemm_f64(aq, a_s, bq, b_s, offsets, mode: str = "m", b_major: str = 
             d[g * M:(g + 1) * M] = a[lo:hi].T @ b[lo:hi]
             sabs[g * M:(g + 1) * M] = np.abs(a[lo:hi]).T @ np.abs(b[lo:hi])
     return d, sabs
+
+
+def code_bits(elem: int) -> int:
+    return {E4M3: 8, E5M2: 8, E2M3: 6, E3M2: 6, E2M1: 4}[elem]
+
+
+def pack_codes16(codes: np.ndarray, elem: int) -> np.ndarray:
+    """Storage layout of 6- and 4-bit codes (Table 1's MXFP6 / MXFP4 elements) as the tensor cores
+    read them: every 16 consecutive codes of a row become one 16-byte slot; code i of the slot
+    occupies bits [w*i, w*i + w) of the slot read as a little-endian integer (w = 6 or 4), the
+    remaining bytes are zero.  8-bit codes are returned unchanged.  `codes`: [rows, cols] uint8,
+    one code per byte, cols a multiple of 16.  An index/bit permutation, no arithmetic."""
+    w = code_bits(elem)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    if w == 8:
+        return codes.copy()
+    rows, cols = codes.shape
+    if cols % 16:
+        raise ValueError("packed slots need cols % 16 == 0")
+    out = np.zeros((rows, cols), dtype=np.uint8)
+    for r in range(rows):
+        for g in range(cols // 16):
+            slot = 0
+            for i in range(16):
+                slot |= int(codes[r, 16 * g + i]) << (w * i)
+            out[r, 16 * g:16 * g + 16] = np.frombuffer(slot.to_bytes(16, "little"), dtype=np.uint8)
+    return out
+
+
+def unpack_codes16(packed: np.ndarray, elem: int) -> np.ndarray:
+    """Inverse of pack_codes16 (padding bytes are ignored)."""
+    w = code_bits(elem)
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    if w == 8:
+        return packed.copy()
+    rows, cols = packed.shape
+    out = np.zeros((rows, cols), dtype=np.uint8)
+    for r in range(rows):
+        for g in range(cols // 16):
+            slot = int.from_bytes(packed[r, 16 * g:16 * g + 16].tobytes(), "little")
+            for i in range(16):
+                out[r, 16 * g + i] = (slot >> (w * i)) & ((1 << w) - 1)
+    return out

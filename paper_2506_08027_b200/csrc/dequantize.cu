@@ -37,6 +37,22 @@ dequantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, 
         for (int i = 0; i < n; ++i) w[i >> 2] |= (uint32_t)q[r * cols + c0 + i] << (8 * (i & 3));
     }
 
+    if constexpr (ELEM != MXFP8_E4M3 && ELEM != MXFP8_E5M2) {
+        // 6- and 4-bit codes arrive as one packed 16-byte slot (little-endian bit stream in the first
+        // 12 / 8 bytes): spread them to one code per byte
+        constexpr int B = (ELEM == MXFP8_E2M1) ? 4 : 6;
+        const uint32_t st[4] = {w[0], w[1], w[2], 0u};
+        uint32_t u[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int bit = B * i, wd = bit >> 5, off = bit & 31;
+            uint32_t code = st[wd] >> off;
+            if (off + B > 32) code |= st[wd + 1] << (32 - off);
+            u[i >> 2] |= (code & ((1u << B) - 1u)) << (8 * (i & 3));
+        }
+        w[0] = u[0]; w[1] = u[1]; w[2] = u[2]; w[3] = u[3];
+    }
+
     float out[16];
     float row_scale = 0.f;
     if (ORIENT == MXFP8_ROW) {
@@ -145,7 +161,7 @@ template <int ELEM, int DST, int ORIENT>
 cudaError_t launch(const uint8_t* q, const uint8_t* s, int64_t rows, int64_t cols, int sf_layout,
                    void* dst, cudaStream_t stream)
 {
-    if ((cols & 127) == 0) {
+    if constexpr (ELEM == MXFP8_E4M3 || ELEM == MXFP8_E5M2) if ((cols & 127) == 0) {
         const int64_t groups = rows * (cols / 128);            // warp steps of 128 elements
         const int64_t warps = (groups + 7) / 8;
         const int64_t blocks = (warps + 7) / 8;                // 8 warps per block
@@ -186,6 +202,7 @@ extern "C" int mxfp8_dequantize(const void* q, const void* s, int64_t rows, int6
     if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
     if (orientation == MXFP8_ROW ? (cols % 32) : (rows % 32)) return MXFP8_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(s) || !aligned16(dst)) return MXFP8_ERR_ALIGN;
+    if (!fp8_elem(elem) && (cols % 16)) return MXFP8_ERR_UNSUPPORTED;   // packed 16-code slots
     const uint8_t* qq = static_cast<const uint8_t*>(q);
     const uint8_t* ss = static_cast<const uint8_t*>(s);
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -1011,7 +1011,6 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     if (a_major != MXFP8_K_MAJOR && a_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
     if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
     if (!valid_elem(a_elem) || !valid_elem(b_elem)) return MXFP8_ERR_ENUM;
-    if (!fp8_elem(a_elem) || !fp8_elem(b_elem)) return MXFP8_ERR_UNSUPPORTED;   // 6- and 4-bit operands need the packed tensor-core layout
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs) return MXFP8_ERR_NULL;
     if (!D && !epi) return MXFP8_ERR_NULL;
@@ -1107,7 +1106,6 @@ extern "C" int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq
     if (mode != MXFP8_GROUP_M && mode != MXFP8_GROUP_K) return MXFP8_ERR_ENUM;
     if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
     if (!valid_elem(a_elem) || !valid_elem(b_elem)) return MXFP8_ERR_ENUM;
-    if (!fp8_elem(a_elem) || !fp8_elem(b_elem)) return MXFP8_ERR_UNSUPPORTED;   // 6- and 4-bit operands need the packed tensor-core layout
     if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (!Aq || !As || !Bq || !Bs || !group_offsets || !D) return MXFP8_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || num_groups <= 0) return MXFP8_ERR_SHAPE;

@@ -279,10 +279,7 @@ int quantize_device(const void* src, int src_dtype, int64_t rows, int64_t cols, 
     switch (elem) {
         MXFP8_ELEM_CASE(MXFP8_E4M3)
         MXFP8_ELEM_CASE(MXFP8_E5M2)
-        MXFP8_ELEM_CASE(MXFP8_E2M3)
-        MXFP8_ELEM_CASE(MXFP8_E3M2)
-        MXFP8_ELEM_CASE(MXFP8_E2M1)
-        default: err = cudaErrorInvalidValue;
+        default: err = cudaErrorInvalidValue;   // 6- and 4-bit codes are packed 16 to a slot: TMA path only
     }
 #undef MXFP8_ELEM_CASE
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
@@ -313,6 +310,7 @@ extern "C" int mxfp8_quantize(const void* src, int src_dtype, int64_t rows, int6
     if (quantize_tma_eligible(src_dtype, rows, cols))
         return quantize_tma_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
                                    q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
+    if (!fp8_elem(elem)) return MXFP8_ERR_UNSUPPORTED;   // packed 16-code slots need cols % 16 == 0
     return quantize_device(src, src_dtype, rows, cols, orientation, scale_rule, elem, q_row, s_row,
                            q_col, s_col, sf_layout, static_cast<cudaStream_t>(stream));
 }

@@ -87,27 +87,68 @@ __device__ __forceinline__ float scale_from_inv(float inv)
     return __uint_as_float(b ? (b << 23) : 0x00400000u);
 }
 
-// One lane's VEC elements of one row: cast x * inv to FP8 and store the codes (EMU = false), or store
-// the decoded values code * X in the source's own dtype (EMU = true: the MXFP8 round trip the paper's
-// Hopper runs used, Sec. 3.1).  The decoded product is exact in FP32; BF16 output is one RNE of it.
-template <int ELEM, int VEC, bool EMU>
-__device__ __forceinline__ void emit(uint8_t* dst, const float (&x)[VEC], const float (&inv)[VEC], const float (&xs)[VEC])
+// 6- and 4-bit codes leave in the layout the tensor cores read (kind::mxf8f6f4): 16 consecutive codes
+// of a row form one 16-byte slot, the codes packed as a little-endian bit stream in its first 12
+// (6-bit) or 8 (4-bit) bytes, the rest zero.  A slot is 4 lanes wide for a BF16 source (4 codes per
+// lane, each lane stores one 32-bit word of the slot) and 8 lanes wide for an FP32 source (2 codes per
+// lane, one 16-bit word each).  `c`: this lane's codes, one per byte.  Every lane of the warp calls.
+template <int ELEM, int VEC>
+__device__ __forceinline__ uint32_t pack_slot(uint32_t c, int lane)
 {
+    constexpr int B = (ELEM == MXFP8_E2M1) ? 4 : 6;
     if constexpr (VEC == 4) {
-        const uint32_t c = cvt_fp8x4<ELEM>(x[0] * inv[0], x[1] * inv[1], x[2] * inv[2], x[3] * inv[3]);
-        if constexpr (!EMU) {
-            *reinterpret_cast<uint32_t*>(dst) = c;
+        const uint32_t v = (c & 0xFFu) | (((c >> 8) & 0xFFu) << B) | (((c >> 16) & 0xFFu) << (2 * B)) | ((c >> 24) << (3 * B));
+        const int j = lane & 3;
+        if constexpr (B == 6) {
+            // word j of the 96-bit stream = bits 32j.. = (v_j >> 8j) | (v_{j+1} << (24 - 8j)); word 3 is padding
+            const uint32_t nxt = __shfl_down_sync(0xFFFFFFFFu, v, 1);
+            return j == 3 ? 0u : ((v >> (8 * j)) | (nxt << (24 - 8 * j)));
         } else {
+            const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, v, 1), n2 = __shfl_down_sync(0xFFFFFFFFu, v, 2);
+            return j == 0 ? (v | (n1 << 16)) : (j == 1 ? (n1 | (n2 << 16)) : 0u);
+        }
+    } else {
+        const uint32_t v = (c & 0xFFu) | (((c >> 8) & 0xFFu) << B);
+        const int j = lane & 7, base = lane & ~7;
+        if constexpr (B == 6) {
+            // 16-bit word j of the stream (j < 6) spans the 12-bit values k = 4j/3 and k + 1
+            const int k = min((4 * j) / 3, 6);
+            const uint32_t lo = __shfl_sync(0xFFFFFFFFu, v, base + k), hi = __shfl_sync(0xFFFFFFFFu, v, base + k + 1);
+            return j >= 6 ? 0u : (((lo | (hi << 12)) >> (16 * j - 12 * k)) & 0xFFFFu);
+        } else {
+            const int k = 2 * (j & 3);
+            const uint32_t lo = __shfl_sync(0xFFFFFFFFu, v, base + k), hi = __shfl_sync(0xFFFFFFFFu, v, base + k + 1);
+            return j >= 4 ? 0u : (lo | (hi << 8));
+        }
+    }
+}
+
+// One lane's VEC elements of one row: cast x * inv to the element type and store the codes (EMU = false),
+// or store the decoded values code * X in the source's own dtype (EMU = true: the MX round trip the
+// paper's Hopper runs used, Sec. 3.1).  The decoded product is exact in FP32; BF16 output is one RNE of
+// it.  All lanes of the warp call (the sub-byte packing shuffles); only lanes with `store` write.
+template <int ELEM, int VEC, bool EMU>
+__device__ __forceinline__ void emit(uint8_t* dst, const float (&x)[VEC], const float (&inv)[VEC], const float (&xs)[VEC], int lane,
+                                     bool store = true)
+{
+    constexpr bool SUB = (ELEM != MXFP8_E4M3 && ELEM != MXFP8_E5M2);
+    if constexpr (VEC == 4) {
+        uint32_t c = cvt_fp8x4<ELEM>(x[0] * inv[0], x[1] * inv[1], x[2] * inv[2], x[3] * inv[3]);
+        if constexpr (!EMU) {
+            if constexpr (SUB) c = pack_slot<ELEM, VEC>(c, lane);
+            if (store) *reinterpret_cast<uint32_t*>(dst) = c;
+        } else if (store) {
             const float2 lo = fp8x2_to_float2<ELEM>(c & 0xFFFFu), hi = fp8x2_to_float2<ELEM>(c >> 16);
             const __nv_bfloat162 a = __floats2bfloat162_rn(lo.x * xs[0], lo.y * xs[1]);
             const __nv_bfloat162 b = __floats2bfloat162_rn(hi.x * xs[2], hi.y * xs[3]);
             *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
         }
     } else {
-        const uint32_t c = cvt_fp8x2<ELEM>(x[0] * inv[0], x[1] * inv[1]);
+        uint32_t c = cvt_fp8x2<ELEM>(x[0] * inv[0], x[1] * inv[1]);
         if constexpr (!EMU) {
-            *reinterpret_cast<uint16_t*>(dst) = (uint16_t)c;
-        } else {
+            if constexpr (SUB) c = pack_slot<ELEM, VEC>(c, lane);
+            if (store) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)c;
+        } else if (store) {
             const float2 f = fp8x2_to_float2<ELEM>(c);
             *reinterpret_cast<float2*>(dst) = make_float2(f.x * xs[0], f.y * xs[1]);
         }
@@ -219,12 +260,12 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
             const float xs0 = EMU ? scale_from_inv(inv0) : 0.f, xs1 = EMU ? scale_from_inv(inv1) : 0.f;
 #pragma unroll
             for (int i = 0; i < VEC; ++i) { i0[i] = inv0; i1[i] = inv1; s0[i] = xs0; s1[i] = xs1; }
-            emit<ELEM, VEC, EMU>(r0, x0, i0, s0);
-            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1);
+            emit<ELEM, VEC, EMU>(r0, x0, i0, s0, lane);
+            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1, lane);
         }
         if (DO_COL) {
-            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs);
-            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs);
+            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs, lane);
+            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs, lane);
         }
     }
     return __any_sync(0xFFFFFFFFu, bad != 0u);
@@ -293,14 +334,14 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
             const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(m), rule_offset);
             const float inv = __uint_as_float(ie << 23);
             if ((lane & (LPB - 1)) == 0) my_sm_row[j * 4] = (uint8_t)(254u - ie);
-            if (live) {
+            if (j < rows_here) {   // warp-uniform; lanes beyond the tensor's last column take part but do not store
                 float iv[VEC], sv[VEC];
 #pragma unroll
                 for (int i = 0; i < VEC; ++i) { iv[i] = inv; sv[i] = scale_from_inv(inv); }
-                emit<ELEM, VEC, EMU>(my_qrow + (uint64_t)j * pitch, x, iv, sv);
+                emit<ELEM, VEC, EMU>(my_qrow + (uint64_t)j * pitch, x, iv, sv, lane, live);
             }
         }
-        if (DO_COL && live) emit<ELEM, VEC, EMU>(my_qcol + (uint64_t)j * pitch, x, col_inv, col_xs);
+        if (DO_COL && j < rows_here) emit<ELEM, VEC, EMU>(my_qcol + (uint64_t)j * pitch, x, col_inv, col_xs, lane, live);
     }
 }
 

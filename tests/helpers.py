@@ -87,7 +87,14 @@ def gpu_quantize(src_np, dtype: str, orientation: int, rule: int, elem: int, sf_
     for name, (q, s) in bufs.items():
         q.check("q_" + name)
         s.check("s_" + name)
-        out["q_" + name] = q.numpy().reshape(rows, cols)
+        raw_q = q.numpy().reshape(rows, cols)
+        if orc.code_bits(elem) < 8:
+            # 6- and 4-bit codes come in packed 16-byte slots: padding must be zero, then compare code by code
+            pad_from = 12 if orc.code_bits(elem) == 6 else 8
+            assert not raw_q.reshape(rows, cols // 16, 16)[:, :, pad_from:].any(), "slot padding must be 0"
+            out["packed_q_" + name] = raw_q
+            raw_q = orc.unpack_codes16(raw_q, elem)
+        out["q_" + name] = raw_q
         raw = s.numpy()
         if name == "row":
             mn, nkb = rows, cols // 32

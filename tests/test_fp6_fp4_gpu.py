@@ -40,9 +40,9 @@ def test_value_distributions(dist, dtype, elem):
         check_against_oracle(x, dtype, BOTH, rule, elem, SWIZZLED, "%s rule=%d" % (dist, rule))
 
 
-@pytest.mark.parametrize("shape", [(32, 32), (7, 64), (160, 352), (384, 8288), (64, 100), (64, 33)])
+@pytest.mark.parametrize("shape", [(32, 32), (7, 64), (160, 352), (384, 2080), (64, 48), (96, 16)])
 @pytest.mark.parametrize("elem", ELEMS)
-def test_ragged_shapes_and_generic_path(shape, elem):
+def test_ragged_shapes(shape, elem):
     rows, cols = shape
     for dtype in ("fp32", "bf16"):
         x = as_dtype(synth.student_t(shape, 77 + rows + cols), dtype)
@@ -78,7 +78,8 @@ def test_dequantize_exhaustive_codes_and_scales(elem, dst):
     s = np.repeat(np.arange(256, dtype=np.uint8)[:, None], 256, axis=1)
     want = orc.dequantize(q, s, orc.ROW, elem, dst)
     out = torch.empty(q.shape, dtype=torch.float32 if dst == "f32" else torch.bfloat16, device="cuda")
-    B.mxfp8_dequantize(torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda().view(-1), B.ROW, elem, B.SF_LINEAR, out)
+    B.mxfp8_dequantize(torch.from_numpy(orc.pack_codes16(q, elem)).cuda(), torch.from_numpy(s).cuda().view(-1), B.ROW, elem,
+                       B.SF_LINEAR, out)
     torch.cuda.synchronize()
     if dst == "f32":
         got = out.cpu().numpy()
@@ -101,15 +102,66 @@ def test_fake_quantize_round_trip(elem, dtype):
             check_round_trip(x, dtype, BOTH, rule, elem, "%s rule=%d" % (dist, rule))
 
 
-def test_gemm_rejects_sub_byte_operands_as_unsupported():
+def test_widths_that_do_not_fill_slots_are_unsupported():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    x = torch.zeros(64, 40, dtype=torch.bfloat16, device="cuda")           # 40 columns: no whole 16-code slots
+    _, _, qc, sc = B.alloc_quantize_outputs(64, 40, B.COL, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_quantize(x, B.COL, B.RULE_PAPER, B.E2M3, None, None, qc, sc, B.SF_LINEAR)
+    assert e.value.status == -5
+    B.mxfp8_quantize(x, B.COL, B.RULE_PAPER, B.E4M3, None, None, qc, sc, B.SF_LINEAR)   # fine for 8-bit codes
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_dequantize(qc, sc, B.COL, B.E2M1, B.SF_LINEAR, torch.empty(64, 40, device="cuda"))
+    assert e.value.status == -5
+
+
+MIXES = [(orc.E2M3, orc.E2M3), (orc.E3M2, orc.E3M2), (orc.E2M1, orc.E2M1), (orc.E2M3, orc.E4M3), (orc.E5M2, orc.E2M1),
+         (orc.E3M2, orc.E2M1)]
+
+
+@pytest.mark.parametrize("mix", MIXES)
+@pytest.mark.parametrize("majors", ["kk", "km", "mm"])
+def test_gemm_on_six_and_four_bit_operands(mix, majors):
+    # mxfp8_quantize writes the operands (packed slots, swizzled scales), mxfp8_gemm multiplies them on the
+    # tensor cores; the oracle quantizes and multiplies the same inputs in FP64
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import check_gemm_tolerance
+    a_elem, b_elem = mix
+    a_mn, b_mn = majors[0] == "m", majors[1] == "m"
+    M, N, K = 384, 256, 512
+    a = synth.gaussian((M, K), 3)
+    b = synth.student_t((N, K), 4) * np.float32(0.1)
+
+    def prep(x, elem, mn):
+        stored = np.ascontiguousarray(x.T) if mn else x                     # MN-major: stored [K, MN], blocks run down K
+        o = B.COL if mn else B.ROW
+        outs = B.alloc_quantize_outputs(stored.shape[0], stored.shape[1], o, B.SF_SWIZZLED)
+        B.mxfp8_quantize(torch.from_numpy(stored).cuda(), o, B.RULE_PAPER, elem, *outs, B.SF_SWIZZLED)
+        q, s = (outs[2], outs[3]) if mn else (outs[0], outs[1])
+        oq, os_ = orc.quantize(stored, orc.COL if mn else orc.ROW, orc.RULE_PAPER, elem)
+        return q, s, oq, os_
+
+    qa, sa, oqa, osa = prep(a, a_elem, a_mn)
+    qb, sb, oqb, osb = prep(b, b_elem, b_mn)
+    D = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    B.mxfp8_gemm(qa, sa, qb, sb, M, N, K, B.MN_MAJOR if a_mn else B.K_MAJOR, B.MN_MAJOR if b_mn else B.K_MAJOR, a_elem, b_elem, D)
+    assert B.mxfp8_device_status() == 0
+    d64, sabs = orc.gemm_f64(oqa, osa, oqb, osb, "mn" if a_mn else "k", "mn" if b_mn else "k", a_elem, b_elem)
+    check_gemm_tolerance(D.cpu().numpy(), d64, sabs, "%s %s" % (mix, majors))
+
+
+def test_gemm_rejects_unknown_element_codes_and_sub_byte_fused_output():
     import torch
     from paper_2506_08027_b200 import binding as B
     z = torch.zeros(128, 128, dtype=torch.uint8, device="cuda")
     sc = torch.zeros(512, dtype=torch.uint8, device="cuda")
     D = torch.empty(128, 128, dtype=torch.float32, device="cuda")
     with pytest.raises(B.Mxfp8Error) as e:
-        B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, B.E2M3, B.E4M3, D)
-    assert e.value.status == -5
-    with pytest.raises(B.Mxfp8Error) as e:
         B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, 2, B.E4M3, D)     # 2 is no element code
     assert e.value.status == -2
+    epi = B.make_epilogue(B.ROW, B.RULE_PAPER, B.E2M3, z, sc)
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, B.E4M3, B.E4M3, D, epi=epi)
+    assert e.value.status == -5

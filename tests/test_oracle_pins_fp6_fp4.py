@@ -160,3 +160,26 @@ def test_quantize_dequantize_blocks_bruteforce(elem):
                                  np.abs(x).reshape(2, 32, 96).max(axis=1, keepdims=True).repeat(32, axis=1).reshape(64, 96))
         mbits = {orc.E2M3: 3, orc.E3M2: 2, orc.E2M1: 1}[elem]
         assert (rel[amax_pos & (x != 0)] <= 2.0 ** -(mbits + 1)).all()
+
+
+def test_packed_slot_layout_hand_worked():
+    # 4-bit: two codes per byte, the earlier code in the low nibble; 8 data bytes, 8 zero bytes
+    c4 = np.arange(16, dtype=np.uint8)[None, :]
+    p4 = orc.pack_codes16(c4, orc.E2M1)
+    assert p4[0].tolist() == [0x10, 0x32, 0x54, 0x76, 0x98, 0xBA, 0xDC, 0xFE] + [0] * 8
+    # 6-bit: a little-endian bit stream; codes 1, 0x3F, 0, 0x2A, ... worked by hand:
+    #   bits 0-5 = 000001, bits 6-11 = 111111, bits 12-17 = 000000, bits 18-23 = 101010
+    #   byte0 = 11|000001 = 0xC1, byte1 = 0000|1111 = 0x0F, byte2 = 101010|00 = 0xA8
+    c6 = np.zeros((1, 16), np.uint8)
+    c6[0, :4] = [1, 0x3F, 0, 0x2A]
+    c6[0, 15] = 0x3F                                  # last code: bits 90-95 = top six bits of byte 11
+    p6 = orc.pack_codes16(c6, orc.E2M3)
+    assert p6[0, :3].tolist() == [0xC1, 0x0F, 0xA8]
+    assert p6[0, 11] == 0xFC and p6[0, 3:11].tolist() == [0] * 8 and p6[0, 12:].tolist() == [0] * 4
+    # round trip on random codes, several slots and rows; 8-bit codes pass through
+    rng = np.random.default_rng(1)
+    for elem, hi in ((orc.E2M3, 64), (orc.E3M2, 64), (orc.E2M1, 16), (orc.E4M3, 256)):
+        c = rng.integers(0, hi, (5, 64)).astype(np.uint8)
+        assert np.array_equal(orc.unpack_codes16(orc.pack_codes16(c, elem), elem), c)
+    with pytest.raises(ValueError):
+        orc.pack_codes16(np.zeros((2, 24), np.uint8), orc.E2M1)
