@@ -195,6 +195,25 @@ size_t mxfp8_scale_bytes(int64_t rows, int64_t cols, int orientation, int sf_lay
 int64_t mxfp8_sf_offset(int64_t mn, int64_t kblock, int64_t n_kblocks, int sf_layout);
 
 /*
+ * mxfp8_gemm_multi -- up to 3 independent block-scaled products in ONE launch.  FPROP, DGRAD and WGRAD of
+ * a layer (Sec. 3.2) are independent once the MXFP8 copies exist; dealt out as one pool of tiles they fill
+ * the machine evenly where each alone would end on a partly idle wave.  Every product follows
+ * mxfp8_gemm's definition, argument rules and tolerance (no fused MXFP8 output here); the outputs share
+ * `out_dtype`.  `problems`: HOST array of `count` entries with device pointers; outputs must not
+ * overlap each other or any operand.  (The batching itself has no counterpart in the paper.)
+ */
+typedef struct mxfp8_gemm_problem {
+    const void* Aq;
+    const void* As;
+    const void* Bq;
+    const void* Bs;
+    int64_t M, N, K;
+    int a_major, b_major, a_elem, b_elem;
+    void* D;
+} mxfp8_gemm_problem;
+int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, int out_dtype, void* stream);
+
+/*
  * mxfp8_grouped_gemm -- the per-expert products of a mixture-of-experts layer in one launch (App. A.4
  * trains a mixture-of-experts model with the same recipe; each expert's FPROP / DGRAD / WGRAD is the
  * block-scaled product of Sec. 2 restricted to the tokens routed to that expert).
@@ -261,8 +280,8 @@ int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64
  *     FPROP  Y  [T, F] = X  * W^T   (row-blocked X,  row-blocked W)
  *     DGRAD  dX [T, H] = dY * W     (row-blocked dY, column-blocked W)
  *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
- * run as block-scaled GEMMs with BF16 output: four kernel launches on `stream` (the three casts
- * share one), no wait.
+ * run as block-scaled GEMMs with BF16 output: two kernel launches on `stream` (the three casts
+ * share one, the three GEMMs share one), no wait.  Y, dX, dW must not overlap.
  * T, H, F must be multiples of 128 (ERR_UNSUPPORTED).  ws: device scratch for the quantized
  * copies, mxfp8_linear_ws_bytes() bytes, 256-byte aligned, owned by the caller.  All tensors
  * 16-byte aligned, row-major, dense.

@@ -27,7 +27,7 @@ EXPORTS = (
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
-    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi",
+    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi",
 )
 
 
@@ -41,6 +41,13 @@ class _QuantizeItem(ctypes.Structure):
     _fields_ = [("src", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
                 ("q_row", ctypes.c_void_p), ("s_row", ctypes.c_void_p),
                 ("q_col", ctypes.c_void_p), ("s_col", ctypes.c_void_p)]
+
+
+class _GemmProblem(ctypes.Structure):
+    _fields_ = [("Aq", ctypes.c_void_p), ("As", ctypes.c_void_p), ("Bq", ctypes.c_void_p), ("Bs", ctypes.c_void_p),
+                ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("a_major", ctypes.c_int), ("b_major", ctypes.c_int), ("a_elem", ctypes.c_int), ("b_elem", ctypes.c_int),
+                ("D", ctypes.c_void_p)]
 
 
 class _Epilogue(ctypes.Structure):
@@ -87,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
         L.mxfp8_fake_quantize.restype = i
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_gemm_multi.restype = i
+        L.mxfp8_gemm_multi.argtypes = [ctypes.POINTER(_GemmProblem), i, i, p]
         L.mxfp8_quantize_multi.restype = i
         L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
         L.mxfp8_grouped_gemm.restype = i
@@ -272,3 +281,19 @@ def mxfp8_quantize_multi(items, src_dtype: int, orientation: int, scale_rule: in
                          stream=None) -> None:
     _check(lib().mxfp8_quantize_multi(items, len(items), src_dtype, orientation, scale_rule, elem, sf_layout,
                                       _stream(stream)), "mxfp8_quantize_multi")
+
+
+def make_gemm_problems(entries):
+    """entries: sequence of (Aq, As, Bq, Bs, M, N, K, a_major, b_major, a_elem, b_elem, D).  Returns the ctypes
+    array mxfp8_gemm_multi takes; build it once and reuse it while the tensors live."""
+    arr = (_GemmProblem * len(entries))()
+    for k, (aq, a_s, bq, b_s, M, N, K, a_major, b_major, a_elem, b_elem, D) in enumerate(entries):
+        arr[k].Aq, arr[k].As, arr[k].Bq, arr[k].Bs = aq.data_ptr(), a_s.data_ptr(), bq.data_ptr(), b_s.data_ptr()
+        arr[k].M, arr[k].N, arr[k].K = M, N, K
+        arr[k].a_major, arr[k].b_major, arr[k].a_elem, arr[k].b_elem = a_major, b_major, a_elem, b_elem
+        arr[k].D = D.data_ptr()
+    return arr
+
+
+def mxfp8_gemm_multi(problems, out_dtype: int, stream=None) -> None:
+    _check(lib().mxfp8_gemm_multi(problems, len(problems), out_dtype, _stream(stream)), "mxfp8_gemm_multi")

@@ -129,8 +129,8 @@ LinearWs plan_linear(char* base, int64_t T, int64_t H, int64_t F, bool staging)
     return w;
 }
 
-// The four launches of one step on device buffers: the three BOTH-orientation conversions in one, then
-// FPROP, DGRAD and WGRAD (Sec. 3.2).
+// The two launches of one step on device buffers: the three BOTH-orientation conversions in one, then
+// FPROP, DGRAD and WGRAD in one (Sec. 3.2).
 int linear_device(const LinearWs& w, const void* x, const void* wt, const void* dy, int64_t T, int64_t H, int64_t F,
                   int scale_rule, void* y, void* dx, void* dw, void* stream)
 {
@@ -143,14 +143,13 @@ int linear_device(const LinearWs& w, const void* x, const void* wt, const void* 
         if (rc != MXFP8_OK) return rc;
     }
     enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
-    int rc = mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR,
-                        MXFP8_E4M3, MXFP8_E4M3, y, MXFP8_BF16, nullptr, nullptr, 0, stream);
-    if (rc != MXFP8_OK) return rc;
-    rc = mxfp8_gemm(w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR,
-                    MXFP8_E4M3, MXFP8_E4M3, dx, MXFP8_BF16, nullptr, nullptr, 0, stream);
-    if (rc != MXFP8_OK) return rc;
-    return mxfp8_gemm(w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR,
-                      MXFP8_E4M3, MXFP8_E4M3, dw, MXFP8_BF16, nullptr, nullptr, 0, stream);
+    // FPROP, DGRAD, WGRAD are independent once the copies exist: one launch over the tiles of all three
+    const mxfp8_gemm_problem gemms[3] = {
+        {w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR, MXFP8_E4M3, MXFP8_E4M3, y},
+        {w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, dx},
+        {w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, dw},
+    };
+    return mxfp8_gemm_multi(gemms, 3, MXFP8_BF16, stream);
 }
 
 int linear_check(int64_t T, int64_t H, int64_t F, int scale_rule)

@@ -56,6 +56,18 @@ constexpr int EPI_BUF_BYTES = 2048;   // 32 rows x 64 bytes per epilogue warp
 constexpr int TMEM_COLS = 512;
 constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;  // bounded waits give up after 1 s
 
+// MULTI mode: several independent products share one launch (one pool of tiles over all of them)
+constexpr int MAX_PROBLEMS = 3;
+struct MultiProblem {
+    int M, N;             // output extent
+    int a_mn, b_mn, a_elem, b_elem;
+    int tiles_m, tiles_n, num_kb;
+    int tile_start;       // first tile of this problem in the launch-wide numbering
+    uint32_t stage_tx;
+};
+struct ProblemMaps { CUtensorMap a, b, sfa, sfb, d; };
+struct MultiMaps { ProblemMaps p[MAX_PROBLEMS]; };
+
 struct GemmParams {
     int64_t M, N, K;
     int a_mn, b_mn;       // 1 = MN-major storage
@@ -73,13 +85,16 @@ struct GemmParams {
     const int32_t* group_offsets;
     int num_groups;
     int token_limit;      // offsets may not pass this (tokens in the grouped tensor)
+    int num_problems;     // MULTI
+    MultiProblem mp[MAX_PROBLEMS];
 };
 
 constexpr int MAX_GROUPS = 256;
 // MODE of the kernel: one dense product, or one product per expert of a mixture-of-experts layer
 //   GROUP_M: the rows of A (tokens) are grouped, B holds one matrix per expert   (fprop, dgrad)
 //   GROUP_K: the reduction axis (tokens) is grouped, D holds one matrix per expert (wgrad)
-enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2 };
+//   MULTI  : up to MAX_PROBLEMS independent dense products, tiles of all of them dealt out as one pool
+enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2, MULTI = 3 };
 
 // BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
 // tile has 2*BM rows.  BN = 256 leaves room for one accumulator only (2 x 256 columns would fill
@@ -468,13 +483,21 @@ struct TileCtx {
     int bn_off;         // added to B's MN coordinate
     int sfb_atom_off;   // added to the MN atom index of B's scales
     int nkb;            // K blocks of this tile
+    int prob;           // MULTI: which product the tile belongs to
 };
 
 template <int MODE, int TM>
 __device__ __forceinline__ TileCtx decode_tile(const GemmParams& p, const int* goff, const int* tstart, int tile, int& g)
 {
     TileCtx t;
-    if constexpr (MODE == DENSE) {
+    t.prob = 0;
+    if constexpr (MODE == MULTI) {
+        while (g + 1 < p.num_problems && tile >= p.mp[g + 1].tile_start) ++g;      // tiles only move forward: g is a cursor
+        const MultiProblem& q = p.mp[g];
+        tile_coords(p.group_m, q.tiles_m, q.tiles_n, tile - q.tile_start, t.tm, t.tn);
+        t.row0 = 0; t.d_row_extra = 0; t.rows_end = q.M; t.ka0 = 0; t.kb0 = 0; t.bn_off = 0; t.sfb_atom_off = 0;
+        t.nkb = q.num_kb; t.prob = g;
+    } else if constexpr (MODE == DENSE) {
         tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile, t.tm, t.tn);
         t.row0 = 0; t.d_row_extra = 0; t.rows_end = (int)p.M; t.ka0 = 0; t.kb0 = 0; t.bn_off = 0; t.sfb_atom_off = 0;
         t.nkb = p.num_kb;
@@ -502,7 +525,15 @@ template <int MODE>
 __device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const int* goff, int num_tiles, int worker, int workers)
 {
     if (num_tiles <= worker) return 0u;
-    if constexpr (MODE != GROUP_K) {
+    if constexpr (MODE == MULTI) {
+        uint32_t total = 0;
+        int g = 0;
+        for (int tile = worker; tile < num_tiles; tile += workers) {
+            while (g + 1 < p.num_problems && tile >= p.mp[g + 1].tile_start) ++g;
+            total += (uint32_t)p.mp[g].num_kb;
+        }
+        return total;
+    } else if constexpr (MODE != GROUP_K) {
         return (uint32_t)((num_tiles - worker + workers - 1) / workers) * (uint32_t)p.num_kb;
     } else {
         const int per_expert = p.tiles_m * p.tiles_n;
@@ -520,7 +551,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
             const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_qrow,
-            const __grid_constant__ CUtensorMap tmap_qcol, const GemmParams p)
+            const __grid_constant__ CUtensorMap tmap_qcol, const __grid_constant__ MultiMaps mmaps,
+            const __grid_constant__ GemmParams p)
 {
     using C = Cfg<BN, PAIR>;
     extern __shared__ uint8_t smem_raw[];
@@ -558,7 +590,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         *bad_groups = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if constexpr (MODE != DENSE) {
+    if constexpr (MODE == GROUP_M || MODE == GROUP_K) {
         // every CTA reads the offsets, checks them (non-negative, non-decreasing, multiples of 128,
         // inside the tensor) and, for GROUP_M, turns them into the first tile index of each group
         const int G = p.num_groups;
@@ -608,7 +640,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // tiles of the whole launch (none when the offsets were rejected)
-    const int num_tiles = MODE == DENSE ? p.num_tiles
+    const int num_tiles = (MODE == DENSE || MODE == MULTI) ? p.num_tiles
                         : (*bad_groups ? 0 : (MODE == GROUP_M ? tstart[p.num_groups] : p.num_groups * p.tiles_m * p.tiles_n));
 
     if (warp == 0) {
@@ -616,7 +648,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
         // ring-depth-unrolled loop as the MMA warp.
         {
-            const int a_mn = p.a_mn, b_mn = p.b_mn;
+            int a_mn = p.a_mn, b_mn = p.b_mn;
+            uint32_t stage_tx = p.stage_tx;
+            const CUtensorMap *ma = &tmap_a, *mb = &tmap_b, *msfa = &tmap_sfa, *msfb = &tmap_sfb;
             const uint32_t total = worker_k_blocks<MODE>(p, goff, num_tiles, worker, workers);
             int kb = 0, tile = worker, gcur = 0;
             int m_atom = 0, m0 = 0, n0 = 0, sfb_atom0 = 0, ka0 = 0, kb0 = 0, nkb = p.num_kb;
@@ -636,6 +670,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                         n0 = t.bn_off + t.tn * BN + (PAIR ? (int)cta_rank * C::B_ROWS : 0);    // first B row this CTA loads
                         sfb_atom0 = t.sfb_atom_off + ((t.tn * BN) >> 7);              // scale atom holding the tile's first column
                         ka0 = t.ka0; kb0 = t.kb0; nkb = t.nkb;
+                        if constexpr (MODE == MULTI) {
+                            const MultiProblem& q = p.mp[t.prob];
+                            a_mn = q.a_mn; b_mn = q.b_mn; stage_tx = q.stage_tx;
+                            ma = &mmaps.p[t.prob].a; mb = &mmaps.p[t.prob].b; msfa = &mmaps.p[t.prob].sfa; msfb = &mmaps.p[t.prob].sfb;
+                        }
                     }
                     ok = warp_wait(empty_bar(s), ph ^ 1u, abort_flag);
                     if (!ok) break;
@@ -645,19 +684,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     const uint32_t sb = base + C::SMEM_B + s * C::B_BYTES;
                     const int k0a = (ka0 + kb) * BK, k0b = (kb0 + kb) * BK;
                     if (elect_one()) {
-                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), p.stage_tx);
-                        if (!a_mn) tma_load_2d<PAIR>(sa, &tmap_a, fb, k0a, m0);
-                        else tma_load_2d<PAIR>(sa, &tmap_a, fb, m0, k0a);
+                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
+                        if (!a_mn) tma_load_2d<PAIR>(sa, ma, fb, k0a, m0);
+                        else tma_load_2d<PAIR>(sa, ma, fb, m0, k0a);
                         if (!b_mn) {
-                            tma_load_2d<PAIR>(sb, &tmap_b, fb, k0b, n0);
+                            tma_load_2d<PAIR>(sb, mb, fb, k0b, n0);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < C::B_SLABS; ++j) tma_load_2d<PAIR>(sb + j * 16384, &tmap_b, fb, n0 + j * 128, k0b);
+                            for (int j = 0; j < C::B_SLABS; ++j) tma_load_2d<PAIR>(sb + j * 16384, mb, fb, n0 + j * 128, k0b);
                         }
-                        tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, &tmap_sfa, fb, 0, ka0 + kb, m_atom);
+                        tma_load_3d<PAIR>(base + C::SMEM_SFA + s * 512, msfa, fb, 0, ka0 + kb, m_atom);
 #pragma unroll
                         for (int j = 0; j < C::SFB_ATOMS; ++j)      // every CTA needs the scales of all BN columns
-                            tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, &tmap_sfb, fb, 0, kb0 + kb,
+                            tma_load_3d<PAIR>(base + C::SMEM_SFB + (s * C::SFB_ATOMS + j) * 512, msfb, fb, 0, kb0 + kb,
                                               sfb_atom0 + j);
                     }
                     __syncwarp();
@@ -677,16 +716,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // tiles of this worker and is unrolled by the ring depth, so the stage index is a
         // compile-time constant and every descriptor is "loop-invariant base + immediate".
         if (cta_rank == 0) {
-            const uint32_t idesc0 = make_idesc(p.a_elem, p.b_elem, p.a_mn, p.b_mn, PAIR ? 2 * BM : BM, BN);
+            uint32_t idesc0 = make_idesc(p.a_elem, p.b_elem, p.a_mn, p.b_mn, PAIR ? 2 * BM : BM, BN);
             // Descriptors differ between stages and K steps only in the 14-bit start-address
             // field (16-byte units): keep the constant upper word and step the lower one.
             //   K-major : next K step = 32 bytes along the swizzled row (2 units); 8-row groups 1024 B apart.
             //   MN-major: next K step = 32 K-rows = 4096 bytes (256 units); 8-K-row groups 1024 B apart,
             //             128-wide MN slabs 16384 B apart.
             const uint32_t op_hi = (uint32_t)(smem_desc(0, 0, 1024, 2) >> 32);
-            const uint32_t a_lo0 = ((base + C::SMEM_A) >> 4) | (p.a_mn ? (16384u >> 4) << 16 : 0u);
-            const uint32_t b_lo0 = ((base + C::SMEM_B) >> 4) | (p.b_mn ? (16384u >> 4) << 16 : 0u);
-            const uint32_t a_kstep = p.a_mn ? 256u : 2u, b_kstep = p.b_mn ? 256u : 2u;
+            uint32_t a_lo0 = ((base + C::SMEM_A) >> 4) | (p.a_mn ? (16384u >> 4) << 16 : 0u);
+            uint32_t b_lo0 = ((base + C::SMEM_B) >> 4) | (p.b_mn ? (16384u >> 4) << 16 : 0u);
+            uint32_t a_kstep = p.a_mn ? 256u : 2u, b_kstep = p.b_mn ? 256u : 2u;
             const uint32_t sf_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);   // scales: 32 rows x 16 B, 8-row groups 128 B apart
             const uint32_t sfa_lo0 = (base + C::SMEM_SFA) >> 4, sfb_lo0 = (base + C::SMEM_SFB) >> 4;
             auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
@@ -706,6 +745,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                             while (t.nkb == 0) { tile += workers; t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur); }   // expert without tokens
                         }
                         num_kb = t.nkb;
+                        if constexpr (MODE == MULTI) {   // the product's own formats and majors
+                            const MultiProblem& q = p.mp[t.prob];
+                            idesc0 = make_idesc(q.a_elem, q.b_elem, q.a_mn, q.b_mn, PAIR ? 2 * BM : BM, BN);
+                            a_lo0 = ((base + C::SMEM_A) >> 4) | (q.a_mn ? (16384u >> 4) << 16 : 0u);
+                            b_lo0 = ((base + C::SMEM_B) >> 4) | (q.b_mn ? (16384u >> 4) << 16 : 0u);
+                            a_kstep = q.a_mn ? 256u : 2u;
+                            b_kstep = q.b_mn ? 256u : 2u;
+                        }
                         // a tile that starts in the middle of a 128-wide scale atom reads its B scales from
                         // the matching TMEM column of the copied atoms (32 columns of B per TMEM column)
                         sfb_skip = (uint32_t)(((t.tn * BN) & 127) >> 5);
@@ -760,11 +807,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         const uint32_t sw = (uint32_t)((lane >> 1) & 3);
         uint32_t acc_it = 0;
         bool ok = true;
-        const int n_total = (int)p.N;
+        int n_total = (int)p.N;
+        const CUtensorMap* md = &tmap_d;
         int gcur = 0;
         for (int tile = worker; tile < num_tiles && ok; tile += workers) {
             const TileCtx t = decode_tile<MODE, TM>(p, goff, tstart, tile, gcur);
             const int tm = t.tm, tn = t.tn;
+            if constexpr (MODE == MULTI) { n_total = p.mp[t.prob].N; md = &mmaps.p[t.prob].d; }
             uint32_t v[CW];
             if (MODE == GROUP_K && t.nkb == 0) {
                 // an expert without tokens: its product is all zeros and no MMA ran for this tile
@@ -823,7 +872,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     __syncwarp();
                     if (lane == 0) {
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&tmap_d), "r"(col0 + ch * 32), "r"(row0), "r"(buf) : "memory");
+                                     ::"l"(md), "r"(col0 + ch * 32), "r"(row0), "r"(buf) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
@@ -842,7 +891,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     __syncwarp();
                     if (lane == 0) {
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&tmap_d), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
+                                     ::"l"(md), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
@@ -951,7 +1000,7 @@ int sm_count()
     return n;
 }
 
-struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; };
+struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; MultiMaps multi; };
 
 template <int BN, bool PAIR, int MODE = DENSE>
 int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
@@ -966,6 +1015,19 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.num_kb = (int)((p.K + BK - 1) / BK);   // a ragged K tail is zero-filled by TMA (operands) and by the scale pads
     p.group_m = 16;
+    if (MODE == MULTI) {
+        int64_t tiles = 0;
+        for (int i = 0; i < p.num_problems; ++i) {
+            MultiProblem& q = p.mp[i];
+            q.tiles_m = (q.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM);
+            q.tiles_n = (q.N + BN - 1) / BN;
+            q.stage_tx = (PAIR ? 2u : 1u) * (uint32_t)(C::A_BYTES + (q.b_mn ? C::B_BYTES_MN : C::B_BYTES_K) + 512 + 512 * C::SFB_ATOMS);
+            q.tile_start = (int)tiles;
+            tiles += (int64_t)q.tiles_m * q.tiles_n;
+            if (tiles > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
+        }
+        p.num_tiles = (int)tiles;
+    }
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
     const int max_workers = PAIR ? sms / 2 : sms;
@@ -987,7 +1049,7 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, m.multi, p);
     if (getenv("MXFP8_LOG"))
         fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d -> %s\n", cfg.gridDim.x, GEMM_THREADS,
                 C::SMEM_TOTAL, p.tiles_m, p.tiles_n, p.num_kb, cudaGetErrorString(err));
@@ -1168,4 +1230,50 @@ extern "C" int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (mode == MXFP8_GROUP_M) return pair ? launch_gemm<256, true, GROUP_M>(m, p, st) : launch_gemm<256, false, GROUP_M>(m, p, st);
     return pair ? launch_gemm<256, true, GROUP_K>(m, p, st) : launch_gemm<256, false, GROUP_K>(m, p, st);
+}
+
+extern "C" int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, int out_dtype, void* stream)
+{
+    using namespace mxfp8;
+    if (!problems) return MXFP8_ERR_NULL;
+    if (count < 1) return MXFP8_ERR_SHAPE;
+    if (count > MAX_PROBLEMS) return MXFP8_ERR_UNSUPPORTED;
+    if (out_dtype != MXFP8_FP32 && out_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    GemmParams p{};
+    p.out_dtype = out_dtype;
+    p.store_d = 1;
+    p.num_problems = count;
+    GemmMaps m;
+    for (int i = 0; i < MAX_PROBLEMS; ++i) {
+        const mxfp8_gemm_problem& g = problems[i < count ? i : 0];   // unused slots repeat the first product: every map stays valid
+        if (i < count) {
+            if (g.a_major != MXFP8_K_MAJOR && g.a_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
+            if (g.b_major != MXFP8_K_MAJOR && g.b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
+            if (!valid_elem(g.a_elem) || !valid_elem(g.b_elem)) return MXFP8_ERR_ENUM;
+            if (!g.Aq || !g.As || !g.Bq || !g.Bs || !g.D) return MXFP8_ERR_NULL;
+            if (g.M <= 0 || g.N <= 0 || g.K <= 0 || (g.K % 32)) return MXFP8_ERR_SHAPE;
+            if (g.a_major == MXFP8_MN_MAJOR && (g.M % 16)) return MXFP8_ERR_UNSUPPORTED;
+            if (g.b_major == MXFP8_MN_MAJOR && (g.N % 16)) return MXFP8_ERR_UNSUPPORTED;
+            if (g.N % (out_dtype == MXFP8_FP32 ? 4 : 8)) return MXFP8_ERR_UNSUPPORTED;
+            if (g.M > 0x3FFFFFFF || g.N > 0x3FFFFFFF || g.K > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
+            if (!aligned16(g.Aq) || !aligned16(g.As) || !aligned16(g.Bq) || !aligned16(g.Bs) || !aligned16(g.D)) return MXFP8_ERR_ALIGN;
+            MultiProblem& q = p.mp[i];
+            q.M = (int)g.M; q.N = (int)g.N; q.num_kb = (int)((g.K + BK - 1) / BK);
+            q.a_mn = g.a_major; q.b_mn = g.b_major; q.a_elem = g.a_elem; q.b_elem = g.b_elem;
+        }
+        ProblemMaps& pm = m.multi.p[i];
+        bool ok = g.a_major == MXFP8_K_MAJOR ? make_tmap(&pm.a, g.Aq, (uint64_t)g.K, (uint64_t)g.M, 128, 128)
+                                             : make_tmap(&pm.a, g.Aq, (uint64_t)g.M, (uint64_t)g.K, 128, 128);
+        ok = ok && (g.b_major == MXFP8_K_MAJOR ? make_tmap(&pm.b, g.Bq, (uint64_t)g.K, (uint64_t)g.N, 128, 128)   // pair tiles: 128 B rows per CTA
+                                               : make_tmap(&pm.b, g.Bq, (uint64_t)g.N, (uint64_t)g.K, 128, 128));
+        ok = ok && make_tmap_sf(&pm.sfa, g.As, (uint64_t)((g.M + 127) / 128), (uint64_t)((g.K + 127) / 128));
+        ok = ok && make_tmap_sf(&pm.sfb, g.Bs, (uint64_t)((g.N + 127) / 128), (uint64_t)((g.K + 127) / 128));
+        ok = ok && make_tmap_d(&pm.d, g.D, (uint64_t)g.M, (uint64_t)g.N, out_dtype);
+        if (!ok) return MXFP8_ERR_CUDA;
+    }
+    // the single-product parameters and maps are unused in this mode but must be valid
+    p.M = problems[0].M; p.N = problems[0].N; p.K = problems[0].K;
+    m.a = m.multi.p[0].a; m.b = m.multi.p[0].b; m.sfa = m.multi.p[0].sfa; m.sfb = m.multi.p[0].sfb; m.d = m.multi.p[0].d;
+    m.qrow = m.d; m.qcol = m.d;
+    return launch_gemm<256, true, MULTI>(m, p, static_cast<cudaStream_t>(stream));
 }

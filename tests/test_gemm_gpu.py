@@ -327,3 +327,81 @@ def test_ragged_shapes(shape, majors):
         gotb = gpu_gemm(A, SA, B_, SB, majors[0], majors[1], out="bf16")
         import torch
         assert np.array_equal(gotb, torch.from_numpy(got).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+
+
+def _multi_case(M, N, K, a_mn, b_mn, a_elem, b_elem, seed):
+    """Operands quantized by the oracle; returns device tensors, problem tuple pieces and the FP64 result."""
+    import torch
+    from helpers import swizzle_np
+    a = synth.gaussian((M, K), seed)
+    b = synth.student_t((N, K), seed + 1) * np.float32(0.05)
+    def prep(x, elem, mn):
+        stored = np.ascontiguousarray(x.T) if mn else x
+        q, s = orc.quantize(stored, orc.COL if mn else orc.ROW, orc.RULE_PAPER, elem)
+        logical = np.ascontiguousarray(s.T) if mn else s
+        return q, s, torch.from_numpy(orc.pack_codes16(q, elem)).cuda(), torch.from_numpy(swizzle_np(logical)).cuda()
+    aq, a_s, da, dsa = prep(a, a_elem, a_mn)
+    bq, b_s, db, dsb = prep(b, b_elem, b_mn)
+    d64, sabs = orc.gemm_f64(aq, a_s, bq, b_s, "mn" if a_mn else "k", "mn" if b_mn else "k", a_elem, b_elem)
+    return da, dsa, db, dsb, d64, sabs
+
+
+@pytest.mark.parametrize("out", ["fp32", "bf16"])
+def test_gemm_multi_equals_separate_products_and_oracle(out):
+    # three products of different shapes, majors and element types (one ragged, one with 6-bit operands) in one
+    # launch: each output equals the single-product launch bit for bit and the oracle within the tolerance
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    specs = [(512, 768, 256, False, False, orc.E4M3, orc.E4M3),
+             (384, 256, 1024, False, True, orc.E5M2, orc.E4M3),
+             (336, 208, 512, True, True, orc.E2M3, orc.E4M3)]
+    dt = torch.float32 if out == "fp32" else torch.bfloat16
+    cases, entries, outs = [], [], []
+    for i, (M, N, K, a_mn, b_mn, ae, be) in enumerate(specs):
+        c = _multi_case(M, N, K, a_mn, b_mn, ae, be, 40 + 3 * i)
+        D = torch.full((M, N), float("nan"), dtype=dt, device="cuda")
+        cases.append(c); outs.append(D)
+        entries.append((c[0], c[1], c[2], c[3], M, N, K, int(a_mn), int(b_mn), ae, be, D))
+    before = B.mxfp8_launch_count()
+    B.mxfp8_gemm_multi(B.make_gemm_problems(entries), B.FP32 if out == "fp32" else B.BF16)
+    assert B.mxfp8_device_status() == 0
+    assert B.mxfp8_launch_count() - before == 1
+    for (M, N, K, a_mn, b_mn, ae, be), c, D in zip(specs, cases, outs):
+        single = torch.full((M, N), float("nan"), dtype=dt, device="cuda")
+        B.mxfp8_gemm(c[0], c[1], c[2], c[3], M, N, K, int(a_mn), int(b_mn), ae, be, single)
+        torch.cuda.synchronize()
+        assert torch.equal(D.view(torch.int32 if out == "fp32" else torch.int16), single.view(torch.int32 if out == "fp32" else torch.int16))
+        if out == "fp32":
+            check_gemm_tolerance(D.cpu().numpy(), c[4], c[5], "multi %s" % ((M, N, K),))
+
+
+def test_gemm_multi_many_tiles_and_uneven_depths():
+    # the benchmark's mix in small: a shallow wide product and two deep narrow ones, more tiles than workers
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    specs = [(2048, 2048, 256, False, False), (2048, 512, 1024, False, True), (2048, 512, 1024, True, True)]
+    entries, keep = [], []
+    for i, (M, N, K, a_mn, b_mn) in enumerate(specs):
+        c = _multi_case(M, N, K, a_mn, b_mn, orc.E4M3, orc.E4M3, 70 + 3 * i)
+        D = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        keep.append((c, D))
+        entries.append((c[0], c[1], c[2], c[3], M, N, K, int(a_mn), int(b_mn), orc.E4M3, orc.E4M3, D))
+    B.mxfp8_gemm_multi(B.make_gemm_problems(entries), B.FP32)
+    assert B.mxfp8_device_status() == 0
+    for (M, N, K, _, _), (c, D) in zip(specs, keep):
+        check_gemm_tolerance(D.cpu().numpy(), c[4], c[5], "multi deep %s" % ((M, N, K),))
+
+
+def test_gemm_multi_argument_errors():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    z = torch.zeros(128, 128, dtype=torch.uint8, device="cuda")
+    sc = torch.zeros(512, dtype=torch.uint8, device="cuda")
+    D = torch.empty(128, 128, dtype=torch.float32, device="cuda")
+    good = (z, sc, z, sc, 128, 128, 128, 0, 0, 0, 0, D)
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_gemm_multi(B.make_gemm_problems([good] * 4), B.FP32)                 # more than three products
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_gemm_multi(B.make_gemm_problems([good, (z, sc, z, sc, 128, 128, 100, 0, 0, 0, 0, D)]), B.FP32)   # K % 32
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_gemm_multi(B.make_gemm_problems([good]), 7)                           # unknown output dtype
