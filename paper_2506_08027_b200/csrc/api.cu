@@ -1,5 +1,7 @@
 // Host helpers of the C ABI: sizes, layout offsets, status strings, host-buffer variant.
 #include "mxfp8_device.cuh"
+#include <mutex>
+
 #include "mxfp8_host.h"
 
 extern "C" size_t mxfp8_scale_bytes(int64_t rows, int64_t cols, int orientation, int sf_layout)
@@ -184,6 +186,36 @@ extern "C" size_t mxfp8_linear_host_ws_bytes(int64_t T, int64_t H, int64_t F)
     return plan_linear(nullptr, T, H, F, true).total;
 }
 
+namespace {
+// Two helper streams and the events that tie them to the caller's stream, one set per device, made on
+// first use and kept for the life of the process: the host variant overlaps the upload of dY with the
+// download of Y (PCIe carries both directions at once).
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, xw_in = nullptr, dy_in = nullptr, y_ready = nullptr, y_out = nullptr;
+    bool ok = false;
+};
+
+HostPipe* host_pipe()
+{
+    static HostPipe pipes[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    HostPipe& p = pipes[dev];
+    if (!p.ok) {
+        bool good = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess;
+        cudaEvent_t* evs[5] = {&p.start, &p.xw_in, &p.dy_in, &p.y_ready, &p.y_out};
+        for (cudaEvent_t* e : evs) good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+        if (!good) return nullptr;
+        p.ok = true;
+    }
+    return &p;
+}
+}  // namespace
+
 extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const void* dy_host,
                                  int64_t T, int64_t H, int64_t F, int scale_rule,
                                  void* y_host, void* dx_host, void* dw_host,
@@ -194,19 +226,49 @@ extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const v
     if ((reinterpret_cast<uintptr_t>(dev_ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
     if (dev_ws_bytes < mxfp8_linear_host_ws_bytes(T, H, F)) return MXFP8_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    HostPipe* hp = host_pipe();
+    if (!hp) return MXFP8_ERR_CUDA;
     const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F, true);
-    const int64_t shp[3][2] = {{T, H}, {F, H}, {T, F}};
-    const void* hsrc[3] = {x_host, w_host, dy_host};
-    for (int t = 0; t < 3; ++t)
-        if (cudaMemcpyAsync(w.src[t], hsrc[t], (size_t)shp[t][0] * shp[t][1] * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return MXFP8_ERR_CUDA;
-    const int rc = linear_device(w, w.src[0], w.src[1], w.src[2], T, H, F, scale_rule, w.out[0], w.out[1], w.out[2], stream);
-    if (rc != MXFP8_OK) return rc;
-    void* hout[3] = {y_host, dx_host, dw_host};
-    const int64_t outs[3][2] = {{T, F}, {T, H}, {F, H}};
-    for (int t = 0; t < 3; ++t)
-        if (cudaMemcpyAsync(hout[t], w.out[t], (size_t)outs[t][0] * outs[t][1] * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-            return MXFP8_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return MXFP8_ERR_CUDA;
+    enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
+    const size_t xb = (size_t)T * H * 2, wb = (size_t)F * H * 2, yb = (size_t)T * F * 2;
+#define MXFP8_TRY(call) do { if ((call) != cudaSuccess) return MXFP8_ERR_CUDA; } while (0)
+#define MXFP8_RC(call) do { const int rc_ = (call); if (rc_ != MXFP8_OK) return rc_; } while (0)
+    // uploads on the helper stream, behind whatever the caller's stream holds: X and W first, dY behind them
+    MXFP8_TRY(cudaEventRecord(hp->start, st));
+    MXFP8_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+    MXFP8_TRY(cudaMemcpyAsync(w.src[W], w_host, wb, cudaMemcpyHostToDevice, hp->in));
+    MXFP8_TRY(cudaMemcpyAsync(w.src[X], x_host, xb, cudaMemcpyHostToDevice, hp->in));
+    MXFP8_TRY(cudaEventRecord(hp->xw_in, hp->in));
+    MXFP8_TRY(cudaMemcpyAsync(w.src[DY], dy_host, yb, cudaMemcpyHostToDevice, hp->in));
+    MXFP8_TRY(cudaEventRecord(hp->dy_in, hp->in));
+    // FPROP as soon as X and W are on the device
+    MXFP8_TRY(cudaStreamWaitEvent(st, hp->xw_in, 0));
+    const mxfp8_quantize_item xw[2] = {
+        {w.src[X], T, H, w.q[X][R], w.s[X][R], w.q[X][C], w.s[X][C]},
+        {w.src[W], F, H, w.q[W][R], w.s[W][R], w.q[W][C], w.s[W][C]},
+    };
+    MXFP8_RC(mxfp8_quantize_multi(xw, 2, MXFP8_BF16, MXFP8_BOTH, scale_rule, MXFP8_E4M3, MXFP8_SF_SWIZZLED, stream));
+    MXFP8_RC(mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR, MXFP8_E4M3,
+                        MXFP8_E4M3, w.out[0], MXFP8_BF16, nullptr, nullptr, 0, stream));
+    MXFP8_TRY(cudaEventRecord(hp->y_ready, st));
+    // Y goes back on the second helper stream while dY is still coming in
+    MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->y_ready, 0));
+    MXFP8_TRY(cudaMemcpyAsync(y_host, w.out[0], yb, cudaMemcpyDeviceToHost, hp->out));
+    MXFP8_TRY(cudaEventRecord(hp->y_out, hp->out));
+    // DGRAD and WGRAD once dY has arrived
+    MXFP8_TRY(cudaStreamWaitEvent(st, hp->dy_in, 0));
+    MXFP8_RC(mxfp8_quantize(w.src[DY], MXFP8_BF16, T, F, MXFP8_BOTH, scale_rule, MXFP8_E4M3, w.q[DY][R], w.s[DY][R], w.q[DY][C],
+                            w.s[DY][C], MXFP8_SF_SWIZZLED, stream));
+    const mxfp8_gemm_problem grads[2] = {
+        {w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, w.out[1]},
+        {w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, w.out[2]},
+    };
+    MXFP8_RC(mxfp8_gemm_multi(grads, 2, MXFP8_BF16, stream));
+    MXFP8_TRY(cudaMemcpyAsync(dx_host, w.out[1], xb, cudaMemcpyDeviceToHost, st));
+    MXFP8_TRY(cudaMemcpyAsync(dw_host, w.out[2], wb, cudaMemcpyDeviceToHost, st));
+    MXFP8_TRY(cudaStreamWaitEvent(st, hp->y_out, 0));
+    MXFP8_TRY(cudaStreamSynchronize(st));
+#undef MXFP8_TRY
+#undef MXFP8_RC
     return mxfp8_device_status(stream);
 }
