@@ -297,3 +297,36 @@ def unpack_codes16(packed: np.ndarray, elem: int) -> np.ndarray:
             for i in range(16):
                 out[r, 16 * g + i] = (slot >> (w * i)) & ((1 << w) - 1)
     return out
+
+
+ACT_NONE, ACT_RELU, ACT_RELU2, ACT_SILU, ACT_GELU_TANH = 0, 1, 2, 3, 4
+
+
+def activation(x: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
+    """Elementwise activation ahead of the conversion (Sec. 3.2 keeps the activation function in high
+    precision and converts its result): the function's plain definition in binary64, rounded once to
+    binary32 and, for dst "bf16", once more to bfloat16 (returned as float32 values / uint16 patterns).
+        relu: x > 0 ? x : 0 (NaN -> 0);  relu2: x > 0 ? x*x : 0;  silu: x / (1 + exp(-x));
+        gelu_tanh: 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
+    """
+    v = np.asarray(x, dtype=np.float64)
+    with np.errstate(over="ignore", invalid="ignore"):
+        if act == ACT_NONE:
+            y = v.copy()
+        elif act == ACT_RELU:
+            y = np.where(v > 0, v, 0.0)
+        elif act == ACT_RELU2:
+            y = np.where(v > 0, v * v, 0.0)
+        elif act == ACT_SILU:
+            y = v / (1.0 + np.exp(-v))
+        elif act == ACT_GELU_TANH:
+            y = 0.5 * v * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (v + 0.044715 * v * v * v)))
+        else:
+            raise ValueError(act)
+        y32 = y.astype(np.float32)
+    if dst == "f32":
+        return y32
+    out = np.empty(y32.shape, dtype=np.uint16)
+    y64 = np.ascontiguousarray(y32, dtype=np.float64)
+    _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
+    return out

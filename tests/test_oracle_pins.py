@@ -585,3 +585,28 @@ def test_grouped_gemm_oracle_against_integer_loops_and_dense_special_cases():
         xz[offsets[g]:offsets[g + 1]] = xq[offsets[g]:offsets[g + 1]]
         dz, sz = orc.gemm_f64(xz, x_s, yq, y_s, "mn", "mn")
         assert np.array_equal(dk[g * M:(g + 1) * M], dz) and np.array_equal(sk[g * M:(g + 1) * M], sz)
+
+
+def test_activation_oracle_against_closed_forms_and_library():
+    import torch
+    x = np.array([-np.inf, -3.5, -1.0, -0.0, 0.0, 2.0 ** -20, 0.5, 1.0, 3.0, 1e20, np.inf, np.nan], np.float32)
+    relu = orc.activation(x, orc.ACT_RELU)
+    assert relu.tolist()[:10] == [0.0, 0.0, 0.0, 0.0, 0.0, 2.0 ** -20, 0.5, 1.0, 3.0, float(np.float32(1e20))] and relu[10] == np.inf and relu[11] == 0.0
+    relu2 = orc.activation(x, orc.ACT_RELU2)
+    assert relu2[:9].tolist() == [0.0, 0.0, 0.0, 0.0, 0.0, 2.0 ** -40, 0.25, 1.0, 9.0] and relu2[9] == np.inf and relu2[11] == 0.0
+    # x*x rounded once to binary32: against Python's exact rationals
+    rng = np.random.default_rng(2)
+    v = rng.standard_normal(200).astype(np.float32) * 100
+    for a, got in zip(v, orc.activation(v, orc.ACT_RELU2)):
+        want = np.float32(float(Fraction(float(a)) ** 2)) if a > 0 else np.float32(0)      # float() of an exact rational rounds once to binary64, exact here (48 bits)
+        assert got == want
+    # library routines (binary64) for the two transcendental ones
+    t = torch.from_numpy(np.linspace(-12, 12, 4001))
+    assert np.array_equal(orc.activation(t.numpy(), orc.ACT_SILU), torch.nn.functional.silu(t).numpy().astype(np.float32))
+    lib = torch.nn.functional.gelu(t, approximate="tanh").numpy()
+    mine = orc.activation(t.numpy(), orc.ACT_GELU_TANH).astype(np.float64)
+    assert np.abs(mine - lib).max() <= 2.0 ** -22 * np.abs(lib).max()
+    assert orc.activation(np.zeros(3, np.float32), orc.ACT_SILU).tolist() == [0.0, 0.0, 0.0]
+    # BF16 destination: one more round-to-nearest-even
+    b = orc.activation(np.array([1.0 + 2.0 ** -8, 3.0], np.float32), orc.ACT_RELU, "bf16")
+    assert b.tolist() == [0x3F80, 0x4040]                 # 1 + 2^-8 ties to even (1.0)
