@@ -545,6 +545,18 @@ def run_sweep(args):
                     print("| %s | %d x %d | %s | %.1f | %.0f | %.2f |" % (dtype, rows, cols, oname, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
                 del src, dr, dc
                 torch.cuda.empty_cache()
+        # an activation fused ahead of the conversion (mxfp8_act_quantize): same bytes as the plain conversion
+        print()
+        print("| activation + conversion, BF16 16384 x 8192, both orientations | us | GB/s | of measured copy |")
+        print("|---|---|---|---|")
+        rows, cols = 16384, 8192
+        src = synth.device_tensor("gaussian", (rows, cols), 12, "bf16")
+        outs = B.alloc_quantize_outputs(rows, cols, B.BOTH, S)
+        for act, name in ((B.ACT_NONE, "none (plain mxfp8_quantize path)"), (B.ACT_RELU, "relu"), (B.ACT_RELU2, "squared relu"),
+                          (B.ACT_SILU, "silu"), (B.ACT_GELU_TANH, "gelu (tanh)")):
+            ms = _time_calls(lambda i: B.mxfp8_act_quantize(src, act, B.BOTH, P, B.E4M3, *outs, S), 1)
+            gbs = rows * cols * (2 + 2 * (1 + 1 / 32)) / ms / 1e6
+            print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
         return
     shapes = [("square", n, n, n, 0, 0) for n in (1024, 2048, 4096, 8192, 16384)]
     shapes.append(("skinny wgrad", 4096, 4096, 65536, 1, 1))

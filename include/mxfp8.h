@@ -129,6 +129,26 @@ int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count, int src_dt
                          int orientation, int scale_rule, int elem, int sf_layout, void* stream);
 
 /*
+ * mxfp8_act_quantize -- an elementwise activation fused ahead of the conversion.  Sec. 3.2 keeps the
+ * activation function in high precision and converts its result for the next GEMM; this call reads
+ * the pre-activation once and writes only the MXFP8 copies: y = act(x) evaluated in FP32 and rounded
+ * once to the source dtype (BF16 round-to-nearest-even; unchanged for FP32), then exactly
+ * mxfp8_quantize(y).  The paper names no particular function; provided are
+ *   MXFP8_ACT_RELU       x > 0 ? x : 0            (NaN -> 0)
+ *   MXFP8_ACT_RELU2      x > 0 ? x * x : 0
+ *   MXFP8_ACT_SILU       x / (1 + exp(-x))
+ *   MXFP8_ACT_GELU_TANH  0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
+ * The first two are exact FP32 arithmetic (bit-reproducible); the last two use the device's fast FP32
+ * exponential and division (relative error of a few 2^-22 before the rounding to the source dtype).
+ * Arguments as mxfp8_quantize; needs cols % 16 == 0 (ERR_UNSUPPORTED otherwise).
+ */
+enum { MXFP8_ACT_NONE = 0, MXFP8_ACT_RELU = 1, MXFP8_ACT_RELU2 = 2, MXFP8_ACT_SILU = 3, MXFP8_ACT_GELU_TANH = 4 };
+int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int act,
+                       int orientation, int scale_rule, int elem,
+                       void* q_row, void* s_row, void* q_col, void* s_col,
+                       int sf_layout, void* stream);
+
+/*
  * mxfp8_fake_quantize -- the MXFP8 round trip in one pass: dst = decode(quantize(src)) in the source's
  * own dtype (BF16 -> MXFP8 -> BF16 is how the paper's accuracy runs emulated MX arithmetic ahead of
  * BF16 GEMMs, Sec. 3.1).  Same block / scale / cast rules and the same special-value handling as

@@ -21,13 +21,14 @@ E2M3, E3M2, E2M1 = 3, 4, 5          # MXFP6 / MXFP4 elements: conversion kernels
 SF_LINEAR, SF_SWIZZLED = 0, 1
 K_MAJOR, MN_MAJOR = 0, 1
 ERR_DEVICE_TIMEOUT, ERR_DEVICE_ARGS = -7, -9
+ACT_NONE, ACT_RELU, ACT_RELU2, ACT_SILU, ACT_GELU_TANH = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "mxfp8_quantize", "mxfp8_dequantize", "mxfp8_gemm", "mxfp8_scale_bytes", "mxfp8_sf_offset",
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
-    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi",
+    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize",
 )
 
 
@@ -94,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
         L.mxfp8_fake_quantize.restype = i
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_act_quantize.restype = i
+        L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_gemm_multi.restype = i
         L.mxfp8_gemm_multi.argtypes = [ctypes.POINTER(_GemmProblem), i, i, p]
         L.mxfp8_quantize_multi.restype = i
@@ -297,3 +300,12 @@ def make_gemm_problems(entries):
 
 def mxfp8_gemm_multi(problems, out_dtype: int, stream=None) -> None:
     _check(lib().mxfp8_gemm_multi(problems, len(problems), out_dtype, _stream(stream)), "mxfp8_gemm_multi")
+
+
+def mxfp8_act_quantize(src: torch.Tensor, act: int, orientation: int, scale_rule: int, elem: int,
+                       q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    rows, cols = src.shape
+    assert src.is_contiguous()
+    _check(lib().mxfp8_act_quantize(_ptr(src), _dtype_code(src), rows, cols, act, orientation, scale_rule, elem,
+                                    _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
+                                    _stream(stream)), "mxfp8_act_quantize")

@@ -40,12 +40,48 @@ struct QParams {
     uint8_t* s_col;
 };
 
+// Elementwise activation ahead of the conversion (Sec. 3.2 keeps the activation function in high
+// precision; its result is what gets converted): evaluated in FP32.  relu(x) = x > 0 ? x : 0 (NaN -> 0).
+template <int ACT>
+__device__ __forceinline__ float apply_act(float x)
+{
+    if constexpr (ACT == MXFP8_ACT_RELU) return x > 0.f ? x : 0.f;
+    else if constexpr (ACT == MXFP8_ACT_RELU2) return x > 0.f ? x * x : 0.f;
+    else if constexpr (ACT == MXFP8_ACT_SILU) return __fdividef(x, 1.f + __expf(-x));
+    else if constexpr (ACT == MXFP8_ACT_GELU_TANH) {
+        // 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)), u = sqrt(2/pi) (x + 0.044715 x^3)
+        const float u2 = 1.5957691216057308f * (x + 0.044715f * x * x * x);
+        return __fdividef(x, 1.f + __expf(-u2));
+    } else return x;
+}
+
+// Applies ACT in place to the 8 bytes per row this lane owns in its 32-row slab, rounding once to the source dtype.
+template <int ACT, bool BF>
+__device__ __forceinline__ void act_slab(uint8_t* mine)
+{
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+        uint2 w = *reinterpret_cast<const uint2*>(mine + j * T_BYTES);
+        if constexpr (BF) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(apply_act<ACT>(__uint_as_float(w.x << 16)), apply_act<ACT>(__uint_as_float(w.x & 0xFFFF0000u)));
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(apply_act<ACT>(__uint_as_float(w.y << 16)), apply_act<ACT>(__uint_as_float(w.y & 0xFFFF0000u)));
+            w.x = *reinterpret_cast<const uint32_t*>(&lo);
+            w.y = *reinterpret_cast<const uint32_t*>(&hi);
+        } else {
+            w.x = __float_as_uint(apply_act<ACT>(__uint_as_float(w.x)));
+            w.y = __float_as_uint(apply_act<ACT>(__uint_as_float(w.y)));
+        }
+        *reinterpret_cast<uint2*>(mine + j * T_BYTES) = w;
+    }
+}
+
 // One launch converts up to QT_MAX_TENSORS tensors: their tiles are numbered one tensor after the
 // other and dealt out to the CTAs as one pool, so small tensors share one ramp-up and one tail and
 // the per-CTA tile counts even out.
 constexpr int QT_MAX_TENSORS = 8;
 struct QBatch {
     int* status;                          // device status word of the library (bounded waits report here)
+    int act;                              // MXFP8_ACT_*: applied to every element before the conversion
     int count;
     int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
     QParams t[QT_MAX_TENSORS];
@@ -419,6 +455,19 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                 if (tid == 0) atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
                 return;
             }
+        }
+        if (batch.act != MXFP8_ACT_NONE) {
+            // activation in place: every lane rewrites exactly the 8 bytes per row it reads below, rounded once
+            // to the source dtype, so what follows equals the conversion of a tensor that holds act(x)
+            uint8_t* mine = in_tile + warp * 32 * T_BYTES + lane * 8;
+            switch (batch.act) {
+                case MXFP8_ACT_RELU: act_slab<MXFP8_ACT_RELU, BF>(mine); break;
+                case MXFP8_ACT_RELU2: act_slab<MXFP8_ACT_RELU2, BF>(mine); break;
+                case MXFP8_ACT_SILU: act_slab<MXFP8_ACT_SILU, BF>(mine); break;
+                default: act_slab<MXFP8_ACT_GELU_TANH, BF>(mine); break;
+            }
+            // the slot is refilled by a bulk copy later: order these generic-proxy writes before it
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         // this warp's slab: 32 rows; first the fully unrolled fast path (no special values, whole
         // slab inside the tensor), and if it saw an Inf / NaN or the slab is ragged, the careful path
