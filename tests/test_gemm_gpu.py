@@ -405,3 +405,29 @@ def test_gemm_multi_argument_errors():
         B.mxfp8_gemm_multi(B.make_gemm_problems([good, (z, sc, z, sc, 128, 128, 100, 0, 0, 0, 0, D)]), B.FP32)   # K % 32
     with pytest.raises(B.Mxfp8Error):
         B.mxfp8_gemm_multi(B.make_gemm_problems([good]), 7)                           # unknown output dtype
+
+
+def test_output_with_more_than_2_to_31_elements_sampled():
+    # D is 65536 x 40960 = 2.7e9 BF16 elements (5.4 GB); K is small so the oracle can check whole 128-row slabs
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    M, N, K = 65536, 40960, 256
+    a = synth.device_tensor("activation", (M, K), 5)
+    b = synth.device_tensor("weight", (N, K), 6)
+    qa = B.alloc_quantize_outputs(M, K, B.ROW, B.SF_SWIZZLED)
+    qb = B.alloc_quantize_outputs(N, K, B.ROW, B.SF_SWIZZLED)
+    B.mxfp8_quantize(a, B.ROW, B.RULE_PAPER, B.E4M3, *qa, B.SF_SWIZZLED)
+    B.mxfp8_quantize(b, B.ROW, B.RULE_PAPER, B.E4M3, *qb, B.SF_SWIZZLED)
+    D = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    B.mxfp8_gemm(qa[0], qa[1], qb[0], qb[1], M, N, K, B.K_MAJOR, B.K_MAJOR, B.E4M3, B.E4M3, D)
+    assert B.mxfp8_device_status() == 0
+    bf = orc.bf16_bits_to_f32(b.view(torch.int16).cpu().numpy().view(np.uint16))
+    bq, bs = orc.quantize(bf, orc.ROW)
+    mark = (2 ** 31) // N // 128 * 128
+    for r0 in (0, mark, M - 128):
+        af = orc.bf16_bits_to_f32(a[r0:r0 + 128].view(torch.int16).cpu().numpy().view(np.uint16))
+        aq, a_s = orc.quantize(af, orc.ROW)
+        d64, sabs = orc.gemm_f64(aq, a_s, bq, bs)
+        got = orc.bf16_bits_to_f32(D[r0:r0 + 128].view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+        err = np.abs(got - d64)
+        assert (err <= 2.0 ** -16 * sabs + 2.0 ** -8 * np.abs(d64) + 2.0 ** -126).all(), "slab %d" % r0

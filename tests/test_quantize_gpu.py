@@ -298,3 +298,48 @@ def test_quantize_multi_argument_errors():
     _, _, qc, sc = B.alloc_quantize_outputs(64, 40, B.COL, B.SF_LINEAR)
     with pytest.raises(B.Mxfp8Error):                      # cols % 16 != 0 has no batched path
         B.mxfp8_quantize_multi(B.make_quantize_items([(y, None, None, qc, sc)]), B.BF16, B.COL, B.RULE_PAPER, B.E4M3, B.SF_LINEAR)
+
+
+def test_more_than_2_to_31_elements_sampled():
+    # 40960 x 53248 = 2.18e9 elements (4.4 GB of BF16): every index computation has to be 64-bit.  The oracle
+    # checks 128-row slabs at the start, across the 2^31-element mark, and at the very end, for the conversion
+    # in both orientations (swizzled scales), the decode of the row copy and the one-pass round trip.
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import logical_scales_from_swizzled
+    rows, cols = 40960, 53248
+    assert rows * cols > 2 ** 31
+    g = torch.Generator(device="cuda"); g.manual_seed(31)
+    src = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    for r0 in range(0, rows, 4096):                     # drawn in pieces: no FP32 temporary of the whole tensor
+        src[r0:r0 + 4096] = (torch.randn((4096, cols), generator=g, device="cuda") *
+                             torch.exp2(torch.randint(-8, 8, (4096, 1), generator=g, device="cuda").float())).to(torch.bfloat16)
+    qr, sr, qc, sc = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_SWIZZLED)
+    B.mxfp8_quantize(src, B.BOTH, B.RULE_PAPER, B.E4M3, qr, sr, qc, sc, B.SF_SWIZZLED)
+    back = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    B.mxfp8_dequantize(qr, sr, B.ROW, B.E4M3, B.SF_SWIZZLED, back)
+    fq = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    B.mxfp8_fake_quantize(src, B.ROW, B.RULE_PAPER, B.E4M3, fq, None)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    mark = (2 ** 31) // cols // 128 * 128               # the slab that contains element 2^31
+    s_row_raw, s_col_raw = sr.cpu().numpy(), sc.cpu().numpy()
+    for r0 in (0, mark, rows - 128):
+        sl = slice(r0, r0 + 128)
+        x = orc.bf16_bits_to_f32(src[sl].view(torch.int16).cpu().numpy().view(np.uint16))
+        wq, ws = orc.quantize(x, orc.ROW)
+        m_idx, k_idx = np.meshgrid(np.arange(r0, r0 + 128), np.arange(cols // 32), indexing="ij")
+        atoms_k = (cols // 32 + 3) // 4
+        off = ((m_idx // 128) * atoms_k + k_idx // 4) * 512 + (m_idx % 32) * 16 + ((m_idx % 128) // 32) * 4 + k_idx % 4
+        assert off[-1, -1] == orc.sf_offset_swizzled(r0 + 127, cols // 32 - 1, cols // 32)
+        assert np.array_equal(s_row_raw[off], ws)
+        assert_q_equal(qr[sl].cpu().numpy(), wq, orc.E4M3, "row slab %d" % r0)
+        want = orc.dequantize(wq, ws, orc.ROW, orc.E4M3, "bf16")
+        assert np.array_equal(back[sl].view(torch.int16).cpu().numpy().view(np.uint16), want)
+        assert np.array_equal(fq[sl].view(torch.int16).cpu().numpy().view(np.uint16), want)
+        wq, ws = orc.quantize(x, orc.COL)                # [4, cols] scales of these four 32-row blocks
+        c_idx, b_idx = np.meshgrid(np.arange(cols), np.arange(r0 // 32, r0 // 32 + 4), indexing="ij")
+        atoms_kc = (rows // 32 + 3) // 4
+        offc = ((c_idx // 128) * atoms_kc + b_idx // 4) * 512 + (c_idx % 32) * 16 + ((c_idx % 128) // 32) * 4 + b_idx % 4
+        assert np.array_equal(s_col_raw[offc].T, ws)
+        assert_q_equal(qc[sl].cpu().numpy(), wq, orc.E4M3, "col slab %d" % r0)
