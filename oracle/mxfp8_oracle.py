@@ -330,3 +330,24 @@ def activation(x: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
     y64 = np.ascontiguousarray(y32, dtype=np.float64)
     _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
     return out
+
+
+def rmsnorm(x: np.ndarray, gamma: np.ndarray, eps: float, dst: str = "f32", rstd: np.ndarray | None = None):
+    """RMS normalisation ahead of the conversion (Sec. 3.2 keeps normalisation in high precision and converts its
+    output).  rstd[r] = 1 / sqrt(mean_c x[r,c]^2 + eps) in binary64, rounded to binary32 (or the `rstd` passed in, one
+    binary32 value per row); y = (x * rstd) * gamma as two binary32 products in that order, rounded once more to
+    bfloat16 for dst "bf16".  Returns (y, rstd): y as float32 values ("f32") or uint16 patterns ("bf16")."""
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    g32 = np.ascontiguousarray(gamma, dtype=np.float32)
+    if rstd is None:
+        v = x32.astype(np.float64)
+        rstd = (1.0 / np.sqrt((v * v).mean(axis=1) + float(eps))).astype(np.float32)
+    rstd = np.ascontiguousarray(rstd, dtype=np.float32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        y32 = (x32 * rstd[:, None]) * g32[None, :]          # numpy float32 products are IEEE single operations
+    if dst == "f32":
+        return y32, rstd
+    out = np.empty(y32.shape, dtype=np.uint16)
+    y64 = np.ascontiguousarray(y32, dtype=np.float64)
+    _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
+    return out, rstd

@@ -610,3 +610,26 @@ def test_activation_oracle_against_closed_forms_and_library():
     # BF16 destination: one more round-to-nearest-even
     b = orc.activation(np.array([1.0 + 2.0 ** -8, 3.0], np.float32), orc.ACT_RELU, "bf16")
     assert b.tolist() == [0x3F80, 0x4040]                 # 1 + 2^-8 ties to even (1.0)
+
+
+def test_rmsnorm_oracle_against_exact_cases_and_library():
+    import torch
+    # rows of +-c with c a power of two and eps = 0: rms = c exactly, so y = sign(x) * gamma exactly
+    x = np.array([[4.0, -4.0, 4.0, -4.0], [0.25, 0.25, -0.25, 0.25]], np.float32)
+    gamma = np.array([1.5, 2.0, -3.0, 0.125], np.float32)
+    y, rstd = orc.rmsnorm(x, gamma, 0.0)
+    assert rstd.tolist() == [0.25, 4.0]
+    assert np.array_equal(y, np.sign(x) * gamma[None, :])
+    # a 3-4-0-0 row: mean square 25/4, rms 5/2
+    y, rstd = orc.rmsnorm(np.array([[3.0, 4.0, 0.0, 0.0]], np.float32), np.ones(4, np.float32), 0.0)
+    assert rstd[0] == np.float32(0.4) and y[0].tolist() == [float(np.float32(3.0) * np.float32(0.4)), float(np.float32(4.0) * np.float32(0.4)), 0.0, 0.0]
+    # against the library's float64 rms_norm: equal up to the binary32 roundings of rstd and of the two products
+    rng = np.random.default_rng(8)
+    xr = rng.standard_normal((64, 256)).astype(np.float32) * 3
+    g = (1 + 0.1 * rng.standard_normal(256)).astype(np.float32)
+    y, _ = orc.rmsnorm(xr, g, 1e-5)
+    lib = torch.nn.functional.rms_norm(torch.from_numpy(xr).double(), (256,), torch.from_numpy(g).double(), 1e-5).numpy()
+    assert np.abs(y - lib).max() <= 3 * 2.0 ** -24 * np.abs(lib).max()
+    # a supplied rstd is used as is; BF16 destination rounds once more (ties to even)
+    y2, r2 = orc.rmsnorm(np.array([[1.0 + 2.0 ** -8, 3.0]], np.float32), np.ones(2, np.float32), 0.0, "bf16", np.array([1.0], np.float32))
+    assert y2[0].tolist() == [0x3F80, 0x4040] and r2[0] == 1.0
