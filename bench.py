@@ -557,6 +557,12 @@ def run_sweep(args):
             ms = _time_calls(lambda i: B.mxfp8_act_quantize(src, act, B.BOTH, P, B.E4M3, *outs, S), 1)
             gbs = rows * cols * (2 + 2 * (1 + 1 / 32)) / ms / 1e6
             print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+        gamma = torch.ones(cols, dtype=torch.bfloat16, device="cuda")
+        rstd = torch.empty(rows, dtype=torch.float32, device="cuda")
+        ms = _time_calls(lambda i: B.mxfp8_rmsnorm_quantize(src, gamma, 1e-5, rstd, B.BOTH, P, B.E4M3, *outs, S), 1)
+        gbs = rows * cols * (2 + 2 + 2 * (1 + 1 / 32)) / ms / 1e6       # the source is read twice (statistics, conversion)
+        print("| rms normalisation (statistics launch + fused conversion; source read twice) | %.1f | %.0f | %.2f |" % (
+            ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
         return
     shapes = [("square", n, n, n, 0, 0) for n in (1024, 2048, 4096, 8192, 16384)]
     shapes.append(("skinny wgrad", 4096, 4096, 65536, 1, 1))

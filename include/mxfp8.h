@@ -149,6 +149,24 @@ int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, int64_t col
                        int sf_layout, void* stream);
 
 /*
+ * mxfp8_rmsnorm_quantize -- RMS normalisation fused ahead of the conversion (Sec. 3.2 keeps the
+ * normalisation layers in high precision and converts their output for the next GEMM).  Two launches:
+ *   rstd[r] = 1 / sqrt(mean_c(x[r, c]^2) + eps)     FP32 accumulation over the row, written to `rstd`
+ *                                                    (device, `rows` floats; the backward pass wants it)
+ *   y[r, c] = (x[r, c] * rstd[r]) * gamma[c]        two FP32 products in this order, rounded once to the
+ *                                                    source dtype, then exactly mxfp8_quantize(y)
+ * gamma: device, `cols` values of the source dtype, 16-byte aligned.  eps >= 0.  The sum of squares is
+ * accumulated in FP32 in a fixed order (reproducible run to run), so rstd agrees with an FP64 evaluation
+ * to FP32 rounding, not bit for bit.  Other arguments as mxfp8_quantize; needs cols % 16 == 0.
+ * The source is read twice (statistics, then conversion) and no normalised tensor is written.
+ */
+int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                           const void* gamma, float eps, float* rstd,
+                           int orientation, int scale_rule, int elem,
+                           void* q_row, void* s_row, void* q_col, void* s_col,
+                           int sf_layout, void* stream);
+
+/*
  * mxfp8_fake_quantize -- the MXFP8 round trip in one pass: dst = decode(quantize(src)) in the source's
  * own dtype (BF16 -> MXFP8 -> BF16 is how the paper's accuracy runs emulated MX arithmetic ahead of
  * BF16 GEMMs, Sec. 3.1).  Same block / scale / cast rules and the same special-value handling as

@@ -28,7 +28,7 @@ EXPORTS = (
     "mxfp8_gemm_workspace_bytes", "mxfp8_device_status", "mxfp8_status_string",
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
-    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize",
+    "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
 )
 
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
         L.mxfp8_fake_quantize.restype = i
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+        L.mxfp8_rmsnorm_quantize.restype = i
+        L.mxfp8_rmsnorm_quantize.argtypes = [p, i, i64, i64, p, ctypes.c_float, p, i, i, i, p, p, p, p, i, p]
         L.mxfp8_act_quantize.restype = i
         L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_gemm_multi.restype = i
@@ -309,3 +311,14 @@ def mxfp8_act_quantize(src: torch.Tensor, act: int, orientation: int, scale_rule
     _check(lib().mxfp8_act_quantize(_ptr(src), _dtype_code(src), rows, cols, act, orientation, scale_rule, elem,
                                     _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
                                     _stream(stream)), "mxfp8_act_quantize")
+
+
+def mxfp8_rmsnorm_quantize(src: torch.Tensor, gamma: torch.Tensor, eps: float, rstd: torch.Tensor,
+                           orientation: int, scale_rule: int, elem: int,
+                           q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    rows, cols = src.shape
+    assert src.is_contiguous() and gamma.dtype == src.dtype and gamma.numel() == cols
+    assert rstd.dtype == torch.float32 and rstd.numel() == rows
+    _check(lib().mxfp8_rmsnorm_quantize(_ptr(src), _dtype_code(src), rows, cols, _ptr(gamma), eps, _ptr(rstd),
+                                        orientation, scale_rule, elem, _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col),
+                                        sf_layout, _stream(stream)), "mxfp8_rmsnorm_quantize")

@@ -367,6 +367,76 @@ extern "C" int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count,
     return quantize_tma_batch(batch, count, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream));
 }
 
+namespace mxfp8 {
+namespace {
+// 1/rms of every row: one warp per row, 16-byte loads, FP32 accumulation (lane-strided partial sums, then a
+// butterfly), rstd = 1 / sqrt(sum / cols + eps) with IEEE square root and division.
+template <int DTYPE>
+__global__ void __launch_bounds__(256) rms_stats_kernel(const void* __restrict__ src, int64_t rows, int64_t cols, float eps,
+                                                        float* __restrict__ rstd)
+{
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    constexpr int PER = (DTYPE == MXFP8_BF16) ? 8 : 4;            // elements per 16-byte load
+    const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(src) + row * cols * (DTYPE == MXFP8_BF16 ? 2 : 4));
+    const int64_t chunks = cols / PER;
+    float acc = 0.f;
+    for (int64_t c = lane; c < chunks; c += 32) {
+        const uint4 w = p[c];
+        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (DTYPE == MXFP8_BF16) {
+                const float a = __uint_as_float(u[i] << 16), b = __uint_as_float(u[i] & 0xFFFF0000u);
+                acc = fmaf(a, a, acc);
+                acc = fmaf(b, b, acc);
+            } else {
+                const float a = __uint_as_float(u[i]);
+                acc = fmaf(a, a, acc);
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+    if (lane == 0) rstd[row] = 1.0f / sqrtf(acc / (float)cols + eps);
+}
+}  // namespace
+}  // namespace mxfp8
+
+extern "C" int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                      const void* gamma, float eps, float* rstd,
+                                      int orientation, int scale_rule, int elem,
+                                      void* q_row, void* s_row, void* q_col, void* s_col,
+                                      int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!src || !gamma || !rstd) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col || !s_col)) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || !(eps >= 0.f)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(src) || !aligned16(gamma) || (reinterpret_cast<uintptr_t>(rstd) & 3u)) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
+    if ((rows + 7) / 8 > 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned blocks = (unsigned)((rows + 7) / 8);
+    if (src_dtype == MXFP8_BF16) rms_stats_kernel<MXFP8_BF16><<<blocks, 256, 0, st>>>(src, rows, cols, eps, rstd);
+    else rms_stats_kernel<MXFP8_FP32><<<blocks, 256, 0, st>>>(src, rows, cols, eps, rstd);
+    count_launch(1);
+    if (cudaGetLastError() != cudaSuccess) return MXFP8_ERR_CUDA;
+    const QuantizeItem item{src, rows, cols, q_row, s_row, q_col, s_col};
+    return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, st, false, MXFP8_ACT_NONE, rstd, gamma);
+}
+
 extern "C" int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int act,
                                   int orientation, int scale_rule, int elem,
                                   void* q_row, void* s_row, void* q_col, void* s_col,

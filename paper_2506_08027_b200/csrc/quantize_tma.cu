@@ -62,7 +62,7 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
 }
 
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
-                       int sf_layout, cudaStream_t stream, bool emulate, int act)
+                       int sf_layout, cudaStream_t stream, bool emulate, int act, const float* rstd, const void* gamma)
 {
     if (count < 1 || count > QT_MAX_TENSORS) return MXFP8_ERR_UNSUPPORTED;
     const bool bf = src_dtype == MXFP8_BF16;
@@ -71,6 +71,8 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
     QBatch p{};
     p.count = count;
     p.act = act;
+    p.rstd = rstd;
+    p.gamma = gamma;
     int64_t tiles = 0;
     for (int i = 0; i < QT_MAX_TENSORS; ++i) {
         const QuantizeItem& it = items[i < count ? i : 0];   // unused slots repeat the first tensor: every map stays valid

@@ -75,6 +75,41 @@ __device__ __forceinline__ void act_slab(uint8_t* mine)
     }
 }
 
+// RMS normalisation in place, same ownership as act_slab: y = (x * rstd[row]) * gamma[col], two FP32 products
+// in that order, rounded once to the source dtype.  Rows and columns beyond the tensor hold TMA's zero fill and
+// are left alone (their statistics and weights do not exist).
+template <bool BF>
+__device__ __forceinline__ void norm_slab(uint8_t* mine, const float* __restrict__ rstd, const void* __restrict__ gamma_col,
+                                          int rows_here, bool col_ok)
+{
+    if (!col_ok) return;
+    float g[4];
+    if constexpr (BF) {
+        const uint2 w = *reinterpret_cast<const uint2*>(gamma_col);
+        g[0] = __uint_as_float(w.x << 16); g[1] = __uint_as_float(w.x & 0xFFFF0000u);
+        g[2] = __uint_as_float(w.y << 16); g[3] = __uint_as_float(w.y & 0xFFFF0000u);
+    } else {
+        const float2 w = *reinterpret_cast<const float2*>(gamma_col);
+        g[0] = w.x; g[1] = w.y; g[2] = 0.f; g[3] = 0.f;
+    }
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+        if (j >= rows_here) break;
+        const float r = rstd[j];
+        uint2 w = *reinterpret_cast<const uint2*>(mine + j * T_BYTES);
+        if constexpr (BF) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn((__uint_as_float(w.x << 16) * r) * g[0], (__uint_as_float(w.x & 0xFFFF0000u) * r) * g[1]);
+            const __nv_bfloat162 hi = __floats2bfloat162_rn((__uint_as_float(w.y << 16) * r) * g[2], (__uint_as_float(w.y & 0xFFFF0000u) * r) * g[3]);
+            w.x = *reinterpret_cast<const uint32_t*>(&lo);
+            w.y = *reinterpret_cast<const uint32_t*>(&hi);
+        } else {
+            w.x = __float_as_uint((__uint_as_float(w.x) * r) * g[0]);
+            w.y = __float_as_uint((__uint_as_float(w.y) * r) * g[1]);
+        }
+        *reinterpret_cast<uint2*>(mine + j * T_BYTES) = w;
+    }
+}
+
 // One launch converts up to QT_MAX_TENSORS tensors: their tiles are numbered one tensor after the
 // other and dealt out to the CTAs as one pool, so small tensors share one ramp-up and one tail and
 // the per-CTA tile counts even out.
@@ -82,6 +117,8 @@ constexpr int QT_MAX_TENSORS = 8;
 struct QBatch {
     int* status;                          // device status word of the library (bounded waits report here)
     int act;                              // MXFP8_ACT_*: applied to every element before the conversion
+    const float* rstd;                    // RMS normalisation ahead of the conversion (first tensor only): 1/rms per row,
+    const void* gamma;                    //   and the per-column weight in the source dtype; both null when unused
     int count;
     int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
     QParams t[QT_MAX_TENSORS];
@@ -455,6 +492,15 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                 if (tid == 0) atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
                 return;
             }
+        }
+        if (batch.rstd != nullptr) {
+            // RMS normalisation in place (single-tensor launches only), then the unchanged conversion
+            const int64_t row_first = grow0 + warp * 32;
+            const int rows_in = (int)max((int64_t)0, min((int64_t)32, p.rows - row_first));
+            const int64_t col_first = gcol0 + lane * VEC;
+            norm_slab<BF>(in_tile + warp * 32 * T_BYTES + lane * 8, batch.rstd + row_first,
+                          static_cast<const uint8_t*>(batch.gamma) + col_first * (BF ? 2 : 4), rows_in, col_first < p.cols);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         if (batch.act != MXFP8_ACT_NONE) {
             // activation in place: every lane rewrites exactly the 8 bytes per row it reads below, rounded once

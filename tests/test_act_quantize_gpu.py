@@ -135,3 +135,75 @@ def test_argument_errors():
     _, _, qc, sc = B.alloc_quantize_outputs(64, 40, B.COL, B.SF_LINEAR)
     with pytest.raises(B.Mxfp8Error):
         B.mxfp8_act_quantize(y, B.ACT_RELU, B.COL, B.RULE_PAPER, B.E4M3, None, None, qc, sc, B.SF_LINEAR)
+
+
+# ------------------------------------------------------------------------------------------ RMS normalisation
+
+def gpu_rmsnorm_quantize(src_np, gamma_np, dtype, eps, orientation, elem=orc.E4M3):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = src_np.shape
+    if dtype == "bf16":
+        src = torch.from_numpy(src_np.view(np.int16)).cuda().view(torch.bfloat16)
+        gamma = torch.from_numpy(gamma_np.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        src, gamma = torch.from_numpy(src_np).cuda(), torch.from_numpy(gamma_np).cuda()
+    rstd = Guarded(rows * 4)
+    bufs, args = {}, []
+    for o, name in ((B.ROW, "row"), (B.COL, "col")):
+        if orientation & o:
+            bufs[name] = (Guarded(rows * cols), Guarded(B.mxfp8_scale_bytes(rows, cols, o, B.SF_SWIZZLED)))
+            args += [bufs[name][0].view.view(rows, cols), bufs[name][1].view]
+        else:
+            args += [None, None]
+    before = B.mxfp8_launch_count()
+    B.mxfp8_rmsnorm_quantize(src, gamma, eps, rstd.view.view(torch.float32), orientation, B.RULE_PAPER, elem, *args, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0 and B.mxfp8_launch_count() - before == 2
+    rstd.check()
+    out = {"rstd": rstd.numpy().view(np.float32).copy()}
+    for name, (q, s) in bufs.items():
+        q.check(); s.check()
+        mn, nkb = (rows, cols // 32) if name == "row" else (cols, rows // 32)
+        logical = logical_scales_from_swizzled(s.numpy(), mn, nkb)
+        out[name] = (orc.unpack_codes16(q.numpy().reshape(rows, cols), elem), logical if name == "row" else np.ascontiguousarray(logical.T))
+    return out
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(256, 512), (160, 352), (96, 4096 + 128), (32, 2048)])
+def test_rmsnorm_quantize(dtype, shape):
+    rows, cols = shape
+    x32 = synth.gaussian(shape, 3 + rows) * np.exp2(np.random.default_rng(rows).integers(-6, 6, (rows, 1))).astype(np.float32)
+    g32 = (1.0 + 0.2 * synth.gaussian((1, cols), 4)[0]).astype(np.float32)
+    x, g = as_dtype(x32, dtype), as_dtype(g32, dtype)
+    xv = orc.bf16_bits_to_f32(x) if dtype == "bf16" else x
+    gv = orc.bf16_bits_to_f32(g) if dtype == "bf16" else g
+    got = gpu_rmsnorm_quantize(x, g, dtype, 1e-5, BOTH)
+    # the statistics: FP32 accumulation against the FP64 definition
+    _, want_rstd = orc.rmsnorm(xv, gv, 1e-5)
+    assert np.abs(got["rstd"] - want_rstd).max() <= 2.0 ** -20 * np.abs(want_rstd).max()
+    # given those statistics everything after is exact arithmetic: bit-exact against the oracle
+    y, _ = orc.rmsnorm(xv, gv, 1e-5, "bf16" if dtype == "bf16" else "f32", got["rstd"])
+    y = orc.bf16_bits_to_f32(y) if dtype == "bf16" else y
+    for o, name in ((orc.ROW, "row"), (orc.COL, "col")):
+        wq, ws = orc.quantize(y, o, orc.RULE_PAPER, orc.E4M3)
+        assert np.array_equal(got[name][1], ws), "scales %s" % name
+        assert_q_equal(got[name][0], wq, orc.E4M3, name)
+
+
+def test_rmsnorm_argument_errors():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    x = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    g = torch.ones(64, dtype=torch.bfloat16, device="cuda")
+    r = torch.empty(64, dtype=torch.float32, device="cuda")
+    q, s, _, _ = B.alloc_quantize_outputs(64, 64, B.ROW, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_rmsnorm_quantize(x, g, -1.0, r, B.ROW, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_rmsnorm_quantize(x, g, 1e-5, r, B.COL, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
+    # an all-zero row with eps = 0 has rstd = Inf and 0 * Inf = NaN elements: they become NaN codes, nothing faults
+    B.mxfp8_rmsnorm_quantize(x, g, 0.0, r, B.ROW, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
+    torch.cuda.synchronize()
+    assert torch.isinf(r).all() and (q == 0x7F).all()
