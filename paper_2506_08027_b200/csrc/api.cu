@@ -194,6 +194,7 @@ struct HostPipe {
     cudaStream_t in = nullptr, out = nullptr;
     cudaEvent_t start = nullptr, xw_in = nullptr, dy_in = nullptr, y_ready = nullptr, y_out = nullptr;
     bool ok = false;
+    std::mutex busy;   // one host-buffer step at a time per device: the events above are shared
 };
 
 HostPipe* host_pipe()
@@ -228,6 +229,7 @@ extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     HostPipe* hp = host_pipe();
     if (!hp) return MXFP8_ERR_CUDA;
+    std::lock_guard<std::mutex> one_at_a_time(hp->busy);
     const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F, true);
     enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
     const size_t xb = (size_t)T * H * 2, wb = (size_t)F * H * 2, yb = (size_t)T * F * 2;
