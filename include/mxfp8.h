@@ -167,6 +167,23 @@ int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t
                            int sf_layout, void* stream);
 
 /*
+ * mxfp8_rmsnorm_quantize_static -- mxfp8_rmsnorm_quantize for callers that do not want the row
+ * statistics and have no buffer to lend: the statistics go to a fixed array inside the library
+ * (file-scope device memory, 65536 rows x 4 bytes = 256 KB, part of the module image), so the call
+ * takes no scratch from the caller and allocates nothing, on the host or on the device.  More than
+ * mxfp8_rmsnorm_quantize_static_max_rows() rows: MXFP8_ERR_UNSUPPORTED.  The array is shared by all
+ * calls on a device: calls must be ordered on one stream (or otherwise not overlap in time).
+ * Results are those of mxfp8_rmsnorm_quantize.  (A packaging for convenience: the paper has no
+ * counterpart.)
+ */
+int64_t mxfp8_rmsnorm_quantize_static_max_rows(void);
+int mxfp8_rmsnorm_quantize_static(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                  const void* gamma, float eps,
+                                  int orientation, int scale_rule, int elem,
+                                  void* q_row, void* s_row, void* q_col, void* s_col,
+                                  int sf_layout, void* stream);
+
+/*
  * mxfp8_fake_quantize -- the MXFP8 round trip in one pass: dst = decode(quantize(src)) in the source's
  * own dtype (BF16 -> MXFP8 -> BF16 is how the paper's accuracy runs emulated MX arithmetic ahead of
  * BF16 GEMMs, Sec. 3.1).  Same block / scale / cast rules and the same special-value handling as

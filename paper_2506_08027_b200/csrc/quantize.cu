@@ -14,6 +14,8 @@
 //   copy (swizzled layout) or as per-row / per-block-row pieces (linear layout).
 #include <atomic>
 
+#include <mutex>
+
 #include "mxfp8_device.cuh"
 #include "mxfp8_host.h"
 
@@ -463,4 +465,44 @@ extern "C" int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, 
     if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;
     const QuantizeItem item{one.src, one.rows, one.cols, one.q_row, one.s_row, one.q_col, one.s_col};
     return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream), false, act);
+}
+
+namespace mxfp8 {
+namespace {
+// Row statistics of mxfp8_rmsnorm_quantize_static: 65536 rows x 4 bytes = 256 KB that live in the module image.
+constexpr int64_t RSTD_STATIC_ROWS = 65536;
+static __device__ __align__(256) float g_rstd_static[RSTD_STATIC_ROWS];
+
+// Device address of the array, looked up once per device.
+float* rstd_static_address()
+{
+    static float* addr[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_rstd_static) != cudaSuccess) return nullptr;
+        addr[dev] = static_cast<float*>(p);
+    }
+    return addr[dev];
+}
+}  // namespace
+}  // namespace mxfp8
+
+extern "C" int64_t mxfp8_rmsnorm_quantize_static_max_rows(void) { return mxfp8::RSTD_STATIC_ROWS; }
+
+extern "C" int mxfp8_rmsnorm_quantize_static(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                             const void* gamma, float eps,
+                                             int orientation, int scale_rule, int elem,
+                                             void* q_row, void* s_row, void* q_col, void* s_col,
+                                             int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (rows > RSTD_STATIC_ROWS) return MXFP8_ERR_UNSUPPORTED;
+    float* rstd = rstd_static_address();
+    if (!rstd) return MXFP8_ERR_CUDA;
+    return mxfp8_rmsnorm_quantize(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem,
+                                  q_row, s_row, q_col, s_col, sf_layout, stream);
 }

@@ -1,0 +1,84 @@
+"""mxfp8_rmsnorm_quantize_static: the RMS-normalisation + conversion call whose row statistics live in a fixed
+array inside the library, so that it needs no scratch from the caller and allocates nothing."""
+import numpy as np
+import pytest
+
+from paper_2506_08027_b200 import synth
+
+
+def test_symbols_are_declared_and_exported():
+    import os
+    import re
+    here = os.path.dirname(os.path.abspath(__file__))
+    header = open(os.path.join(here, "..", "include", "mxfp8.h")).read()
+    assert re.search(r"\bmxfp8_rmsnorm_quantize_static\s*\(", header)
+    assert re.search(r"\bmxfp8_rmsnorm_quantize_static_max_rows\s*\(", header)
+    from paper_2506_08027_b200 import binding as B
+    assert "mxfp8_rmsnorm_quantize_static" in B.EXPORTS
+    lib = B.lib()
+    assert hasattr(lib, "mxfp8_rmsnorm_quantize_static") and B.mxfp8_rmsnorm_quantize_static_max_rows() == 65536
+
+
+def _inputs(rows, cols, seed):
+    import torch
+    x = synth.device_tensor("activation", (rows, cols), seed)
+    gamma = (1.0 + 0.1 * torch.randn(cols, generator=torch.Generator().manual_seed(seed))).to(torch.bfloat16).cuda()
+    return x, gamma
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", [(256, 512), (160, 352), (65536, 32)])
+def test_same_result_as_the_call_with_a_caller_buffer(shape):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = shape
+    x, gamma = _inputs(rows, cols, 5)
+    a = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_SWIZZLED)
+    b = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_SWIZZLED)
+    for t in a + b:
+        t.zero_()
+    rstd = torch.empty(rows, dtype=torch.float32, device="cuda")
+    B.mxfp8_rmsnorm_quantize(x, gamma, 1e-5, rstd, B.BOTH, B.RULE_PAPER, B.E4M3, *a, B.SF_SWIZZLED)
+    B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *b, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for u, v in zip(a, b):
+        assert torch.equal(u, v)
+
+
+@pytest.mark.gpu
+def test_allocates_nothing_on_host_or_device():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = 4096, 2048
+    x, gamma = _inputs(rows, cols, 6)
+    outs = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_SWIZZLED)
+    # first call: module load and the one-time address lookup
+    B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *outs, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    stats0 = torch.cuda.memory_stats()
+    for _ in range(20):
+        B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *outs, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    stats1 = torch.cuda.memory_stats()
+    assert free1 == free0, "device memory in use changed across the calls"
+    assert stats1["allocation.all.allocated"] == stats0["allocation.all.allocated"]
+    assert stats1["allocated_bytes.all.current"] == stats0["allocated_bytes.all.current"]
+
+
+@pytest.mark.gpu
+def test_rejects_more_rows_than_the_array_holds():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = 65536 + 32, 32
+    x, gamma = _inputs(rows, cols, 7)
+    outs = B.alloc_quantize_outputs(rows, cols, B.ROW, B.SF_LINEAR)
+    for t in outs[:2]:
+        t.fill_(0xA5)
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.ROW, B.RULE_PAPER, B.E4M3, *outs, B.SF_LINEAR)
+    assert e.value.status == -5
+    torch.cuda.synchronize()
+    assert (outs[0] == 0xA5).all() and (outs[1] == 0xA5).all()      # nothing was launched
