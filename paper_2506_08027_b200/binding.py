@@ -132,7 +132,11 @@ def _check(status: int, what: str) -> None:
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("the C entry points take dense row-major buffers: pass a contiguous tensor")
+    return ctypes.c_void_p(t.data_ptr())
 
 
 def _stream(stream=None):

@@ -151,7 +151,7 @@ def gpu_gemm(aq, a_s, bq, b_s, a_major="k", b_major="k", a_elem=0, b_elem=0, out
     else:
         _, N = bq.shape
         sb_log = np.ascontiguousarray(b_s.T)
-    dA, dB = torch.from_numpy(aq).cuda(), torch.from_numpy(bq).cuda()
+    dA, dB = torch.from_numpy(np.ascontiguousarray(aq)).cuda(), torch.from_numpy(np.ascontiguousarray(bq)).cuda()   # fancy-indexed inputs may be strided
     dSA, dSB = torch.from_numpy(swizzle_np(sa_log)).cuda(), torch.from_numpy(swizzle_np(sb_log)).cuda()
     D = torch.full((M, N), float("nan"), dtype=torch.float32 if out == "fp32" else torch.bfloat16, device="cuda")
     B.mxfp8_gemm(dA, dSA, dB, dSB, M, N, K, B.MN_MAJOR if a_major == "mn" else B.K_MAJOR,

@@ -431,3 +431,29 @@ def test_output_with_more_than_2_to_31_elements_sampled():
         got = orc.bf16_bits_to_f32(D[r0:r0 + 128].view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
         err = np.abs(got - d64)
         assert (err <= 2.0 ** -16 * sabs + 2.0 ** -8 * np.abs(d64) + 2.0 ** -126).all(), "slab %d" % r0
+
+
+@pytest.mark.parametrize("majors", [("k", "k"), ("mn", "mn")])
+def test_k_permutation_leaves_exact_products_unchanged(majors):
+    # the same permutation of the K axis in both operands (elements together with their blocks' scales): shuffling
+    # inside blocks, shuffling whole blocks, and both.  Small integers and power-of-two scales keep every partial
+    # sum exact in FP32, so the result must not change by a single bit, whatever the order of accumulation.
+    m, n, k = 256, 384, 512
+    rng = np.random.default_rng(91)
+    ai, aq = int_operand(rng, m, k)
+    bi, bq = int_operand(rng, n, k)
+    a_s = rng.integers(126, 129, (m, k // 32)).astype(np.uint8)      # 1/2, 1, 2: sums stay below 2^24 units
+    b_s = rng.integers(126, 129, (n, k // 32)).astype(np.uint8)
+    base = gpu_gemm(*stored(aq, a_s, majors[0]), *stored(bq, b_s, majors[1]), majors[0], majors[1])
+    d64, _ = orc.gemm_f64(*stored(aq, a_s, majors[0]), *stored(bq, b_s, majors[1]), majors[0], majors[1])
+    assert np.array_equal(base.astype(np.float64), d64)
+    within = np.concatenate([32 * b + rng.permutation(32) for b in range(k // 32)])     # inside each block
+    blocks = rng.permutation(k // 32)
+    across = np.concatenate([32 * b + np.arange(32) for b in blocks])                   # whole blocks
+    for perm, sperm in ((within, np.arange(k // 32)), (across, blocks), (across[within], blocks)):
+        if perm is not within and perm is not across:
+            # across[within]: first shuffle inside blocks, then move the blocks
+            perm = np.concatenate([32 * b + rng.permutation(32) for b in blocks])
+        got = gpu_gemm(*stored(aq[:, perm], a_s[:, sperm], majors[0]), *stored(bq[:, perm], b_s[:, sperm], majors[1]),
+                       majors[0], majors[1])
+        assert np.array_equal(got, base)
