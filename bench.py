@@ -148,6 +148,9 @@ def oracle_sample_seconds(sample_rows: int = 256):
         gemm_full = t_gemm * STEP_FLOP / (2.0 * r * r * H)
         desc = ("%d rows of X, W, dY quantized in both orientations on %d threads; %dx%dx%d FP64 product "
                 "(+|A||B| bound product) via numpy; scaled linearly to the full step" % (r, threads, r, r, H))
+    oracle_sample_seconds.split = {   # the two halves of the metric for the oracle (same byte and FLOP counts as the GPU arm)
+        "cast_gbs": CAST_BYTES / cast_full / 1e9, "gemm_tflops": STEP_FLOP / gemm_full / 1e12,
+        "cast_seconds_full_step": cast_full, "gemm_seconds_full_step": gemm_full}
     return t_cast + t_gemm, cast_full + gemm_full, desc, threads
 
 
@@ -342,7 +345,7 @@ def run_ours(args):
     if world == 1 and not args.no_cpu_baseline:
         s, f, desc, threads = oracle_sample_seconds(8192)
         cpu = {"value": STEP_FLOP / f / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
-               "sample": desc, "sample_seconds": s}
+               "sample": desc, "sample_seconds": s, **getattr(oracle_sample_seconds, "split", {})}
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
