@@ -56,14 +56,19 @@ def test_allocates_nothing_on_host_or_device():
     # first call: module load and the one-time address lookup
     B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *outs, B.SF_SWIZZLED)
     torch.cuda.synchronize()
-    free0, _ = torch.cuda.mem_get_info()
     stats0 = torch.cuda.memory_stats()
-    for _ in range(20):
-        B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *outs, B.SF_SWIZZLED)
-    torch.cuda.synchronize()
-    free1, _ = torch.cuda.mem_get_info()
+    unchanged = False
+    for _ in range(3):          # the free-memory figure is device-wide: repeat if something else moved it meanwhile
+        free0, _ = torch.cuda.mem_get_info()
+        for _ in range(20):
+            B.mxfp8_rmsnorm_quantize_static(x, gamma, 1e-5, B.BOTH, B.RULE_PAPER, B.E4M3, *outs, B.SF_SWIZZLED)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        if free1 == free0:
+            unchanged = True
+            break
+    assert unchanged, "device memory in use changed across the calls"
     stats1 = torch.cuda.memory_stats()
-    assert free1 == free0, "device memory in use changed across the calls"
     assert stats1["allocation.all.allocated"] == stats0["allocation.all.allocated"]
     assert stats1["allocated_bytes.all.current"] == stats0["allocated_bytes.all.current"]
 
