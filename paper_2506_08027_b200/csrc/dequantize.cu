@@ -157,10 +157,108 @@ dequantize_vec_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__
     }
 }
 
+// Four decoded elements of one lane: codes -> FP32 (exact), times the scales, one rounding if BF16 is asked.
+template <int ELEM, int DST>
+__device__ __forceinline__ void decode_store4(uint32_t codes, float s0, float s1, float s2, float s3, void* dst_elem)
+{
+    const float2 lo = fp8x2_to_float2<ELEM>(codes & 0xFFFFu), hi = fp8x2_to_float2<ELEM>(codes >> 16);
+    const float o0 = lo.x * s0, o1 = lo.y * s1, o2 = hi.x * s2, o3 = hi.y * s3;
+    if (DST == MXFP8_FP32) {
+        __stcs(reinterpret_cast<float4*>(dst_elem), make_float4(o0, o1, o2, o3));
+    } else {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b2 = __floats2bfloat162_rn(o2, o3);
+        __stcs(reinterpret_cast<uint2*>(dst_elem), make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b2)));
+    }
+}
+
+// Row blocks, cols % 1024 == 0: a warp owns 1024 consecutive elements of one row = 32 blocks.  Lane l fetches
+// and decodes the scale of block l once; in step u (128 elements) lane l owns elements 4l..4l+3 of block
+// 4u + l/8 and takes its scale by shuffle.  One 4-byte load and one 8/16-byte store per lane and step.
+template <int ELEM, int DST>
+__global__ void __launch_bounds__(256)
+dequantize_row1024_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, int64_t cols, int sf_layout,
+                          void* __restrict__ dst_v, int64_t chunks)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;     // 1024-element chunk
+    if (chunk >= chunks) return;
+    const int64_t per_row = cols >> 10;
+    const int64_t r = chunk / per_row;
+    const int64_t c0 = (chunk - r * per_row) << 10;
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(q + r * cols + c0) + lane;
+    uint32_t w[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) w[u] = __ldcs(src + u * 32);
+    const int64_t ncb = cols >> 5, kb = (c0 >> 5) + lane;
+    const float mine = scale_value(s[(sf_layout == MXFP8_SF_SWIZZLED) ? sf_swizzled_offset(r, kb, ncb) : r * ncb + kb]);
+    constexpr int ESZ = (DST == MXFP8_FP32) ? 4 : 2;
+    uint8_t* out = static_cast<uint8_t*>(dst_v) + (r * cols + c0 + lane * 4) * ESZ;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const float sc = __shfl_sync(0xFFFFFFFFu, mine, 4 * u + (lane >> 3));
+        decode_store4<ELEM, DST>(w[u], sc, sc, sc, sc, out + u * 128 * ESZ);
+    }
+}
+
+// Column blocks: a warp owns a strip of 128 columns x 32 rows = one block of every column of the strip, so
+// each lane fetches and decodes the four scales of its columns once and reuses them for the 32 rows.
+template <int ELEM, int DST>
+__global__ void __launch_bounds__(256)
+dequantize_colstrip_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ s, int64_t rows, int64_t cols,
+                           int sf_layout, void* __restrict__ dst_v, int64_t strips)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t strip = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (strip >= strips) return;
+    const int64_t strips_per_band = cols >> 7;
+    const int64_t kb = strip / strips_per_band;                       // 32-row band = block index along the rows
+    const int64_t c = ((strip - kb * strips_per_band) << 7) + lane * 4;
+    const int64_t nrb = rows >> 5;
+    float sc[4];
+    if (sf_layout == MXFP8_SF_SWIZZLED) {
+        const uint8_t* base = s + sf_swizzled_offset(c, kb, nrb);    // columns c..c+3 sit 16 bytes apart in their atom
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sc[i] = scale_value(base[i * 16]);
+    } else {
+        const uint32_t four = *reinterpret_cast<const uint32_t*>(s + kb * cols + c);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sc[i] = scale_value((four >> (8 * i)) & 0xFFu);
+    }
+    constexpr int ESZ = (DST == MXFP8_FP32) ? 4 : 2;
+    const uint8_t* src = q + (kb * 32) * cols + c;
+    uint8_t* out = static_cast<uint8_t*>(dst_v) + ((kb * 32) * cols + c) * ESZ;
+#pragma unroll
+    for (int j0 = 0; j0 < 32; j0 += 8) {
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w[j] = __ldcs(reinterpret_cast<const uint32_t*>(src + (int64_t)(j0 + j) * cols));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) decode_store4<ELEM, DST>(w[j], sc[0], sc[1], sc[2], sc[3], out + (int64_t)(j0 + j) * cols * ESZ);
+    }
+}
+
 template <int ELEM, int DST, int ORIENT>
 cudaError_t launch(const uint8_t* q, const uint8_t* s, int64_t rows, int64_t cols, int sf_layout,
                    void* dst, cudaStream_t stream)
 {
+    if constexpr (ELEM == MXFP8_E4M3 || ELEM == MXFP8_E5M2) {
+        if (ORIENT == MXFP8_ROW && (cols & 1023) == 0) {
+            const int64_t chunks = rows * (cols >> 10);
+            const int64_t blocks = (chunks + 7) / 8;               // 8 warps per block
+            if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+            dequantize_row1024_kernel<ELEM, DST><<<(unsigned)blocks, 256, 0, stream>>>(q, s, cols, sf_layout, dst, chunks);
+            count_launch(1);
+            return cudaGetLastError();
+        }
+        if (ORIENT == MXFP8_COL && (cols & 127) == 0) {
+            const int64_t strips = (rows >> 5) * (cols >> 7);
+            const int64_t blocks = (strips + 7) / 8;
+            if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+            dequantize_colstrip_kernel<ELEM, DST><<<(unsigned)blocks, 256, 0, stream>>>(q, s, rows, cols, sf_layout, dst, strips);
+            count_launch(1);
+            return cudaGetLastError();
+        }
+    }
     if constexpr (ELEM == MXFP8_E4M3 || ELEM == MXFP8_E5M2) if ((cols & 127) == 0) {
         const int64_t groups = rows * (cols / 128);            // warp steps of 128 elements
         const int64_t warps = (groups + 7) / 8;
