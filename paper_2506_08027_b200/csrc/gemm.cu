@@ -22,6 +22,13 @@
 //   byte per row per MMA = one 4-byte TMEM column entry per K step).
 //   Every mbarrier wait is bounded: on expiry the kernel records MXFP8_ERR_DEVICE_TIMEOUT in
 //   the device status word, raises an abort flag that all roles poll, drains and exits.
+//   The same kernel runs, by template parameter MODE, one dense product, up to three independent
+//   products as one pool of tiles (MULTI: mxfp8_gemm_multi), or the per-expert products of a
+//   mixture-of-experts layer with the token axis split by device-side offsets (GROUP_M: tokens are
+//   the rows of A; GROUP_K: tokens are the reduction axis): every role decodes "where does tile t
+//   sit" through decode_tile() and shifts its TMA coordinates, K range and output rows accordingly.
+//   Operands of any of the five element types of Table 1: the format codes go into the
+//   instruction descriptor, 6- and 4-bit codes arrive in packed 16-byte slots.
 #include <cuda.h>
 #include <cstdio>
 #include <cstdlib>

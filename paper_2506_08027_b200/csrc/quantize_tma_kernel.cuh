@@ -13,7 +13,11 @@
 //   pass B (row blocks)   : amax across the lanes of a 32-column block by xor-shuffles; BF16 rows
 //                           go through the shuffles two at a time (one in each half of a register)
 //   scale: integer form of Algorithm 1 / App. A.1 on the amax bit pattern (see mxfp8_device.cuh)
-//   cast : x * 2^-e in FP32 (exact), cvt.rn.satfinite to e4m3x2 / e5m2x2
+//   cast : x * 2^-e in FP32 (exact), cvt.rn.satfinite to the element type (e4m3x2 / e5m2x2, or the
+//          6- / 4-bit types, whose codes are then packed 16 to a 16-byte slot across the lanes)
+//   One launch takes up to 8 tensors (their tiles form one pool); optional in-place prologues on the
+//   tile in shared memory: an activation function or an RMS normalisation ahead of the conversion;
+//   optional store mode that writes the decoded values back instead of the codes (round trip).
 #pragma once
 
 #include <cuda.h>
