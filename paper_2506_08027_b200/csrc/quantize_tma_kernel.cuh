@@ -238,7 +238,7 @@ __device__ __forceinline__ void emit(uint8_t* dst, const float (&x)[VEC], const 
 template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
 __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uint8_t* __restrict__ my_qrow,
                                           uint8_t* __restrict__ my_qcol, uint32_t pitch, uint8_t* my_sm_row,
-                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset, bool col_ok)
+                                          uint8_t* my_sm_col, int lane, uint32_t rule_offset)
 {
     constexpr bool BF = (DTYPE == MXFP8_BF16);
     constexpr int VEC = BF ? 4 : 2;
@@ -337,12 +337,12 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
             const float xs0 = EMU ? scale_from_inv(inv0) : 0.f, xs1 = EMU ? scale_from_inv(inv1) : 0.f;
 #pragma unroll
             for (int i = 0; i < VEC; ++i) { i0[i] = inv0; i1[i] = inv1; s0[i] = xs0; s1[i] = xs1; }
-            emit<ELEM, VEC, EMU>(r0, x0, i0, s0, lane, col_ok);
-            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1, lane, col_ok);
+            emit<ELEM, VEC, EMU>(r0, x0, i0, s0, lane);
+            emit<ELEM, VEC, EMU>(r0 + pitch, x1, i1, s1, lane);
         }
         if (DO_COL) {
-            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs, lane, col_ok);
-            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs, lane, col_ok);
+            emit<ELEM, VEC, EMU>(c0, x0, col_inv, col_xs, lane);
+            emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs, lane);
         }
     }
     return __any_sync(0xFFFFFFFFu, bad != 0u);
@@ -532,12 +532,10 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         const uint32_t pitch = (uint32_t)p.cols * OUT_ESZ;
         uint8_t* my_sm_row = sm_row + warp * 128 + lane / LPB;
         uint8_t* my_sm_col = sm_col + lane * VEC * 4 + warp;
-        // columns beyond the tensor hold TMA's zero fill: they cannot raise an amax, and their lanes simply do not
-        // store, so the fast path also serves the ragged last tile column; ragged rows take the careful path
-        const bool whole = rows_here == 32;
+        const bool whole = __all_sync(0xFFFFFFFFu, col_ok) && rows_here == 32;
         bool special = !whole;
         if (whole)
-            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset, col_ok);
+            special = slab_fast<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset);
         if (special && rows_here > 0)
             slab_careful<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
                                                        rows_here, col_ok);
