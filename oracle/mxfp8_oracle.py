@@ -351,3 +351,20 @@ def rmsnorm(x: np.ndarray, gamma: np.ndarray, eps: float, dst: str = "f32", rstd
     y64 = np.ascontiguousarray(y32, dtype=np.float64)
     _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
     return out, rstd
+
+
+def glu(x: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
+    """Gated activation ahead of the conversion: x is [rows, 2*cols] = (gate | up); y = act(gate) * up, with act(gate)
+    as in `activation` (binary64 definition rounded to binary32), then one binary32 product, then one rounding to
+    bfloat16 for dst "bf16".  Returns [rows, cols] float32 values ("f32") or uint16 patterns ("bf16")."""
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    cols = x32.shape[1] // 2
+    a = activation(x32[:, :cols], act, "f32")
+    with np.errstate(over="ignore", invalid="ignore"):
+        y32 = a * x32[:, cols:]                 # numpy float32 product: one IEEE single operation
+    if dst == "f32":
+        return y32
+    out = np.empty(y32.shape, dtype=np.uint16)
+    y64 = np.ascontiguousarray(y32, dtype=np.float64)
+    _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
+    return out

@@ -633,3 +633,21 @@ def test_rmsnorm_oracle_against_exact_cases_and_library():
     # a supplied rstd is used as is; BF16 destination rounds once more (ties to even)
     y2, r2 = orc.rmsnorm(np.array([[1.0 + 2.0 ** -8, 3.0]], np.float32), np.ones(2, np.float32), 0.0, "bf16", np.array([1.0], np.float32))
     assert y2[0].tolist() == [0x3F80, 0x4040] and r2[0] == 1.0
+
+
+def test_glu_oracle_against_hand_values_and_library():
+    import torch
+    # (gate | up) = ([-2, 3] | [5, 0.5]): relu gate -> [0*5, 3*0.5]; bilinear -> [-10, 1.5]
+    x = np.array([[-2.0, 3.0, 5.0, 0.5]], np.float32)
+    assert orc.glu(x, orc.ACT_RELU).tolist() == [[0.0, 1.5]]
+    assert orc.glu(x, orc.ACT_NONE).tolist() == [[-10.0, 1.5]]
+    assert orc.glu(x, orc.ACT_RELU2).tolist() == [[0.0, 4.5]]
+    rng = np.random.default_rng(4)
+    g = rng.standard_normal((32, 64)) * 3
+    u = rng.standard_normal((32, 64))
+    xx = np.concatenate([g, u], axis=1).astype(np.float32)
+    lib = (torch.nn.functional.silu(torch.from_numpy(xx[:, :64]).double()) * torch.from_numpy(xx[:, 64:]).double()).numpy()
+    mine = orc.glu(xx, orc.ACT_SILU).astype(np.float64)
+    assert np.abs(mine - lib).max() <= 2.0 ** -22 * np.abs(lib).max()          # two binary32 roundings
+    b = orc.glu(np.array([[1.0 + 2.0 ** -8, 1.0]], np.float32), orc.ACT_NONE, "bf16")
+    assert b.tolist() == [[0x3F80]]
