@@ -560,6 +560,12 @@ def run_sweep(args):
             ms = _time_calls(lambda i: B.mxfp8_act_quantize(src, act, B.BOTH, P, B.E4M3, *outs, S), 1)
             gbs = rows * cols * (2 + 2 * (1 + 1 / 32)) / ms / 1e6
             print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+        src2 = synth.device_tensor("gaussian", (rows, 2 * cols), 13, "bf16")
+        for act, name in ((B.ACT_SILU, "gated silu (SwiGLU): source 16384 x 16384 = (gate | up)"), (B.ACT_RELU, "gated relu (ReGLU)")):
+            ms = _time_calls(lambda i: B.mxfp8_glu_quantize(src2, act, B.BOTH, P, B.E4M3, *outs, S), 1)
+            gbs = rows * cols * (4 + 2 * (1 + 1 / 32)) / ms / 1e6       # gate and up are read, one [rows, cols] result in both orientations written
+            print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+        del src2
         gamma = torch.ones(cols, dtype=torch.bfloat16, device="cuda")
         rstd = torch.empty(rows, dtype=torch.float32, device="cuda")
         ms = _time_calls(lambda i: B.mxfp8_rmsnorm_quantize(src, gamma, 1e-5, rstd, B.BOTH, P, B.E4M3, *outs, S), 1)

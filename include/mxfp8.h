@@ -149,6 +149,22 @@ int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, int64_t col
                        int sf_layout, void* stream);
 
 /*
+ * mxfp8_glu_quantize -- a gated activation fused ahead of the conversion: the source is [rows, 2 * cols]
+ * with the gate in columns 0 .. cols-1 and the up projection in columns cols .. 2*cols-1 (one tensor,
+ * as a fused gate/up GEMM writes it), and
+ *     y[r, c] = act(gate[r, c]) * up[r, c]
+ * is evaluated in FP32 (act as in mxfp8_act_quantize, then one FP32 product), rounded once to the source
+ * dtype, and converted exactly as mxfp8_quantize(y) of the [rows, cols] result (MXFP8_ACT_SILU: SwiGLU,
+ * MXFP8_ACT_GELU_TANH: GeGLU, MXFP8_ACT_RELU: ReGLU, MXFP8_ACT_NONE: the bilinear form).  Same place in
+ * the recipe as mxfp8_act_quantize (Sec. 3.2).  cols must be a multiple of 128 (BF16 source) or 64 (FP32
+ * source) -- MXFP8_ERR_UNSUPPORTED otherwise; other arguments as mxfp8_quantize.
+ */
+int mxfp8_glu_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int act,
+                       int orientation, int scale_rule, int elem,
+                       void* q_row, void* s_row, void* q_col, void* s_col,
+                       int sf_layout, void* stream);
+
+/*
  * mxfp8_rmsnorm_quantize -- RMS normalisation fused ahead of the conversion (Sec. 3.2 keeps the
  * normalisation layers in high precision and converts their output for the next GEMM).  Two launches:
  *   rstd[r] = 1 / sqrt(mean_c(x[r, c]^2) + eps)     FP32 accumulation over the row, written to `rstd`

@@ -29,7 +29,7 @@ EXPORTS = (
     "mxfp8_launch_count", "mxfp8_quantize_host_ws_bytes", "mxfp8_quantize_host",
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
-    "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows",
+    "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
 )
 
 
@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_rmsnorm_quantize_static.argtypes = [p, i, i64, i64, p, ctypes.c_float, i, i, i, p, p, p, p, i, p]
         L.mxfp8_rmsnorm_quantize_static_max_rows.restype = i64
         L.mxfp8_rmsnorm_quantize_static_max_rows.argtypes = []
+        L.mxfp8_glu_quantize.restype = i
+        L.mxfp8_glu_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_act_quantize.restype = i
         L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_gemm_multi.restype = i
@@ -345,3 +347,13 @@ def mxfp8_rmsnorm_quantize_static(src: torch.Tensor, gamma: torch.Tensor, eps: f
     _check(lib().mxfp8_rmsnorm_quantize_static(_ptr(src), _dtype_code(src), rows, cols, _ptr(gamma), eps,
                                                orientation, scale_rule, elem, _ptr(q_row), _ptr(s_row), _ptr(q_col),
                                                _ptr(s_col), sf_layout, _stream(stream)), "mxfp8_rmsnorm_quantize_static")
+
+
+def mxfp8_glu_quantize(src: torch.Tensor, act: int, orientation: int, scale_rule: int, elem: int,
+                       q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    """src: [rows, 2 * cols] = (gate | up); the outputs have shape [rows, cols]."""
+    rows, two_cols = src.shape
+    assert src.is_contiguous() and two_cols % 2 == 0
+    _check(lib().mxfp8_glu_quantize(_ptr(src), _dtype_code(src), rows, two_cols // 2, act, orientation, scale_rule, elem,
+                                    _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
+                                    _stream(stream)), "mxfp8_glu_quantize")

@@ -369,6 +369,35 @@ extern "C" int mxfp8_quantize_multi(const mxfp8_quantize_item* items, int count,
     return quantize_tma_batch(batch, count, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int mxfp8_glu_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int act,
+                                  int orientation, int scale_rule, int elem,
+                                  void* q_row, void* s_row, void* q_col, void* s_col,
+                                  int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (act < MXFP8_ACT_NONE || act > MXFP8_ACT_GELU_TANH) return MXFP8_ERR_ENUM;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!src) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col || !s_col)) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(src)) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    // whole tiles along the columns: a tile of the gate half must not reach into the up half
+    if (cols % (src_dtype == MXFP8_BF16 ? 128 : 64)) return MXFP8_ERR_UNSUPPORTED;
+    if (!quantize_tma_eligible(src_dtype, rows, 2 * cols)) return MXFP8_ERR_UNSUPPORTED;
+    const QuantizeItem item{src, rows, cols, q_row, s_row, q_col, s_col};
+    return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream), false, act,
+                              nullptr, nullptr, true);
+}
+
 namespace mxfp8 {
 namespace {
 // 1/rms of every row: one warp per row, 16-byte loads, FP32 accumulation (lane-strided partial sums, then a

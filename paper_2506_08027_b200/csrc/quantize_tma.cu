@@ -62,7 +62,8 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
 }
 
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
-                       int sf_layout, cudaStream_t stream, bool emulate, int act, const float* rstd, const void* gamma)
+                       int sf_layout, cudaStream_t stream, bool emulate, int act, const float* rstd, const void* gamma,
+                       bool gated)
 {
     if (count < 1 || count > QT_MAX_TENSORS) return MXFP8_ERR_UNSUPPORTED;
     const bool bf = src_dtype == MXFP8_BF16;
@@ -73,11 +74,12 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
     p.act = act;
     p.rstd = rstd;
     p.gamma = gamma;
+    p.glu_cols = gated ? (int)items[0].cols : 0;     // gated: one tensor, source [rows, 2 * cols]
     int64_t tiles = 0;
     for (int i = 0; i < QT_MAX_TENSORS; ++i) {
         const QuantizeItem& it = items[i < count ? i : 0];   // unused slots repeat the first tensor: every map stays valid
         if (!make_map_2d(&ms.m[i], bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
-                         const_cast<void*>(it.src), (uint64_t)it.cols, (uint64_t)it.rows, t_cols, T_ROWS))
+                         const_cast<void*>(it.src), (uint64_t)(gated ? 2 * it.cols : it.cols), (uint64_t)it.rows, t_cols, T_ROWS))
             return MXFP8_ERR_CUDA;
         if (i >= count) continue;
         QParams& q = p.t[i];

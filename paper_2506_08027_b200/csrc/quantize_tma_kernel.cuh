@@ -114,6 +114,29 @@ __device__ __forceinline__ void norm_slab(uint8_t* mine, const float* __restrict
     }
 }
 
+// Gated activation in place: gate tile <- act(gate) * up (FP32 product), rounded once to the source dtype.
+template <int ACT, bool BF>
+__device__ __forceinline__ void glu_slab(uint8_t* gate, const uint8_t* up)
+{
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+        uint2 g = *reinterpret_cast<const uint2*>(gate + j * T_BYTES);
+        const uint2 u = *reinterpret_cast<const uint2*>(up + j * T_BYTES);
+        if constexpr (BF) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(apply_act<ACT>(__uint_as_float(g.x << 16)) * __uint_as_float(u.x << 16),
+                                                            apply_act<ACT>(__uint_as_float(g.x & 0xFFFF0000u)) * __uint_as_float(u.x & 0xFFFF0000u));
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(apply_act<ACT>(__uint_as_float(g.y << 16)) * __uint_as_float(u.y << 16),
+                                                            apply_act<ACT>(__uint_as_float(g.y & 0xFFFF0000u)) * __uint_as_float(u.y & 0xFFFF0000u));
+            g.x = *reinterpret_cast<const uint32_t*>(&lo);
+            g.y = *reinterpret_cast<const uint32_t*>(&hi);
+        } else {
+            g.x = __float_as_uint(apply_act<ACT>(__uint_as_float(g.x)) * __uint_as_float(u.x));
+            g.y = __float_as_uint(apply_act<ACT>(__uint_as_float(g.y)) * __uint_as_float(u.y));
+        }
+        *reinterpret_cast<uint2*>(gate + j * T_BYTES) = g;
+    }
+}
+
 // One launch converts up to QT_MAX_TENSORS tensors: their tiles are numbered one tensor after the
 // other and dealt out to the CTAs as one pool, so small tensors share one ramp-up and one tail and
 // the per-CTA tile counts even out.
@@ -123,6 +146,7 @@ struct QBatch {
     int act;                              // MXFP8_ACT_*: applied to every element before the conversion
     const float* rstd;                    // RMS normalisation ahead of the conversion (first tensor only): 1/rms per row,
     const void* gamma;                    //   and the per-column weight in the source dtype; both null when unused
+    int glu_cols;                         // gated activation: the source is [rows, 2 * glu_cols] = (gate | up); 0 when unused
     int count;
     int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
     QParams t[QT_MAX_TENSORS];
@@ -422,7 +446,7 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
     }
 }
 
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU>
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU, bool GLU>
 __global__ void __launch_bounds__(QT_THREADS, 3)
 quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QBatch batch)
 {
@@ -435,7 +459,9 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* in_ring = smem;                               // 2 x [128][256]
     uint8_t* sm_scales = smem + 2 * IN_BYTES;              // 2 x ([128][4] row scales + [T_COLS][4] column scales)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);   // [0], [1]: ring slots; [2]: the up tile (gated mode)
+    uint8_t* up_buf = sm_scales + 2048 + 128;                         // gated mode only: [128][256], allocated by such launches
+    const int glu_cols = GLU ? batch.glu_cols : 0;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;   // warp = 32-row slab of the tile
     const uint32_t rule_offset = (batch.t[0].rule == MXFP8_RULE_PAPER) ? paper_offset<ELEM>() : 0u;
@@ -443,6 +469,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
+        if (GLU) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[2])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -458,10 +485,36 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                      ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&maps.m[load_ti]), "r"(b), "r"((lt % tx) * T_COLS), "r"((lt / tx) * T_ROWS)
                      : "memory");
     };
+    auto issue_up = [&](int t) {              // gated mode (one tensor per launch): the up half of tile t
+        const int tx = batch.t[0].tiles_x;
+        const uint32_t b = smem_addr(&bars[2]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                     ::"r"(smem_addr(up_buf)), "l"(&maps.m[0]), "r"(b), "r"(glu_cols + (t % tx) * T_COLS), "r"((t / tx) * T_ROWS)
+                     : "memory");
+    };
+    // bounded wait on one of the barriers: false when the limit passed
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+        uint32_t ok = 0, spins = 0;
+        uint64_t t0 = 0;
+        while (true) {
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+            if (ok) break;
+            if ((++spins & 0xFFu) == 0) {
+                uint64_t now;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > QT_WAIT_LIMIT_NS) break;
+            }
+        }
+        return ok != 0;
+    };
     int tile = blockIdx.x, ti = 0;
     if (tid == 0) {
         if (tile < num_tiles) issue_load(tile, 0);
         if (tile + (int)gridDim.x < num_tiles) issue_load(tile + gridDim.x, 1);
+        if (GLU && tile < num_tiles) issue_up(tile);
     }
 
     for (int it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
@@ -479,23 +532,27 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
 
         // wait for the tile (bounded: on expiry report through the status word and leave)
         {
-            uint32_t ok = 0, spins = 0;
-            uint64_t t0 = 0;
-            while (true) {
-                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                             : "=r"(ok) : "r"(bar_a), "r"(phase) : "memory");
-                if (ok) break;
-                if ((++spins & 0xFFu) == 0) {
-                    uint64_t now;
-                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > QT_WAIT_LIMIT_NS) break;
-                }
-            }
+            bool ok = wait_bar(bar_a, phase);
+            if constexpr (GLU) ok = wait_bar(smem_addr(&bars[2]), (uint32_t)it & 1u) && ok;
             if (!__syncthreads_and((int)ok)) {
                 if (tid == 0) atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
                 return;
             }
+        }
+        if constexpr (GLU) {
+            // gated activation: the slot holds the gate tile, up_buf the up tile; the slot becomes act(gate) * up
+            uint8_t* mine = in_tile + warp * 32 * T_BYTES + lane * 8;
+            const uint8_t* mine_up = up_buf + warp * 32 * T_BYTES + lane * 8;
+            switch (batch.act) {
+                case MXFP8_ACT_NONE: glu_slab<MXFP8_ACT_NONE, BF>(mine, mine_up); break;
+                case MXFP8_ACT_RELU: glu_slab<MXFP8_ACT_RELU, BF>(mine, mine_up); break;
+                case MXFP8_ACT_RELU2: glu_slab<MXFP8_ACT_RELU2, BF>(mine, mine_up); break;
+                case MXFP8_ACT_SILU: glu_slab<MXFP8_ACT_SILU, BF>(mine, mine_up); break;
+                default: glu_slab<MXFP8_ACT_GELU_TANH, BF>(mine, mine_up); break;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();                     // every warp has consumed the up tile: fetch the next one under the conversion
+            if (tid == 0 && tile + (int)gridDim.x < num_tiles) issue_up(tile + gridDim.x);
         }
         if (batch.rstd != nullptr) {
             // RMS normalisation in place (single-tensor launches only), then the unchanged conversion
@@ -506,7 +563,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                           static_cast<const uint8_t*>(batch.gamma) + col_first * (BF ? 2 : 4), rows_in, col_first < p.cols);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        if (batch.act != MXFP8_ACT_NONE) {
+        if (!GLU && batch.act != MXFP8_ACT_NONE) {
             // activation in place: every lane rewrites exactly the 8 bytes per row it reads below, rounded once
             // to the source dtype, so what follows equals the conversion of a tensor that holds act(x)
             uint8_t* mine = in_tile + warp * 32 * T_BYTES + lane * 8;
@@ -599,28 +656,29 @@ int qt_sm_count()
     return n;
 }
 
-template <int DTYPE, int ELEM, bool R, bool C, bool EMU>
+template <int DTYPE, int ELEM, bool R, bool C, bool EMU, bool GLU>
 cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
 {
-    constexpr int SMEM = 2 * IN_BYTES + 2048 + 16;
-    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU>;
+    constexpr int SMEM = 2 * IN_BYTES + 2048 + 128;          // ring, scale staging, barriers
+    constexpr int SMEM_USED = GLU ? SMEM + IN_BYTES : SMEM;  // + the up tile of the gated mode
+    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU, GLU>;
     static unsigned long long smem_set = 0;
-    cudaError_t err = ensure_dynamic_smem(kernel, SMEM, smem_set);
+    cudaError_t err = ensure_dynamic_smem(kernel, SMEM_USED, smem_set);
     if (err != cudaSuccess) return err;
     const int tiles = p.tile_start[p.count];
-    const int max_ctas = qt_sm_count() * 3;
+    const int max_ctas = qt_sm_count() * (GLU ? 2 : 3);
     const int grid = tiles < max_ctas ? tiles : max_ctas;
-    kernel<<<grid, QT_THREADS, SMEM, stream>>>(ms, p);
+    kernel<<<grid, QT_THREADS, SMEM_USED, stream>>>(ms, p);
     count_launch(1);
     return cudaGetLastError();
 }
 
-template <int DTYPE, int ELEM, bool EMU>
+template <int DTYPE, int ELEM, bool EMU, bool GLU = false>
 cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
-    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU>(ms, p, st);
-    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU>(ms, p, st);
-    return launch<DTYPE, ELEM, true, true, EMU>(ms, p, st);
+    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU, GLU>(ms, p, st);
+    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU, GLU>(ms, p, st);
+    return launch<DTYPE, ELEM, true, true, EMU, GLU>(ms, p, st);
 }
 
 
@@ -629,6 +687,8 @@ cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStre
 template <int ELEM>
 cudaError_t quantize_tma_launch(bool bf16_src, int orientation, bool emulate, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
+    if (p.glu_cols)
+        return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, true>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false, true>(orientation, ms, p, st);
     if (emulate)
         return bf16_src ? launch_o<MXFP8_BF16, ELEM, true>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, true>(orientation, ms, p, st);
     return bf16_src ? launch_o<MXFP8_BF16, ELEM, false>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false>(orientation, ms, p, st);

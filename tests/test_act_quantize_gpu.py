@@ -207,3 +207,96 @@ def test_rmsnorm_argument_errors():
     B.mxfp8_rmsnorm_quantize(x, g, 0.0, r, B.ROW, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
     torch.cuda.synchronize()
     assert torch.isinf(r).all() and (q == 0x7F).all()
+
+
+# ------------------------------------------------------------------------------------------ gated activation
+
+def gpu_glu_quantize(src_np, dtype, act, orientation, elem=orc.E4M3):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, two_cols = src_np.shape
+    cols = two_cols // 2
+    src = torch.from_numpy(src_np.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(src_np).cuda()
+    bufs, args = {}, []
+    for o, name in ((B.ROW, "row"), (B.COL, "col")):
+        if orientation & o:
+            bufs[name] = (Guarded(rows * cols), Guarded(B.mxfp8_scale_bytes(rows, cols, o, B.SF_SWIZZLED)))
+            args += [bufs[name][0].view.view(rows, cols), bufs[name][1].view]
+        else:
+            args += [None, None]
+    B.mxfp8_glu_quantize(src, act, orientation, B.RULE_PAPER, elem, *args, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    out = {}
+    for name, (q, s) in bufs.items():
+        q.check(); s.check()
+        mn, nkb = (rows, cols // 32) if name == "row" else (cols, rows // 32)
+        logical = logical_scales_from_swizzled(s.numpy(), mn, nkb)
+        out[name] = (orc.unpack_codes16(q.numpy().reshape(rows, cols), elem), logical if name == "row" else np.ascontiguousarray(logical.T))
+    return out
+
+
+@pytest.mark.parametrize("act", [orc.ACT_RELU, orc.ACT_NONE, orc.ACT_RELU2])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(256, 2 * 256), (160, 2 * 384), (96, 2 * 1408), (1056, 2 * 128)])
+def test_gated_exact_activations_bit_exact(act, dtype, shape):
+    # many tiles per CTA on the last shape: the up tile is prefetched one tile ahead
+    x = as_dtype(synth.gaussian(shape, 21 + act + shape[0]) * np.float32(2.0), dtype)
+    xv = orc.bf16_bits_to_f32(x) if dtype == "bf16" else x
+    y = orc.glu(xv, act, "bf16" if dtype == "bf16" else "f32")
+    y = orc.bf16_bits_to_f32(y) if dtype == "bf16" else y
+    got = gpu_glu_quantize(x, dtype, act, BOTH)
+    for o, name in ((orc.ROW, "row"), (orc.COL, "col")):
+        wq, ws = orc.quantize(y, o, orc.RULE_PAPER, orc.E4M3)
+        assert np.array_equal(got[name][1], ws), "scales %s" % name
+        assert_q_equal(got[name][0], wq, orc.E4M3, name)
+
+
+def test_swiglu_matches_up_to_rounding_boundaries_and_many_tiles():
+    x = as_dtype(synth.gaussian((2048, 2 * 1408), 8) * np.float32(2.0), "bf16")         # 16 x 11 tiles on 296 CTAs? no: 176 tiles
+    xv = orc.bf16_bits_to_f32(x)
+    y = orc.bf16_bits_to_f32(orc.glu(xv, orc.ACT_SILU, "bf16"))
+    got = gpu_glu_quantize(x, "bf16", orc.ACT_SILU, BOTH)
+    for o, name in ((orc.ROW, "row"), (orc.COL, "col")):
+        wq, ws = orc.quantize(y, o, orc.RULE_PAPER, orc.E4M3)
+        gq, gs = got[name]
+        same_scale = gs == ws
+        assert same_scale.mean() >= 0.999
+        blk = np.repeat(same_scale, 32, axis=1) if o == orc.ROW else np.repeat(same_scale, 32, axis=0)
+        diff = (gq != wq) & blk
+        assert diff.mean() <= 2e-3
+        a, b = gq[diff].astype(np.int32), wq[diff].astype(np.int32)
+        assert (np.abs((a & 0x7F) - (b & 0x7F)) <= 1).all()
+
+
+def test_gated_equals_torch_reglu_then_quantize_on_device_large():
+    # 8192 x (2 x 4096): more tiles than resident CTAs, every CTA walks several tiles
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    x = synth.device_tensor("activation", (8192, 2 * 4096), 12)
+    xf = x.float()
+    y = (torch.relu(xf[:, :4096]) * xf[:, 4096:]).to(torch.bfloat16).contiguous()
+    a = B.alloc_quantize_outputs(8192, 4096, B.BOTH, B.SF_SWIZZLED)
+    b = B.alloc_quantize_outputs(8192, 4096, B.BOTH, B.SF_SWIZZLED)
+    for t in a + b:
+        t.zero_()
+    B.mxfp8_glu_quantize(x, B.ACT_RELU, B.BOTH, B.RULE_PAPER, B.E4M3, *a, B.SF_SWIZZLED)
+    B.mxfp8_quantize(y, B.BOTH, B.RULE_PAPER, B.E4M3, *b, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for u, v in zip(a, b):
+        assert torch.equal(u, v)
+
+
+def test_gated_argument_errors():
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    x = torch.zeros(64, 2 * 96, dtype=torch.bfloat16, device="cuda")          # 96 output columns: not whole tiles
+    q, s, _, _ = B.alloc_quantize_outputs(64, 96, B.ROW, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error) as e:
+        B.mxfp8_glu_quantize(x, B.ACT_SILU, B.ROW, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
+    assert e.value.status == -5
+    x = torch.zeros(64, 2 * 128, dtype=torch.bfloat16, device="cuda")
+    q, s, _, _ = B.alloc_quantize_outputs(64, 128, B.ROW, B.SF_LINEAR)
+    with pytest.raises(B.Mxfp8Error):
+        B.mxfp8_glu_quantize(x, 11, B.ROW, B.RULE_PAPER, B.E4M3, q, s, None, None, B.SF_LINEAR)
