@@ -446,7 +446,11 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
     }
 }
 
-template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU, bool GLU>
+// PRO: what runs on a tile before the conversion.  Separate instantiations, so that the plain conversion carries
+// none of the prologue code (folding the prologues in at run time cost the plain kernels 2-5 %).
+enum { PRO_NONE = 0, PRO_ELEMENTWISE = 1 /* activation or RMS normalisation */, PRO_GLU = 2 /* gated activation */ };
+
+template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU, int PRO>
 __global__ void __launch_bounds__(QT_THREADS, 3)
 quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QBatch batch)
 {
@@ -455,6 +459,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     constexpr int T_COLS = T_BYTES / (BF ? 2 : 4);  // 128 or 64
     constexpr int NKB = T_COLS / 32;                // row blocks per tile row: 4 or 2
     constexpr int LPB = 32 / VEC;                   // lanes per row block: 8 or 16
+    constexpr bool GLU = (PRO == PRO_GLU);
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* in_ring = smem;                               // 2 x [128][256]
@@ -554,7 +559,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
             __syncthreads();                     // every warp has consumed the up tile: fetch the next one under the conversion
             if (tid == 0 && tile + (int)gridDim.x < num_tiles) issue_up(tile + gridDim.x);
         }
-        if (batch.rstd != nullptr) {
+        if (PRO == PRO_ELEMENTWISE && batch.rstd != nullptr) {
             // RMS normalisation in place (single-tensor launches only), then the unchanged conversion
             const int64_t row_first = grow0 + warp * 32;
             const int rows_in = (int)max((int64_t)0, min((int64_t)32, p.rows - row_first));
@@ -563,7 +568,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                           static_cast<const uint8_t*>(batch.gamma) + col_first * (BF ? 2 : 4), rows_in, col_first < p.cols);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        if (!GLU && batch.act != MXFP8_ACT_NONE) {
+        if (PRO == PRO_ELEMENTWISE && batch.act != MXFP8_ACT_NONE) {
             // activation in place: every lane rewrites exactly the 8 bytes per row it reads below, rounded once
             // to the source dtype, so what follows equals the conversion of a tensor that holds act(x)
             uint8_t* mine = in_tile + warp * 32 * T_BYTES + lane * 8;
@@ -656,12 +661,13 @@ int qt_sm_count()
     return n;
 }
 
-template <int DTYPE, int ELEM, bool R, bool C, bool EMU, bool GLU>
+template <int DTYPE, int ELEM, bool R, bool C, bool EMU, int PRO>
 cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
 {
+    constexpr bool GLU = (PRO == PRO_GLU);
     constexpr int SMEM = 2 * IN_BYTES + 2048 + 128;          // ring, scale staging, barriers
     constexpr int SMEM_USED = GLU ? SMEM + IN_BYTES : SMEM;  // + the up tile of the gated mode
-    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU, GLU>;
+    auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU, PRO>;
     static unsigned long long smem_set = 0;
     cudaError_t err = ensure_dynamic_smem(kernel, SMEM_USED, smem_set);
     if (err != cudaSuccess) return err;
@@ -673,12 +679,12 @@ cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
     return cudaGetLastError();
 }
 
-template <int DTYPE, int ELEM, bool EMU, bool GLU = false>
+template <int DTYPE, int ELEM, bool EMU, int PRO = PRO_NONE>
 cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
-    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU, GLU>(ms, p, st);
-    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU, GLU>(ms, p, st);
-    return launch<DTYPE, ELEM, true, true, EMU, GLU>(ms, p, st);
+    if (orientation == MXFP8_ROW) return launch<DTYPE, ELEM, true, false, EMU, PRO>(ms, p, st);
+    if (orientation == MXFP8_COL) return launch<DTYPE, ELEM, false, true, EMU, PRO>(ms, p, st);
+    return launch<DTYPE, ELEM, true, true, EMU, PRO>(ms, p, st);
 }
 
 
@@ -688,7 +694,10 @@ template <int ELEM>
 cudaError_t quantize_tma_launch(bool bf16_src, int orientation, bool emulate, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
     if (p.glu_cols)
-        return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, true>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false, true>(orientation, ms, p, st);
+        return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, PRO_GLU>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false, PRO_GLU>(orientation, ms, p, st);
+    if (p.rstd != nullptr || p.act != MXFP8_ACT_NONE)
+        return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, PRO_ELEMENTWISE>(orientation, ms, p, st)
+                        : launch_o<MXFP8_FP32, ELEM, false, PRO_ELEMENTWISE>(orientation, ms, p, st);
     if (emulate)
         return bf16_src ? launch_o<MXFP8_BF16, ELEM, true>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, true>(orientation, ms, p, st);
     return bf16_src ? launch_o<MXFP8_BF16, ELEM, false>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false>(orientation, ms, p, st);
