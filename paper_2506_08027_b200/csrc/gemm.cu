@@ -553,7 +553,8 @@ __device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const i
     }
 }
 
-template <int BN, bool PAIR, int MODE>
+// EPI: with the fused MXFP8 output compiled in (a separate instantiation: the plain kernels carry none of its code)
+template <int BN, bool PAIR, int MODE, bool EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
@@ -850,7 +851,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const int row0 = t.row0 + t.d_row_extra + (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
             const bool rows_inside = row0 < t.rows_end;      // ragged last M tile / rows of the next expert: a 32-row box entirely outside stores nothing
-            if constexpr (CW % 64 == 0) {
+            if constexpr (EPI && CW % 64 == 0) {
                 if (p.epi_orient && rows_inside) {
                     if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
                     else epi_mx<CW, MXFP8_E5M2>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
@@ -1009,11 +1010,11 @@ int sm_count()
 
 struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; MultiMaps multi; };
 
-template <int BN, bool PAIR, int MODE = DENSE>
+template <int BN, bool PAIR, int MODE = DENSE, bool EPI = false>
 int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
 {
     using C = Cfg<BN, PAIR>;
-    auto kernel = gemm_kernel<BN, PAIR, MODE>;
+    auto kernel = gemm_kernel<BN, PAIR, MODE, EPI>;
     static unsigned long long smem_set = 0;
     if (ensure_dynamic_smem(kernel, C::SMEM_TOTAL, smem_set) != cudaSuccess) return MXFP8_ERR_CUDA;
     p.tiles_m = (int)((p.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM));
@@ -1161,6 +1162,10 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
                 (long long)K, best_bn, best_pair ? "p" : "", (int)oka, (int)okb, (int)oks, (int)okd, (int)okq);
     if (!oka || !okb || !oks || !okd || !okq) return MXFP8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (epi) {   // 192-wide tiles are never chosen with a fused output
+        if (best_pair) return launch_gemm<256, true, DENSE, true>(m, p, st);
+        return best_bn == 256 ? launch_gemm<256, false, DENSE, true>(m, p, st) : launch_gemm<128, false, DENSE, true>(m, p, st);
+    }
     if (best_pair) return best_bn == 256 ? launch_gemm<256, true>(m, p, st) : launch_gemm<192, true>(m, p, st);
     if (best_bn == 256) return launch_gemm<256, false>(m, p, st);
     return best_bn == 192 ? launch_gemm<192, false>(m, p, st) : launch_gemm<128, false>(m, p, st);
