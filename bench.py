@@ -411,6 +411,27 @@ def run_case(args):
         for _ in range(reps):
             B.mxfp8_quantize_multi(items, B.BF16, B.BOTH, P, E, S)
             B.mxfp8_gemm_multi(gemms, B.BF16)
+    elif args.case == "grouped":
+        # per-expert fprop of a 64-expert layer (hidden 2048, expert FFN 1408, 49152 routed tokens, uniform routing)
+        import numpy as np
+        Hd, Fe, G = 2048, 1408, 64
+        rng = np.random.default_rng(2506)
+        padded = (rng.multinomial(8192 * 6, np.full(G, 1.0 / G)) + 127) // 128 * 128
+        offs = np.concatenate([[0], np.cumsum(padded)]).astype(np.int32)
+        Tt = int(offs[-1])
+        xa = synth.device_tensor("activation", (Tt, Hd), 21)
+        wst = synth.device_tensor("weight", (G * Fe, Hd), 23)
+        qx = B.alloc_quantize_outputs(Tt, Hd, B.ROW, S); B.mxfp8_quantize(xa, B.ROW, P, E, *qx, S)
+        qw = B.alloc_quantize_outputs(G * Fe, Hd, B.ROW, S); B.mxfp8_quantize(wst, B.ROW, P, E, *qw, S)
+        yg = torch.empty((Tt, Fe), dtype=torch.bfloat16, device="cuda")
+        off_d = torch.from_numpy(offs).cuda()
+        for _ in range(reps):
+            B.mxfp8_grouped_gemm(qx[0], qx[1], qw[0], qw[1], off_d, B.GROUP_M, Tt, Fe, Hd, B.K_MAJOR, E, E, yg)
+    elif args.case == "glu":
+        # SwiGLU fused ahead of the conversion: source 8192 x (2 x 8192) BF16, both orientations
+        src2 = synth.device_tensor("gaussian", (n, 2 * n), 13, "bf16")
+        for _ in range(reps):
+            B.mxfp8_glu_quantize(src2, B.ACT_SILU, B.BOTH, P, E, *q, S)
     elif args.case == "fake_quantize":
         dst = torch.empty_like(x)
         for _ in range(reps):
@@ -626,7 +647,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "step"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "step", "grouped", "glu"],
                     help="run one kernel on one small case and exit (for profiler captures)")
     ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
