@@ -651,3 +651,32 @@ def test_glu_oracle_against_hand_values_and_library():
     assert np.abs(mine - lib).max() <= 2.0 ** -22 * np.abs(lib).max()          # two binary32 roundings
     b = orc.glu(np.array([[1.0 + 2.0 ** -8, 1.0]], np.float32), orc.ACT_NONE, "bf16")
     assert b.tolist() == [[0x3F80]]
+
+
+def test_property_error_bound_and_no_saturation_under_the_paper_rule():
+    # Property check over generated blocks (all five element types): with the paper's scale rule no element
+    # saturates, so every finite element is reproduced to half a unit in the last place of its own binade on the
+    # element grid, or to half the smallest subnormal step, whichever is larger (Sec. 3.3: round to nearest).
+    from hypothesis import given, settings, strategies as st
+    fmt = {orc.E4M3: (3, -6, 448.0), orc.E5M2: (2, -14, 57344.0), orc.E2M3: (3, 0, 7.5), orc.E3M2: (2, -2, 28.0), orc.E2M1: (1, 0, 6.0)}
+
+    @settings(max_examples=120, deadline=None)
+    @given(st.integers(0, 4), st.integers(-60, 60), st.lists(st.floats(-1.0, 1.0, width=32), min_size=32, max_size=32),
+           st.integers(0, 31), st.floats(0.5, 1.0, width=32))
+    def check(elem_i, expo, body, pos, top):
+        elem = list(fmt)[elem_i]
+        mbits, emin, destmax = fmt[elem]
+        v = (np.array(body, np.float32) * np.float32(0.999)).astype(np.float32)
+        v[pos] = np.float32(top)                                   # the block maximum
+        x = (v * np.float32(2.0) ** expo).astype(np.float32).reshape(1, 32)
+        q, s = orc.quantize(x, orc.ROW, orc.RULE_PAPER, elem)
+        d = orc.dequantize_f64(q, s, orc.ROW, elem)
+        X = 2.0 ** (int(s[0, 0]) - 127)
+        y = x.astype(np.float64) / X
+        assert np.abs(y).max() <= destmax                          # no overflow: Sec. 3.3's point about rounding up
+        with np.errstate(divide="ignore"):
+            binade = np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** emin)))
+        half_ulp = 2.0 ** (binade - mbits - 1)
+        assert (np.abs(d / X - y) <= half_ulp * (1 + 1e-12)).all()
+
+    check()
