@@ -457,3 +457,29 @@ def test_k_permutation_leaves_exact_products_unchanged(majors):
         got = gpu_gemm(*stored(aq[:, perm], a_s[:, sperm], majors[0]), *stored(bq[:, perm], b_s[:, sperm], majors[1]),
                        majors[0], majors[1])
         assert np.array_equal(got, base)
+
+
+def test_bench_step_joint_launch_equals_single_launches_at_full_size():
+    # the benchmark's GEMM launch: fprop + dgrad + wgrad (tokens 8192, hidden 2048, FFN 8192) as one pool of tiles.
+    # Every output must equal, bit for bit, the single-product launch that test_bench_step_shapes_sampled_rows
+    # checks against the oracle.
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    T, H, F = 8192, 2048, 8192
+    E, S = B.E4M3, B.SF_SWIZZLED
+    X = synth.device_tensor("activation", (T, H), synth.seed_for(2, 0))
+    W = synth.device_tensor("weight", (F, H), synth.seed_for(2, 1))
+    dY = synth.device_tensor("output_gradient", (T, F), synth.seed_for(2, 2))
+    qX, qW, qdY = (B.alloc_quantize_outputs(t.shape[0], t.shape[1], B.BOTH, S) for t in (X, W, dY))
+    B.mxfp8_quantize_multi(B.make_quantize_items([(X,) + qX, (W,) + qW, (dY,) + qdY]), B.BF16, B.BOTH, B.RULE_PAPER, E, S)
+    specs = [(qX[0], qX[1], qW[0], qW[1], T, F, H, B.K_MAJOR, B.K_MAJOR),
+             (qdY[0], qdY[1], qW[2], qW[3], T, H, F, B.K_MAJOR, B.MN_MAJOR),
+             (qdY[2], qdY[3], qX[2], qX[3], F, H, T, B.MN_MAJOR, B.MN_MAJOR)]
+    joint = [torch.full((m, n), float("nan"), dtype=torch.bfloat16, device="cuda") for (_, _, _, _, m, n, _, _, _) in specs]
+    B.mxfp8_gemm_multi(B.make_gemm_problems([s + (E, E, d) for s, d in zip(specs, joint)]), B.BF16)
+    assert B.mxfp8_device_status() == 0
+    for (aq, a_s, bq, b_s, m, n, k, am, bm), d in zip(specs, joint):
+        single = torch.full((m, n), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.mxfp8_gemm(aq, a_s, bq, b_s, m, n, k, am, bm, E, E, single)
+        torch.cuda.synchronize()
+        assert torch.equal(d.view(torch.int16), single.view(torch.int16))
