@@ -483,3 +483,41 @@ def test_bench_step_joint_launch_equals_single_launches_at_full_size():
         B.mxfp8_gemm(aq, a_s, bq, b_s, m, n, k, am, bm, E, E, single)
         torch.cuda.synchronize()
         assert torch.equal(d.view(torch.int16), single.view(torch.int16))
+
+
+@pytest.mark.parametrize("case", ["ffn_up fprop", "qkv wgrad"])
+def test_fused_output_at_decoder_block_sizes_equals_quantize_of_unfused_output(case):
+    # two GEMMs of the 8B-class decoder block at full size (tokens 16384): the fused row+column MXFP8 output must
+    # be byte for byte what mxfp8_quantize makes of the same product's FP32 output (all on the device)
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    E, S = B.E4M3, B.SF_SWIZZLED
+    Tk = 16384
+    if case == "ffn_up fprop":
+        M, N, K, am, bm = Tk, 28672, 4096, B.K_MAJOR, B.K_MAJOR
+        a = synth.device_tensor("activation", (M, K), 41)
+        b = synth.device_tensor("weight", (N, K), 42)
+        qa = B.alloc_quantize_outputs(M, K, B.ROW, S); B.mxfp8_quantize(a, B.ROW, B.RULE_PAPER, E, *qa, S)
+        qb = B.alloc_quantize_outputs(N, K, B.ROW, S); B.mxfp8_quantize(b, B.ROW, B.RULE_PAPER, E, *qb, S)
+        ops = (qa[0], qa[1], qb[0], qb[1])
+    else:
+        M, N, K, am, bm = 6144, 4096, Tk, B.MN_MAJOR, B.MN_MAJOR            # dW = dY^T X, both operands token-major
+        dy = synth.device_tensor("output_gradient", (K, M), 43)
+        x = synth.device_tensor("activation", (K, N), 44)
+        qa = B.alloc_quantize_outputs(K, M, B.COL, S); B.mxfp8_quantize(dy, B.COL, B.RULE_PAPER, E, *qa, S)
+        qb = B.alloc_quantize_outputs(K, N, B.COL, S); B.mxfp8_quantize(x, B.COL, B.RULE_PAPER, E, *qb, S)
+        ops = (qa[2], qa[3], qb[2], qb[3])
+    d32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    B.mxfp8_gemm(*ops, M, N, K, am, bm, E, E, d32)
+    ref = B.alloc_quantize_outputs(M, N, B.BOTH, S)
+    B.mxfp8_quantize(d32, B.BOTH, B.RULE_PAPER, E, *ref, S)
+    fused = B.alloc_quantize_outputs(M, N, B.BOTH, S)
+    for t in fused:
+        t.zero_()
+    epi = B.make_epilogue(B.BOTH, B.RULE_PAPER, E, *fused)
+    d16 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    B.mxfp8_gemm(*ops, M, N, K, am, bm, E, E, d16, epi=epi)
+    assert B.mxfp8_device_status() == 0
+    for name, u, v in zip(("q_row", "s_row", "q_col", "s_col"), fused, ref):
+        assert torch.equal(u, v), name
+    assert torch.equal(d16, d32.to(torch.bfloat16))
