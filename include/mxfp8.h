@@ -351,7 +351,8 @@ int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t rows, int64
  *     FPROP  Y  [T, F] = X  * W^T   (row-blocked X,  row-blocked W)
  *     DGRAD  dX [T, H] = dY * W     (row-blocked dY, column-blocked W)
  *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
- * run as block-scaled GEMMs with BF16 output: two kernel launches on `stream` (the three casts
+ * run as block-scaled GEMMs with BF16 output (the call only enqueues work: it can be captured in a CUDA
+ * graph and replayed): two kernel launches on `stream` (the three casts
  * share one, the three GEMMs share one), no wait.  Y, dX, dW must not overlap.
  * T, H, F must be multiples of 128 (ERR_UNSUPPORTED).  ws: device scratch for the quantized
  * copies, mxfp8_linear_ws_bytes() bytes, 256-byte aligned, owned by the caller.  All tensors

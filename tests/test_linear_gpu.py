@@ -124,3 +124,38 @@ def test_linear_argument_errors():
     with pytest.raises(B.Mxfp8Error):        # unknown rule
         B.mxfp8_linear(z(T, H), z(F, H), z(T, F), 9, z(T, F), z(T, H), z(F, H), ws)
     assert B.mxfp8_linear_ws_bytes(0, 1, 1) == 0
+
+
+def test_linear_step_can_be_captured_in_a_cuda_graph():
+    # the device-pointer entry points only enqueue work on the caller's stream (no allocation, no synchronisation),
+    # so a step can be captured once and replayed: replay on new inputs must equal the eager call bit for bit
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    T, H, F = 512, 256, 384
+    xb, wb, dyb = inputs(T, H, F, 11)
+    x, w, dy = to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(dyb)
+    outs = [torch.empty(s, dtype=torch.bfloat16, device="cuda") for s in ((T, F), (T, H), (F, H))]
+    ws = torch.empty(B.mxfp8_linear_ws_bytes(T, H, F), dtype=torch.uint8, device="cuda")
+    B.mxfp8_linear(x, w, dy, B.RULE_PAPER, *outs, ws)                 # first use outside the capture (kernel attributes)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.mxfp8_linear(x, w, dy, B.RULE_PAPER, *outs, ws)
+    # new inputs into the captured buffers, replay, and compare with an eager call on copies
+    xb2, wb2, dyb2 = inputs(T, H, F, 12)
+    x.copy_(to_dev_bf16(xb2)); w.copy_(to_dev_bf16(wb2)); dy.copy_(to_dev_bf16(dyb2))
+    for o in outs:
+        o.zero_()
+    launches = B.mxfp8_launch_count()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert B.mxfp8_launch_count() == launches                          # nothing went through the host entry points
+    replayed = [o.clone() for o in outs]
+    eager = [torch.empty_like(o) for o in outs]
+    ws2 = torch.empty_like(ws)
+    B.mxfp8_linear(x, w, dy, B.RULE_PAPER, *eager, ws2)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for a, b in zip(replayed, eager):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        assert a.float().abs().sum() > 0
