@@ -70,3 +70,61 @@ def test_argument_validation_happens_on_the_host():
     assert g(p, p, p, p, 100, 128, 128, 1, 0, 0, 0, p, 0, None, None, 0, None) == -5   # MN-major A needs M % 16 == 0
     assert g(p, p, p, p, 128, 130, 128, 0, 0, 0, 0, p, 1, None, None, 0, None) == -5   # BF16 output needs N % 8 == 0
     assert "timeout" in B.status_string(-7) or "wait" in B.status_string(-7)
+
+
+def test_argument_validation_of_the_widened_entry_points():
+    L = B.lib()
+    p = ctypes.c_void_p(0x1000)          # never dereferenced: every call below fails validation first
+    odd = ctypes.c_void_p(0x1004)
+    # round trip
+    f = L.mxfp8_fake_quantize
+    assert f(None, B.BF16, 32, 32, B.ROW, 0, 0, p, None, None) == -1
+    assert f(p, B.BF16, 32, 32, B.ROW, 0, 9, p, None, None) == -2
+    assert f(p, B.BF16, 32, 48, B.ROW, 0, 0, p, None, None) == -3
+    assert f(p, B.BF16, 32, 32, B.COL, 0, 0, p, None, None) == -1            # column output missing
+    # activation / gated activation / normalisation ahead of the conversion
+    a = L.mxfp8_act_quantize
+    assert a(p, B.BF16, 32, 32, 9, B.ROW, 0, 0, p, p, None, None, 0, None) == -2
+    assert a(p, B.BF16, 32, 32, B.ACT_RELU, B.ROW, 0, 0, p, None, None, None, 0, None) == -1
+    assert a(odd, B.BF16, 32, 32, B.ACT_RELU, B.ROW, 0, 0, p, p, None, None, 0, None) == -4
+    g = L.mxfp8_glu_quantize
+    assert g(p, B.BF16, 32, 96, B.ACT_SILU, B.ROW, 0, 0, p, p, None, None, 0, None) == -5    # not whole 128-column tiles
+    assert g(p, B.FP32, 32, 96, B.ACT_SILU, B.ROW, 0, 0, p, p, None, None, 0, None) == -5    # not whole 64-column tiles
+    assert g(p, B.BF16, 32, 128, -1, B.ROW, 0, 0, p, p, None, None, 0, None) == -2
+    r = L.mxfp8_rmsnorm_quantize
+    assert r(p, B.BF16, 32, 32, None, 1e-5, p, B.ROW, 0, 0, p, p, None, None, 0, None) == -1
+    assert r(p, B.BF16, 32, 32, p, -1.0, p, B.ROW, 0, 0, p, p, None, None, 0, None) == -3
+    assert r(p, B.BF16, 32, 32, p, float("nan"), p, B.ROW, 0, 0, p, p, None, None, 0, None) == -3
+    rs = L.mxfp8_rmsnorm_quantize_static
+    assert rs(p, B.BF16, 65536 + 32, 32, p, 1e-5, B.ROW, 0, 0, p, p, None, None, 0, None) == -5
+    # batched conversion
+    items = (B._QuantizeItem * 9)()
+    qm = L.mxfp8_quantize_multi
+    assert qm(items, 9, B.BF16, B.ROW, 0, 0, 0, None) == -5
+    assert qm(items, 0, B.BF16, B.ROW, 0, 0, 0, None) == -3
+    assert qm(None, 1, B.BF16, B.ROW, 0, 0, 0, None) == -1
+    assert qm(items, 1, B.BF16, B.ROW, 0, 0, 0, None) == -1                   # null source in the first item
+    # several products in one launch
+    probs = (B._GemmProblem * 4)()
+    gm = L.mxfp8_gemm_multi
+    assert gm(probs, 4, B.BF16, None) == -5
+    assert gm(probs, 0, B.BF16, None) == -3
+    assert gm(None, 1, B.BF16, None) == -1
+    assert gm(probs, 1, 5, None) == -2
+    assert gm(probs, 1, B.BF16, None) == -1                                   # null operands in the first product
+    # per-expert products
+    gg = L.mxfp8_grouped_gemm
+    assert gg(p, p, p, p, None, 4, B.GROUP_M, 512, 128, 128, 0, 0, 0, p, 1, None) == -1
+    assert gg(p, p, p, p, p, 4, 3, 512, 128, 128, 0, 0, 0, p, 1, None) == -2
+    assert gg(p, p, p, p, p, 0, B.GROUP_M, 512, 128, 128, 0, 0, 0, p, 1, None) == -3
+    assert gg(p, p, p, p, p, 300, B.GROUP_M, 512, 128, 128, 0, 0, 0, p, 1, None) == -5
+    assert gg(p, p, p, p, p, 4, B.GROUP_M, 512, 96, 128, 0, 0, 0, p, 1, None) == -5
+    assert gg(p, p, p, p, p, 4, B.GROUP_K, 128, 128, 512, 0, 0, 0, p, 1, None) == -5    # GROUP_K needs token-major B
+    assert gg(p, p, p, p, ctypes.c_void_p(0x1002), 4, B.GROUP_M, 512, 128, 128, 0, 0, 0, p, 1, None) == -4   # offsets need 4-byte alignment
+    # linear-layer step
+    ln = L.mxfp8_linear
+    assert ln(p, p, p, 128, 128, 128, 0, p, p, p, None, 0, None) == -1
+    assert ln(p, p, p, 96, 128, 128, 0, p, p, p, p, 1 << 30, None) == -5
+    assert ln(p, p, p, 128, 128, 128, 7, p, p, p, p, 1 << 30, None) == -2
+    assert ln(p, p, p, 128, 128, 128, 0, p, p, p, ctypes.c_void_p(0x1100), 16, None) == -8
+    assert B.status_string(-9).startswith("invalid values")
