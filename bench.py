@@ -442,7 +442,7 @@ def run_case(args):
         for _ in range(reps):
             B.mxfp8_dequantize(q[0], q[1], B.ROW, E, S, dst)
     else:
-        m_, n_, k_ = (T, F, H) if args.case == "gemm" else (8192, 8192, 8192)
+        m_, n_, k_ = (8192, 8192, 8192) if args.case == "gemm8k" else (T, F, H)
         a = synth.device_tensor("activation", (m_, k_), 2)
         w = synth.device_tensor("weight", (n_, k_), 3)
         qa = B.alloc_quantize_outputs(m_, k_, B.ROW, S)
@@ -450,8 +450,12 @@ def run_case(args):
         B.mxfp8_quantize(a, B.ROW, P, E, *qa, S)
         B.mxfp8_quantize(w, B.ROW, P, E, *qw, S)
         y = torch.empty((m_, n_), dtype=torch.bfloat16, device="cuda")
+        epi = None
+        if args.case == "gemm_fused":        # the fprop product with the row + column MXFP8 output next to D
+            keep = B.alloc_quantize_outputs(m_, n_, B.BOTH, S)
+            epi = B.make_epilogue(B.BOTH, P, E, *keep)
         for _ in range(reps):
-            B.mxfp8_gemm(qa[0], qa[1], qw[0], qw[1], m_, n_, k_, B.K_MAJOR, B.K_MAJOR, E, E, y)
+            B.mxfp8_gemm(qa[0], qa[1], qw[0], qw[1], m_, n_, k_, B.K_MAJOR, B.K_MAJOR, E, E, y, epi=epi)
     torch.cuda.synchronize()
     print(json.dumps({"case": args.case, "launches": int(B.mxfp8_launch_count()), "device_status": B.mxfp8_device_status()}))
 
@@ -647,7 +651,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "step", "grouped", "glu"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu"],
                     help="run one kernel on one small case and exit (for profiler captures)")
     ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
