@@ -521,3 +521,29 @@ def test_fused_output_at_decoder_block_sizes_equals_quantize_of_unfused_output(c
     for name, u, v in zip(("q_row", "s_row", "q_col", "s_col"), fused, ref):
         assert torch.equal(u, v), name
     assert torch.equal(d16, d32.to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("tile", ["256p", "192p", "256", "192", "128"])
+@pytest.mark.parametrize("majors", [("k", "k"), ("mn", "mn")])
+def test_every_tile_shape_against_the_oracle(tile, majors):
+    # the tile shape is normally chosen by a cost model; here each of the five kernel shapes is forced in turn on a
+    # product with ragged M, N and K tails (several tiles in both directions, two K blocks plus a tail)
+    import os
+    m, n, k = 656, 720, 352
+    a = synth.gaussian((m, k), 61)
+    b = synth.student_t((n, k), 62) * np.float32(0.1)
+    def prep(x, major):
+        stored_x = np.ascontiguousarray(x.T) if major == "mn" else x
+        return orc.quantize(stored_x, orc.COL if major == "mn" else orc.ROW)
+    aq, a_s = prep(a, majors[0])
+    bq, b_s = prep(b, majors[1])
+    d64, sabs = orc.gemm_f64(aq, a_s, bq, b_s, majors[0], majors[1])
+    old = os.environ.pop("MXFP8_GEMM_TILE", None)
+    os.environ["MXFP8_GEMM_TILE"] = tile
+    try:
+        got = gpu_gemm(aq, a_s, bq, b_s, majors[0], majors[1])
+    finally:
+        os.environ.pop("MXFP8_GEMM_TILE", None)
+        if old is not None:
+            os.environ["MXFP8_GEMM_TILE"] = old
+    check_gemm_tolerance(got, d64, sabs, "tile %s %s" % (tile, majors))
