@@ -193,3 +193,19 @@ def test_argument_errors():
     big = torch.zeros(300, dtype=torch.int32, device="cuda")
     with pytest.raises(B.Mxfp8Error):      # more than 256 experts
         B.mxfp8_grouped_gemm(z(128, 128), sc, z(128, 128), sc, big, B.GROUP_M, 128, 128, 128, B.K_MAJOR, B.E4M3, B.E4M3, D)
+
+
+def test_no_tokens_at_all():
+    # every expert empty: the token-grouped product stores nothing, the reduction-grouped one stores zeros
+    T, K, N = 256, 128, 128
+    offsets = [128, 128, 128, 128]
+    G = 3
+    one = lambda r, c: np.full((r, c), 127, np.uint8)
+    aq = np.full((T, K), 0x38, np.uint8)
+    bq = np.full((G * N, K), 0x38, np.uint8)
+    d, status = run_grouped(aq, one(T, K // 32), bq, one(G * N, K // 32), offsets, "m", T, N, K, "k", T)
+    assert status == 0 and np.isnan(d).all()
+    M = 128
+    d, status = run_grouped(np.full((T, M), 0x38, np.uint8), one(M, T // 32), np.full((T, N), 0x38, np.uint8), one(N, T // 32),
+                            offsets, "k", M, N, T, "mn", G * M)
+    assert status == 0 and not d.any() and not np.isnan(d).any()
