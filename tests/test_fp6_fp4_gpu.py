@@ -165,3 +165,40 @@ def test_gemm_rejects_unknown_element_codes_and_sub_byte_fused_output():
     with pytest.raises(B.Mxfp8Error) as e:
         B.mxfp8_gemm(z, sc, z, sc, 128, 128, 128, B.K_MAJOR, B.K_MAJOR, B.E4M3, B.E4M3, D, epi=epi)
     assert e.value.status == -5
+
+
+@pytest.mark.parametrize("elem", ELEMS)
+def test_batched_and_fused_conversions_take_the_small_formats(elem):
+    # the batched launch, the activation prologue and the gated prologue with 6- / 4-bit elements: same results as the
+    # plain conversion of the corresponding tensor (which the tests above check against the oracle)
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    S = B.SF_SWIZZLED
+    xs = [synth.device_tensor("gaussian", shp, 70 + i) for i, shp in enumerate(((256, 512), (160, 352)))]
+    single = [B.alloc_quantize_outputs(t.shape[0], t.shape[1], B.BOTH, S) for t in xs]
+    multi = [B.alloc_quantize_outputs(t.shape[0], t.shape[1], B.BOTH, S) for t in xs]
+    for t, o in zip(xs, single):
+        B.mxfp8_quantize(t, B.BOTH, B.RULE_PAPER, elem, *o, S)
+    B.mxfp8_quantize_multi(B.make_quantize_items([(t,) + o for t, o in zip(xs, multi)]), B.BF16, B.BOTH, B.RULE_PAPER, elem, S)
+    torch.cuda.synchronize()
+    for a, b in zip(single, multi):
+        for u, v in zip(a, b):
+            assert torch.equal(u, v)
+    # relu ahead of the conversion == conversion of relu(x)
+    x = xs[0]
+    want = B.alloc_quantize_outputs(256, 512, B.BOTH, S)
+    got = B.alloc_quantize_outputs(256, 512, B.BOTH, S)
+    B.mxfp8_quantize(torch.relu(x).contiguous(), B.BOTH, B.RULE_PAPER, elem, *want, S)
+    B.mxfp8_act_quantize(x, B.ACT_RELU, B.BOTH, B.RULE_PAPER, elem, *got, S)
+    # relu(gate) * up == conversion of the BF16 product (FP32 product rounded once, as torch does for BF16 operands)
+    g2 = synth.device_tensor("gaussian", (256, 2 * 512), 75)
+    y = (torch.relu(g2[:, :512].float()) * g2[:, 512:].float()).to(torch.bfloat16).contiguous()
+    want2 = B.alloc_quantize_outputs(256, 512, B.BOTH, S)
+    got2 = B.alloc_quantize_outputs(256, 512, B.BOTH, S)
+    B.mxfp8_quantize(y, B.BOTH, B.RULE_PAPER, elem, *want2, S)
+    B.mxfp8_glu_quantize(g2, B.ACT_RELU, B.BOTH, B.RULE_PAPER, elem, *got2, S)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for a, b in ((want, got), (want2, got2)):
+        for u, v in zip(a, b):
+            assert torch.equal(u, v)
