@@ -373,9 +373,11 @@ int mxfp8_linear(const void* x, const void* w, const void* dy,
  *     WGRAD  dW [F, H] = dY^T * X   (column-blocked dY, column-blocked X)
  *   run as block-scaled GEMMs with BF16 output, and Y, dX, dW are copied back to the host.
  * T, H, F must be multiples of 128.  dev_ws: device scratch of mxfp8_linear_host_ws_bytes(),
- * 256-byte aligned.  Waits for `stream` before returning.  The upload of dY overlaps FPROP and the
- * download of Y (two helper streams per device, created on first use, ordered after the work already
- * in `stream`); launches: cast(X, W), FPROP, cast(dY), DGRAD + WGRAD.  (The composition is the paper's
+ * 256-byte aligned.  Waits for `stream` before returning.  The token axis goes through in four row
+ * chunks when T is a multiple of 512, so that uploads, products and downloads overlap (two helper
+ * streams per device, created on first use, ordered after the work already in `stream`): FPROP and
+ * DGRAD run per chunk, the column-blocked copies and WGRAD once everything is there; same results as
+ * mxfp8_linear, bit for bit.  (The composition is the paper's
  * workflow; the host-buffer packaging has no counterpart in the paper.)
  */
 size_t mxfp8_linear_host_ws_bytes(int64_t T, int64_t H, int64_t F);

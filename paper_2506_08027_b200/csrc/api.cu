@@ -190,9 +190,12 @@ namespace {
 // Two helper streams and the events that tie them to the caller's stream, one set per device, made on
 // first use and kept for the life of the process: the host variant overlaps the upload of dY with the
 // download of Y (PCIe carries both directions at once).
+constexpr int HOST_CHUNKS = 4;   // row chunks of the token axis in the host-buffer step
+
 struct HostPipe {
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, xw_in = nullptr, dy_in = nullptr, y_ready = nullptr, y_out = nullptr;
+    cudaEvent_t start = nullptr, w_in = nullptr, out_done = nullptr, dw_ready = nullptr;
+    cudaEvent_t x_in[HOST_CHUNKS] = {}, dy_in[HOST_CHUNKS] = {}, y_ready[HOST_CHUNKS] = {}, dx_ready[HOST_CHUNKS] = {};
     bool ok = false;
     std::mutex busy;   // one host-buffer step at a time per device: the events above are shared
 };
@@ -208,8 +211,9 @@ HostPipe* host_pipe()
     if (!p.ok) {
         bool good = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess;
-        cudaEvent_t* evs[5] = {&p.start, &p.xw_in, &p.dy_in, &p.y_ready, &p.y_out};
-        for (cudaEvent_t* e : evs) good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+        auto make = [&](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+        make(&p.start); make(&p.w_in); make(&p.out_done); make(&p.dw_ready);
+        for (int c = 0; c < HOST_CHUNKS; ++c) { make(&p.x_in[c]); make(&p.dy_in[c]); make(&p.y_ready[c]); make(&p.dx_ready[c]); }
         if (!good) return nullptr;
         p.ok = true;
     }
@@ -232,43 +236,75 @@ extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const v
     std::lock_guard<std::mutex> one_at_a_time(hp->busy);
     const LinearWs w = plan_linear(static_cast<char*>(dev_ws), T, H, F, true);
     enum { X = 0, W = 1, DY = 2, R = 0, C = 1 };
-    const size_t xb = (size_t)T * H * 2, wb = (size_t)F * H * 2, yb = (size_t)T * F * 2;
+    // The token axis goes through in row chunks (whole 128-row scale atoms each), so that PCIe carries both directions
+    // for most of the call: FPROP of a chunk starts when its rows of X have arrived and its rows of Y leave at once,
+    // while dY is still coming in; DGRAD likewise per chunk of dY.  Row-blocked copies are made per chunk, the
+    // column-blocked ones (blocks run down the token axis) once per tensor when all of it is there.  Every product
+    // is the same tile arithmetic as in mxfp8_linear, so the results are bit-identical.
+    const int chunks = (T % (128 * HOST_CHUNKS) == 0) ? HOST_CHUNKS : 1;
+    const int64_t Tc = T / chunks;
+    const int64_t s_row_chunk_x = (Tc / 128) * ((H / 32 + 3) / 4) * 512;    // bytes of swizzled row scales per chunk of X
+    const int64_t s_row_chunk_dy = (Tc / 128) * ((F / 32 + 3) / 4) * 512;   // ... and of dY
+    const size_t wb = (size_t)F * H * 2;
 #define MXFP8_TRY(call) do { if ((call) != cudaSuccess) return MXFP8_ERR_CUDA; } while (0)
 #define MXFP8_RC(call) do { const int rc_ = (call); if (rc_ != MXFP8_OK) return rc_; } while (0)
-    // uploads on the helper stream, behind whatever the caller's stream holds: X and W first, dY behind them
+    // uploads on the helper stream, behind whatever the caller's stream holds: W, then X and dY chunk by chunk
     MXFP8_TRY(cudaEventRecord(hp->start, st));
     MXFP8_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+    MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->start, 0));
     MXFP8_TRY(cudaMemcpyAsync(w.src[W], w_host, wb, cudaMemcpyHostToDevice, hp->in));
-    MXFP8_TRY(cudaMemcpyAsync(w.src[X], x_host, xb, cudaMemcpyHostToDevice, hp->in));
-    MXFP8_TRY(cudaEventRecord(hp->xw_in, hp->in));
-    MXFP8_TRY(cudaMemcpyAsync(w.src[DY], dy_host, yb, cudaMemcpyHostToDevice, hp->in));
-    MXFP8_TRY(cudaEventRecord(hp->dy_in, hp->in));
-    // FPROP as soon as X and W are on the device
-    MXFP8_TRY(cudaStreamWaitEvent(st, hp->xw_in, 0));
-    const mxfp8_quantize_item xw[2] = {
-        {w.src[X], T, H, w.q[X][R], w.s[X][R], w.q[X][C], w.s[X][C]},
-        {w.src[W], F, H, w.q[W][R], w.s[W][R], w.q[W][C], w.s[W][C]},
-    };
-    MXFP8_RC(mxfp8_quantize_multi(xw, 2, MXFP8_BF16, MXFP8_BOTH, scale_rule, MXFP8_E4M3, MXFP8_SF_SWIZZLED, stream));
-    MXFP8_RC(mxfp8_gemm(w.q[X][R], w.s[X][R], w.q[W][R], w.s[W][R], T, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR, MXFP8_E4M3,
-                        MXFP8_E4M3, w.out[0], MXFP8_BF16, nullptr, nullptr, 0, stream));
-    MXFP8_TRY(cudaEventRecord(hp->y_ready, st));
-    // Y goes back on the second helper stream while dY is still coming in
-    MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->y_ready, 0));
-    MXFP8_TRY(cudaMemcpyAsync(y_host, w.out[0], yb, cudaMemcpyDeviceToHost, hp->out));
-    MXFP8_TRY(cudaEventRecord(hp->y_out, hp->out));
-    // DGRAD and WGRAD once dY has arrived
-    MXFP8_TRY(cudaStreamWaitEvent(st, hp->dy_in, 0));
-    MXFP8_RC(mxfp8_quantize(w.src[DY], MXFP8_BF16, T, F, MXFP8_BOTH, scale_rule, MXFP8_E4M3, w.q[DY][R], w.s[DY][R], w.q[DY][C],
-                            w.s[DY][C], MXFP8_SF_SWIZZLED, stream));
-    const mxfp8_gemm_problem grads[2] = {
-        {w.q[DY][R], w.s[DY][R], w.q[W][C], w.s[W][C], T, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, w.out[1]},
-        {w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3, w.out[2]},
-    };
-    MXFP8_RC(mxfp8_gemm_multi(grads, 2, MXFP8_BF16, stream));
-    MXFP8_TRY(cudaMemcpyAsync(dx_host, w.out[1], xb, cudaMemcpyDeviceToHost, st));
-    MXFP8_TRY(cudaMemcpyAsync(dw_host, w.out[2], wb, cudaMemcpyDeviceToHost, st));
-    MXFP8_TRY(cudaStreamWaitEvent(st, hp->y_out, 0));
+    MXFP8_TRY(cudaEventRecord(hp->w_in, hp->in));
+    for (int c = 0; c < chunks; ++c) {
+        const size_t off = (size_t)c * Tc * H * 2;
+        MXFP8_TRY(cudaMemcpyAsync(w.src[X] + off, static_cast<const char*>(x_host) + off, (size_t)Tc * H * 2, cudaMemcpyHostToDevice, hp->in));
+        MXFP8_TRY(cudaEventRecord(hp->x_in[c], hp->in));
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const size_t off = (size_t)c * Tc * F * 2;
+        MXFP8_TRY(cudaMemcpyAsync(w.src[DY] + off, static_cast<const char*>(dy_host) + off, (size_t)Tc * F * 2, cudaMemcpyHostToDevice, hp->in));
+        MXFP8_TRY(cudaEventRecord(hp->dy_in[c], hp->in));
+    }
+    // W: both orientations as soon as it is there
+    MXFP8_TRY(cudaStreamWaitEvent(st, hp->w_in, 0));
+    MXFP8_RC(mxfp8_quantize(w.src[W], MXFP8_BF16, F, H, MXFP8_BOTH, scale_rule, MXFP8_E4M3, w.q[W][R], w.s[W][R], w.q[W][C], w.s[W][C],
+                            MXFP8_SF_SWIZZLED, stream));
+    // FPROP chunk by chunk; Y rows leave on the second helper stream
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t r0 = (int64_t)c * Tc;
+        MXFP8_TRY(cudaStreamWaitEvent(st, hp->x_in[c], 0));
+        MXFP8_RC(mxfp8_quantize(w.src[X] + r0 * H * 2, MXFP8_BF16, Tc, H, MXFP8_ROW, scale_rule, MXFP8_E4M3, w.q[X][R] + r0 * H,
+                                w.s[X][R] + c * s_row_chunk_x, nullptr, nullptr, MXFP8_SF_SWIZZLED, stream));
+        MXFP8_RC(mxfp8_gemm(w.q[X][R] + r0 * H, w.s[X][R] + c * s_row_chunk_x, w.q[W][R], w.s[W][R], Tc, F, H, MXFP8_K_MAJOR, MXFP8_K_MAJOR,
+                            MXFP8_E4M3, MXFP8_E4M3, w.out[0] + r0 * F * 2, MXFP8_BF16, nullptr, nullptr, 0, stream));
+        MXFP8_TRY(cudaEventRecord(hp->y_ready[c], st));
+        MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->y_ready[c], 0));
+        MXFP8_TRY(cudaMemcpyAsync(static_cast<char*>(y_host) + r0 * F * 2, w.out[0] + r0 * F * 2, (size_t)Tc * F * 2, cudaMemcpyDeviceToHost, hp->out));
+    }
+    // the column-blocked copy of X (for WGRAD) once all of X is there
+    MXFP8_RC(mxfp8_quantize(w.src[X], MXFP8_BF16, T, H, MXFP8_COL, scale_rule, MXFP8_E4M3, nullptr, nullptr, w.q[X][C], w.s[X][C],
+                            MXFP8_SF_SWIZZLED, stream));
+    // DGRAD chunk by chunk as dY arrives
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t r0 = (int64_t)c * Tc;
+        MXFP8_TRY(cudaStreamWaitEvent(st, hp->dy_in[c], 0));
+        MXFP8_RC(mxfp8_quantize(w.src[DY] + r0 * F * 2, MXFP8_BF16, Tc, F, MXFP8_ROW, scale_rule, MXFP8_E4M3, w.q[DY][R] + r0 * F,
+                                w.s[DY][R] + c * s_row_chunk_dy, nullptr, nullptr, MXFP8_SF_SWIZZLED, stream));
+        MXFP8_RC(mxfp8_gemm(w.q[DY][R] + r0 * F, w.s[DY][R] + c * s_row_chunk_dy, w.q[W][C], w.s[W][C], Tc, H, F, MXFP8_K_MAJOR, MXFP8_MN_MAJOR,
+                            MXFP8_E4M3, MXFP8_E4M3, w.out[1] + r0 * H * 2, MXFP8_BF16, nullptr, nullptr, 0, stream));
+        MXFP8_TRY(cudaEventRecord(hp->dx_ready[c], st));
+        MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->dx_ready[c], 0));
+        MXFP8_TRY(cudaMemcpyAsync(static_cast<char*>(dx_host) + r0 * H * 2, w.out[1] + r0 * H * 2, (size_t)Tc * H * 2, cudaMemcpyDeviceToHost, hp->out));
+    }
+    // WGRAD needs every token: column-blocked dY, then the product, then dW leaves
+    MXFP8_RC(mxfp8_quantize(w.src[DY], MXFP8_BF16, T, F, MXFP8_COL, scale_rule, MXFP8_E4M3, nullptr, nullptr, w.q[DY][C], w.s[DY][C],
+                            MXFP8_SF_SWIZZLED, stream));
+    MXFP8_RC(mxfp8_gemm(w.q[DY][C], w.s[DY][C], w.q[X][C], w.s[X][C], F, H, T, MXFP8_MN_MAJOR, MXFP8_MN_MAJOR, MXFP8_E4M3, MXFP8_E4M3,
+                        w.out[2], MXFP8_BF16, nullptr, nullptr, 0, stream));
+    MXFP8_TRY(cudaEventRecord(hp->dw_ready, st));
+    MXFP8_TRY(cudaStreamWaitEvent(hp->out, hp->dw_ready, 0));
+    MXFP8_TRY(cudaMemcpyAsync(dw_host, w.out[2], wb, cudaMemcpyDeviceToHost, hp->out));
+    MXFP8_TRY(cudaEventRecord(hp->out_done, hp->out));
+    MXFP8_TRY(cudaStreamWaitEvent(st, hp->out_done, 0));
     MXFP8_TRY(cudaStreamSynchronize(st));
 #undef MXFP8_TRY
 #undef MXFP8_RC
