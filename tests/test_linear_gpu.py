@@ -68,10 +68,12 @@ def test_linear_device_matches_oracle_chain(shape, rule):
         check_bf16_result(from_dev_bf16(got), d64, sabs, name)
 
 
-def test_linear_host_equals_device_variant():
+@pytest.mark.parametrize("shape", [(256, 256, 384), (512, 128, 128), (1024, 384, 640), (2048, 512, 1152)])
+def test_linear_host_equals_device_variant(shape):
+    """T = 256 goes through in one piece; multiples of 512 tokens go through in four row chunks whose copies overlap."""
     import torch
     from paper_2506_08027_b200 import binding as B
-    T, H, F = 256, 256, 384
+    T, H, F = shape
     xb, wb, dyb = inputs(T, H, F, 77)
     x, w, dy = to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(dyb)
     outs = [torch.empty(s, dtype=torch.bfloat16, device="cuda") for s in ((T, F), (T, H), (F, H))]
