@@ -256,6 +256,50 @@ def grouped_gemm_f64(aq, a_s, bq, b_s, offsets, mode: str = "m", b_major: str = 
     return d, sabs
 
 
+def concat_swizzled_scales_k(parts, mn: int, nkb_part: int) -> np.ndarray:
+    """Swizzled scales of logical [mn, len(parts) * nkb_part] from the swizzled arrays of its parts, each logical
+    [mn, nkb_part]: byte by byte through the layout's offset formula."""
+    nkb = len(parts) * nkb_part
+    out = np.zeros(((mn + 127) // 128) * ((nkb + 3) // 4) * 512, dtype=np.uint8)
+    for r, part in enumerate(parts):
+        for m in range(mn):
+            for kb in range(nkb_part):
+                out[sf_offset_swizzled(m, r * nkb_part + kb, nkb)] = part[sf_offset_swizzled(m, kb, nkb_part)]
+    return out
+
+
+def data_parallel_linear_f64(xs, w_shards, dys, rule: int = RULE_PAPER, elem: int = E4M3):
+    """One linear-layer step (Sec. 3.2: FPROP, DGRAD and WGRAD on MXFP8 copies blocked along each product's
+    reduction axis) when rank r holds tokens xs[r] [T_r, H] with output gradients dys[r] [T_r, F] and owns
+    rows w_shards[r] [F_r, H] of the weight.  The paper states the single-device arithmetic only; sharded, it
+    reads: every rank converts its own tensors (blocks never cross a shard: T_r and F_r are multiples of 32);
+    the weight operand of every rank is the shards' conversions one under another; Y_r and dX_r use the rank's
+    own tokens; dW sums the ranks' partial products over their tokens and rank r keeps its rows.
+
+    Returns (ys, dxs, dw_shards, sabs) as lists per rank of float64 arrays; sabs = matching lists of |a*b| sums
+    (for dW the sum over ranks)."""
+    R, C = ROW, COL
+    wq = {o: [quantize(w, o, rule, elem) for w in w_shards] for o in (R, C)}
+    w_row = (np.concatenate([q for q, _ in wq[R]]), np.concatenate([sc for _, sc in wq[R]]))     # [F, H], [F, H/32]
+    w_col = (np.concatenate([q for q, _ in wq[C]]), np.concatenate([sc for _, sc in wq[C]]))     # [F, H], [F/32, H]
+    ys, dxs, s_y, s_dx = [], [], [], []
+    dw = None
+    s_dw = None
+    for x, dy in zip(xs, dys):
+        xq = {o: quantize(x, o, rule, elem) for o in (R, C)}
+        dyq = {o: quantize(dy, o, rule, elem) for o in (R, C)}
+        y, sy = gemm_f64(xq[R][0], xq[R][1], w_row[0], w_row[1], "k", "k", elem, elem)
+        dx, sdx = gemm_f64(dyq[R][0], dyq[R][1], w_col[0], w_col[1], "k", "mn", elem, elem)
+        part, spart = gemm_f64(dyq[C][0], dyq[C][1], xq[C][0], xq[C][1], "mn", "mn", elem, elem)
+        ys.append(y); dxs.append(dx); s_y.append(sy); s_dx.append(sdx)
+        dw = part if dw is None else dw + part
+        s_dw = spart if s_dw is None else s_dw + spart
+    bounds = np.cumsum([0] + [w.shape[0] for w in w_shards])
+    dw_shards = [dw[bounds[r]:bounds[r + 1]] for r in range(len(w_shards))]
+    s_dw_shards = [s_dw[bounds[r]:bounds[r + 1]] for r in range(len(w_shards))]
+    return ys, dxs, dw_shards, (s_y, s_dx, s_dw_shards)
+
+
 def code_bits(elem: int) -> int:
     return {E4M3: 8, E5M2: 8, E2M3: 6, E3M2: 6, E2M1: 4}[elem]
 
