@@ -316,6 +316,41 @@ int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq, const voi
                        int64_t M, int64_t N, int64_t K, int b_major, int a_elem, int b_elem,
                        void* D, int out_dtype, void* stream);
 
+/*
+ * Data-parallel exchange.  The recipe casts weights, activations and output gradients (Sec. 3.2); when
+ * the tokens of a step are split over GPUs and every GPU owns a row range of each weight, two exchanges
+ * follow from that arithmetic: the MXFP8 copies of the weight shards are gathered (1 + 1/32 bytes per
+ * element and orientation instead of 2 for BF16), and the WGRAD partial results, one per GPU over its
+ * own tokens, are summed and scattered to the owners of the rows.  (The paper states no multi-GPU
+ * algorithm; these two calls are what its per-tensor arithmetic needs when the tensors are sharded.)
+ *
+ * mxfp8_sf_concat_k -- joins swizzled scale arrays along the block axis.  `parts` holds `num_parts`
+ * swizzled arrays one after another, each for logical [mn, k_part/32] scales (k_part a multiple of 128,
+ * so every part is whole 512-byte atoms); `dst` receives the swizzled array for logical
+ * [mn, num_parts * k_part/32], part r supplying blocks r*k_part/32 .. .  This is what the column-blocked
+ * scales of row-sharded weights need after an all-gather (blocks run down the sharded axis); the element
+ * bytes of both orientations and the row-blocked scales of row shards are already in place when
+ * each shard is written at its row offset.  Device pointers, 16-byte aligned; one launch; a pure permutation of bytes.
+ *
+ * mxfp8_gemm_reduce_scatter -- D_owner[r][m - r*M/num_owners, n] += sum_k A[m,k] * B[n,k] for every m:
+ * the block-scaled product of mxfp8_gemm (operands as there) whose FP32 result is ADDED, tile by tile
+ * while the product runs, into one FP32 buffer [M/num_owners, N] per owner of a row range.  `D_owner`
+ * is a HOST array of `num_owners` (1..8) device pointers; a pointer may be another GPU's memory mapped
+ * into this process (peer access or an IPC mapping): the additions then cross NVLink as they are produced.
+ * `first_owner` (0 .. num_owners-1) is the owner whose tiles this launch produces first; giving each
+ * rank its own index spreads the traffic over the owners.  The caller zeroes the buffers, makes sure every rank has done so before any
+ * rank launches, and waits for all ranks' launches before reading its own buffer; the order in
+ * which different launches' contributions are added is not fixed (two contributions: exact and order-free;
+ * more: equal up to FP32 rounding order).  M a multiple of 128 * num_owners, N of 4 (16 with an MN-major B), K of 32.
+ * Nothing is allocated; never waits on another GPU inside the kernel.
+ */
+int mxfp8_sf_concat_k(const void* parts, int num_parts, int64_t mn, int64_t k_part, void* dst, void* stream);
+#define MXFP8_REDUCE_SCATTER_MAX_OWNERS 8
+int mxfp8_gemm_reduce_scatter(const void* Aq, const void* As, const void* Bq, const void* Bs,
+                              int64_t M, int64_t N, int64_t K,
+                              int a_major, int b_major, int a_elem, int b_elem,
+                              void* const* D_owner, int num_owners, int first_owner, void* stream);
+
 /* Scratch bytes mxfp8_gemm needs for this problem (0 when none). */
 size_t mxfp8_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int out_dtype, int has_epilogue);
 

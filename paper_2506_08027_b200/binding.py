@@ -20,7 +20,8 @@ E4M3, E5M2 = 0, 1
 E2M3, E3M2, E2M1 = 3, 4, 5          # MXFP6 / MXFP4 elements: conversion kernels only
 SF_LINEAR, SF_SWIZZLED = 0, 1
 K_MAJOR, MN_MAJOR = 0, 1
-ERR_DEVICE_TIMEOUT, ERR_DEVICE_ARGS = -7, -9
+ERR_NULL, ERR_ENUM, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA = -1, -2, -3, -4, -5, -6
+ERR_DEVICE_TIMEOUT, ERR_WORKSPACE, ERR_DEVICE_ARGS = -7, -8, -9
 ACT_NONE, ACT_RELU, ACT_RELU2, ACT_SILU, ACT_GELU_TANH = 0, 1, 2, 3, 4
 
 EXPORTS = (
@@ -30,6 +31,7 @@ EXPORTS = (
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
     "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
+    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter",
 )
 
 
@@ -112,6 +114,10 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
         L.mxfp8_grouped_gemm.restype = i
         L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
+        L.mxfp8_sf_concat_k.restype = i
+        L.mxfp8_sf_concat_k.argtypes = [p, i, i64, i64, p, p]
+        L.mxfp8_gemm_reduce_scatter.restype = i
+        L.mxfp8_gemm_reduce_scatter.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, ctypes.POINTER(ctypes.c_void_p), i, i, p]
         L.mxfp8_linear_ws_bytes.restype = sz
         L.mxfp8_linear_ws_bytes.argtypes = [i64, i64, i64]
         L.mxfp8_linear.restype = i
@@ -279,6 +285,25 @@ def mxfp8_grouped_gemm(aq, a_s, bq, b_s, group_offsets: torch.Tensor, mode: int,
     _check(lib().mxfp8_grouped_gemm(_ptr(aq), _ptr(a_s), _ptr(bq), _ptr(b_s), _ptr(group_offsets),
                                     group_offsets.numel() - 1, mode, M, N, K, b_major, a_elem, b_elem,
                                     _ptr(D), _dtype_code(D), _stream(stream)), "mxfp8_grouped_gemm")
+
+
+def mxfp8_sf_concat_k(parts: torch.Tensor, num_parts: int, mn: int, k_part: int, dst: torch.Tensor, stream=None) -> None:
+    _check(lib().mxfp8_sf_concat_k(_ptr(parts), num_parts, mn, k_part, _ptr(dst), _stream(stream)), "mxfp8_sf_concat_k")
+
+
+def make_owner_pointers(addresses):
+    """addresses: one device address per owner (int, or a tensor whose data_ptr() is taken).  Returns the
+    host pointer array mxfp8_gemm_reduce_scatter takes; build it once per set of buffers."""
+    arr = (ctypes.c_void_p * len(addresses))()
+    for k, a in enumerate(addresses):
+        arr[k] = a.data_ptr() if isinstance(a, torch.Tensor) else int(a)
+    return arr
+
+
+def mxfp8_gemm_reduce_scatter(aq, a_s, bq, b_s, M: int, N: int, K: int, a_major: int, b_major: int, a_elem: int, b_elem: int,
+                              owners, first_owner: int, stream=None) -> None:
+    _check(lib().mxfp8_gemm_reduce_scatter(_ptr(aq), _ptr(a_s), _ptr(bq), _ptr(b_s), M, N, K, a_major, b_major, a_elem, b_elem,
+                                           owners, len(owners), first_owner, _stream(stream)), "mxfp8_gemm_reduce_scatter")
 
 
 def make_quantize_items(entries):

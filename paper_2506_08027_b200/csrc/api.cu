@@ -48,6 +48,35 @@ extern "C" int mxfp8_device_status(void* stream)
 }
 
 namespace {
+// One 16-byte piece per thread: atom (i, j) of part r goes to atom (i, r * atoms_part + j) of the whole.
+__global__ void __launch_bounds__(256)
+sf_concat_k_kernel(const uint4* __restrict__ parts, uint4* __restrict__ dst, int64_t atom_rows, int64_t atoms_part, int num_parts)
+{
+    const int64_t pieces = atom_rows * atoms_part * num_parts * 32;   // 32 pieces of 16 bytes per 512-byte atom
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < pieces; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t atom = t >> 5, piece = t & 31;
+        const int64_t j = atom % atoms_part, ri = atom / atoms_part;   // destination order: (i, r, j)
+        const int64_t r = ri % num_parts, i = ri / num_parts;
+        dst[t] = parts[(((r * atom_rows + i) * atoms_part + j) << 5) + piece];
+    }
+}
+}  // namespace
+
+extern "C" int mxfp8_sf_concat_k(const void* parts, int num_parts, int64_t mn, int64_t k_part, void* dst, void* stream)
+{
+    if (!parts || !dst) return MXFP8_ERR_NULL;
+    if (num_parts < 1 || mn <= 0 || k_part <= 0 || (k_part % 128)) return MXFP8_ERR_SHAPE;
+    if (!mxfp8::aligned16(parts) || !mxfp8::aligned16(dst)) return MXFP8_ERR_ALIGN;
+    const int64_t atom_rows = (mn + 127) / 128, atoms_part = k_part / 128;
+    const int64_t pieces = atom_rows * atoms_part * num_parts * 32;
+    const int64_t blocks = (pieces + 255) / 256;
+    sf_concat_k_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(parts), static_cast<uint4*>(dst), atom_rows, atoms_part, num_parts);
+    mxfp8::count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}
+
+namespace {
 inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 }
 

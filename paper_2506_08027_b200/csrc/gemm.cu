@@ -94,6 +94,8 @@ struct GemmParams {
     int token_limit;      // offsets may not pass this (tokens in the grouped tensor)
     int num_problems;     // MULTI
     MultiProblem mp[MAX_PROBLEMS];
+    int rows_per_owner;   // SCATTER: D rows [r * rows_per_owner, (r + 1) * rows_per_owner) are added into owner r's buffer
+    int tm_rot;           // SCATTER: M-tile this launch starts with (ranks start at different owners)
 };
 
 constexpr int MAX_GROUPS = 256;
@@ -101,7 +103,12 @@ constexpr int MAX_GROUPS = 256;
 //   GROUP_M: the rows of A (tokens) are grouped, B holds one matrix per expert   (fprop, dgrad)
 //   GROUP_K: the reduction axis (tokens) is grouped, D holds one matrix per expert (wgrad)
 //   MULTI  : up to MAX_PROBLEMS independent dense products, tiles of all of them dealt out as one pool
-enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2, MULTI = 3 };
+//   SCATTER: one dense product whose FP32 result is ADDED (TMA reduce) into per-owner buffers, row range by row
+//            range; the buffers may be other GPUs' memory, so that the data-parallel sum of WGRAD partial
+//            results and its scatter to the owners of the weight shards happen tile by tile inside the product
+enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2, MULTI = 3, SCATTER = 4 };
+constexpr int MAX_OWNERS = 8;   // the owners' output maps take the place of MultiMaps (15 maps)
+static_assert(sizeof(MultiMaps) >= MAX_OWNERS * sizeof(CUtensorMap), "owner maps must fit where the MULTI maps go");
 
 // BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
 // tile has 2*BM rows.  BN = 256 leaves room for one accumulator only (2 x 256 columns would fill
@@ -504,8 +511,9 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmParams& p, const int* g
         tile_coords(p.group_m, q.tiles_m, q.tiles_n, tile - q.tile_start, t.tm, t.tn);
         t.row0 = 0; t.d_row_extra = 0; t.rows_end = q.M; t.ka0 = 0; t.kb0 = 0; t.bn_off = 0; t.sfb_atom_off = 0;
         t.nkb = q.num_kb; t.prob = g;
-    } else if constexpr (MODE == DENSE) {
+    } else if constexpr (MODE == DENSE || MODE == SCATTER) {
         tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile, t.tm, t.tn);
+        if constexpr (MODE == SCATTER) { t.tm += p.tm_rot; if (t.tm >= p.tiles_m) t.tm -= p.tiles_m; }
         t.row0 = 0; t.d_row_extra = 0; t.rows_end = (int)p.M; t.ka0 = 0; t.kb0 = 0; t.bn_off = 0; t.sfb_atom_off = 0;
         t.nkb = p.num_kb;
     } else if constexpr (MODE == GROUP_M) {
@@ -648,7 +656,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // tiles of the whole launch (none when the offsets were rejected)
-    const int num_tiles = (MODE == DENSE || MODE == MULTI) ? p.num_tiles
+    const int num_tiles = (MODE == DENSE || MODE == MULTI || MODE == SCATTER) ? p.num_tiles
                         : (*bad_groups ? 0 : (MODE == GROUP_M ? tstart[p.num_groups] : p.num_groups * p.tiles_m * p.tiles_n));
 
     if (warp == 0) {
@@ -848,13 +856,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 }
             }
 
-            const int row0 = t.row0 + t.d_row_extra + (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
+            int row0 = t.row0 + t.d_row_extra + (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
             const bool rows_inside = row0 < t.rows_end;      // ragged last M tile / rows of the next expert: a 32-row box entirely outside stores nothing
             if constexpr (EPI && CW % 64 == 0) {
                 if (p.epi_orient && rows_inside) {
                     if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
                     else epi_mx<CW, MXFP8_E5M2>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
+                }
+            }
+            if constexpr (MODE == SCATTER) {
+                if (rows_inside) {   // this 32-row box lies inside one owner's row range (ranges are multiples of 128 rows)
+                    const int owner = row0 / p.rows_per_owner;
+                    md = reinterpret_cast<const CUtensorMap*>(&mmaps) + owner;
+                    row0 -= owner * p.rows_per_owner;
                 }
             }
             if (!p.store_d || !rows_inside) {
@@ -898,8 +913,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
-                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(md), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
+                        if constexpr (MODE == SCATTER)
+                            asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(md), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
+                        else
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(md), "r"(col0 + ch * 16), "r"(row0), "r"(buf) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
@@ -1065,6 +1084,37 @@ int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
+// Tile shape: estimated cycles = waves x (MMA cycles per tile + what the epilogue adds when it cannot run
+// under the next tile's MMAs).  False when a forced shape (testing aid) does not apply to this problem.
+bool choose_tile(int64_t M, int64_t N, int64_t K, bool epi, int sms, int& best_bn, bool& best_pair)
+{
+    best_bn = 128;
+    best_pair = false;
+    double best_cost = 1e300;
+    // testing aid: MXFP8_GEMM_TILE = "256p" | "192p" | "256" | "192" | "128" forces a shape ("p" = CTA pair)
+    const char* force = getenv("MXFP8_GEMM_TILE");
+    for (int pass = force ? 0 : 1; pass < 2 && best_cost >= 1e300; ++pass)
+    for (int bn : {256, 192, 128}) {
+        for (int pr = 1; pr >= 0; --pr) {
+            if (pr && (M <= 128 || bn == 128)) continue;
+            if (epi && bn == 192) continue;   // the fused output works on 64-column chunks per epilogue warp
+            if (pass == 0) {   // forced shape, when it applies to this problem
+                if (atoi(force) != bn || (strchr(force, 'p') != nullptr) != (pr != 0)) continue;
+            }
+            const int64_t tiles = ((M + (pr ? 255 : 127)) / (pr ? 256 : 128)) * ((N + bn - 1) / bn);
+            const int64_t workers = pr ? sms / 2 : sms;
+            const int64_t waves = (tiles + workers - 1) / workers;
+            // cycles per 128-deep K block measured on B200 for each shape (TMA feed and MMA issue
+            // included), plus the part of the epilogue that cannot run under the next tile's MMAs
+            const double kblock = pr ? (bn == 256 ? 624.0 : 747.0) : (bn == 256 ? 759.0 : (bn == 192 ? 770.0 : 450.0));
+            const double per_tile = (double)(K / 128) * kblock + (bn == 256 ? 1600.0 : 300.0);
+            const double cost = (double)waves * per_tile;
+            if (cost < best_cost) { best_cost = cost; best_bn = bn; best_pair = pr != 0; }
+        }
+    }
+    return best_cost < 1e300;
+}
+
 }  // namespace
 }  // namespace mxfp8
 
@@ -1112,35 +1162,11 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
         p.epi_s_row = static_cast<uint8_t*>(epi->s_row);
         p.epi_s_col = static_cast<uint8_t*>(epi->s_col);
     }
-    // tile shape: estimated cycles = waves x (MMA cycles per tile + what the epilogue adds when it
-    // cannot run under the next tile's MMAs)
     const int sms = sm_count();
     if (sms <= 0) return MXFP8_ERR_CUDA;
     int best_bn = 128;
     bool best_pair = false;
-    double best_cost = 1e300;
-    // testing aid: MXFP8_GEMM_TILE = "256p" | "192p" | "256" | "192" | "128" forces a shape ("p" = CTA pair)
-    const char* force = getenv("MXFP8_GEMM_TILE");
-    for (int pass = force ? 0 : 1; pass < 2 && best_cost >= 1e300; ++pass)
-    for (int bn : {256, 192, 128}) {
-        for (int pr = 1; pr >= 0; --pr) {
-            if (pr && (M <= 128 || bn == 128)) continue;
-            if (epi && bn == 192) continue;   // the fused output works on 64-column chunks per epilogue warp
-            if (pass == 0) {   // forced shape, when it applies to this problem
-                if (atoi(force) != bn || (strchr(force, 'p') != nullptr) != (pr != 0)) continue;
-            }
-            const int64_t tiles = ((M + (pr ? 255 : 127)) / (pr ? 256 : 128)) * ((N + bn - 1) / bn);
-            const int64_t workers = pr ? sms / 2 : sms;
-            const int64_t waves = (tiles + workers - 1) / workers;
-            // cycles per 128-deep K block measured on B200 for each shape (TMA feed and MMA issue
-            // included), plus the part of the epilogue that cannot run under the next tile's MMAs
-            const double kblock = pr ? (bn == 256 ? 624.0 : 747.0) : (bn == 256 ? 759.0 : (bn == 192 ? 770.0 : 450.0));
-            const double per_tile = (double)(K / 128) * kblock + (bn == 256 ? 1600.0 : 300.0);
-            const double cost = (double)waves * per_tile;
-            if (cost < best_cost) { best_cost = cost; best_bn = bn; best_pair = pr != 0; }
-        }
-    }
-    if (best_cost >= 1e300) return MXFP8_ERR_UNSUPPORTED;
+    if (!choose_tile(M, N, K, epi != nullptr, sms, best_bn, best_pair)) return MXFP8_ERR_UNSUPPORTED;
     const uint32_t b_box_rows = (uint32_t)(best_pair ? best_bn / 2 : best_bn);   // K-major B rows per TMA box
     GemmMaps m;
     const bool oka = a_major == MXFP8_K_MAJOR ? make_tmap(&m.a, Aq, (uint64_t)K, (uint64_t)M, 128, 128)
@@ -1288,4 +1314,57 @@ extern "C" int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, i
     m.a = m.multi.p[0].a; m.b = m.multi.p[0].b; m.sfa = m.multi.p[0].sfa; m.sfb = m.multi.p[0].sfb; m.d = m.multi.p[0].d;
     m.qrow = m.d; m.qcol = m.d;
     return launch_gemm<256, true, MULTI>(m, p, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int mxfp8_gemm_reduce_scatter(const void* Aq, const void* As, const void* Bq, const void* Bs,
+                                         int64_t M, int64_t N, int64_t K,
+                                         int a_major, int b_major, int a_elem, int b_elem,
+                                         void* const* D_owner, int num_owners, int first_owner, void* stream)
+{
+    using namespace mxfp8;
+    if (a_major != MXFP8_K_MAJOR && a_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
+    if (b_major != MXFP8_K_MAJOR && b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
+    if (!valid_elem(a_elem) || !valid_elem(b_elem)) return MXFP8_ERR_ENUM;
+    if (!Aq || !As || !Bq || !Bs || !D_owner) return MXFP8_ERR_NULL;
+    if (num_owners < 1 || num_owners > MAX_OWNERS || first_owner < 0 || first_owner >= num_owners) return MXFP8_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || K <= 0 || (K % 32)) return MXFP8_ERR_SHAPE;
+    if (M % ((int64_t)num_owners * 128)) return MXFP8_ERR_UNSUPPORTED;   // every owner holds whole 128-row tiles
+    if (a_major == MXFP8_MN_MAJOR && (M % 16)) return MXFP8_ERR_UNSUPPORTED;
+    if (b_major == MXFP8_MN_MAJOR && (N % 16)) return MXFP8_ERR_UNSUPPORTED;
+    if (N % 4) return MXFP8_ERR_UNSUPPORTED;
+    if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF) return MXFP8_ERR_UNSUPPORTED;
+    if (!aligned16(Aq) || !aligned16(As) || !aligned16(Bq) || !aligned16(Bs)) return MXFP8_ERR_ALIGN;
+    for (int r = 0; r < num_owners; ++r) {
+        if (!D_owner[r]) return MXFP8_ERR_NULL;
+        if (!aligned16(D_owner[r])) return MXFP8_ERR_ALIGN;
+    }
+    GemmParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.a_mn = a_major; p.b_mn = b_major; p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = MXFP8_FP32;
+    p.store_d = 1;
+    p.rows_per_owner = (int)(M / num_owners);
+    const int sms = sm_count();
+    if (sms <= 0) return MXFP8_ERR_CUDA;
+    int bn = 128;
+    bool pair = false;
+    if (!choose_tile(M, N, K, false, sms, bn, pair)) return MXFP8_ERR_UNSUPPORTED;
+    if (!pair && bn != 128) { pair = M > 128; bn = pair ? bn : 128; }   // shapes built for this mode: 256p, 192p, 128
+    // this launch begins with the tiles of owner `first_owner`, so that ranks do not all send to one GPU at a time
+    p.tm_rot = (int)(((int64_t)first_owner * p.rows_per_owner) / (pair ? 2 * BM : BM));
+    const uint32_t b_box_rows = (uint32_t)(pair ? bn / 2 : bn);
+    GemmMaps m;
+    bool ok = a_major == MXFP8_K_MAJOR ? make_tmap(&m.a, Aq, (uint64_t)K, (uint64_t)M, 128, 128)
+                                       : make_tmap(&m.a, Aq, (uint64_t)M, (uint64_t)K, 128, 128);
+    ok = ok && (b_major == MXFP8_K_MAJOR ? make_tmap(&m.b, Bq, (uint64_t)K, (uint64_t)N, 128, b_box_rows)
+                                         : make_tmap(&m.b, Bq, (uint64_t)N, (uint64_t)K, 128, 128));
+    ok = ok && make_tmap_sf(&m.sfa, As, (uint64_t)((M + 127) / 128), (uint64_t)((K + 127) / 128)) &&
+         make_tmap_sf(&m.sfb, Bs, (uint64_t)((N + 127) / 128), (uint64_t)((K + 127) / 128));
+    CUtensorMap* owner_maps = reinterpret_cast<CUtensorMap*>(&m.multi);
+    for (int r = 0; r < num_owners && ok; ++r)
+        ok = make_tmap_d(&owner_maps[r], D_owner[r], (uint64_t)p.rows_per_owner, (uint64_t)N, MXFP8_FP32);
+    if (!ok) return MXFP8_ERR_CUDA;
+    m.d = owner_maps[0]; m.qrow = m.d; m.qcol = m.d;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (pair) return bn == 256 ? launch_gemm<256, true, SCATTER>(m, p, st) : launch_gemm<192, true, SCATTER>(m, p, st);
+    return launch_gemm<128, false, SCATTER>(m, p, st);
 }
