@@ -344,6 +344,11 @@ int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq, const voi
  * more: equal up to FP32 rounding order).  M a multiple of 128 * num_owners, N of 4 (16 with an MN-major B), K of 32.
  * Nothing is allocated; never waits on another GPU inside the kernel.
  */
+/* Lets kernels launched on the current device read and write memory of `peer_device` (needed once per pair of
+ * devices before a pointer into the peer's memory is given to mxfp8_gemm_reduce_scatter).  MXFP8_OK when access
+ * is, or already was, enabled or the peer is the current device; MXFP8_ERR_SHAPE for a device that does not
+ * exist; MXFP8_ERR_UNSUPPORTED when the two devices have no peer path.  Changes this process's context only. */
+int mxfp8_enable_peer_access(int peer_device);
 int mxfp8_sf_concat_k(const void* parts, int num_parts, int64_t mn, int64_t k_part, void* dst, void* stream);
 #define MXFP8_REDUCE_SCATTER_MAX_OWNERS 8
 int mxfp8_gemm_reduce_scatter(const void* Aq, const void* As, const void* Bq, const void* Bs,

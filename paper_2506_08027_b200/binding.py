@@ -31,7 +31,7 @@ EXPORTS = (
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
     "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
-    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter",
+    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access",
 )
 
 
@@ -114,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
         L.mxfp8_grouped_gemm.restype = i
         L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
+        L.mxfp8_enable_peer_access.restype = i
+        L.mxfp8_enable_peer_access.argtypes = [i]
         L.mxfp8_sf_concat_k.restype = i
         L.mxfp8_sf_concat_k.argtypes = [p, i, i64, i64, p, p]
         L.mxfp8_gemm_reduce_scatter.restype = i
@@ -289,6 +291,10 @@ def mxfp8_grouped_gemm(aq, a_s, bq, b_s, group_offsets: torch.Tensor, mode: int,
 
 def mxfp8_sf_concat_k(parts: torch.Tensor, num_parts: int, mn: int, k_part: int, dst: torch.Tensor, stream=None) -> None:
     _check(lib().mxfp8_sf_concat_k(_ptr(parts), num_parts, mn, k_part, _ptr(dst), _stream(stream)), "mxfp8_sf_concat_k")
+
+
+def mxfp8_enable_peer_access(peer_device: int) -> None:
+    _check(lib().mxfp8_enable_peer_access(peer_device), "mxfp8_enable_peer_access")
 
 
 def make_owner_pointers(addresses):

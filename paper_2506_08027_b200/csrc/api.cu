@@ -76,6 +76,18 @@ extern "C" int mxfp8_sf_concat_k(const void* parts, int num_parts, int64_t mn, i
     return cudaGetLastError() == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
 
+extern "C" int mxfp8_enable_peer_access(int peer_device)
+{
+    int dev = 0, can = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MXFP8_ERR_CUDA;
+    if (peer_device == dev) return MXFP8_OK;
+    if (cudaDeviceCanAccessPeer(&can, dev, peer_device) != cudaSuccess) { cudaGetLastError(); return MXFP8_ERR_SHAPE; }
+    if (!can) return MXFP8_ERR_UNSUPPORTED;
+    const cudaError_t err = cudaDeviceEnablePeerAccess(peer_device, 0);
+    if (err == cudaErrorPeerAccessAlreadyEnabled) { cudaGetLastError(); return MXFP8_OK; }
+    return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
+}
+
 namespace {
 inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 }
