@@ -558,6 +558,41 @@ def run_sweep(args):
                     tf / (2 * peaks["bf16_tflops"]), ms_dense * 1e3), flush=True)
             assert B.mxfp8_device_status() == 0
         return
+    if args.sweep == "dp":
+        # the data-parallel exchange kernels on ONE GPU (all owners' buffers on this device: the additions go to local
+        # memory instead of NVLink, everything else is what a rank of a multi-GPU job launches)
+        from paper_2506_08027_b200.dp import DataParallelLinear
+        E, MN = B.E4M3, B.MN_MAJOR
+        x = synth.device_tensor("activation", (T, H), 31)
+        w = synth.device_tensor("weight", (F, H), 32)
+        dy = synth.device_tensor("output_gradient", (T, F), 33)
+        qx = B.alloc_quantize_outputs(T, H, B.COL, S); B.mxfp8_quantize(x, B.COL, P, E, *qx, S)
+        qdy = B.alloc_quantize_outputs(T, F, B.COL, S); B.mxfp8_quantize(dy, B.COL, P, E, *qdy, S)
+        dw32 = torch.zeros((F, H), dtype=torch.float32, device="cuda")
+        print("| WGRAD %d x %d x %d (tokens), FP32 result | us | TFLOP/s | of 2x measured BF16 |" % (F, H, T))
+        print("|---|---|---|---|")
+        cases = [("mxfp8_gemm, result stored", lambda i: B.mxfp8_gemm(qdy[2], qdy[3], qx[2], qx[3], F, H, T, MN, MN, E, E, dw32))]
+        for owners_n in (1, 2, 8):
+            ptrs = B.make_owner_pointers([dw32[r * (F // owners_n):] for r in range(owners_n)])
+            cases.append(("mxfp8_gemm_reduce_scatter, result added into %d owner buffer%s" % (owners_n, "" if owners_n == 1 else "s"),
+                          lambda i, ptrs=ptrs: B.mxfp8_gemm_reduce_scatter(qdy[2], qdy[3], qx[2], qx[3], F, H, T, MN, MN, E, E, ptrs, len(ptrs) // 2)))
+        for name, fn in cases:
+            ms = _time_calls(fn, 1)
+            tf = 2.0 * F * H * T / ms / 1e9
+            print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, tf, tf / (2 * peaks["bf16_tflops"])), flush=True)
+        y = torch.empty((T, F), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+        dw = torch.empty((F, H), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(B.mxfp8_linear_ws_bytes(T, H, F), dtype=torch.uint8, device="cuda")
+        layer = DataParallelLinear(T, H, F)
+        print()
+        print("| whole step, T %d, H %d, F %d, one rank | launches | us |" % (T, H, F))
+        print("|---|---|---|")
+        print("| mxfp8_linear (dW in BF16) | 2 | %.1f |" % (1e3 * _time_calls(lambda i: B.mxfp8_linear(x, w, dy, P, y, dx, dw, ws), 1)), flush=True)
+        print("| DataParallelLinear.step (dW added into the FP32 shard, zeroed every step) | 5 + memset | %.1f |" % (
+            1e3 * _time_calls(lambda i: layer.step(x, w, dy), 1)), flush=True)
+        assert B.mxfp8_device_status() == 0
+        return
     if args.sweep == "emu":
         # the MXFP8 round trip (Sec. 3.1): reads the source once, writes one same-dtype tensor per orientation
         print("| dtype | rows x cols | orient | us | GB/s | of measured copy |")
@@ -653,7 +688,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu"],
                     help="run one kernel on one small case and exit (for profiler captures)")
-    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe"],
+    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe", "dp"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
     args = ap.parse_args()
     if args.sweep:

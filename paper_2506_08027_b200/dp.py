@@ -105,7 +105,7 @@ class DataParallelLinear:
     and valid, in stream order, until the next step.  Every rank calls step() the same number of times.
     """
 
-    def __init__(self, T: int, H: int, F: int, scale_rule: int = B.RULE_PAPER, group=None, device=None):
+    def __init__(self, T: int, H: int, F: int, scale_rule: int = B.RULE_PAPER, group=None, device=None, exchange_when_alone: bool = False):
         self.group = group
         self.world = dist.get_world_size(group) if dist.is_initialized() else 1
         self.rank = dist.get_rank(group) if dist.is_initialized() else 0
@@ -114,7 +114,9 @@ class DataParallelLinear:
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         B.lib()   # fails loudly when the CUDA library is missing
         # NCCL moves device memory in stream order; any other backend (two ranks sharing one GPU in a test) goes through the host
-        self.on_stream = self.world == 1 or dist.get_backend(group) == "nccl"
+        self.on_stream = not dist.is_initialized() or dist.get_backend(group) == "nccl"
+        # a single rank has nothing to exchange; `exchange_when_alone` issues the collectives all the same (a one-rank group must exist)
+        self.exchange = self.world > 1 or exchange_when_alone
         u8 = dict(dtype=torch.uint8, device=self.device)
         self.wq_row, self.wq_col = torch.empty(F, H, **u8), torch.empty(F, H, **u8)
         self.ws_row, self.ws_col = torch.empty(p.s_row_bytes, **u8), torch.empty(p.s_col_bytes, **u8)
@@ -145,7 +147,7 @@ class DataParallelLinear:
 
     # ------------------------------------------------------------------ exchanges
     def _all_gather_slots(self):
-        if self.world == 1:
+        if not self.exchange:
             return []
         if self.on_stream:
             return [dist.all_gather_into_tensor(full, mine, group=self.group, async_op=True) for full, mine in self._gathers]
@@ -158,7 +160,7 @@ class DataParallelLinear:
 
     def _everyone_arrived(self):
         """Returns, in stream order, only after every rank's work queued so far has finished."""
-        if self.world == 1:
+        if not self.exchange:
             return
         if self.on_stream:
             dist.all_reduce(self._token, group=self.group)

@@ -48,6 +48,35 @@ def test_one_rank_equals_the_single_device_step(shape):
         assert torch.equal(gdw.to(torch.bfloat16).view(torch.int16), dw.view(torch.int16))   # FP32 here, BF16 (one rounding) there
 
 
+def test_one_rank_group_runs_the_collectives_on_the_stream():
+    """A one-rank NCCL group: the in-place all-gathers and the closing all-reduce are issued as on many GPUs."""
+    import torch
+    import torch.distributed as dist
+    from paper_2506_08027_b200 import binding as B
+    from paper_2506_08027_b200.dp import DataParallelLinear
+    T, H, F = 256, 256, 384
+    x = _bf16(synth.f32_to_bf16_bits(synth.gaussian((T, H), 15)))
+    w = _bf16(synth.f32_to_bf16_bits(0.02 * synth.gaussian((F, H), 16)))
+    dy = _bf16(synth.f32_to_bf16_bits(synth.output_gradient((T, F), 17)))
+    alone = DataParallelLinear(T, H, F)
+    want = [t.clone() for t in alone.step(x, w, dy)]
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % port, rank=0, world_size=1)
+    try:
+        layer = DataParallelLinear(T, H, F, exchange_when_alone=True)
+        assert layer.on_stream and layer.exchange
+        for _ in range(2):
+            got = layer.step(x, w, dy)
+            torch.cuda.synchronize()
+            assert B.mxfp8_device_status() == 0
+            for g, t in zip(got, want):
+                assert torch.equal(g, t)
+    finally:
+        dist.destroy_process_group()
+
+
 WORKER = r'''
 import os, sys, json
 sys.path.insert(0, os.environ["REPO_ROOT"]); sys.path.insert(0, os.path.join(os.environ["REPO_ROOT"], "tests"))
