@@ -427,6 +427,16 @@ def run_case(args):
         off_d = torch.from_numpy(offs).cuda()
         for _ in range(reps):
             B.mxfp8_grouped_gemm(qx[0], qx[1], qw[0], qw[1], off_d, B.GROUP_M, Tt, Fe, Hd, B.K_MAJOR, E, E, yg)
+    elif args.case == "scatter":
+        # the WGRAD product of the benchmark layer, its FP32 result added into 8 owner buffers (all on this device)
+        xs = synth.device_tensor("activation", (T, H), 2)
+        dys = synth.device_tensor("output_gradient", (T, F), 3)
+        qx = B.alloc_quantize_outputs(T, H, B.COL, S); B.mxfp8_quantize(xs, B.COL, P, E, *qx, S)
+        qdy = B.alloc_quantize_outputs(T, F, B.COL, S); B.mxfp8_quantize(dys, B.COL, P, E, *qdy, S)
+        dw32 = torch.zeros((F, H), dtype=torch.float32, device="cuda")
+        ptrs = B.make_owner_pointers([dw32[r * (F // 8):] for r in range(8)])
+        for _ in range(reps):
+            B.mxfp8_gemm_reduce_scatter(qdy[2], qdy[3], qx[2], qx[3], F, H, T, B.MN_MAJOR, B.MN_MAJOR, E, E, ptrs, 3)
     elif args.case == "glu":
         # SwiGLU fused ahead of the conversion: source 8192 x (2 x 8192) BF16, both orientations
         src2 = synth.device_tensor("gaussian", (n, 2 * n), 13, "bf16")
@@ -686,7 +696,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu", "scatter"],
                     help="run one kernel on one small case and exit (for profiler captures)")
     ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe", "dp"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
