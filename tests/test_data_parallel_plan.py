@@ -95,6 +95,7 @@ def _free_port():
 
 
 def test_two_gloo_ranks_assemble_the_whole_weight_and_their_rows_of_dw():
+    orc.build_oracle()          # once, before the ranks start
     port = _free_port()
     procs = []
     for r in range(2):

@@ -125,6 +125,7 @@ def _free_port():
 
 
 def test_two_processes_on_one_gpu_exchange_through_ipc_mappings():
+    orc.build_oracle()          # once, before the ranks start
     port = _free_port()
     procs = []
     for r in range(2):
