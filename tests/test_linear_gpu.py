@@ -68,7 +68,7 @@ def test_linear_device_matches_oracle_chain(shape, rule):
         check_bf16_result(from_dev_bf16(got), d64, sabs, name)
 
 
-@pytest.mark.parametrize("shape", [(256, 256, 384), (512, 128, 128), (1024, 384, 640), (2048, 512, 1152)])
+@pytest.mark.parametrize("shape", [(256, 256, 384), (512, 128, 128), (1024, 384, 640), (2048, 512, 1152), (512, 256, 1024), (384, 128, 512), (1024, 256, 2048)])
 def test_linear_host_equals_device_variant(shape):
     """T = 256 goes through in one piece; multiples of 512 tokens go through in four row chunks whose copies overlap."""
     import torch
