@@ -163,7 +163,7 @@ def gpu_gemm(aq, a_s, bq, b_s, a_major="k", b_major="k", a_elem=0, b_elem=0, out
 
 
 def check_gemm_tolerance(d_gpu, d64, sabs, what=""):
-    """spec bounds: relative Frobenius error <= 1e-5 and every element within
+    """The GEMM acceptance bounds: relative Frobenius error <= 1e-5 and every element within
     2^-16 * sum_k |a_k b_k| (plus an absolute floor of 2^-126 at the edge of the FP32 range)."""
     d = d_gpu.astype(np.float64)
     assert np.array_equal(np.isnan(d), np.isnan(d64)), "NaN positions differ " + what
