@@ -278,6 +278,8 @@ def run_ours(args):
     launches = B.mxfp8_launch_count() - launches0
     ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     ms_step = ms_total / args.steps
+    # the SM clock the last GEMM launch of the timed region really ran at (cycles / nanoseconds read inside the kernel)
+    gemm_clock_mhz, gemm_probe_us = B.mxfp8_gemm_last_clock()
 
     # ---- timed region 2: the same steps with an event before every launch -> per-kernel durations
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
@@ -326,6 +328,10 @@ def run_ours(args):
         del ws
 
     clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["sm_mhz_inside_gemm_kernel"] = round(gemm_clock_mhz, 1)
+        clocks["note"] = ("sm_mhz is the driver's sampled clock (200 ms period, longer than the timed region); sm_mhz_inside_gemm_kernel is "
+                          "SM cycles / wall time read by the last timed GEMM launch itself (%.0f us alive)" % gemm_probe_us)
     if world > 1:
         dist.barrier()
     if rank != 0:

@@ -364,6 +364,12 @@ size_t mxfp8_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int out_dtype
  * This is the only device-pointer call that synchronises. */
 int mxfp8_device_status(void* stream);
 
+/* Measurement aid (no counterpart in the paper): waits for `stream`, then reports the SM clock that the most recent
+ * GEMM launch of this library on the current device really ran at -- SM cycles divided by wall nanoseconds, both read
+ * by the kernel's first CTA at its start and end -- and that CTA's lifetime in microseconds.  A sampled
+ * driver clock cannot resolve a kernel of a few hundred microseconds; this can, and shows a power-capped run. */
+int mxfp8_gemm_last_clock(void* stream, double* sm_mhz, double* kernel_us);
+
 /* Human-readable name of a status code (static string). */
 const char* mxfp8_status_string(int status);
 

@@ -31,7 +31,7 @@ EXPORTS = (
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
     "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
-    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access",
+    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access", "mxfp8_gemm_last_clock",
 )
 
 
@@ -114,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
         L.mxfp8_grouped_gemm.restype = i
         L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
+        L.mxfp8_gemm_last_clock.restype = i
+        L.mxfp8_gemm_last_clock.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.mxfp8_enable_peer_access.restype = i
         L.mxfp8_enable_peer_access.argtypes = [i]
         L.mxfp8_sf_concat_k.restype = i
@@ -291,6 +293,13 @@ def mxfp8_grouped_gemm(aq, a_s, bq, b_s, group_offsets: torch.Tensor, mode: int,
 
 def mxfp8_sf_concat_k(parts: torch.Tensor, num_parts: int, mn: int, k_part: int, dst: torch.Tensor, stream=None) -> None:
     _check(lib().mxfp8_sf_concat_k(_ptr(parts), num_parts, mn, k_part, _ptr(dst), _stream(stream)), "mxfp8_sf_concat_k")
+
+
+def mxfp8_gemm_last_clock(stream=None):
+    """(SM MHz, microseconds) of the most recent GEMM launch, measured by the kernel itself; waits for the stream."""
+    mhz, us = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().mxfp8_gemm_last_clock(_stream(stream), ctypes.byref(mhz), ctypes.byref(us)), "mxfp8_gemm_last_clock")
+    return mhz.value, us.value
 
 
 def mxfp8_enable_peer_access(peer_device: int) -> None:

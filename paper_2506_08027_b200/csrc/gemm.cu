@@ -40,6 +40,8 @@
 namespace mxfp8 {
 
 __device__ int g_device_status = 0;
+// SM cycles and nanoseconds that the last GEMM launch's first CTA was alive: gives the SM clock the kernel really ran at
+__device__ unsigned long long g_gemm_clock_probe[2] = {0ull, 0ull};
 
 int read_and_clear_device_status(cudaStream_t stream)
 {
@@ -595,6 +597,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
+    const bool probe = blockIdx.x == 0 && threadIdx.x == 0;
+    long long probe_c0 = 0;
+    uint64_t probe_t0 = 0;
+    if (probe) { probe_c0 = clock64(); probe_t0 = global_timer(); }
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < C::ACC_STAGES; ++a) {
@@ -931,6 +937,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
     tc_fence_before();
     __syncthreads();
+    if (probe) {
+        g_gemm_clock_probe[0] = (unsigned long long)(clock64() - probe_c0);
+        g_gemm_clock_probe[1] = (unsigned long long)(global_timer() - probe_t0);
+    }
     if (PAIR) cluster_sync_all();      // nobody leaves while the peer may still signal this CTA's barriers
     if (warp == 1) {
         __syncwarp();
@@ -1367,4 +1377,15 @@ extern "C" int mxfp8_gemm_reduce_scatter(const void* Aq, const void* As, const v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (pair) return bn == 256 ? launch_gemm<256, true, SCATTER>(m, p, st) : launch_gemm<192, true, SCATTER>(m, p, st);
     return launch_gemm<128, false, SCATTER>(m, p, st);
+}
+
+extern "C" int mxfp8_gemm_last_clock(void* stream, double* sm_mhz, double* kernel_us)
+{
+    if (!sm_mhz || !kernel_us) return MXFP8_ERR_NULL;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return MXFP8_ERR_CUDA;
+    unsigned long long h[2] = {0ull, 0ull};
+    if (cudaMemcpyFromSymbol(h, mxfp8::g_gemm_clock_probe, sizeof(h)) != cudaSuccess) return MXFP8_ERR_CUDA;
+    *kernel_us = (double)h[1] * 1e-3;
+    *sm_mhz = h[1] ? (double)h[0] * 1e3 / (double)h[1] : 0.0;
+    return MXFP8_OK;
 }

@@ -547,3 +547,17 @@ def test_every_tile_shape_against_the_oracle(tile, majors):
         if old is not None:
             os.environ["MXFP8_GEMM_TILE"] = old
     check_gemm_tolerance(got, d64, sabs, "tile %s %s" % (tile, majors))
+
+
+def test_clock_probe_reports_a_plausible_sm_clock():
+    """The kernel's own cycles / wall time: between the idle floor and the boost clock, for a launch long enough to measure."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    n = 4096
+    q = torch.zeros(n, n, dtype=torch.uint8, device="cuda")
+    sf = torch.full((B.mxfp8_scale_bytes(n, n, B.ROW, B.SF_SWIZZLED),), 127, dtype=torch.uint8, device="cuda")
+    d = torch.empty(n, n, dtype=torch.bfloat16, device="cuda")
+    for _ in range(3):
+        B.mxfp8_gemm(q, sf, q, sf, n, n, n, B.K_MAJOR, B.K_MAJOR, B.E4M3, B.E4M3, d)
+    mhz, us = B.mxfp8_gemm_last_clock()
+    assert 300.0 < mhz < 2500.0 and 5.0 < us < 5000.0, (mhz, us)
