@@ -526,9 +526,12 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmParams& p, const int* g
         if (p.b_mn) { t.kb0 = g * p.num_kb; t.bn_off = 0; t.sfb_atom_off = 0; }
         else { t.kb0 = 0; t.bn_off = g * (int)p.N; t.sfb_atom_off = (g * (int)p.N) >> 7; }
     } else {
+        // experts are visited longest first (tstart[] holds that order here): the tiles that run side by side in
+        // the persistent workers then have nearly the same K depth, and the short ones fill the end
         const int per_expert = p.tiles_m * p.tiles_n;
-        g = tile / per_expert;
-        tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile - g * per_expert, t.tm, t.tn);
+        const int slot = tile / per_expert;
+        g = tstart[slot];
+        tile_coords(p.group_m, p.tiles_m, p.tiles_n, tile - slot * per_expert, t.tm, t.tn);
         const int lo = goff[g], hi = goff[g + 1];
         t.row0 = 0; t.d_row_extra = g * (int)p.M; t.rows_end = (g + 1) * (int)p.M;
         t.ka0 = lo >> 7; t.kb0 = lo >> 7; t.bn_off = 0; t.sfb_atom_off = 0;
@@ -539,7 +542,7 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmParams& p, const int* g
 
 // K blocks this worker will run through: the flat loops of the producer and the MMA issuer count them.
 template <int MODE>
-__device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const int* goff, int num_tiles, int worker, int workers)
+__device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const int* goff, const int* tstart, int num_tiles, int worker, int workers)
 {
     if (num_tiles <= worker) return 0u;
     if constexpr (MODE == MULTI) {
@@ -556,7 +559,7 @@ __device__ __forceinline__ uint32_t worker_k_blocks(const GemmParams& p, const i
         const int per_expert = p.tiles_m * p.tiles_n;
         uint32_t total = 0;
         for (int tile = worker; tile < num_tiles; tile += workers) {
-            const int g = tile / per_expert;
+            const int g = tstart[tile / per_expert];
             total += (uint32_t)((goff[g + 1] - goff[g]) >> 7);
         }
         return total;
@@ -635,13 +638,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     const int y = __shfl_up_sync(0xFFFFFFFFu, x, d);
                     if (lane >= d) x += y;
                 }
-                if (i < G) tstart[i + 1] = run + x;
+                if (MODE == GROUP_M && i < G) tstart[i + 1] = run + x;
                 run += __shfl_sync(0xFFFFFFFFu, x, 31);
             }
             bad = __any_sync(0xFFFFFFFFu, bad);
             if (lane == 0) {
-                tstart[0] = 0;
+                if (MODE == GROUP_M) tstart[0] = 0;
                 if (bad) { *bad_groups = 1; atomicExch(&g_device_status, (int)MXFP8_ERR_DEVICE_ARGS); }
+            }
+        }
+        if (MODE == GROUP_K && warp >= 2) {
+            // tstart[k] = the expert with the k-th most tokens (ties by index): one thread per expert counts who comes before it
+            const int i = (int)threadIdx.x - 64;
+            if (i < G) {
+                const int len = goff[i + 1] - goff[i];
+                int rank = 0;
+                for (int j = 0; j < G; ++j) {
+                    const int other = goff[j + 1] - goff[j];
+                    rank += (other > len || (other == len && j < i)) ? 1 : 0;
+                }
+                tstart[rank] = i;
             }
         }
     }
@@ -673,7 +689,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             int a_mn = p.a_mn, b_mn = p.b_mn;
             uint32_t stage_tx = p.stage_tx;
             const CUtensorMap *ma = &tmap_a, *mb = &tmap_b, *msfa = &tmap_sfa, *msfb = &tmap_sfb;
-            const uint32_t total = worker_k_blocks<MODE>(p, goff, num_tiles, worker, workers);
+            const uint32_t total = worker_k_blocks<MODE>(p, goff, tstart, num_tiles, worker, workers);
             int kb = 0, tile = worker, gcur = 0;
             int m_atom = 0, m0 = 0, n0 = 0, sfb_atom0 = 0, ka0 = 0, kb0 = 0, nkb = p.num_kb;
             uint32_t ph = 0;
@@ -751,7 +767,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t sf_hi = (uint32_t)(smem_desc(0, 0, 128, 0) >> 32);   // scales: 32 rows x 16 B, 8-row groups 128 B apart
             const uint32_t sfa_lo0 = (base + C::SMEM_SFA) >> 4, sfb_lo0 = (base + C::SMEM_SFB) >> 4;
             auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
-            const uint32_t total = worker_k_blocks<MODE>(p, goff, num_tiles, worker, workers);
+            const uint32_t total = worker_k_blocks<MODE>(p, goff, tstart, num_tiles, worker, workers);
             int kb = 0, tile = worker, gcur = 0, num_kb = p.num_kb;
             uint32_t ph = 0, acc_it = 0, d_tmem = tmem_base, sfb_skip = 0;
             int as = 0;
