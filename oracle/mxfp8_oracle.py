@@ -397,6 +397,34 @@ def rmsnorm(x: np.ndarray, gamma: np.ndarray, eps: float, dst: str = "f32", rstd
     return out, rstd
 
 
+def layernorm(x: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float, dst: str = "f32",
+              mean: np.ndarray | None = None, rstd: np.ndarray | None = None):
+    """Layer normalisation ahead of the conversion (Sec. 3.2 keeps normalisation in high precision and converts its
+    output).  mean[r] = mean_c x[r,c] and rstd[r] = 1 / sqrt(mean_c (x[r,c] - mean[r])^2 + eps) in binary64, each
+    rounded to binary32 (or the values passed in); y = ((x - mean) * rstd) * gamma + beta as binary32 operations in
+    that order (a subtraction, two products, an addition: four roundings), rounded once more to bfloat16 for dst
+    "bf16".  Returns (y, mean, rstd)."""
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    g32 = np.ascontiguousarray(gamma, dtype=np.float32)
+    b32 = np.ascontiguousarray(beta, dtype=np.float32)
+    v = x32.astype(np.float64)
+    if mean is None:
+        mean = v.mean(axis=1).astype(np.float32)
+    mean = np.ascontiguousarray(mean, dtype=np.float32)
+    if rstd is None:
+        d = v - v.mean(axis=1)[:, None]
+        rstd = (1.0 / np.sqrt((d * d).mean(axis=1) + float(eps))).astype(np.float32)
+    rstd = np.ascontiguousarray(rstd, dtype=np.float32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        y32 = ((x32 - mean[:, None]) * rstd[:, None]) * g32[None, :] + b32[None, :]   # numpy float32 operations are IEEE single operations
+    if dst == "f32":
+        return y32, mean, rstd
+    out = np.empty(y32.shape, dtype=np.uint16)
+    y64 = np.ascontiguousarray(y32, dtype=np.float64)
+    _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
+    return out, mean, rstd
+
+
 def glu(x: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
     """Gated activation ahead of the conversion: x is [rows, 2*cols] = (gate | up); y = act(gate) * up, with act(gate)
     as in `activation` (binary64 definition rounded to binary32), then one binary32 product, then one rounding to

@@ -635,6 +635,37 @@ def test_rmsnorm_oracle_against_exact_cases_and_library():
     assert y2[0].tolist() == [0x3F80, 0x4040] and r2[0] == 1.0
 
 
+def test_layernorm_oracle_against_exact_cases_and_library():
+    import torch
+    # rows mean +- c with c a power of two and eps = 0: deviations are +-c, so y = sign(x - mean) * gamma + beta exactly
+    x = np.array([[10.0 + 4.0, 10.0 - 4.0, 10.0 + 4.0, 10.0 - 4.0], [-3.0 + 0.25, -3.0 + 0.25, -3.0 - 0.25, -3.0 - 0.25]], np.float32)
+    gamma = np.array([1.5, 2.0, -3.0, 0.125], np.float32)
+    beta = np.array([0.5, -1.0, 2.0, 0.0], np.float32)
+    y, mean, rstd = orc.layernorm(x, gamma, beta, 0.0)
+    assert mean.tolist() == [10.0, -3.0] and rstd.tolist() == [0.25, 4.0]
+    assert np.array_equal(y, np.sign(x - mean[:, None]) * gamma[None, :] + beta[None, :])
+    # a constant row has no deviation: y = beta whatever gamma is (eps keeps rstd finite)
+    y, mean, rstd = orc.layernorm(np.full((1, 4), 7.0, np.float32), gamma, beta, 1e-5)
+    assert mean[0] == 7.0 and np.array_equal(y[0], beta) and rstd[0] == np.float32(1.0 / np.sqrt(1e-5))
+    # shifting a row by a constant changes the mean only (exactly representable shift)
+    rng = np.random.default_rng(9)
+    xr = (rng.integers(-64, 64, (8, 32)) / 16.0).astype(np.float32)
+    y0, m0, r0 = orc.layernorm(xr, np.ones(32, np.float32), np.zeros(32, np.float32), 1e-5)
+    y1, m1, r1 = orc.layernorm(xr + 32.0, np.ones(32, np.float32), np.zeros(32, np.float32), 1e-5)
+    assert np.array_equal(m1, m0 + 32.0) and np.array_equal(r1, r0) and np.array_equal(y1, y0)
+    # against the library's float64 layer_norm: equal up to the binary32 roundings of the statistics and the four operations
+    xg = (rng.standard_normal((64, 256)) * 3 + 1.5).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(256)).astype(np.float32)
+    b = (0.2 * rng.standard_normal(256)).astype(np.float32)
+    y, _, _ = orc.layernorm(xg, g, b, 1e-5)
+    lib = torch.nn.functional.layer_norm(torch.from_numpy(xg).double(), (256,), torch.from_numpy(g).double(), torch.from_numpy(b).double(), 1e-5).numpy()
+    assert np.abs(y - lib).max() <= 6 * 2.0 ** -24 * max(np.abs(lib).max(), np.abs(xg).max())
+    # supplied statistics are used as they are; BF16 destination rounds once more (ties to even)
+    y2, m2, r2 = orc.layernorm(np.array([[2.0 + 2.0 ** -8, 4.0]], np.float32), np.ones(2, np.float32), np.zeros(2, np.float32), 0.0, "bf16",
+                               np.array([1.0], np.float32), np.array([1.0], np.float32))
+    assert y2[0].tolist() == [0x3F80, 0x4040] and m2[0] == 1.0 and r2[0] == 1.0
+
+
 def test_glu_oracle_against_hand_values_and_library():
     import torch
     # (gate | up) = ([-2, 3] | [5, 0.5]): relu gate -> [0*5, 3*0.5]; bilinear -> [-10, 1.5]
