@@ -648,6 +648,12 @@ def run_sweep(args):
         gbs = rows * cols * (2 + 2 + 2 * (1 + 1 / 32)) / ms / 1e6       # the source is read twice (statistics, conversion)
         print("| rms normalisation (statistics launch + fused conversion; source read twice) | %.1f | %.0f | %.2f |" % (
             ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+        beta = torch.zeros(cols, dtype=torch.bfloat16, device="cuda")
+        mean = torch.empty(rows, dtype=torch.float32, device="cuda")
+        ms = _time_calls(lambda i: B.mxfp8_layernorm_quantize(src, gamma, beta, 1e-5, mean, rstd, B.BOTH, P, B.E4M3, *outs, S), 1)
+        gbs = rows * cols * (2 + 2 + 2 * (1 + 1 / 32)) / ms / 1e6       # the statistics launch reads each row twice, the second time from cache
+        print("| layer normalisation (statistics launch + fused conversion; source read twice from memory) | %.1f | %.0f | %.2f |" % (
+            ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
         return
     shapes = [("square", n, n, n, 0, 0) for n in (1024, 2048, 4096, 8192, 16384)]
     shapes.append(("skinny wgrad", 4096, 4096, 65536, 1, 1))

@@ -183,6 +183,20 @@ int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t
                            int sf_layout, void* stream);
 
 /*
+ * mxfp8_layernorm_quantize -- the same with a layer normalisation: y = ((x - mean[row]) * rstd[row]) * gamma[col] + beta[col],
+ * four FP32 operations in that order (no fused multiply-add), rounded once to the source dtype, then converted.
+ * mean[row] and rstd[row] = 1 / sqrt(mean_c (x - mean)^2 + eps) are computed by a statistics launch (two passes
+ * over the row, FP32 sums in a fixed order) and written to `mean` and `rstd` (device, FP32 [rows]) for the backward
+ * pass.  `gamma`, `beta`: device, source dtype, [cols], 16-byte aligned.  Everything else as mxfp8_rmsnorm_quantize.
+ * (Sec. 3.2 keeps normalisation in high precision and converts its output; the paper names no particular one.)
+ */
+int mxfp8_layernorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                             const void* gamma, const void* beta, float eps, float* mean, float* rstd,
+                             int orientation, int scale_rule, int elem,
+                             void* q_row, void* s_row, void* q_col, void* s_col,
+                             int sf_layout, void* stream);
+
+/*
  * mxfp8_rmsnorm_quantize_static -- mxfp8_rmsnorm_quantize for callers that do not want the row
  * statistics and have no buffer to lend: the statistics go to a fixed array inside the library
  * (file-scope device memory, 65536 rows x 4 bytes = 256 KB, part of the module image), so the call

@@ -31,7 +31,7 @@ EXPORTS = (
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
     "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
-    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access", "mxfp8_gemm_last_clock",
+    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access", "mxfp8_gemm_last_clock", "mxfp8_layernorm_quantize",
 )
 
 
@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
         L.mxfp8_rmsnorm_quantize.restype = i
         L.mxfp8_rmsnorm_quantize.argtypes = [p, i, i64, i64, p, ctypes.c_float, p, i, i, i, p, p, p, p, i, p]
+        L.mxfp8_layernorm_quantize.restype = i
+        L.mxfp8_layernorm_quantize.argtypes = [p, i, i64, i64, p, p, ctypes.c_float, p, p, i, i, i, p, p, p, p, i, p]
         L.mxfp8_rmsnorm_quantize_static.restype = i
         L.mxfp8_rmsnorm_quantize_static.argtypes = [p, i, i64, i64, p, ctypes.c_float, i, i, i, p, p, p, p, i, p]
         L.mxfp8_rmsnorm_quantize_static_max_rows.restype = i64
@@ -362,6 +364,17 @@ def mxfp8_act_quantize(src: torch.Tensor, act: int, orientation: int, scale_rule
     _check(lib().mxfp8_act_quantize(_ptr(src), _dtype_code(src), rows, cols, act, orientation, scale_rule, elem,
                                     _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
                                     _stream(stream)), "mxfp8_act_quantize")
+
+
+def mxfp8_layernorm_quantize(src: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: float, mean: torch.Tensor, rstd: torch.Tensor,
+                             orientation: int, scale_rule: int, elem: int,
+                             q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    rows, cols = src.shape
+    assert src.is_contiguous() and gamma.dtype == src.dtype and beta.dtype == src.dtype
+    assert mean.dtype == torch.float32 and rstd.dtype == torch.float32
+    _check(lib().mxfp8_layernorm_quantize(_ptr(src), _dtype_code(src), rows, cols, _ptr(gamma), _ptr(beta), eps, _ptr(mean), _ptr(rstd),
+                                          orientation, scale_rule, elem, _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
+                                          _stream(stream)), "mxfp8_layernorm_quantize")
 
 
 def mxfp8_rmsnorm_quantize(src: torch.Tensor, gamma: torch.Tensor, eps: float, rstd: torch.Tensor,

@@ -400,8 +400,9 @@ extern "C" int mxfp8_glu_quantize(const void* src, int src_dtype, int64_t rows, 
 
 namespace mxfp8 {
 namespace {
-// 1/rms of every row: one warp per row, 16-byte loads, FP32 accumulation (lane-strided partial sums, then a
-// butterfly), rstd = 1 / sqrt(sum / cols + eps) with IEEE square root and division.
+// 1/rms of every row: one warp per row, four 16-byte loads in flight per lane, FP32 accumulation (four lane-strided
+// partial sums per lane in a fixed order, then a butterfly), rstd = 1 / sqrt(sum / cols + eps) with IEEE square root
+// and division.
 template <int DTYPE>
 __global__ void __launch_bounds__(256) rms_stats_kernel(const void* __restrict__ src, int64_t rows, int64_t cols, float eps,
                                                         float* __restrict__ rstd)
@@ -412,28 +413,123 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const void* __restrict__
     constexpr int PER = (DTYPE == MXFP8_BF16) ? 8 : 4;            // elements per 16-byte load
     const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(src) + row * cols * (DTYPE == MXFP8_BF16 ? 2 : 4));
     const int64_t chunks = cols / PER;
-    float acc = 0.f;
-    for (int64_t c = lane; c < chunks; c += 32) {
-        const uint4 w = p[c];
+    float part[4] = {0.f, 0.f, 0.f, 0.f};
+    auto add = [&](const uint4& w, int k) {
         const uint32_t u[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (DTYPE == MXFP8_BF16) {
                 const float a = __uint_as_float(u[i] << 16), b = __uint_as_float(u[i] & 0xFFFF0000u);
-                acc = fmaf(a, a, acc);
-                acc = fmaf(b, b, acc);
+                part[k] = fmaf(a, a, part[k]);
+                part[k] = fmaf(b, b, part[k]);
             } else {
                 const float a = __uint_as_float(u[i]);
-                acc = fmaf(a, a, acc);
+                part[k] = fmaf(a, a, part[k]);
             }
         }
+    };
+    int64_t c = lane;
+    for (; c + 96 < chunks; c += 128) {          // four 16-byte loads in flight per lane
+        const uint4 w0 = p[c], w1 = p[c + 32], w2 = p[c + 64], w3 = p[c + 96];
+        add(w0, 0); add(w1, 1); add(w2, 2); add(w3, 3);
     }
+    if (c < chunks) { add(p[c], 0); c += 32; }    // up to three 16-byte pieces per lane are left
+    if (c < chunks) { add(p[c], 1); c += 32; }
+    if (c < chunks) add(p[c], 2);
+    float acc = (part[0] + part[1]) + (part[2] + part[3]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
     if (lane == 0) rstd[row] = 1.0f / sqrtf(acc / (float)cols + eps);
 }
+
+// Row statistics of the layer normalisation, one warp per row, ONE pass: sums of d = x - pivot and of d^2 with the
+// row's first element as pivot (a value within a few standard deviations of the mean, so the subtraction
+// S2 - S1^2 / n cancels little), four 16-byte loads in flight per lane, four partial sums per lane in a fixed order,
+// xor butterflies; mean = pivot + S1 / n, rstd = 1 / sqrt((S2 - S1^2 / n) / n + eps) with IEEE square root and division.
+template <int DTYPE>
+__global__ void __launch_bounds__(256) ln_stats_kernel(const void* __restrict__ src, int64_t rows, int64_t cols, float eps,
+                                                       float* __restrict__ mean, float* __restrict__ rstd)
+{
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    constexpr int PER = (DTYPE == MXFP8_BF16) ? 8 : 4;            // elements per 16-byte load
+    const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(src) + row * cols * (DTYPE == MXFP8_BF16 ? 2 : 4));
+    const int64_t chunks = cols / PER;
+    const uint32_t first = *reinterpret_cast<const uint32_t*>(p);
+    const float pivot = (DTYPE == MXFP8_BF16) ? __uint_as_float(first << 16) : __uint_as_float(first);
+    float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+    auto add = [&](const uint4& w, int k) {
+        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (DTYPE == MXFP8_BF16) {
+                const float a = __uint_as_float(u[i] << 16) - pivot, b = __uint_as_float(u[i] & 0xFFFF0000u) - pivot;
+                s1[k] += a; s2[k] = fmaf(a, a, s2[k]);
+                s1[k] += b; s2[k] = fmaf(b, b, s2[k]);
+            } else {
+                const float a = __uint_as_float(u[i]) - pivot;
+                s1[k] += a; s2[k] = fmaf(a, a, s2[k]);
+            }
+        }
+    };
+    int64_t c = lane;
+    for (; c + 96 < chunks; c += 128) {
+        const uint4 w0 = p[c], w1 = p[c + 32], w2 = p[c + 64], w3 = p[c + 96];
+        add(w0, 0); add(w1, 1); add(w2, 2); add(w3, 3);
+    }
+    if (c < chunks) { add(p[c], 0); c += 32; }    // up to three 16-byte pieces per lane are left
+    if (c < chunks) { add(p[c], 1); c += 32; }
+    if (c < chunks) add(p[c], 2);
+    float a1 = (s1[0] + s1[1]) + (s1[2] + s1[3]), a2 = (s2[0] + s2[1]) + (s2[2] + s2[3]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, off);
+        a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, off);
+    }
+    if (lane == 0) {
+        const float n = (float)cols;
+        const float var = fmaxf((a2 - a1 * a1 / n) / n, 0.f);
+        mean[row] = pivot + a1 / n;
+        rstd[row] = 1.0f / sqrtf(var + eps);
+    }
+}
 }  // namespace
 }  // namespace mxfp8
+
+extern "C" int mxfp8_layernorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                        const void* gamma, const void* beta, float eps, float* mean, float* rstd,
+                                        int orientation, int scale_rule, int elem,
+                                        void* q_row, void* s_row, void* q_col, void* s_col,
+                                        int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!src || !gamma || !beta || !mean || !rstd) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col || !s_col)) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || !(eps >= 0.f)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(src) || !aligned16(gamma) || !aligned16(beta)) return MXFP8_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(rstd) & 3u) || (reinterpret_cast<uintptr_t>(mean) & 3u)) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
+    if ((rows + 7) / 8 > 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned blocks = (unsigned)((rows + 7) / 8);
+    if (src_dtype == MXFP8_BF16) ln_stats_kernel<MXFP8_BF16><<<blocks, 256, 0, st>>>(src, rows, cols, eps, mean, rstd);
+    else ln_stats_kernel<MXFP8_FP32><<<blocks, 256, 0, st>>>(src, rows, cols, eps, mean, rstd);
+    count_launch(1);
+    if (cudaGetLastError() != cudaSuccess) return MXFP8_ERR_CUDA;
+    const QuantizeItem item{src, rows, cols, q_row, s_row, q_col, s_col};
+    return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, st, false, MXFP8_ACT_NONE, rstd, gamma, false, mean, beta);
+}
 
 extern "C" int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
                                       const void* gamma, float eps, float* rstd,

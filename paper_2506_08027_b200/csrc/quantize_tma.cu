@@ -63,7 +63,7 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
 
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
                        int sf_layout, cudaStream_t stream, bool emulate, int act, const float* rstd, const void* gamma,
-                       bool gated)
+                       bool gated, const float* mean, const void* beta)
 {
     if (count < 1 || count > QT_MAX_TENSORS) return MXFP8_ERR_UNSUPPORTED;
     const bool bf = src_dtype == MXFP8_BF16;
@@ -74,6 +74,8 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
     p.act = act;
     p.rstd = rstd;
     p.gamma = gamma;
+    p.mean = mean;
+    p.beta = beta;
     p.glu_cols = gated ? (int)items[0].cols : 0;     // gated: one tensor, source [rows, 2 * cols]
     int64_t tiles = 0;
     for (int i = 0; i < QT_MAX_TENSORS; ++i) {

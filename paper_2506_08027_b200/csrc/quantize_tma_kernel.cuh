@@ -79,36 +79,49 @@ __device__ __forceinline__ void act_slab(uint8_t* mine)
     }
 }
 
-// RMS normalisation in place, same ownership as act_slab: y = (x * rstd[row]) * gamma[col], two FP32 products
+// Normalisation in place, same ownership as act_slab: RMS y = (x * rstd[row]) * gamma[col], two FP32 products; layer
+// normalisation y = ((x - mean[row]) * rstd[row]) * gamma[col] + beta[col], four FP32 operations
 // in that order, rounded once to the source dtype.  Rows and columns beyond the tensor hold TMA's zero fill and
 // are left alone (their statistics and weights do not exist).
 template <bool BF>
 __device__ __forceinline__ void norm_slab(uint8_t* mine, const float* __restrict__ rstd, const void* __restrict__ gamma_col,
-                                          int rows_here, bool col_ok)
+                                          int rows_here, bool col_ok, const float* __restrict__ mean, const void* __restrict__ beta_col)
 {
     if (!col_ok) return;
-    float g[4];
-    if constexpr (BF) {
-        const uint2 w = *reinterpret_cast<const uint2*>(gamma_col);
-        g[0] = __uint_as_float(w.x << 16); g[1] = __uint_as_float(w.x & 0xFFFF0000u);
-        g[2] = __uint_as_float(w.y << 16); g[3] = __uint_as_float(w.y & 0xFFFF0000u);
-    } else {
-        const float2 w = *reinterpret_cast<const float2*>(gamma_col);
-        g[0] = w.x; g[1] = w.y; g[2] = 0.f; g[3] = 0.f;
-    }
+    auto weights = [](const void* ptr, float (&g)[4]) {
+        if constexpr (BF) {
+            const uint2 w = *reinterpret_cast<const uint2*>(ptr);
+            g[0] = __uint_as_float(w.x << 16); g[1] = __uint_as_float(w.x & 0xFFFF0000u);
+            g[2] = __uint_as_float(w.y << 16); g[3] = __uint_as_float(w.y & 0xFFFF0000u);
+        } else {
+            const float2 w = *reinterpret_cast<const float2*>(ptr);
+            g[0] = w.x; g[1] = w.y; g[2] = 0.f; g[3] = 0.f;
+        }
+    };
+    float g[4], b[4] = {0.f, 0.f, 0.f, 0.f};
+    weights(gamma_col, g);
+    const bool layer = mean != nullptr;      // layer normalisation: subtract the row mean first, add the per-column bias last
+    if (layer) weights(beta_col, b);
+    // one value: a subtraction (layer normalisation only), two products and an addition (layer normalisation only),
+    // each rounded to FP32 on its own (no fused multiply-add: the definition has four roundings)
+    auto one = [&](float x, float m, float r, int i) {
+        const float t = __fmul_rn(__fmul_rn(layer ? __fsub_rn(x, m) : x, r), g[i]);
+        return layer ? __fadd_rn(t, b[i]) : t;
+    };
 #pragma unroll 8
     for (int j = 0; j < 32; ++j) {
         if (j >= rows_here) break;
         const float r = rstd[j];
+        const float m = layer ? mean[j] : 0.f;
         uint2 w = *reinterpret_cast<const uint2*>(mine + j * T_BYTES);
         if constexpr (BF) {
-            const __nv_bfloat162 lo = __floats2bfloat162_rn((__uint_as_float(w.x << 16) * r) * g[0], (__uint_as_float(w.x & 0xFFFF0000u) * r) * g[1]);
-            const __nv_bfloat162 hi = __floats2bfloat162_rn((__uint_as_float(w.y << 16) * r) * g[2], (__uint_as_float(w.y & 0xFFFF0000u) * r) * g[3]);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(one(__uint_as_float(w.x << 16), m, r, 0), one(__uint_as_float(w.x & 0xFFFF0000u), m, r, 1));
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(one(__uint_as_float(w.y << 16), m, r, 2), one(__uint_as_float(w.y & 0xFFFF0000u), m, r, 3));
             w.x = *reinterpret_cast<const uint32_t*>(&lo);
             w.y = *reinterpret_cast<const uint32_t*>(&hi);
         } else {
-            w.x = __float_as_uint((__uint_as_float(w.x) * r) * g[0]);
-            w.y = __float_as_uint((__uint_as_float(w.y) * r) * g[1]);
+            w.x = __float_as_uint(one(__uint_as_float(w.x), m, r, 0));
+            w.y = __float_as_uint(one(__uint_as_float(w.y), m, r, 1));
         }
         *reinterpret_cast<uint2*>(mine + j * T_BYTES) = w;
     }
@@ -146,6 +159,8 @@ struct QBatch {
     int act;                              // MXFP8_ACT_*: applied to every element before the conversion
     const float* rstd;                    // RMS normalisation ahead of the conversion (first tensor only): 1/rms per row,
     const void* gamma;                    //   and the per-column weight in the source dtype; both null when unused
+    const float* mean;                    // layer normalisation: the row means (subtracted first) and the per-column bias in the
+    const void* beta;                     //   source dtype (added last); both null for RMS normalisation
     int glu_cols;                         // gated activation: the source is [rows, 2 * glu_cols] = (gate | up); 0 when unused
     int count;
     int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
@@ -565,7 +580,9 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
             const int rows_in = (int)max((int64_t)0, min((int64_t)32, p.rows - row_first));
             const int64_t col_first = gcol0 + lane * VEC;
             norm_slab<BF>(in_tile + warp * 32 * T_BYTES + lane * 8, batch.rstd + row_first,
-                          static_cast<const uint8_t*>(batch.gamma) + col_first * (BF ? 2 : 4), rows_in, col_first < p.cols);
+                          static_cast<const uint8_t*>(batch.gamma) + col_first * (BF ? 2 : 4), rows_in, col_first < p.cols,
+                          batch.mean ? batch.mean + row_first : nullptr,
+                          batch.beta ? static_cast<const uint8_t*>(batch.beta) + col_first * (BF ? 2 : 4) : nullptr);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         if (PRO == PRO_ELEMENTWISE && batch.act != MXFP8_ACT_NONE) {

@@ -192,6 +192,80 @@ def test_rmsnorm_quantize(dtype, shape):
         assert_q_equal(got[name][0], wq, orc.E4M3, name)
 
 
+# ------------------------------------------------------------------------------------------ layer normalisation
+
+def gpu_layernorm_quantize(src_np, gamma_np, beta_np, dtype, eps, orientation, elem=orc.E4M3):
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = src_np.shape
+
+    def dev(a):
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(a).cuda()
+    src, gamma, beta = dev(src_np), dev(gamma_np), dev(beta_np)
+    mean, rstd = Guarded(rows * 4), Guarded(rows * 4)
+    bufs, args = {}, []
+    for o, name in ((B.ROW, "row"), (B.COL, "col")):
+        if orientation & o:
+            bufs[name] = (Guarded(rows * cols), Guarded(B.mxfp8_scale_bytes(rows, cols, o, B.SF_SWIZZLED)))
+            args += [bufs[name][0].view.view(rows, cols), bufs[name][1].view]
+        else:
+            args += [None, None]
+    before = B.mxfp8_launch_count()
+    B.mxfp8_layernorm_quantize(src, gamma, beta, eps, mean.view.view(torch.float32), rstd.view.view(torch.float32), orientation,
+                               B.RULE_PAPER, elem, *args, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0 and B.mxfp8_launch_count() - before == 2
+    mean.check(); rstd.check()
+    out = {"mean": mean.numpy().view(np.float32).copy(), "rstd": rstd.numpy().view(np.float32).copy()}
+    for name, (q, s) in bufs.items():
+        q.check(); s.check()
+        mn, nkb = (rows, cols // 32) if name == "row" else (cols, rows // 32)
+        logical = logical_scales_from_swizzled(s.numpy(), mn, nkb)
+        out[name] = (orc.unpack_codes16(q.numpy().reshape(rows, cols), elem), logical if name == "row" else np.ascontiguousarray(logical.T))
+    return out
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(256, 512), (160, 352), (96, 4096 + 128), (32, 2048)])
+def test_layernorm_quantize(dtype, shape):
+    rows, cols = shape
+    rng = np.random.default_rng(rows)
+    x32 = (synth.gaussian(shape, 13 + rows) * np.exp2(rng.integers(-6, 6, (rows, 1))) + rng.standard_normal((rows, 1)) * 4).astype(np.float32)
+    g32 = (1.0 + 0.2 * synth.gaussian((1, cols), 14)[0]).astype(np.float32)
+    b32 = (0.3 * synth.gaussian((1, cols), 15)[0]).astype(np.float32)
+    x, g, b = as_dtype(x32, dtype), as_dtype(g32, dtype), as_dtype(b32, dtype)
+    val = (lambda a: orc.bf16_bits_to_f32(a)) if dtype == "bf16" else (lambda a: a)
+    xv, gv, bv = val(x), val(g), val(b)
+    got = gpu_layernorm_quantize(x, g, b, dtype, 1e-5, BOTH)
+    # the statistics: FP32 accumulation against the FP64 definition
+    _, want_mean, want_rstd = orc.layernorm(xv, gv, bv, 1e-5)
+    assert np.abs(got["mean"] - want_mean).max() <= 2.0 ** -20 * np.abs(xv).max()
+    assert np.abs(got["rstd"] - want_rstd).max() <= 2.0 ** -18 * np.abs(want_rstd).max()
+    # given those statistics everything after is exact arithmetic: bit-exact against the oracle
+    y, _, _ = orc.layernorm(xv, gv, bv, 1e-5, "bf16" if dtype == "bf16" else "f32", got["mean"], got["rstd"])
+    y = orc.bf16_bits_to_f32(y) if dtype == "bf16" else y
+    for o, name in ((orc.ROW, "row"), (orc.COL, "col")):
+        wq, ws = orc.quantize(y, o, orc.RULE_PAPER, orc.E4M3)
+        assert np.array_equal(got[name][1], ws), "scales %s" % name
+        assert_q_equal(got[name][0], wq, orc.E4M3, name)
+
+
+def test_layernorm_equals_rmsnorm_on_centred_rows_without_bias():
+    """Rows of small multiples of 1/4 in (v, -v) pairs and a zero bias: every sum the two statistics kernels form is exact,
+    the mean is exactly zero, and the two normalisations are the same arithmetic."""
+    rows, cols = 64, 256
+    rng = np.random.default_rng(77)
+    half = (rng.integers(1, 9, (rows, cols // 2)) * rng.choice([-1.0, 1.0], (rows, cols // 2)) / 4.0).astype(np.float32)   # no zeros: -0 + bias 0 = +0
+    x = np.stack([half, -half], axis=2).reshape(rows, cols).copy()
+    g = (1.0 + 0.2 * synth.gaussian((1, cols), 78)[0]).astype(np.float32)
+    ln = gpu_layernorm_quantize(x, g, np.zeros(cols, np.float32), "fp32", 1e-5, BOTH)
+    rms = gpu_rmsnorm_quantize(x, g, "fp32", 1e-5, BOTH)
+    assert not ln["mean"].any()
+    assert np.array_equal(ln["rstd"], rms["rstd"])
+    for name in ("row", "col"):
+        assert np.array_equal(ln[name][0], rms[name][0]) and np.array_equal(ln[name][1], rms[name][1])
+
+
 def test_rmsnorm_argument_errors():
     import torch
     from paper_2506_08027_b200 import binding as B
