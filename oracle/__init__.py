@@ -10,6 +10,6 @@ from .mxfp8_oracle import (  # noqa: F401
     build_oracle, fp8_decode, fp8_encode, scale_byte, quantize, dequantize_f64,
     dequantize, bf16_bits_to_f32, sf_offset_swizzled,
     swizzle_scales, gemm_f64, quantize_threads, grouped_gemm_f64, code_bits, pack_codes16, unpack_codes16,
-    ACT_NONE, ACT_RELU, ACT_RELU2, ACT_SILU, ACT_GELU_TANH, activation, rmsnorm, glu, layernorm,
+    ACT_NONE, ACT_RELU, ACT_RELU2, ACT_SILU, ACT_GELU_TANH, activation, rmsnorm, glu, layernorm, activation_grad,
     concat_swizzled_scales_k, data_parallel_linear_f64,
 )

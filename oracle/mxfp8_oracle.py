@@ -376,6 +376,41 @@ def activation(x: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
     return out
 
 
+def activation_grad(z: np.ndarray, dh: np.ndarray, act: int, dst: str = "f32") -> np.ndarray:
+    """Backward of the elementwise activation ahead of the conversion: the gradient with respect to the activation's
+    input, dz = act'(z) * dh, is an activation gradient and is converted like one (Sec. 3.2).  act'(z) is the plain
+    derivative in binary64 rounded once to binary32; the product with dh is one binary32 operation; for dst "bf16"
+    the result is rounded once more to bfloat16.
+        relu': z > 0 ? 1 : 0;  relu2': z > 0 ? 2z : 0;  silu': s (1 + z (1 - s)) with s = 1 / (1 + exp(-z));
+        gelu_tanh': 0.5 (1 + t) + 0.5 z (1 - t^2) sqrt(2/pi) (1 + 3 * 0.044715 z^2) with t = tanh(sqrt(2/pi) (z + 0.044715 z^3))
+    """
+    v = np.asarray(z, dtype=np.float64)
+    g32 = np.ascontiguousarray(dh, dtype=np.float32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        if act == ACT_NONE:
+            d = np.ones_like(v)
+        elif act == ACT_RELU:
+            d = np.where(v > 0, 1.0, 0.0)
+        elif act == ACT_RELU2:
+            d = np.where(v > 0, 2.0 * v, 0.0)
+        elif act == ACT_SILU:
+            sg = 1.0 / (1.0 + np.exp(-v))
+            d = sg * (1.0 + v * (1.0 - sg))
+        elif act == ACT_GELU_TANH:
+            c = np.sqrt(2.0 / np.pi)
+            t = np.tanh(c * (v + 0.044715 * v * v * v))
+            d = 0.5 * (1.0 + t) + 0.5 * v * (1.0 - t * t) * c * (1.0 + 3.0 * 0.044715 * v * v)
+        else:
+            raise ValueError(act)
+        y32 = d.astype(np.float32) * g32          # one binary32 product
+    if dst == "f32":
+        return y32
+    out = np.empty(y32.shape, dtype=np.uint16)
+    y64 = np.ascontiguousarray(y32, dtype=np.float64)
+    _load().orc_round_to_bf16(_ptr(y64), y64.size, _ptr(out))
+    return out
+
+
 def rmsnorm(x: np.ndarray, gamma: np.ndarray, eps: float, dst: str = "f32", rstd: np.ndarray | None = None):
     """RMS normalisation ahead of the conversion (Sec. 3.2 keeps normalisation in high precision and converts its
     output).  rstd[r] = 1 / sqrt(mean_c x[r,c]^2 + eps) in binary64, rounded to binary32 (or the `rstd` passed in, one

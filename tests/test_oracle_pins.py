@@ -612,6 +612,35 @@ def test_activation_oracle_against_closed_forms_and_library():
     assert b.tolist() == [0x3F80, 0x4040]                 # 1 + 2^-8 ties to even (1.0)
 
 
+def test_activation_grad_oracle_against_closed_forms_autograd_and_differences():
+    import torch
+    z = np.array([-3.5, -1.0, -0.0, 0.0, 2.0 ** -20, 0.5, 1.0, 3.0], np.float32)
+    dh = np.array([2.0, -1.0, 5.0, 5.0, 4.0, -8.0, 0.5, 1.5], np.float32)
+    assert orc.activation_grad(z, dh, orc.ACT_RELU).tolist() == [0.0, -0.0, 0.0, 0.0, 4.0, -8.0, 0.5, 1.5]
+    assert orc.activation_grad(z, dh, orc.ACT_RELU2).tolist() == [0.0, -0.0, 0.0, 0.0, 2.0 ** -17, -8.0, 1.0, 9.0]
+    assert np.array_equal(orc.activation_grad(z, dh, orc.ACT_NONE), dh)
+    # the library's reverse-mode derivative in binary64 for the two transcendental ones
+    t = torch.linspace(-12, 12, 4001, dtype=torch.float64, requires_grad=True)
+    up = np.random.default_rng(3).standard_normal(4001).astype(np.float32)
+    for act, fn in ((orc.ACT_SILU, torch.nn.functional.silu), (orc.ACT_GELU_TANH, lambda v: torch.nn.functional.gelu(v, approximate="tanh"))):
+        (grad,) = torch.autograd.grad(fn(t).sum(), t)
+        want = grad.numpy() * up.astype(np.float64)
+        got = orc.activation_grad(t.detach().numpy(), up, act).astype(np.float64)
+        assert np.abs(got - want).max() <= 2.0 ** -21 * np.abs(want).max()
+    # and the derivative is the derivative of the forward function of this oracle: central differences in binary64
+    zz = np.linspace(-6, 6, 240)          # no grid point on the kink of relu2 at 0
+    h = 1e-5
+    for act in (orc.ACT_RELU2, orc.ACT_SILU, orc.ACT_GELU_TANH):
+        fwd = lambda v: {orc.ACT_RELU2: np.where(v > 0, v * v, 0.0), orc.ACT_SILU: v / (1 + np.exp(-v)),
+                         orc.ACT_GELU_TANH: 0.5 * v * (1 + np.tanh(np.sqrt(2 / np.pi) * (v + 0.044715 * v ** 3)))}[act]
+        num = (fwd(zz + h) - fwd(zz - h)) / (2 * h)
+        got = orc.activation_grad(zz, np.ones(zz.size, np.float32), act).astype(np.float64)
+        assert np.abs(got - num).max() <= 1e-6
+    # BF16 destination: one more round-to-nearest-even
+    b = orc.activation_grad(np.array([1.0, 1.0], np.float32), np.array([1.0 + 2.0 ** -8, 3.0], np.float32), orc.ACT_RELU, "bf16")
+    assert b.tolist() == [0x3F80, 0x4040]
+
+
 def test_rmsnorm_oracle_against_exact_cases_and_library():
     import torch
     # rows of +-c with c a power of two and eps = 0: rms = c exactly, so y = sign(x) * gamma exactly
