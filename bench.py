@@ -642,6 +642,12 @@ def run_sweep(args):
             gbs = rows * cols * (4 + 2 * (1 + 1 / 32)) / ms / 1e6       # gate and up are read, one [rows, cols] result in both orientations written
             print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
         del src2
+        dh = synth.device_tensor("output_gradient", (rows, cols), 14, "bf16")
+        for act, name in ((B.ACT_RELU2, "backward of squared relu: 2 relu(z) * dh, two sources"), (B.ACT_SILU, "backward of silu: silu'(z) * dh, two sources")):
+            ms = _time_calls(lambda i: B.mxfp8_act_grad_quantize(dh, src, act, B.BOTH, P, B.E4M3, *outs, S), 1)
+            gbs = rows * cols * (4 + 2 * (1 + 1 / 32)) / ms / 1e6       # z and dh are read, one [rows, cols] result in both orientations written
+            print("| %s | %.1f | %.0f | %.2f |" % (name, ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
+        del dh
         gamma = torch.ones(cols, dtype=torch.bfloat16, device="cuda")
         rstd = torch.empty(rows, dtype=torch.float32, device="cuda")
         ms = _time_calls(lambda i: B.mxfp8_rmsnorm_quantize(src, gamma, 1e-5, rstd, B.BOTH, P, B.E4M3, *outs, S), 1)

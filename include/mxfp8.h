@@ -165,6 +165,21 @@ int mxfp8_glu_quantize(const void* src, int src_dtype, int64_t rows, int64_t col
                        int sf_layout, void* stream);
 
 /*
+ * mxfp8_act_grad_quantize -- the backward of such an activation ahead of the conversion: dz = act'(z) * dh, the
+ * gradient with respect to the activation's input, is an activation gradient and gets converted (Sec. 3.2).
+ * `z` (the activation's input saved by the forward pass) and `dh` (the incoming gradient) are device tensors
+ * [rows, cols] of `src_dtype`; act is MXFP8_ACT_RELU .. MXFP8_ACT_GELU_TANH.  act'(z) is evaluated in FP32 (relu: 0 or
+ * 1; squared relu: 2z or 0; silu and tanh-gelu with the fast FP32 exponential and division), multiplied by dh (one
+ * FP32 product), rounded once to the source dtype, then converted exactly like mxfp8_quantize of a tensor holding
+ * that value.  One launch; nothing is written besides the MXFP8 outputs; cols a multiple of 16; other arguments,
+ * layouts and errors as mxfp8_quantize.
+ */
+int mxfp8_act_grad_quantize(const void* dh, const void* z, int src_dtype, int64_t rows, int64_t cols, int act,
+                            int orientation, int scale_rule, int elem,
+                            void* q_row, void* s_row, void* q_col, void* s_col,
+                            int sf_layout, void* stream);
+
+/*
  * mxfp8_rmsnorm_quantize -- RMS normalisation fused ahead of the conversion (Sec. 3.2 keeps the
  * normalisation layers in high precision and converts their output for the next GEMM).  Two launches:
  *   rstd[r] = 1 / sqrt(mean_c(x[r, c]^2) + eps)     FP32 accumulation over the row, written to `rstd`

@@ -31,7 +31,7 @@ EXPORTS = (
     "mxfp8_linear_host_ws_bytes", "mxfp8_linear_host", "mxfp8_fake_quantize", "mxfp8_linear_ws_bytes",
     "mxfp8_linear", "mxfp8_grouped_gemm", "mxfp8_quantize_multi", "mxfp8_gemm_multi", "mxfp8_act_quantize", "mxfp8_rmsnorm_quantize",
     "mxfp8_rmsnorm_quantize_static", "mxfp8_rmsnorm_quantize_static_max_rows", "mxfp8_glu_quantize",
-    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access", "mxfp8_gemm_last_clock", "mxfp8_layernorm_quantize",
+    "mxfp8_sf_concat_k", "mxfp8_gemm_reduce_scatter", "mxfp8_enable_peer_access", "mxfp8_gemm_last_clock", "mxfp8_layernorm_quantize", "mxfp8_act_grad_quantize",
 )
 
 
@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.mxfp8_rmsnorm_quantize_static_max_rows.argtypes = []
         L.mxfp8_glu_quantize.restype = i
         L.mxfp8_glu_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
+        L.mxfp8_act_grad_quantize.restype = i
+        L.mxfp8_act_grad_quantize.argtypes = [p, p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_act_quantize.restype = i
         L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
         L.mxfp8_gemm_multi.restype = i
@@ -355,6 +357,15 @@ def make_gemm_problems(entries):
 
 def mxfp8_gemm_multi(problems, out_dtype: int, stream=None) -> None:
     _check(lib().mxfp8_gemm_multi(problems, len(problems), out_dtype, _stream(stream)), "mxfp8_gemm_multi")
+
+
+def mxfp8_act_grad_quantize(dh: torch.Tensor, z: torch.Tensor, act: int, orientation: int, scale_rule: int, elem: int,
+                            q_row, s_row, q_col, s_col, sf_layout: int, stream=None) -> None:
+    rows, cols = z.shape
+    assert z.is_contiguous() and dh.is_contiguous() and dh.shape == z.shape and dh.dtype == z.dtype
+    _check(lib().mxfp8_act_grad_quantize(_ptr(dh), _ptr(z), _dtype_code(z), rows, cols, act, orientation, scale_rule, elem,
+                                         _ptr(q_row), _ptr(s_row), _ptr(q_col), _ptr(s_col), sf_layout,
+                                         _stream(stream)), "mxfp8_act_grad_quantize")
 
 
 def mxfp8_act_quantize(src: torch.Tensor, act: int, orientation: int, scale_rule: int, elem: int,

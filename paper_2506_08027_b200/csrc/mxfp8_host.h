@@ -53,7 +53,7 @@ struct QuantizeItem {
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
                        int sf_layout, cudaStream_t stream, bool emulate = false, int act = MXFP8_ACT_NONE,
                        const float* rstd = nullptr, const void* gamma = nullptr, bool gated = false,
-                       const float* mean = nullptr, const void* beta = nullptr);
+                       const float* mean = nullptr, const void* beta = nullptr, const void* second_src = nullptr);
 int quantize_read_and_clear_status();
 
 // Device status word (bounded waits report here); defined in gemm.cu.

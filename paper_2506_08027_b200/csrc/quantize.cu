@@ -592,6 +592,34 @@ extern "C" int mxfp8_act_quantize(const void* src, int src_dtype, int64_t rows, 
     return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream), false, act);
 }
 
+extern "C" int mxfp8_act_grad_quantize(const void* dh, const void* z, int src_dtype, int64_t rows, int64_t cols, int act,
+                                       int orientation, int scale_rule, int elem,
+                                       void* q_row, void* s_row, void* q_col, void* s_col,
+                                       int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    if (act < MXFP8_ACT_RELU || act > MXFP8_ACT_GELU_TANH) return MXFP8_ERR_ENUM;
+    if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
+    if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
+    if (!valid_elem(elem)) return MXFP8_ERR_ENUM;
+    if (sf_layout != MXFP8_SF_LINEAR && sf_layout != MXFP8_SF_SWIZZLED) return MXFP8_ERR_ENUM;
+    if (!dh || !z) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_ROW) && (!q_row || !s_row)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col || !s_col)) return MXFP8_ERR_NULL;
+    if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_ROW) && (cols % 32)) return MXFP8_ERR_SHAPE;
+    if ((orientation & MXFP8_COL) && (rows % 32)) return MXFP8_ERR_SHAPE;
+    if (!aligned16(dh) || !aligned16(z)) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_ROW) && (!aligned16(q_row) || !aligned16(s_row))) return MXFP8_ERR_ALIGN;
+    if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
+    if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
+    // the z tile rides the ring and is overwritten by act'(z) * dh; dh arrives through the second tensor map
+    const QuantizeItem item{z, rows, cols, q_row, s_row, q_col, s_col};
+    return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, static_cast<cudaStream_t>(stream), false,
+                              4 + act, nullptr, nullptr, false, nullptr, nullptr, dh);
+}
+
 namespace mxfp8 {
 namespace {
 // Row statistics of mxfp8_rmsnorm_quantize_static: 65536 rows x 4 bytes = 256 KB that live in the module image.

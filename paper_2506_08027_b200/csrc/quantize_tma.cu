@@ -63,7 +63,7 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
 
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
                        int sf_layout, cudaStream_t stream, bool emulate, int act, const float* rstd, const void* gamma,
-                       bool gated, const float* mean, const void* beta)
+                       bool gated, const float* mean, const void* beta, const void* second_src)
 {
     if (count < 1 || count > QT_MAX_TENSORS) return MXFP8_ERR_UNSUPPORTED;
     const bool bf = src_dtype == MXFP8_BF16;
@@ -77,9 +77,17 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
     p.mean = mean;
     p.beta = beta;
     p.glu_cols = gated ? (int)items[0].cols : 0;     // gated: one tensor, source [rows, 2 * cols]
+    p.up_map = second_src ? 1 : 0;                   // two sources of one shape: the second one rides in map 1
     int64_t tiles = 0;
     for (int i = 0; i < QT_MAX_TENSORS; ++i) {
         const QuantizeItem& it = items[i < count ? i : 0];   // unused slots repeat the first tensor: every map stays valid
+        if (second_src && i == 1) {
+            if (count != 1 || gated) return MXFP8_ERR_UNSUPPORTED;
+            if (!make_map_2d(&ms.m[1], bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
+                             const_cast<void*>(second_src), (uint64_t)it.cols, (uint64_t)it.rows, t_cols, T_ROWS))
+                return MXFP8_ERR_CUDA;
+            continue;
+        }
         if (!make_map_2d(&ms.m[i], bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
                          const_cast<void*>(it.src), (uint64_t)(gated ? 2 * it.cols : it.cols), (uint64_t)it.rows, t_cols, T_ROWS))
             return MXFP8_ERR_CUDA;

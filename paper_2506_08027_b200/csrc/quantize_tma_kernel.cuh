@@ -44,6 +44,9 @@ struct QParams {
     uint8_t* s_col;
 };
 
+// ACT codes above this offset stand for the derivative of the activation (backward pass: act'(z) * dh)
+constexpr int ACT_GRAD = 4;
+
 // Elementwise activation ahead of the conversion (Sec. 3.2 keeps the activation function in high
 // precision; its result is what gets converted): evaluated in FP32.  relu(x) = x > 0 ? x : 0 (NaN -> 0).
 template <int ACT>
@@ -56,6 +59,17 @@ __device__ __forceinline__ float apply_act(float x)
         // 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)), u = sqrt(2/pi) (x + 0.044715 x^3)
         const float u2 = 1.5957691216057308f * (x + 0.044715f * x * x * x);
         return __fdividef(x, 1.f + __expf(-u2));
+    } else if constexpr (ACT == ACT_GRAD + MXFP8_ACT_RELU) return x > 0.f ? 1.f : 0.f;
+    else if constexpr (ACT == ACT_GRAD + MXFP8_ACT_RELU2) return x > 0.f ? 2.f * x : 0.f;
+    else if constexpr (ACT == ACT_GRAD + MXFP8_ACT_SILU) {
+        const float sg = __fdividef(1.f, 1.f + __expf(-x));
+        return sg * (1.f + x * (1.f - sg));
+    } else if constexpr (ACT == ACT_GRAD + MXFP8_ACT_GELU_TANH) {
+        // with s = 1 / (1 + exp(-2u)): 0.5 (1 + tanh u) = s and 1 - tanh^2 u = 4 s (1 - s), so
+        // gelu'(x) = s + x s (1 - s) * 2 sqrt(2/pi) (1 + 3 * 0.044715 x^2)
+        const float u2 = 1.5957691216057308f * (x + 0.044715f * x * x * x);
+        const float sg = __fdividef(1.f, 1.f + __expf(-u2));
+        return sg + x * sg * (1.f - sg) * (1.5957691216057308f * (1.f + 0.134145f * x * x));
     } else return x;
 }
 
@@ -162,6 +176,7 @@ struct QBatch {
     const float* mean;                    // layer normalisation: the row means (subtracted first) and the per-column bias in the
     const void* beta;                     //   source dtype (added last); both null for RMS normalisation
     int glu_cols;                         // gated activation: the source is [rows, 2 * glu_cols] = (gate | up); 0 when unused
+    int up_map;                           // two-source launches: tensor map of the second factor (1), or 0 when it is the up half of the first
     int count;
     int tile_start[QT_MAX_TENSORS + 1];   // first tile of each tensor; [count] = all tiles
     QParams t[QT_MAX_TENSORS];
@@ -510,7 +525,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         const uint32_t b = smem_addr(&bars[2]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(up_buf)), "l"(&maps.m[0]), "r"(b), "r"(glu_cols + (t % tx) * T_COLS), "r"((t / tx) * T_ROWS)
+                     ::"r"(smem_addr(up_buf)), "l"(&maps.m[batch.up_map]), "r"(b), "r"(glu_cols + (t % tx) * T_COLS), "r"((t / tx) * T_ROWS)
                      : "memory");
     };
     // bounded wait on one of the barriers: false when the limit passed
@@ -568,7 +583,12 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
                 case MXFP8_ACT_RELU: glu_slab<MXFP8_ACT_RELU, BF>(mine, mine_up); break;
                 case MXFP8_ACT_RELU2: glu_slab<MXFP8_ACT_RELU2, BF>(mine, mine_up); break;
                 case MXFP8_ACT_SILU: glu_slab<MXFP8_ACT_SILU, BF>(mine, mine_up); break;
-                default: glu_slab<MXFP8_ACT_GELU_TANH, BF>(mine, mine_up); break;
+                case MXFP8_ACT_GELU_TANH: glu_slab<MXFP8_ACT_GELU_TANH, BF>(mine, mine_up); break;
+                // backward of an activation: the slot holds z, up_buf holds dh; the slot becomes act'(z) * dh
+                case ACT_GRAD + MXFP8_ACT_RELU: glu_slab<ACT_GRAD + MXFP8_ACT_RELU, BF>(mine, mine_up); break;
+                case ACT_GRAD + MXFP8_ACT_RELU2: glu_slab<ACT_GRAD + MXFP8_ACT_RELU2, BF>(mine, mine_up); break;
+                case ACT_GRAD + MXFP8_ACT_SILU: glu_slab<ACT_GRAD + MXFP8_ACT_SILU, BF>(mine, mine_up); break;
+                default: glu_slab<ACT_GRAD + MXFP8_ACT_GELU_TANH, BF>(mine, mine_up); break;
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncthreads();                     // every warp has consumed the up tile: fetch the next one under the conversion
@@ -710,7 +730,7 @@ cudaError_t launch_o(int orientation, const QMaps& ms, const QBatch& p, cudaStre
 template <int ELEM>
 cudaError_t quantize_tma_launch(bool bf16_src, int orientation, bool emulate, const QMaps& ms, const QBatch& p, cudaStream_t st)
 {
-    if (p.glu_cols)
+    if (p.glu_cols || p.up_map)
         return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, PRO_GLU>(orientation, ms, p, st) : launch_o<MXFP8_FP32, ELEM, false, PRO_GLU>(orientation, ms, p, st);
     if (p.rstd != nullptr || p.act != MXFP8_ACT_NONE)
         return bf16_src ? launch_o<MXFP8_BF16, ELEM, false, PRO_ELEMENTWISE>(orientation, ms, p, st)
