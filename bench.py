@@ -131,6 +131,13 @@ def oracle_sample_seconds(sample_rows: int = 256):
         q[name, "c"] = orc.quantize_threads(t, orc.COL, orc.RULE_PAPER, orc.E4M3, threads)
     t_cast = time.perf_counter() - t0
     cast_full = t_cast * (T * H + F * H + T * F) / float(r * H + r * H + r * F)
+    # the same conversion on ONE thread (256 rows of dY, both orientations): the oracle's scalar rate
+    one = dy[:min(r, 256)]
+    t1 = time.perf_counter()
+    orc.quantize(one, orc.ROW, orc.RULE_PAPER, orc.E4M3)
+    orc.quantize(one, orc.COL, orc.RULE_PAPER, orc.E4M3)
+    t_one = time.perf_counter() - t1
+    cast_gbs_one_thread = one.size * (2 + 2 * (1 + 1 / 32)) / t_one / 1e9
     t0 = time.perf_counter()
     if r == T:
         # the whole step: all three products in FP64 over the decoded operands (+ the |A||B| bound products)
@@ -149,7 +156,7 @@ def oracle_sample_seconds(sample_rows: int = 256):
         desc = ("%d rows of X, W, dY quantized in both orientations on %d threads; %dx%dx%d FP64 product "
                 "(+|A||B| bound product) via numpy; scaled linearly to the full step" % (r, threads, r, r, H))
     oracle_sample_seconds.split = {   # the two halves of the metric for the oracle (same byte and FLOP counts as the GPU arm)
-        "cast_gbs": CAST_BYTES / cast_full / 1e9, "gemm_tflops": STEP_FLOP / gemm_full / 1e12,
+        "cast_gbs": CAST_BYTES / cast_full / 1e9, "cast_gbs_one_thread": cast_gbs_one_thread, "gemm_tflops": STEP_FLOP / gemm_full / 1e12,
         "cast_seconds_full_step": cast_full, "gemm_seconds_full_step": gemm_full}
     return t_cast + t_gemm, cast_full + gemm_full, desc, threads
 
