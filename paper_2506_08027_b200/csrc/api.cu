@@ -287,8 +287,16 @@ extern "C" int mxfp8_linear_host(const void* x_host, const void* w_host, const v
     const int64_t s_row_chunk_x = (Tc / 128) * ((H / 32 + 3) / 4) * 512;    // bytes of swizzled row scales per chunk of X
     const int64_t s_row_chunk_dy = (Tc / 128) * ((F / 32 + 3) / 4) * 512;   // ... and of dY
     const size_t wb = (size_t)F * H * 2;
-#define MXFP8_TRY(call) do { if ((call) != cudaSuccess) return MXFP8_ERR_CUDA; } while (0)
-#define MXFP8_RC(call) do { const int rc_ = (call); if (rc_ != MXFP8_OK) return rc_; } while (0)
+    // A failure half way leaves copies to and from the caller's buffers queued on three streams: wait for them before
+    // handing the buffers back with the error.
+    auto fail = [&](int rc) {
+        cudaStreamSynchronize(hp->in);
+        cudaStreamSynchronize(st);
+        cudaStreamSynchronize(hp->out);
+        return rc;
+    };
+#define MXFP8_TRY(call) do { if ((call) != cudaSuccess) return fail(MXFP8_ERR_CUDA); } while (0)
+#define MXFP8_RC(call) do { const int rc_ = (call); if (rc_ != MXFP8_OK) return fail(rc_); } while (0)
     // uploads on the helper stream, behind whatever the caller's stream holds: W, then X and dY chunk by chunk
     MXFP8_TRY(cudaEventRecord(hp->start, st));
     MXFP8_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
