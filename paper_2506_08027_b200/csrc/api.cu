@@ -110,6 +110,8 @@ extern "C" int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t 
     if (!src_host || !dev_ws) return MXFP8_ERR_NULL;
     if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
+    if ((orientation & MXFP8_ROW) && (!q_row_host || !s_row_host)) return MXFP8_ERR_NULL;
+    if ((orientation & MXFP8_COL) && (!q_col_host || !s_col_host)) return MXFP8_ERR_NULL;
     if (rows <= 0 || cols <= 0) return MXFP8_ERR_SHAPE;
     if (dev_ws_bytes < mxfp8_quantize_host_ws_bytes(src_dtype, rows, cols, orientation)) return MXFP8_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(dev_ws) & 255u) != 0) return MXFP8_ERR_ALIGN;
@@ -126,17 +128,18 @@ extern "C" int mxfp8_quantize_host(const void* src_host, int src_dtype, int64_t 
             d_q[o] = p; p += up256(n);
             d_s[o] = p; p += up256(mxfp8_scale_bytes(rows, cols, o + 1, MXFP8_SF_SWIZZLED));
         }
-    if (cudaMemcpyAsync(d_src, src_host, n * esz, cudaMemcpyHostToDevice, st) != cudaSuccess) return MXFP8_ERR_CUDA;
+    // whatever fails after the first copy has been queued: wait for the stream before the caller gets its buffers back
+    auto fail = [&](int rc) { cudaStreamSynchronize(st); return rc; };
+    if (cudaMemcpyAsync(d_src, src_host, n * esz, cudaMemcpyHostToDevice, st) != cudaSuccess) return fail(MXFP8_ERR_CUDA);
     const int rc = mxfp8_quantize(d_src, src_dtype, rows, cols, orientation, scale_rule, elem,
                                   d_q[0], d_s[0], d_q[1], d_s[1], sf_layout, stream);
-    if (rc != MXFP8_OK) return rc;
+    if (rc != MXFP8_OK) return fail(rc);
     void* h_q[2] = {q_row_host, q_col_host};
     void* h_s[2] = {s_row_host, s_col_host};
     for (int o = 0; o < 2; ++o)
         if (orientation & (o + 1)) {
-            if (!h_q[o] || !h_s[o]) return MXFP8_ERR_NULL;
-            if (cudaMemcpyAsync(h_q[o], d_q[o], n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXFP8_ERR_CUDA;
-            if (cudaMemcpyAsync(h_s[o], d_s[o], s_bytes[o], cudaMemcpyDeviceToHost, st) != cudaSuccess) return MXFP8_ERR_CUDA;
+            if (cudaMemcpyAsync(h_q[o], d_q[o], n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(MXFP8_ERR_CUDA);
+            if (cudaMemcpyAsync(h_s[o], d_s[o], s_bytes[o], cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(MXFP8_ERR_CUDA);
         }
     return cudaStreamSynchronize(st) == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
 }
