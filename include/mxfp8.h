@@ -371,7 +371,8 @@ int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq, const voi
  * rank launches, and waits for all ranks' launches before reading its own buffer; the order in
  * which different launches' contributions are added is not fixed (two contributions: exact and order-free;
  * more: equal up to FP32 rounding order).  M a multiple of 128 * num_owners, N of 4 (16 with an MN-major B), K of 32.
- * Nothing is allocated; never waits on another GPU inside the kernel.
+ * Nothing is allocated; never waits on another GPU inside the kernel.  With num_owners = 1 and a local buffer the
+ * call is a product that accumulates into an FP32 output (D += A * B^T): WGRAD summed over micro-batches.
  */
 /* Lets kernels launched on the current device read and write memory of `peer_device` (needed once per pair of
  * devices before a pointer into the peer's memory is given to mxfp8_gemm_reduce_scatter).  MXFP8_OK when access
