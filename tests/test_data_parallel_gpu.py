@@ -120,6 +120,23 @@ def test_reduce_scatter_over_emulated_ranks(world, Tr, H, F):
     check_gemm_tolerance(got, d64, world * sabs, "sum of %d partial products" % world)
 
 
+@pytest.mark.parametrize("tile", ["256p", "192p", "128"])
+def test_reduce_scatter_with_every_tile_shape_built_for_it(tile, monkeypatch):
+    """The three tile shapes of this mode forced in turn (the library reads MXFP8_GEMM_TILE at every launch): owners' row
+    ranges that start inside a 256-row pair tile, a ragged last column tile."""
+    import torch
+    from helpers import gpu_gemm
+    monkeypatch.setenv("MXFP8_GEMM_TILE", tile)
+    world, Tr, H, F = 3, 256, 336, 384                     # 128 rows per owner: every pair tile spans two owners
+    owners = [torch.zeros(F // world, H, dtype=torch.float32, device="cuda") for _ in range(world)]
+    acc = np.zeros((F, H), dtype=np.float32)
+    for r in range(world):
+        dyq, xq = _wgrad_operands(Tr, H, F, 500 + 10 * r)
+        _scatter(dyq, xq, owners, r)
+        acc = acc + gpu_gemm(dyq[0], dyq[1], xq[0], xq[1], "mn", "mn")
+    assert np.array_equal(np.concatenate([o.cpu().numpy() for o in owners]), acc)
+
+
 def test_reduce_scatter_argument_errors():
     import torch
     from paper_2506_08027_b200 import binding as B
