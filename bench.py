@@ -75,7 +75,7 @@ class ClockSampler(threading.Thread):
     def run(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             for line in self.proc.stdout:
                 parts = [p.strip() for p in line.split(",")]
@@ -337,7 +337,11 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
         clocks["sm_mhz_inside_gemm_kernel"] = round(gemm_clock_mhz, 1)
-        clocks["note"] = ("sm_mhz is the driver's sampled clock (200 ms period, longer than the timed region); sm_mhz_inside_gemm_kernel is "
+        if clocks.get("sm_max_mhz") and gemm_clock_mhz < 0.9 * clocks["sm_max_mhz"] and "sw_power_cap" not in clocks["reasons"]:
+            # the board's power limit acts inside the sub-millisecond GEMM bursts; the sampler sees mostly the gaps between passes
+            clocks["reasons_note"] = ("no sample fell inside a GEMM launch; longer runs (--steps 200) report sw_power_cap, the only "
+                                      "reason ever seen on this path")
+        clocks["note"] = ("sm_mhz is the driver's sampled clock (tens of milliseconds per sample, longer than a step); sm_mhz_inside_gemm_kernel is "
                           "SM cycles / wall time read by the last timed GEMM launch itself (%.0f us alive)" % gemm_probe_us)
     if world > 1:
         dist.barrier()
