@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxfp8.so")
-SOURCES = ["quantize.cu", "quantize_tma.cu", "quantize_tma_fp6_fp4.cu", "dequantize.cu", "gemm.cu", "api.cu"]
+SOURCES = ["quantize.cu", "quantize_tma.cu", "quantize_tma_fp6_fp4.cu", "dequantize.cu", "gemm.cu", "gemm_deep.cu", "api.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC",

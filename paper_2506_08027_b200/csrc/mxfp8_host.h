@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/mxfp8.h"
 
@@ -28,6 +29,95 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long l
     err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (err == cudaSuccess) __atomic_fetch_or(&done, bit, __ATOMIC_RELEASE);
     return err;
+}
+
+// A value per device that costs driver calls to find (multiprocessor count, the address of a __device__ symbol:
+// every device holds its own copy of each symbol, at its own address).  get() fills the current device's slot on
+// first use, under a lock, and afterwards reads it without one.  `fill(device, value)` returns false on failure,
+// which is not cached.  The device index can be given (tests); by default it is the calling thread's current device.
+template <typename T>
+class PerDeviceCache {
+public:
+    static constexpr int MAX_DEVICES = 64;
+    template <typename Fill>
+    bool get(T& out, Fill fill, int device = -1)
+    {
+        if (device < 0 && cudaGetDevice(&device) != cudaSuccess) return false;
+        if (device < 0 || device >= MAX_DEVICES) return false;
+        const unsigned long long bit = 1ull << device;
+        if (!(__atomic_load_n(&done_, __ATOMIC_ACQUIRE) & bit)) {
+            while (__atomic_exchange_n(&lock_, 1, __ATOMIC_ACQUIRE)) {}
+            bool ok = true;
+            if (!(done_ & bit)) {
+                T v{};
+                ok = fill(device, v);
+                if (ok) {
+                    slot_[device] = v;
+                    __atomic_fetch_or(&done_, bit, __ATOMIC_RELEASE);
+                }
+            }
+            __atomic_store_n(&lock_, 0, __ATOMIC_RELEASE);
+            if (!ok) return false;
+        }
+        out = slot_[device];
+        return true;
+    }
+
+private:
+    T slot_[MAX_DEVICES] = {};
+    unsigned long long done_ = 0;
+    int lock_ = 0;
+};
+
+// Encoded TMA tensor maps, kept in static storage (nothing is allocated) and keyed by every argument of the encode call.  A map is a pure
+// function of those arguments (address, extents, pitches, box, types), so a cached one is valid for as long as
+// the caller's buffer is; the cache owns nothing.  Direct-mapped: a colliding key replaces the entry.
+// One driver call per map costs about a microsecond, and a launch needs 5 to 15 of them.
+struct TensorMapKey {
+    const void* base;
+    uint64_t dim[3], stride[2];
+    uint32_t box[3];
+    uint32_t dtype, rank, swizzle, l2;
+};
+template <typename Map>
+class TensorMapCache {
+public:
+    template <typename Encode>
+    bool get(const TensorMapKey& key, Map* out, Encode encode)
+    {
+        const unsigned char* b = reinterpret_cast<const unsigned char*>(&key);
+        uint64_t h = 1469598103934665603ull;
+        for (size_t i = 0; i < sizeof(key); ++i) h = (h ^ b[i]) * 1099511628211ull;
+        Entry& e = entries_[h % SLOTS];
+        while (__atomic_exchange_n(&lock_, 1, __ATOMIC_ACQUIRE)) {}
+        const bool hit = e.valid && memcmp(&e.key, &key, sizeof(key)) == 0;
+        if (hit) *out = e.map;
+        __atomic_store_n(&lock_, 0, __ATOMIC_RELEASE);
+        if (hit) return true;
+        if (!encode(out)) return false;
+        while (__atomic_exchange_n(&lock_, 1, __ATOMIC_ACQUIRE)) {}
+        e.key = key;
+        e.map = *out;
+        e.valid = true;
+        __atomic_store_n(&lock_, 0, __ATOMIC_RELEASE);
+        return true;
+    }
+
+private:
+    static constexpr int SLOTS = 256;
+    struct Entry { TensorMapKey key; Map map; bool valid; };
+    Entry entries_[SLOTS] = {};
+    int lock_ = 0;
+};
+inline TensorMapKey tensor_map_key(const void* base, uint32_t dtype, uint32_t rank, const uint64_t* dims, const uint64_t* strides,
+                                   const uint32_t* box, uint32_t swizzle, uint32_t l2)
+{
+    TensorMapKey k;
+    memset(&k, 0, sizeof(k));   // padding bytes take part in the comparison
+    k.base = base; k.dtype = dtype; k.rank = rank; k.swizzle = swizzle; k.l2 = l2;
+    for (uint32_t i = 0; i < rank; ++i) { k.dim[i] = dims[i]; k.box[i] = box[i]; }
+    for (uint32_t i = 0; i + 1 < rank; ++i) k.stride[i] = strides[i];
+    return k;
 }
 
 // Launch accounting (mxfp8_launch_count).

@@ -45,9 +45,14 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t esz, void* bas
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * esz};
     const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    static TensorMapCache<CUtensorMap> cache;
+    const uint64_t kd[2] = {cols, rows}, ks[1] = {cols * esz};
+    return cache.get(tensor_map_key(base, (uint32_t)dt, 2, kd, ks, box, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B), map,
+                     [&](CUtensorMap* m) {
+                         const cuuint32_t estr[2] = {1, 1};
+                         return fn(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                     });
 }
 
 }  // namespace
@@ -80,7 +85,11 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
     p.up_map = second_src ? 1 : 0;                   // two sources of one shape: the second one rides in map 1
     int64_t tiles = 0;
     for (int i = 0; i < QT_MAX_TENSORS; ++i) {
-        const QuantizeItem& it = items[i < count ? i : 0];   // unused slots repeat the first tensor: every map stays valid
+        const QuantizeItem& it = items[i < count ? i : 0];
+        if (i >= count && !(second_src && i == 1)) {   // unused slots repeat the first tensor's map: every map stays valid
+            ms.m[i] = ms.m[0];
+            continue;
+        }
         if (second_src && i == 1) {
             if (count != 1 || gated) return MXFP8_ERR_UNSUPPORTED;
             if (!make_map_2d(&ms.m[1], bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf ? 2 : 4,
@@ -105,12 +114,15 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
         if (tiles >= 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
     }
     for (int i = count; i <= QT_MAX_TENSORS; ++i) p.tile_start[i] = (int)tiles;
-    static int* status_word = [] {
-        void* ptr = nullptr;
-        return cudaGetSymbolAddress(&ptr, g_quantize_status) == cudaSuccess ? static_cast<int*>(ptr) : nullptr;
-    }();
-    if (!status_word) return MXFP8_ERR_CUDA;
-    p.status = status_word;
+    // every device holds its own copy of the status word, at its own address
+    static PerDeviceCache<int*> status_word;
+    if (!status_word.get(p.status, [](int, int*& addr) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_quantize_status) != cudaSuccess) return false;
+            addr = static_cast<int*>(ptr);
+            return true;
+        }))
+        return MXFP8_ERR_CUDA;
     cudaError_t err;
     switch (elem) {
         case MXFP8_E4M3: err = quantize_tma_launch<MXFP8_E4M3>(bf, orientation, emulate, ms, p, stream); break;

@@ -687,15 +687,14 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     }
 }
 
+// Multiprocessors of the current device (looked up once per device)
 int qt_sm_count()
 {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return v;
-    }();
-    return n;
+    static PerDeviceCache<int> cache;
+    int n = 0;
+    return cache.get(n, [](int dev, int& v) {
+               return cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0;
+           }) ? n : 0;
 }
 
 template <int DTYPE, int ELEM, bool R, bool C, bool EMU, int PRO>
@@ -709,7 +708,9 @@ cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
     cudaError_t err = ensure_dynamic_smem(kernel, SMEM_USED, smem_set);
     if (err != cudaSuccess) return err;
     const int tiles = p.tile_start[p.count];
-    const int max_ctas = qt_sm_count() * (GLU ? 2 : 3);
+    const int sms = qt_sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
+    const int max_ctas = sms * (GLU ? 2 : 3);
     const int grid = tiles < max_ctas ? tiles : max_ctas;
     kernel<<<grid, QT_THREADS, SMEM_USED, stream>>>(ms, p);
     count_launch(1);
