@@ -72,70 +72,75 @@ def lib() -> ctypes.CDLL:
             path = _build.build()
         if not os.path.exists(path):
             raise ImportError("libmxfp8.so is missing: run `python -m paper_2506_08027_b200.build`")
-        L = ctypes.CDLL(path)
-        i, i64, p, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
-        L.mxfp8_quantize.restype = i
-        L.mxfp8_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_dequantize.restype = i
-        L.mxfp8_dequantize.argtypes = [p, p, i64, i64, i, i, i, p, i, p]
-        L.mxfp8_gemm.restype = i
-        L.mxfp8_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, p, i, ctypes.POINTER(_Epilogue), p, sz, p]
-        L.mxfp8_scale_bytes.restype = sz
-        L.mxfp8_scale_bytes.argtypes = [i64, i64, i, i]
-        L.mxfp8_sf_offset.restype = i64
-        L.mxfp8_sf_offset.argtypes = [i64, i64, i64, i]
-        L.mxfp8_gemm_workspace_bytes.restype = sz
-        L.mxfp8_gemm_workspace_bytes.argtypes = [i64, i64, i64, i, i]
-        L.mxfp8_device_status.restype = i
-        L.mxfp8_device_status.argtypes = [p]
-        L.mxfp8_status_string.restype = ctypes.c_char_p
-        L.mxfp8_status_string.argtypes = [i]
-        L.mxfp8_launch_count.restype = i64
-        L.mxfp8_launch_count.argtypes = []
-        L.mxfp8_quantize_host_ws_bytes.restype = sz
-        L.mxfp8_quantize_host_ws_bytes.argtypes = [i, i64, i64, i]
-        L.mxfp8_quantize_host.restype = i
-        L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
-        L.mxfp8_fake_quantize.restype = i
-        L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
-        L.mxfp8_rmsnorm_quantize.restype = i
-        L.mxfp8_rmsnorm_quantize.argtypes = [p, i, i64, i64, p, ctypes.c_float, p, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_layernorm_quantize.restype = i
-        L.mxfp8_layernorm_quantize.argtypes = [p, i, i64, i64, p, p, ctypes.c_float, p, p, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_rmsnorm_quantize_static.restype = i
-        L.mxfp8_rmsnorm_quantize_static.argtypes = [p, i, i64, i64, p, ctypes.c_float, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_rmsnorm_quantize_static_max_rows.restype = i64
-        L.mxfp8_rmsnorm_quantize_static_max_rows.argtypes = []
-        L.mxfp8_glu_quantize.restype = i
-        L.mxfp8_glu_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_act_grad_quantize.restype = i
-        L.mxfp8_act_grad_quantize.argtypes = [p, p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_act_quantize.restype = i
-        L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
-        L.mxfp8_gemm_multi.restype = i
-        L.mxfp8_gemm_multi.argtypes = [ctypes.POINTER(_GemmProblem), i, i, p]
-        L.mxfp8_quantize_multi.restype = i
-        L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
-        L.mxfp8_grouped_gemm.restype = i
-        L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
-        L.mxfp8_gemm_last_clock.restype = i
-        L.mxfp8_gemm_last_clock.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
-        L.mxfp8_enable_peer_access.restype = i
-        L.mxfp8_enable_peer_access.argtypes = [i]
-        L.mxfp8_sf_concat_k.restype = i
-        L.mxfp8_sf_concat_k.argtypes = [p, i, i64, i64, p, p]
-        L.mxfp8_gemm_reduce_scatter.restype = i
-        L.mxfp8_gemm_reduce_scatter.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, ctypes.POINTER(ctypes.c_void_p), i, i, p]
-        L.mxfp8_linear_ws_bytes.restype = sz
-        L.mxfp8_linear_ws_bytes.argtypes = [i64, i64, i64]
-        L.mxfp8_linear.restype = i
-        L.mxfp8_linear.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
-        L.mxfp8_linear_host_ws_bytes.restype = sz
-        L.mxfp8_linear_host_ws_bytes.argtypes = [i64, i64, i64]
-        L.mxfp8_linear_host.restype = i
-        L.mxfp8_linear_host.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
-        _lib = L
+        _lib = load_library(path)
     return _lib
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    """dlopen a build of the library and declare every entry point's signature."""
+    L = ctypes.CDLL(path)
+    i, i64, p, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+    L.mxfp8_quantize.restype = i
+    L.mxfp8_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_dequantize.restype = i
+    L.mxfp8_dequantize.argtypes = [p, p, i64, i64, i, i, i, p, i, p]
+    L.mxfp8_gemm.restype = i
+    L.mxfp8_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, p, i, ctypes.POINTER(_Epilogue), p, sz, p]
+    L.mxfp8_scale_bytes.restype = sz
+    L.mxfp8_scale_bytes.argtypes = [i64, i64, i, i]
+    L.mxfp8_sf_offset.restype = i64
+    L.mxfp8_sf_offset.argtypes = [i64, i64, i64, i]
+    L.mxfp8_gemm_workspace_bytes.restype = sz
+    L.mxfp8_gemm_workspace_bytes.argtypes = [i64, i64, i64, i, i]
+    L.mxfp8_device_status.restype = i
+    L.mxfp8_device_status.argtypes = [p]
+    L.mxfp8_status_string.restype = ctypes.c_char_p
+    L.mxfp8_status_string.argtypes = [i]
+    L.mxfp8_launch_count.restype = i64
+    L.mxfp8_launch_count.argtypes = []
+    L.mxfp8_quantize_host_ws_bytes.restype = sz
+    L.mxfp8_quantize_host_ws_bytes.argtypes = [i, i64, i64, i]
+    L.mxfp8_quantize_host.restype = i
+    L.mxfp8_quantize_host.argtypes = [p, i, i64, i64, i, i, i, p, p, p, p, i, p, sz, p]
+    L.mxfp8_fake_quantize.restype = i
+    L.mxfp8_fake_quantize.argtypes = [p, i, i64, i64, i, i, i, p, p, p]
+    L.mxfp8_rmsnorm_quantize.restype = i
+    L.mxfp8_rmsnorm_quantize.argtypes = [p, i, i64, i64, p, ctypes.c_float, p, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_layernorm_quantize.restype = i
+    L.mxfp8_layernorm_quantize.argtypes = [p, i, i64, i64, p, p, ctypes.c_float, p, p, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_rmsnorm_quantize_static.restype = i
+    L.mxfp8_rmsnorm_quantize_static.argtypes = [p, i, i64, i64, p, ctypes.c_float, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_rmsnorm_quantize_static_max_rows.restype = i64
+    L.mxfp8_rmsnorm_quantize_static_max_rows.argtypes = []
+    L.mxfp8_glu_quantize.restype = i
+    L.mxfp8_glu_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_act_grad_quantize.restype = i
+    L.mxfp8_act_grad_quantize.argtypes = [p, p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_act_quantize.restype = i
+    L.mxfp8_act_quantize.argtypes = [p, i, i64, i64, i, i, i, i, p, p, p, p, i, p]
+    L.mxfp8_gemm_multi.restype = i
+    L.mxfp8_gemm_multi.argtypes = [ctypes.POINTER(_GemmProblem), i, i, p]
+    L.mxfp8_quantize_multi.restype = i
+    L.mxfp8_quantize_multi.argtypes = [ctypes.POINTER(_QuantizeItem), i, i, i, i, i, i, p]
+    L.mxfp8_grouped_gemm.restype = i
+    L.mxfp8_grouped_gemm.argtypes = [p, p, p, p, p, i, i, i64, i64, i64, i, i, i, p, i, p]
+    L.mxfp8_gemm_last_clock.restype = i
+    L.mxfp8_gemm_last_clock.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    L.mxfp8_enable_peer_access.restype = i
+    L.mxfp8_enable_peer_access.argtypes = [i]
+    L.mxfp8_sf_concat_k.restype = i
+    L.mxfp8_sf_concat_k.argtypes = [p, i, i64, i64, p, p]
+    L.mxfp8_gemm_reduce_scatter.restype = i
+    L.mxfp8_gemm_reduce_scatter.argtypes = [p, p, p, p, i64, i64, i64, i, i, i, i, ctypes.POINTER(ctypes.c_void_p), i, i, p]
+    L.mxfp8_linear_ws_bytes.restype = sz
+    L.mxfp8_linear_ws_bytes.argtypes = [i64, i64, i64]
+    L.mxfp8_linear.restype = i
+    L.mxfp8_linear.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
+    L.mxfp8_linear_host_ws_bytes.restype = sz
+    L.mxfp8_linear_host_ws_bytes.argtypes = [i64, i64, i64]
+    L.mxfp8_linear_host.restype = i
+    L.mxfp8_linear_host.argtypes = [p, p, p, i64, i64, i64, i, p, p, p, p, sz, p]
+    return L
 
 
 def status_string(status: int) -> str:

@@ -123,6 +123,9 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
             return true;
         }))
         return MXFP8_ERR_CUDA;
+#ifdef MXFP8_TEST_HOOKS
+    if (const char* skip = getenv("MXFP8_TEST_SKIP_TILE")) p.test_skip_tile = atoi(skip);
+#endif
     cudaError_t err;
     switch (elem) {
         case MXFP8_E4M3: err = quantize_tma_launch<MXFP8_E4M3>(bf, orientation, emulate, ms, p, stream); break;

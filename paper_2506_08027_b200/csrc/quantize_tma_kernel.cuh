@@ -32,7 +32,11 @@ constexpr int T_ROWS = 128;
 constexpr int T_BYTES = 256;                 // source bytes per tile row
 constexpr int IN_BYTES = T_ROWS * T_BYTES;   // 32 KB
 constexpr int QT_THREADS = 128;
+#ifdef MXFP8_TEST_HOOKS
+constexpr uint64_t QT_WAIT_LIMIT_NS = 5000000ull;      // test build: the bounded wait gives up after 5 ms
+#else
 constexpr uint64_t QT_WAIT_LIMIT_NS = 1000000000ull;
+#endif
 
 struct QParams {
     int64_t rows, cols;
@@ -170,6 +174,7 @@ __device__ __forceinline__ void glu_slab(uint8_t* gate, const uint8_t* up)
 constexpr int QT_MAX_TENSORS = 8;
 struct QBatch {
     int* status;                          // device status word of the library (bounded waits report here)
+    int test_skip_tile;                   // test builds only: 1 + index of the tile whose load is left out (0 = none)
     int act;                              // MXFP8_ACT_*: applied to every element before the conversion
     const float* rstd;                    // RMS normalisation ahead of the conversion (first tensor only): 1/rms per row,
     const void* gamma;                    //   and the per-column weight in the source dtype; both null when unused
@@ -512,6 +517,9 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     const int num_tiles = batch.tile_start[batch.count];
     int load_ti = 0;                          // tensor of the tile being loaded (tiles only move forward)
     auto issue_load = [&](int t, int buf) {   // one thread: tile t -> ring slot buf
+#ifdef MXFP8_TEST_HOOKS
+        if (batch.test_skip_tile && t == batch.test_skip_tile - 1) return;   // never issued: the consumer's bounded wait runs out
+#endif
         while (t >= batch.tile_start[load_ti + 1]) ++load_ti;
         const int lt = t - batch.tile_start[load_ti], tx = batch.t[load_ti].tiles_x;
         const uint32_t b = smem_addr(&bars[buf]);

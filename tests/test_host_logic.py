@@ -128,3 +128,19 @@ def test_argument_validation_of_the_widened_entry_points():
     assert ln(p, p, p, 128, 128, 128, 7, p, p, p, p, 1 << 30, None) == -2
     assert ln(p, p, p, 128, 128, 128, 0, p, p, p, ctypes.c_void_p(0x1100), 16, None) == -8
     assert B.status_string(-9).startswith("invalid values")
+
+
+def test_per_device_and_tensor_map_caches(tmp_path):
+    """The status-word / SM-count caches hand every device its own entry (device index given explicitly, no
+    GPU needed), and the tensor-map cache hits only on identical encode arguments."""
+    import subprocess
+    here = os.path.dirname(os.path.abspath(__file__))
+    root = os.path.dirname(here)
+    exe = str(tmp_path / "host_caches_test")
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    subprocess.check_call(["g++", "-std=c++17", "-O1", "-I" + os.path.join(root, "paper_2506_08027_b200", "csrc"),
+                           "-I" + os.path.join(cuda, "include"), os.path.join(here, "cpp", "host_caches_test.cpp"),
+                           "-L" + os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + os.path.join(cuda, "lib64"), "-o", exe])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert "all checks passed" in out.stdout
