@@ -1,10 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the MXFP8 hot path on B200: one training step of a linear layer.
 
-A "step" is one pass of the whole path over one batch of synthetic input, for the
-~800M-parameter GPT-style linear layer (tokens 8192, hidden 2048, FFN 8192): the three BF16
-tensors X, W, dY are each converted to MXFP8-E4M3 in both block orientations (one read each),
-then FPROP, DGRAD and WGRAD run as block-scaled MXFP8 GEMMs with BF16 output.
+One pass of the whole path over one batch of synthetic input, for the ~800M-parameter GPT-style
+linear layer (tokens 8192, hidden 2048, FFN 8192): the three BF16 tensors X, W, dY are each
+converted to MXFP8-E4M3 in both block orientations (one read each), then FPROP, DGRAD and WGRAD run
+as block-scaled MXFP8 GEMMs with BF16 output.  A pass takes 0.4 ms, far too short to time alone, so
+a "step" is PASSES_PER_STEP = 64 such passes back to back (64 micro-batches): the default 20 steps
+then keep the device busy for half a second, which is the power-capped steady state; the first 20
+passes after an idle gap are reported beside it as the burst figure.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -31,6 +34,7 @@ sys.path.insert(0, ROOT)
 T, H, F = 8192, 2048, 8192          # tokens, hidden, FFN of the benchmarked linear layer
 METRIC = "MXFP8 cast GB/s (% HBM peak); MXFP8 GEMM TFLOP/s (% dense FP8 peak)"
 WORKLOAD = "linear layer of a ~800M-param GPT: tokens 8192, hidden 2048, FFN 8192; quantize X,W,dY (both orientations) + fprop/dgrad/wgrad MXFP8 GEMMs, BF16 out"
+L2_NOTE = "inputs larger than L2: 192 MB of BF16 sources and 590 MB of outputs per pass"
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -44,9 +48,16 @@ NCU_TRAFFIC_GEMM_FPROP = 49.8e6 + 85.3e6
 NCU_TRAFFIC_GEMM_MULTI = 293.4e6 + 189.0e6          # the three-product launch of the step (dram read + write, ncu)
 NCU_TRAFFIC_QUANTIZE_STEP = 201.4e6 + 152.5e6       # the batched cast of X, W, dY (408.9 MB algorithmic; part of the output still in L2)
 
-STEP_FLOP = 3 * 2.0 * T * H * F                       # three GEMMs of 275 GFLOP
+PASSES_PER_STEP = 64                                  # micro-batches per timed step (see the module docstring)
+STEP_FLOP = 3 * 2.0 * T * H * F                       # one pass: three GEMMs of 275 GFLOP
 CAST_BYTES = (T * H + F * H + T * F) * (2 + 2 * (1 + 1 / 32))   # src + two orientations x (q + scales)
 GEMM_SHAPES = {"fprop": (T, F, H), "dgrad": (T, H, F), "wgrad": (F, H, T)}
+
+
+def bench_config(n_gpus: int) -> dict:
+    """The `config` object of the JSON line, the same for both arms."""
+    return {"workload": WORKLOAD, "passes_per_step": PASSES_PER_STEP, "l2": L2_NOTE,
+            "parallelism": "dp%d (independent batches, no collective)" % n_gpus}
 
 
 def measured_peaks():
@@ -146,7 +157,7 @@ def oracle_sample_seconds(sample_rows: int = 256):
         orc.gemm_f64(q["dy", "c"][0], q["dy", "c"][1], q["x", "c"][0], q["x", "c"][1], "mn", "mn")        # wgrad
         t_gemm = time.perf_counter() - t0
         gemm_full = t_gemm
-        desc = ("the whole step on the host: X, W, dY quantized in both orientations on %d threads (row slabs), then "
+        desc = ("the whole pass on the host: X, W, dY quantized in both orientations on %d threads (row slabs), then "
                 "fprop, dgrad, wgrad as FP64 products of the decoded operands (+ the |A||B| bound products) via numpy" % threads)
     else:
         # GEMM sample: r x r outputs of fprop over the full K = H (decoded FP64 operands, two products)
@@ -162,25 +173,29 @@ def oracle_sample_seconds(sample_rows: int = 256):
 
 
 def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores: every step is ONE whole pass of the workload
+    (all casts on all threads, the three products in FP64 through numpy), i.e. one of the PASSES_PER_STEP
+    micro-batches that a step of the GPU arm holds; the rate is per pass either way."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample_seconds(64)
-    times, full = [], []
+        oracle_sample_seconds(256)
+    times = []
     desc, threads = "", 1
     for _ in range(args.steps):
-        s, f, desc, threads = oracle_sample_seconds(1024)
-        times.append(s)
-        full.append(f)
-    est = statistics.mean(full)
-    value = STEP_FLOP / est / 1e12
+        _, sec_pass, desc, threads = oracle_sample_seconds(T)     # casts + products; drawing the inputs is not timed
+        times.append(sec_pass)
+    sec = statistics.mean(times)
+    value = STEP_FLOP / sec / 1e12
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sampled": True},
-        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "config": bench_config(args.gpus),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+                         "sample": "each step: one of the %d passes of a step, whole -- %s" % (PASSES_PER_STEP, desc),
+                         "median_seconds_per_pass": statistics.median(times), "best_seconds_per_pass": min(times)},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -201,7 +216,8 @@ def max_over_ranks(ms: float, world: int, device) -> float:
 
 
 def whole_job_value(world: int, ms_step: float) -> float:
-    """TFLOP/s of the whole job: every rank runs the same step on its own batch (weak scaling)."""
+    """TFLOP/s of the whole job: every rank runs the same passes on its own batches (weak scaling).
+    ms_step is the time of ONE pass."""
     return world * STEP_FLOP / (ms_step * 1e-3) / 1e12
 
 
@@ -245,9 +261,24 @@ def run_ours(args):
         (qdY[2], qdY[3], qX[2], qX[3], F, H, T, B.MN_MAJOR, B.MN_MAJOR, E, E, dW),      # wgrad
     ])
 
-    def step():
+    def one_pass():
         B.mxfp8_quantize_multi(items, B.BF16, B.BOTH, P, E, S)
         B.mxfp8_gemm_multi(gemms, B.BF16)
+
+    def step():
+        for _ in range(PASSES_PER_STEP):
+            one_pass()
+
+    def passes_with_events(n):
+        """n passes with an event before and after each of the two launches -> (cast ms, gemm ms, pass ms) lists."""
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n)]
+        for k in range(n):
+            ev[k][0].record(); B.mxfp8_quantize_multi(items, B.BF16, B.BOTH, P, E, S)
+            ev[k][1].record(); B.mxfp8_gemm_multi(gemms, B.BF16)
+            ev[k][2].record()
+        torch.cuda.synchronize()
+        return ([e[0].elapsed_time(e[1]) for e in ev], [e[1].elapsed_time(e[2]) for e in ev],
+                [e[0].elapsed_time(e[2]) for e in ev])
 
     def step_by_kernel(ev):
         # the same work with one launch per GEMM and an event before every launch: per-kernel durations
@@ -262,6 +293,15 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- burst figure: the first 20 passes after an idle gap (boost clock, before the power cap bites)
+    for _ in range(3):
+        one_pass()
+    step_by_kernel([torch.cuda.Event(enable_timing=True) for _ in range(5)])      # first use of the single-product kernels
+    barrier()
+    time.sleep(0.5)
+    b_cast, b_gemm, b_pass = passes_with_events(20)
+    burst_clock_mhz, _ = B.mxfp8_gemm_last_clock()
+
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
@@ -273,7 +313,7 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)
 
-    # ---- timed region 1: K whole steps, device time, max over ranks
+    # ---- timed region 1: K steps of PASSES_PER_STEP passes, device time, max over ranks (no events inside)
     launches0 = B.mxfp8_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -285,28 +325,23 @@ def run_ours(args):
     launches = B.mxfp8_launch_count() - launches0
     ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     ms_step = ms_total / args.steps
+    ms_pass = ms_step / PASSES_PER_STEP
     # the SM clock the last GEMM launch of the timed region really ran at (cycles / nanoseconds read inside the kernel)
     gemm_clock_mhz, gemm_probe_us = B.mxfp8_gemm_last_clock()
 
-    # ---- timed region 2: the same steps with an event before every launch -> per-kernel durations
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
-    step_by_kernel([torch.cuda.Event(enable_timing=True) for _ in range(5)])      # first use of the single-product kernels: untimed
-    for k in range(args.steps):
+    # ---- timed region 2 (continues the steady state): per-launch events on every pass of a few more steps
+    n_ev = PASSES_PER_STEP * max(1, min(args.steps, 8))
+    s_cast, s_gemm, s_pass = passes_with_events(n_ev)
+    steady_clock_mhz, _ = B.mxfp8_gemm_last_clock()
+    cast_ms = statistics.median(s_cast)
+    gemm_multi_ms = statistics.median(s_gemm)
+    # ---- timed region 3: the three GEMMs launched one by one (per-product breakdown)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(PASSES_PER_STEP)]
+    for k in range(PASSES_PER_STEP):
         step_by_kernel(evs[k])
     torch.cuda.synchronize()
-    dur = [[evs[k][i].elapsed_time(evs[k][i + 1]) for i in range(4)] for k in range(args.steps)]
-    mean = [statistics.mean(d[i] for d in dur) for i in range(4)]
-    cast_ms = mean[0]
-    gemm_ms = dict(zip(("fprop", "dgrad", "wgrad"), mean[1:4]))
-    # ---- timed region 3: the step as timed, with an event around each of its two launches
-    ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    for k in range(args.steps):
-        ev3[k][0].record(); B.mxfp8_quantize_multi(items, B.BF16, B.BOTH, P, E, S)
-        ev3[k][1].record(); B.mxfp8_gemm_multi(gemms, B.BF16)
-        ev3[k][2].record()
-    torch.cuda.synchronize()
-    cast_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev3)
-    gemm_multi_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev3)
+    dur = [[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]
+    gemm_ms = dict(zip(("fprop", "dgrad", "wgrad"), (statistics.median(d[i] for d in dur) for i in (1, 2, 3))))
     status = B.mxfp8_device_status()
 
     # ---- end to end through the host-buffer C-ABI call (pinned host memory, copies inside)
@@ -318,31 +353,30 @@ def run_ours(args):
         hdw = torch.empty((F, H), dtype=torch.bfloat16).pin_memory()
         ws = torch.empty(B.mxfp8_linear_host_ws_bytes(T, H, F), dtype=torch.uint8, device=dev)
         B.mxfp8_linear_host(hx, hw, hdy, P, hy, hdx, hdw, ws)
-        n_e2e = max(1, min(args.steps, 5))
+        n_e2e = PASSES_PER_STEP                      # one step of the end-to-end path (about a third of a second)
         barrier()
-        t0 = time.perf_counter()
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record()
         for _ in range(n_e2e):
             B.mxfp8_linear_host(hx, hw, hdy, P, hy, hdx, hdw, ws)
         g1.record()
         barrier()
-        e2e_ms = max_over_ranks(g0.elapsed_time(g1) / n_e2e, world, dev)
+        e2e_ms = max_over_ranks(g0.elapsed_time(g1) / n_e2e, world, dev)     # per pass
         assert torch.equal(hy.cuda(), Y), "host-buffer path and device path disagree"
-        e2e = {"value": whole_job_value(world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": (T * H + F * H + T * F) * 2, "d2h_bytes_per_step": (T * F + T * H + F * H) * 2,
-               "steps": n_e2e}
+        e2e = {"value": whole_job_value(world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms * PASSES_PER_STEP,
+               "ms_per_pass": e2e_ms,
+               "h2d_bytes_per_step": (T * H + F * H + T * F) * 2 * PASSES_PER_STEP,
+               "d2h_bytes_per_step": (T * F + T * H + F * H) * 2 * PASSES_PER_STEP,
+               "steps": 1, "passes": n_e2e}
         del ws
 
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
         clocks["sm_mhz_inside_gemm_kernel"] = round(gemm_clock_mhz, 1)
-        if clocks.get("sm_max_mhz") and gemm_clock_mhz < 0.9 * clocks["sm_max_mhz"] and "sw_power_cap" not in clocks["reasons"]:
-            # the board's power limit acts inside the sub-millisecond GEMM bursts; the sampler sees mostly the gaps between passes
-            clocks["reasons_note"] = ("no sample fell inside a GEMM launch; longer runs (--steps 200) report sw_power_cap, the only "
-                                      "reason ever seen on this path")
-        clocks["note"] = ("sm_mhz is the driver's sampled clock (tens of milliseconds per sample, longer than a step); sm_mhz_inside_gemm_kernel is "
-                          "SM cycles / wall time read by the last timed GEMM launch itself (%.0f us alive)" % gemm_probe_us)
+        clocks["sm_mhz_inside_gemm_kernel_burst"] = round(burst_clock_mhz, 1)
+        clocks["note"] = ("sm_mhz is the driver's sampled clock (20 ms per sample); sm_mhz_inside_gemm_kernel is SM cycles / wall time read "
+                          "by the last GEMM launch of the timed region itself (%.0f us alive), ..._burst the same for the 20th pass after an "
+                          "idle gap" % gemm_probe_us)
     if world > 1:
         dist.barrier()
     if rank != 0:
@@ -351,39 +385,67 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
-    fp8_peak = 2.0 * peaks["bf16_tflops"]                      # FP8 = 2x the BF16 tensor rate (Table 1)
+    fp8_burst = 2.0 * peaks["bf16_tflops"]                     # FP8 = 2x the BF16 tensor rate (Table 1)
+    fp8_sustained = 2.0 * peaks["bf16_tflops_sustained"]
     gemm_tflops = {k: 2.0 * m * n * kk / (gemm_ms[k] * 1e-3) / 1e12 for k, (m, n, kk) in GEMM_SHAPES.items()}
     gemm_all = STEP_FLOP / (sum(gemm_ms.values()) * 1e-3) / 1e12
     cast_gbs = CAST_BYTES / (cast_ms * 1e-3) / 1e9
-    gemm_multi_tflops = STEP_FLOP / (gemm_multi_ms * 1e-3) / 1e12    # the launch the timed step uses: all three products
-    value = whole_job_value(world, ms_step)
+    gemm_multi_tflops = STEP_FLOP / (gemm_multi_ms * 1e-3) / 1e12    # the launch the timed passes use: all three products
+    value = whole_job_value(world, ms_pass)
+
+    def tf(ms):
+        return STEP_FLOP / (ms * 1e-3) / 1e12
+
+    def gbs(ms):
+        return CAST_BYTES / (ms * 1e-3) / 1e9
+
+    b_gemm_ms, b_cast_ms = statistics.median(b_gemm), statistics.median(b_cast)
+    burst = {"passes": len(b_pass), "after_idle_s": 0.5, "ms_per_pass": statistics.median(b_pass), "best_ms_per_pass": min(b_pass),
+             "value": tf(statistics.median(b_pass)), "gemm_tflops": tf(b_gemm_ms), "gemm_ms": b_gemm_ms,
+             "gemm_frac_of_2x_bf16_burst": tf(b_gemm_ms) / fp8_burst, "cast_gbs": gbs(b_cast_ms), "cast_ms": b_cast_ms,
+             "cast_frac_of_measured_copy": gbs(b_cast_ms) / peaks["hbm_gbs"], "sm_mhz_inside_gemm_kernel": round(burst_clock_mhz, 1),
+             "gemm_mcycles": b_gemm_ms * burst_clock_mhz * 1e-3}
+    steady = {"passes": len(s_pass), "ms_per_pass": statistics.median(s_pass), "best_ms_per_pass": min(s_pass),
+              "value": tf(statistics.median(s_pass)), "gemm_tflops": gemm_multi_tflops, "gemm_ms": gemm_multi_ms,
+              "gemm_best_ms": min(s_gemm), "gemm_frac_of_2x_bf16_sustained": gemm_multi_tflops / fp8_sustained,
+              "cast_gbs": cast_gbs, "cast_ms": cast_ms, "cast_best_ms": min(s_cast),
+              "sm_mhz_inside_gemm_kernel": round(steady_clock_mhz, 1), "gemm_mcycles": gemm_multi_ms * steady_clock_mhz * 1e-3,
+              "note": "per-launch CUDA events on every pass, taken right after the timed region (same thermal and power state)"}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         s, f, desc, threads = oracle_sample_seconds(8192)
         cpu = {"value": STEP_FLOP / f / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
-               "sample": desc, "sample_seconds": s, **getattr(oracle_sample_seconds, "split", {})}
+               "sample": "one pass (one of the %d of a step) -- %s" % (PASSES_PER_STEP, desc), "sample_seconds": s,
+               **getattr(oracle_sample_seconds, "split", {})}
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_pass": ms_pass, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "fp8_e4m3 x fp8_e4m3 -> f32 accumulate", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: 192 MB of BF16 sources and 590 MB of outputs per step",
-                   "parallelism": "dp%d (independent batches, no collective)" % world},
+        "config": bench_config(world),
         "cast": {"value": cast_gbs, "unit": "GB/s", "ms": cast_ms, "bytes": CAST_BYTES,
                  "frac_of_measured_copy": cast_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": cast_gbs / NOMINAL_HBM_GBS},
         "gemm": {"value": gemm_multi_tflops, "unit": "TFLOP/s", "ms": gemm_multi_ms,
-                 "frac_of_2x_measured_bf16": gemm_multi_tflops / fp8_peak, "frac_of_nominal_4.5PF": gemm_multi_tflops / NOMINAL_FP8_TFLOPS,
+                 "frac_of_2x_measured_bf16_sustained": gemm_multi_tflops / fp8_sustained,
+                 "frac_of_2x_measured_bf16_burst": gemm_multi_tflops / fp8_burst, "frac_of_nominal_4.5PF": gemm_multi_tflops / NOMINAL_FP8_TFLOPS,
                  "launched_one_by_one": {"value": gemm_all, "ms": gemm_ms, "tflops": gemm_tflops}},
+        "burst": burst, "steady": steady,
+        # the dominant kernel, timed inside the long steady-state run: against the sustained peak
         "roofline": {"bound": "tensor", "kernel": "gemm_kernel<256, pair, multi> (fprop + dgrad + wgrad in one launch)",
-                     "achieved": gemm_multi_tflops, "peak": fp8_peak, "unit": "TFLOP/s", "frac": gemm_multi_tflops / fp8_peak,
-                     "peak_source": "2 x %s bf16 burst TFLOP/s (Table 1: MXFP8 = 2x BF16)" % peaks["source"],
-                     "algorithmic_flop_per_launch": STEP_FLOP,
+                     "achieved": gemm_multi_tflops, "peak": fp8_sustained, "unit": "TFLOP/s", "frac": gemm_multi_tflops / fp8_sustained,
+                     "peak_source": "2 x %s bf16 sustained TFLOP/s (Table 1: MXFP8 = 2x BF16); steady state of a %.2f s timed region"
+                                    % (peaks["source"], ms_total * 1e-3),
+                     "algorithmic_flop_per_launch": STEP_FLOP, "sm_mhz_inside_kernel": round(steady_clock_mhz, 1),
                      "traffic": NCU_TRAFFIC_GEMM_MULTI, "traffic_note": "ncu capture of this launch, see profiles/"},
+        # the same launch in the first 20 passes after an idle gap: against the burst peak
+        "roofline_burst": {"bound": "tensor", "achieved": tf(b_gemm_ms), "peak": fp8_burst, "unit": "TFLOP/s",
+                           "frac": tf(b_gemm_ms) / fp8_burst, "peak_source": "2 x %s bf16 burst TFLOP/s" % peaks["source"],
+                           "sm_mhz_inside_kernel": round(burst_clock_mhz, 1)},
         "roofline_cast": {"bound": "hbm", "kernel": "quantize_tma_kernel<bf16,e4m3,row+col>", "achieved": cast_gbs,
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cast_gbs / peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "algorithmic_bytes_per_element": 4.0625,
-                          "algorithmic_bytes_per_launch": CAST_BYTES,
+                          "algorithmic_bytes_per_launch": CAST_BYTES, "frac_burst": gbs(b_cast_ms) / peaks["hbm_gbs"],
                           "traffic": NCU_TRAFFIC_QUANTIZE_STEP,
                           "traffic_note": "ncu capture of this launch (X, W, dY in one), see profiles/"},
         "e2e": e2e, "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
@@ -518,29 +580,98 @@ def run_sweep(args):
     peaks = measured_peaks()
     P, S = B.RULE_PAPER, B.SF_SWIZZLED
     if args.sweep == "cast":
-        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy |")
-        print("|---|---|---|---|---|---|---|---|---|")
+        # Config-4 sweep.  Part 1: sizes x shapes x dtypes x orientations, each shape with "its" distribution.
+        # Part 2 (at 256 MB): every distribution on every shape, E5M2 beside E4M3 in every orientation; the
+        # distribution with 0.01 % NaN / Inf sends the slabs that meet one through the careful path.
+        # host us/call: wall time of the C-ABI call alone (argument checks, tensor maps, launch), 200 calls.
+        def cell(dtype, esz, nbytes, cols, kind, orients, elems):
+            rows = max(32, (nbytes // (cols * esz)) // 32 * 32)
+            n_bufs = max(1, min(4, int((768 << 20) // (rows * cols * esz)) + 1)) if nbytes < (1 << 30) else 1
+            srcs = [synth.device_tensor(kind, (rows, cols), 7 + i, dtype) for i in range(n_bufs)]
+            for orient, oname in orients:
+                for elem in elems:
+                    outs = B.alloc_quantize_outputs(rows, cols, orient, S)
+                    ms = _time_calls(lambda i: B.mxfp8_quantize(srcs[i], orient, P, elem, *outs, S), n_bufs)
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                    for i in range(200):
+                        B.mxfp8_quantize(srcs[0], orient, P, elem, *outs, S)
+                    host_us = (time.perf_counter() - t0) / 200 * 1e6 if nbytes <= (16 << 20) else float("nan")
+                    torch.cuda.synchronize()
+                    by = rows * cols * (esz + (2 if orient == B.BOTH else 1) * (1 + 1 / 32))
+                    gbs = by / ms / 1e6
+                    print("| %s | %d MB | %d x %d | %s | %s | %s | %.1f | %.0f | %.2f | %s |" % (
+                        dtype, nbytes >> 20, rows, cols, kind, oname, "e4m3" if elem == B.E4M3 else "e5m2",
+                        ms * 1e3, gbs, gbs / peaks["hbm_gbs"], "-" if host_us != host_us else "%.1f" % host_us), flush=True)
+                    del outs
+            del srcs
+            torch.cuda.empty_cache()
+
+        all_o = ((B.ROW, "row"), (B.COL, "col"), (B.BOTH, "both"))
+        own_kind = {4096: "gaussian", 14336: "gradient_like", 8288: "student_t"}
+        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call |")
+        print("|---|---|---|---|---|---|---|---|---|---|")
         for dtype, esz in (("bf16", 2), ("fp32", 4)):
-            for nbytes in (1 << 20, 16 << 20, 256 << 20, 1 << 30, 4 << 30):
+            for nbytes in (1 << 20, 4 << 20, 16 << 20, 64 << 20, 256 << 20, 1 << 30, 4 << 30):
                 for cols in (4096, 14336, 8288):
                     if nbytes >= (1 << 30) and cols != 4096 and dtype == "fp32":
                         continue
-                    rows = max(32, (nbytes // (cols * esz)) // 32 * 32)
-                    kind = "gradient_like" if cols == 14336 else ("student_t" if cols == 8288 else "gaussian")
-                    n_bufs = max(1, min(4, int((768 << 20) // (rows * cols * esz)) + 1)) if nbytes < (1 << 30) else 1
-                    srcs = [synth.device_tensor(kind, (rows, cols), 7 + i, dtype) for i in range(n_bufs)]
-                    for orient, oname in ((B.ROW, "row"), (B.COL, "col"), (B.BOTH, "both")):
-                        for elem in ((B.E4M3, B.E5M2) if (orient == B.BOTH and cols == 4096) else (B.E4M3,)):
-                            outs = B.alloc_quantize_outputs(rows, cols, orient, S)
-                            ms = _time_calls(lambda i: B.mxfp8_quantize(srcs[i], orient, P, elem, *outs, S), n_bufs)
-                            by = rows * cols * (esz + (2 if orient == B.BOTH else 1) * (1 + 1 / 32))
-                            gbs = by / ms / 1e6
-                            print("| %s | %d MB | %d x %d | %s | %s | %s | %.1f | %.0f | %.2f |" % (
-                                dtype, nbytes >> 20, rows, cols, kind, oname, "e4m3" if elem == B.E4M3 else "e5m2",
-                                ms * 1e3, gbs, gbs / peaks["hbm_gbs"]), flush=True)
-                            del outs
-                    del srcs
-                    torch.cuda.empty_cache()
+                    cell(dtype, esz, nbytes, cols, own_kind[cols], all_o, (B.E4M3,))
+        print()
+        print("Every distribution on every shape, both element types, 256 MB sources:")
+        print()
+        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call |")
+        print("|---|---|---|---|---|---|---|---|---|---|")
+        for dtype, esz in (("bf16", 2), ("fp32", 4)):
+            for cols in (4096, 14336, 8288):
+                for kind in ("gaussian", "student_t", "gradient_like", "nonfinite"):
+                    cell(dtype, esz, 256 << 20, cols, kind, all_o if dtype == "bf16" else ((B.BOTH, "both"),), (B.E4M3, B.E5M2))
+        return
+    if args.sweep == "rules":
+        # The comparison of Sec. 3.3 (the paragraph after Algorithm 1; Fig. 5's subject) on synthetic tensors: for each
+        # distribution x source dtype x element type, the share of blocks whose scale differs between the paper's rule
+        # and the OCP one, the share of finite elements that the OCP scale pushes beyond destmax (clamped by the
+        # saturating cast; none under the paper's rule), and the relative Frobenius error of the MXFP8 round trip under
+        # each rule -- all through mxfp8_quantize / mxfp8_fake_quantize on the GPU, with the oracle's figures for the
+        # first 2^22 elements of the same tensor beside them.
+        import numpy as np
+        import oracle as orc
+        rows, cols = 8192, 4096
+        print("| dist | source | elem | blocks with different scales | oracle | elements clamped, OCP | oracle | clamped, paper | round-trip error, paper | oracle | round-trip error, OCP | oracle |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+        for kind in ("gaussian", "student_t", "gradient_like", "nonfinite"):
+            for dtype in ("bf16", "fp32"):
+                src = synth.device_tensor(kind, (rows, cols), 41, dtype)
+                x = src.float()
+                fin = torch.isfinite(x)
+                x0 = torch.where(fin, x, torch.zeros_like(x)).double()
+                norm = float(x0.pow(2).sum().sqrt())
+                host = src[:1024].float().cpu().numpy()
+                hfin = np.isfinite(host)
+                h0 = np.where(hfin, host.astype(np.float64), 0.0)
+                for elem, ename, destmax in ((B.E4M3, "e4m3", 448.0), (B.E5M2, "e5m2", 57344.0)):
+                    res, ores = {}, {}
+                    for rule, rname in ((B.RULE_PAPER, "paper"), (B.RULE_OCP, "ocp")):
+                        q, sc, _, _ = B.alloc_quantize_outputs(rows, cols, B.ROW, B.SF_LINEAR)
+                        B.mxfp8_quantize(src, B.ROW, rule, elem, q, sc, None, None, B.SF_LINEAR)
+                        back = torch.empty_like(src)
+                        B.mxfp8_fake_quantize(src, B.ROW, rule, elem, back, None)
+                        scale = torch.exp2(sc.view(rows, cols // 32).double() - 127.0).repeat_interleave(32, dim=1)
+                        res[rname] = {"s": sc.view(rows, cols // 32).clone(),
+                                      "clamped": float(((x0.abs() / scale) > destmax).sum() / fin.sum()),
+                                      "err": float(torch.where(fin, back.double() - x0, torch.zeros_like(x0)).pow(2).sum().sqrt()) / norm}
+                        oq, osc = orc.quantize_threads(host, orc.ROW, rule, elem, os.cpu_count() or 1)
+                        od = orc.dequantize_f64(oq, osc, orc.ROW, elem)
+                        oscale = np.repeat(np.exp2(osc.astype(np.float64) - 127.0), 32, axis=1)
+                        ores[rname] = {"s": osc, "clamped": float((np.abs(h0) / oscale > destmax).sum() / hfin.sum()),
+                                       "err": float(np.sqrt((np.where(hfin, od - h0, 0.0) ** 2).sum() / (h0 ** 2).sum()))}
+                        del q, sc, back
+                    differ = float((res["paper"]["s"] != res["ocp"]["s"]).float().mean())
+                    odiffer = float((ores["paper"]["s"] != ores["ocp"]["s"]).mean())
+                    print("| %s | %s | %s | %.2f %% | %.2f %% | %.3f %% | %.3f %% | %.3f %% | %.4f | %.4f | %.4f | %.4f |" % (
+                        kind, dtype, ename, 100 * differ, 100 * odiffer, 100 * res["ocp"]["clamped"], 100 * ores["ocp"]["clamped"],
+                        100 * res["paper"]["clamped"], res["paper"]["err"], ores["paper"]["err"], res["ocp"]["err"], ores["ocp"]["err"]), flush=True)
+        assert B.mxfp8_device_status() == 0
         return
     if args.sweep == "moe":
         # per-expert GEMMs of a mixture-of-experts FFN (App. A.4 trains a 16B-total / 2.5B-active model; the layer here
@@ -679,8 +810,11 @@ def run_sweep(args):
         shapes.append((name + " fprop", Tk, fout, fin, 0, 0))
         shapes.append((name + " dgrad", Tk, fin, fout, 0, 1))
         shapes.append((name + " wgrad", fout, fin, Tk, 1, 1))
-    print("| case | M | N | K | majors | out | fused MX out | us | TFLOP/s | of 2x measured BF16 |")
-    print("|---|---|---|---|---|---|---|---|---|---|")
+    # every cell is timed in three rounds, the variants of one shape interleaved inside each round (the launch runs under
+    # the board's power cap and the clock drifts by several percent between rounds): the median of the rounds is
+    # reported, with the SM clock the kernel itself measured and the product of the two in cycles
+    print("| case | M | N | K | majors | out | fused MX out | us (median of 3) | min | max | TFLOP/s | of 2x measured BF16 burst | SM MHz in kernel | Mcycles |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     fp8_peak = 2.0 * peaks["bf16_tflops"]
     for name, M, N, K, am, bm in shapes:
         def operand(mn, k, major, seed):
@@ -695,6 +829,7 @@ def run_sweep(args):
             return o[2], o[3]
         Aq, As = operand(M, K, am, 11)
         Bq, Bs = operand(N, K, bm, 12)
+        cells = []
         for out_dt, oname in ((torch.bfloat16, "bf16"), (torch.float32, "fp32")):
             for epi_o in (0, B.ROW, B.BOTH):
                 if epi_o and out_dt == torch.float32:
@@ -706,13 +841,19 @@ def run_sweep(args):
                 if epi_o:
                     keep = B.alloc_quantize_outputs(M, N, epi_o, S)
                     epi = B.make_epilogue(epi_o, P, B.E4M3, *keep)
-                ms = _time_calls(lambda i: B.mxfp8_gemm(Aq, As, Bq, Bs, M, N, K, am, bm, B.E4M3, B.E4M3, D, epi=epi), 1, 10, 20.0)
-                tf = 2.0 * M * N * K / ms / 1e9
-                print("| %s | %d | %d | %d | %s%s | %s | %s | %.1f | %.0f | %.2f |" % (
-                    name, M, N, K, "kn"[0] if am == 0 else "m", "k" if bm == 0 else "n", oname,
-                    {0: "-", B.ROW: "row", B.BOTH: "row+col"}[epi_o], ms * 1e3, tf, tf / fp8_peak), flush=True)
-                del D, keep, epi
-        del Aq, As, Bq, Bs
+                cells.append({"out": oname, "epi": epi_o, "D": D, "epi_obj": epi, "keep": keep, "ms": [], "mhz": []})
+        for _ in range(3):
+            for c in cells:
+                c["ms"].append(_time_calls(lambda i: B.mxfp8_gemm(Aq, As, Bq, Bs, M, N, K, am, bm, B.E4M3, B.E4M3, c["D"], epi=c["epi_obj"]), 1, 10, 20.0))
+                c["mhz"].append(B.mxfp8_gemm_last_clock()[0])
+        for c in cells:
+            ms, mhz = statistics.median(c["ms"]), statistics.median(c["mhz"])
+            tf = 2.0 * M * N * K / ms / 1e9
+            print("| %s | %d | %d | %d | %s%s | %s | %s | %.1f | %.1f | %.1f | %.0f | %.2f | %.0f | %.2f |" % (
+                name, M, N, K, "kn"[0] if am == 0 else "m", "k" if bm == 0 else "n", c["out"],
+                {0: "-", B.ROW: "row", B.BOTH: "row+col"}[c["epi"]], ms * 1e3, min(c["ms"]) * 1e3, max(c["ms"]) * 1e3, tf, tf / fp8_peak,
+                mhz, ms * mhz * 1e-3), flush=True)
+        del cells, Aq, As, Bq, Bs
         torch.cuda.empty_cache()
     assert B.mxfp8_device_status() == 0
 
@@ -727,7 +868,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu", "scatter"],
                     help="run one kernel on one small case and exit (for profiler captures)")
-    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe", "dp"],
+    ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe", "dp", "rules"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
     args = ap.parse_args()
     if args.sweep:

@@ -124,7 +124,8 @@ def draw(dist: str, shape, seed: int) -> np.ndarray:
 
 def device_tensor(kind: str, shape, seed: int, dtype="bf16", device="cuda"):
     """A seeded tensor drawn on ``device``; kind in {activation, weight, output_gradient,
-    gaussian, student_t, gradient_like}."""
+    gaussian, student_t, gradient_like, nonfinite (Gaussian with 0.01 % of the elements replaced by NaN, +Inf, -Inf
+    in equal thirds)}."""
     import torch
 
     g = torch.Generator(device=device)
@@ -136,6 +137,12 @@ def device_tensor(kind: str, shape, seed: int, dtype="bf16", device="cuda"):
 
     if kind in ("activation", "gaussian"):
         x = randn(*shape)
+    elif kind == "nonfinite":
+        x = randn(*shape)
+        u = torch.rand(*shape, generator=g, device=device, dtype=torch.float32)
+        x = torch.where(u < 1e-4 / 3, torch.full_like(x, float("nan")), x)
+        x = torch.where((u >= 1e-4 / 3) & (u < 2e-4 / 3), torch.full_like(x, float("inf")), x)
+        x = torch.where((u >= 2e-4 / 3) & (u < 1e-4), torch.full_like(x, float("-inf")), x)
     elif kind == "weight":
         x = randn(*shape) * 0.02
     elif kind == "output_gradient":

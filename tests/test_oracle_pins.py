@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 
 import oracle as orc
+from paper_2506_08027_b200 import synth
 
 ELEMS = {"e4m3": orc.E4M3, "e5m2": orc.E5M2}
 DESTMAX = {orc.E4M3: 448, orc.E5M2: 57344}
@@ -740,3 +741,40 @@ def test_property_error_bound_and_no_saturation_under_the_paper_rule():
         assert (np.abs(d / X - y) <= half_ulp * (1 + 1e-12)).all()
 
     check()
+
+
+def _share_of_block_maxima_above_1_75(cdf_abs):
+    """P(mantissa(amax) > 1.75) for the maximum of 32 i.i.d. magnitudes with CDF cdf_abs: the sum over binades of
+    F(2^(n+1)) - F(1.75 * 2^n), F = cdf_abs^32."""
+    F = lambda a: cdf_abs(a) ** 32
+    return sum(F(2.0 ** (n + 1)) - F(1.75 * 2.0 ** n) for n in range(-40, 60))
+
+
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+def test_rule_disagreement_rates_match_the_distribution_of_block_maxima(elem):
+    """Sec. 3.3: the two rules give different scales exactly when the block maximum's mantissa exceeds that of
+    destmax (1.75), where the OCP rule then clamps elements and the paper's rule does not.  How often that happens
+    follows from the distribution of the maximum of 32 magnitudes, in closed form for the Gaussian and Student-t(3)
+    inputs; with per-row scales spread over many binades the mantissa is log-uniform and the share is
+    log2(2 / 1.75) = 19.3 %.  The oracle's rates on 2^22 elements must sit within half a point of those."""
+    import math
+    gauss = _share_of_block_maxima_above_1_75(lambda a: math.erf(a / math.sqrt(2.0)))
+    t3 = _share_of_block_maxima_above_1_75(
+        lambda a: (2.0 / math.pi) * ((a / math.sqrt(3.0)) / (1.0 + a * a / 3.0) + math.atan(a / math.sqrt(3.0))))
+    want = {"gaussian": gauss, "student_t": t3, "gradient_like": math.log2(2.0 / 1.75), "nonfinite": gauss}
+    assert abs(gauss - 0.169) < 0.003 and abs(t3 - 0.195) < 0.004      # the closed forms themselves
+    destmax = 448.0 if elem == orc.E4M3 else 57344.0
+    for dist in synth.DISTRIBUTIONS:
+        x = synth.draw(dist, (1024, 4096), 77)
+        _, sp = orc.quantize(x, orc.ROW, orc.RULE_PAPER, elem)
+        _, so = orc.quantize(x, orc.ROW, orc.RULE_OCP, elem)
+        assert set(np.unique(sp.astype(int) - so.astype(int))) <= {0, 1}
+        differ = float((sp != so).mean())
+        assert abs(differ - want[dist]) < 0.005, (dist, differ, want[dist])
+        # clamped elements: |V / X| above destmax happens under the OCP rule only, and only in the blocks that differ
+        mag = np.where(np.isfinite(x), np.abs(x.astype(np.float64)), 0.0)
+        over_ocp = mag / np.repeat(np.exp2(so.astype(np.float64) - 127), 32, axis=1) > destmax
+        over_paper = mag / np.repeat(np.exp2(sp.astype(np.float64) - 127), 32, axis=1) > destmax
+        assert not over_paper.any()
+        assert 0.005 < over_ocp.mean() < 0.012
+        assert not (over_ocp & np.repeat(sp == so, 32, axis=1)).any()
