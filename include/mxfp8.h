@@ -200,9 +200,11 @@ int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t
 /*
  * mxfp8_layernorm_quantize -- the same with a layer normalisation: y = ((x - mean[row]) * rstd[row]) * gamma[col] + beta[col],
  * four FP32 operations in that order (no fused multiply-add), rounded once to the source dtype, then converted.
- * mean[row] and rstd[row] = 1 / sqrt(mean_c (x - mean)^2 + eps) are computed by a statistics launch (two passes
- * over the row, FP32 sums in a fixed order) and written to `mean` and `rstd` (device, FP32 [rows]) for the backward
- * pass.  `gamma`, `beta`: device, source dtype, [cols], 16-byte aligned.  Everything else as mxfp8_rmsnorm_quantize.
+ * mean[row] and rstd[row] = 1 / sqrt(mean_c (x - mean)^2 + eps) are computed by a statistics launch (FP32 sums in a
+ * fixed order of x - pivot and its square, pivot = the row's first element, in one pass over the row; a row whose
+ * pivot turns out to lie more than about four standard deviations from the mean is summed a second time around
+ * that mean, so an outlier in the first column costs time, not digits) and written to `mean` and `rstd` (device,
+ * FP32 [rows]) for the backward pass.  `gamma`, `beta`: device, source dtype, [cols], 16-byte aligned.  Everything else as mxfp8_rmsnorm_quantize.
  * (Sec. 3.2 keeps normalisation in high precision and converts its output; the paper names no particular one.)
  */
 int mxfp8_layernorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
@@ -215,9 +217,17 @@ int mxfp8_layernorm_quantize(const void* src, int src_dtype, int64_t rows, int64
  * mxfp8_rmsnorm_quantize_static -- mxfp8_rmsnorm_quantize for callers that do not want the row
  * statistics and have no buffer to lend: the statistics go to a fixed array inside the library
  * (file-scope device memory, 65536 rows x 4 bytes = 256 KB, part of the module image), so the call
- * takes no scratch from the caller and allocates nothing, on the host or on the device.  More than
- * mxfp8_rmsnorm_quantize_static_max_rows() rows: MXFP8_ERR_UNSUPPORTED.  The array is shared by all
- * calls on a device: calls must be ordered on one stream (or otherwise not overlap in time).
+ * takes no scratch from the caller and allocates nothing, on the host or on the device.  It is meant
+ * for callers that cannot call cudaMalloc where they stand: code inside a stream capture, a real-time
+ * loop that must not take the allocator's lock, a plugin that was handed its buffers and nothing else.
+ * The array used is the one of the device that is current on the calling thread (every device that
+ * loads the library holds its own copy until the process ends); its address is looked up on the first
+ * call on that device, so make that first call before any stream capture begins.
+ * Errors: those of mxfp8_rmsnorm_quantize, checked in the same order, and after them
+ * MXFP8_ERR_UNSUPPORTED for more than mxfp8_rmsnorm_quantize_static_max_rows() rows (nothing is launched).
+ * The array is shared by all calls on a device and keeps the last call's statistics: every call
+ * overwrites the rows it uses before it reads them, and calls that overlap on the GPU (two streams,
+ * two threads) race on it -- order them on one stream.
  * Results are those of mxfp8_rmsnorm_quantize.  (A packaging for convenience: the paper has no
  * counterpart.)
  */

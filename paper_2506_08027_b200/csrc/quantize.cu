@@ -442,10 +442,13 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const void* __restrict__
     if (lane == 0) rstd[row] = 1.0f / sqrtf(acc / (float)cols + eps);
 }
 
-// Row statistics of the layer normalisation, one warp per row, ONE pass: sums of d = x - pivot and of d^2 with the
-// row's first element as pivot (a value within a few standard deviations of the mean, so the subtraction
-// S2 - S1^2 / n cancels little), four 16-byte loads in flight per lane, four partial sums per lane in a fixed order,
-// xor butterflies; mean = pivot + S1 / n, rstd = 1 / sqrt((S2 - S1^2 / n) / n + eps) with IEEE square root and division.
+// Row statistics of the layer normalisation, one warp per row, as a rule ONE pass: sums of d = x - pivot and of d^2
+// with the row's first element as pivot, four 16-byte loads in flight per lane, four partial sums per lane in a fixed
+// order, xor butterflies; mean = pivot + S1 / n, rstd = 1 / sqrt((S2 - S1^2 / n) / n + eps) with IEEE square root and
+// division.  S2 - S1^2 / n loses log2(1 + (d / sigma)^2) bits when the pivot lies d from the mean: nothing to speak
+// of for a pivot within a few standard deviations, everything for an outlier.  So when S1^2 / n takes more than 15/16
+// of S2 (the pivot is more than about 4 sigma out, one row in ten thousand of Gaussian data) the row is summed once
+// more around the mean just found: the second read comes from cache, and the result is that of a two-pass algorithm.
 template <int DTYPE>
 __global__ void __launch_bounds__(256) ln_stats_kernel(const void* __restrict__ src, int64_t rows, int64_t cols, float eps,
                                                        float* __restrict__ mean, float* __restrict__ rstd)
@@ -457,7 +460,10 @@ __global__ void __launch_bounds__(256) ln_stats_kernel(const void* __restrict__ 
     const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(src) + row * cols * (DTYPE == MXFP8_BF16 ? 2 : 4));
     const int64_t chunks = cols / PER;
     const uint32_t first = *reinterpret_cast<const uint32_t*>(p);
-    const float pivot = (DTYPE == MXFP8_BF16) ? __uint_as_float(first << 16) : __uint_as_float(first);
+    float pivot = (DTYPE == MXFP8_BF16) ? __uint_as_float(first << 16) : __uint_as_float(first);
+    float a1 = 0.f, a2 = 0.f;
+    const float n = (float)cols;
+  for (int pass = 0; pass < 2; ++pass) {
     float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
     auto add = [&](const uint4& w, int k) {
         const uint32_t u[4] = {w.x, w.y, w.z, w.w};
@@ -481,14 +487,18 @@ __global__ void __launch_bounds__(256) ln_stats_kernel(const void* __restrict__ 
     if (c < chunks) { add(p[c], 0); c += 32; }    // up to three 16-byte pieces per lane are left
     if (c < chunks) { add(p[c], 1); c += 32; }
     if (c < chunks) add(p[c], 2);
-    float a1 = (s1[0] + s1[1]) + (s1[2] + s1[3]), a2 = (s2[0] + s2[1]) + (s2[2] + s2[3]);
+    a1 = (s1[0] + s1[1]) + (s1[2] + s1[3]);
+    a2 = (s2[0] + s2[1]) + (s2[2] + s2[3]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, off);
         a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, off);
     }
+    // every lane holds the same sums: the decision is uniform over the warp
+    if (pass == 1 || !(a1 * a1 / n > 0.9375f * a2)) break;
+    pivot = pivot + a1 / n;       // the pivot was far out: once more around the mean
+  }
     if (lane == 0) {
-        const float n = (float)cols;
         const float var = fmaxf((a2 - a1 * a1 / n) / n, 0.f);
         mean[row] = pivot + a1 / n;
         rstd[row] = 1.0f / sqrtf(var + eps);
@@ -531,13 +541,12 @@ extern "C" int mxfp8_layernorm_quantize(const void* src, int src_dtype, int64_t 
     return quantize_tma_batch(&item, 1, src_dtype, orientation, scale_rule, elem, sf_layout, st, false, MXFP8_ACT_NONE, rstd, gamma, false, mean, beta);
 }
 
-extern "C" int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
-                                      const void* gamma, float eps, float* rstd,
-                                      int orientation, int scale_rule, int elem,
-                                      void* q_row, void* s_row, void* q_col, void* s_col,
-                                      int sf_layout, void* stream)
+namespace mxfp8 {
+namespace {
+// Argument checks shared by mxfp8_rmsnorm_quantize and its variant with the library's own statistics array.
+int rmsnorm_check(const void* src, int src_dtype, int64_t rows, int64_t cols, const void* gamma, float eps, const float* rstd,
+                  int orientation, int scale_rule, int elem, void* q_row, void* s_row, void* q_col, void* s_col, int sf_layout)
 {
-    using namespace mxfp8;
     if (src_dtype != MXFP8_FP32 && src_dtype != MXFP8_BF16) return MXFP8_ERR_ENUM;
     if (orientation < MXFP8_ROW || orientation > MXFP8_BOTH) return MXFP8_ERR_ENUM;
     if (scale_rule != MXFP8_RULE_PAPER && scale_rule != MXFP8_RULE_OCP) return MXFP8_ERR_ENUM;
@@ -554,6 +563,20 @@ extern "C" int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t ro
     if ((orientation & MXFP8_COL) && (!aligned16(q_col) || !aligned16(s_col))) return MXFP8_ERR_ALIGN;
     if (!quantize_tma_eligible(src_dtype, rows, cols)) return MXFP8_ERR_UNSUPPORTED;   // needs cols % 16 == 0
     if ((rows + 7) / 8 > 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
+    return MXFP8_OK;
+}
+}  // namespace
+}  // namespace mxfp8
+
+extern "C" int mxfp8_rmsnorm_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols,
+                                      const void* gamma, float eps, float* rstd,
+                                      int orientation, int scale_rule, int elem,
+                                      void* q_row, void* s_row, void* q_col, void* s_col,
+                                      int sf_layout, void* stream)
+{
+    using namespace mxfp8;
+    const int bad = rmsnorm_check(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem, q_row, s_row, q_col, s_col, sf_layout);
+    if (bad != MXFP8_OK) return bad;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const unsigned blocks = (unsigned)((rows + 7) / 8);
     if (src_dtype == MXFP8_BF16) rms_stats_kernel<MXFP8_BF16><<<blocks, 256, 0, st>>>(src, rows, cols, eps, rstd);
@@ -653,9 +676,12 @@ extern "C" int mxfp8_rmsnorm_quantize_static(const void* src, int src_dtype, int
                                              int sf_layout, void* stream)
 {
     using namespace mxfp8;
-    if (rows > RSTD_STATIC_ROWS) return MXFP8_ERR_UNSUPPORTED;
-    float* rstd = rstd_static_address();
+    float* rstd = rstd_static_address();      // the array of the device that is current on this thread
     if (!rstd) return MXFP8_ERR_CUDA;
+    // the same checks, in the same order, as the call with a caller's buffer; then this variant's own limit
+    const int bad = rmsnorm_check(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem, q_row, s_row, q_col, s_col, sf_layout);
+    if (bad != MXFP8_OK) return bad;
+    if (rows > RSTD_STATIC_ROWS) return MXFP8_ERR_UNSUPPORTED;
     return mxfp8_rmsnorm_quantize(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem,
                                   q_row, s_row, q_col, s_col, sf_layout, stream);
 }

@@ -250,6 +250,27 @@ def test_layernorm_quantize(dtype, shape):
         assert_q_equal(got[name][0], wq, orc.E4M3, name)
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_layernorm_statistics_with_an_outlier_in_the_first_column(dtype):
+    """The statistics pass sums around the row's first element; rows that begin with an outlier of 10^3 to 10^4
+    standard deviations (and rows with the outlier elsewhere, or none) must still give the mean and rstd of the
+    FP64 definition."""
+    rows, cols = 96, 2048
+    rng = np.random.default_rng(5)
+    x32 = (synth.gaussian((rows, cols), 31) + rng.standard_normal((rows, 1)) * 3).astype(np.float32)
+    x32[0:32, 0] += np.float32(1e3) * rng.choice([-1.0, 1.0], 32).astype(np.float32)
+    x32[32:64, 0] += np.float32(1e4)
+    x32[64:80, 777] -= np.float32(1e4)
+    g32 = np.ones(cols, np.float32)
+    b32 = np.zeros(cols, np.float32)
+    x, g, b = as_dtype(x32, dtype), as_dtype(g32, dtype), as_dtype(b32, dtype)
+    xv = orc.bf16_bits_to_f32(x) if dtype == "bf16" else x
+    got = gpu_layernorm_quantize(x, g, b, dtype, 1e-5, ROW)
+    _, want_mean, want_rstd = orc.layernorm(xv, g32, b32, 1e-5)
+    assert np.abs(got["mean"] - want_mean).max() <= 2.0 ** -20 * np.abs(xv).max()
+    assert (np.abs(got["rstd"] - want_rstd) <= 2.0 ** -18 * np.abs(want_rstd)).all()
+
+
 def test_layernorm_equals_rmsnorm_on_centred_rows_without_bias():
     """Rows of small multiples of 1/4 in (v, -v) pairs and a zero bias: every sum the two statistics kernels form is exact,
     the mean is exactly zero, and the two normalisations are the same arithmetic."""

@@ -48,8 +48,16 @@ def test_same_result_as_the_call_with_a_caller_buffer(shape):
 
 @pytest.mark.gpu
 def test_allocates_nothing_on_host_or_device():
+    import ctypes
     import torch
     from paper_2506_08027_b200 import binding as B
+
+    class Mallinfo2(ctypes.Structure):        # glibc: bytes in use by the C heap are `uordblks`
+        _fields_ = [(n, ctypes.c_size_t) for n in ("arena", "ordblks", "smblks", "hblks", "hblkhd", "usmblks", "fsmblks",
+                                                    "uordblks", "fordblks", "keepcost")]
+    libc = ctypes.CDLL(None)
+    libc.mallinfo2.restype = Mallinfo2
+    lib = B.lib()
     rows, cols = 4096, 2048
     x, gamma = _inputs(rows, cols, 6)
     outs = B.alloc_quantize_outputs(rows, cols, B.BOTH, B.SF_SWIZZLED)
@@ -71,6 +79,22 @@ def test_allocates_nothing_on_host_or_device():
     stats1 = torch.cuda.memory_stats()
     assert stats1["allocation.all.allocated"] == stats0["allocation.all.allocated"]
     assert stats1["allocated_bytes.all.current"] == stats0["allocated_bytes.all.current"]
+    # the host side: the C heap of this process around 20 calls made straight through the C ABI (arguments
+    # marshalled beforehand, so that nothing of Python's runs between the two readings but the foreign calls)
+    args = (x.data_ptr(), B.BF16, rows, cols, gamma.data_ptr(), ctypes.c_float(1e-5), B.BOTH, B.RULE_PAPER, B.E4M3,
+            outs[0].data_ptr(), outs[1].data_ptr(), outs[2].data_ptr(), outs[3].data_ptr(), B.SF_SWIZZLED, None)
+    call = lib.mxfp8_rmsnorm_quantize_static
+    assert call(*args) == 0
+    grew = []
+    for _ in range(3):
+        before = libc.mallinfo2().uordblks
+        rc = [call(*args) for _ in range(20)]
+        grew.append(libc.mallinfo2().uordblks - before)
+        assert not any(rc)
+    torch.cuda.synchronize()
+    # the list of 20 return codes is Python's own (a few hundred bytes at most): a buffer of any size that the
+    # library allocated and kept per call would show far above that
+    assert max(grew) < 4096, grew
 
 
 @pytest.mark.gpu
