@@ -15,6 +15,9 @@ SOURCES = ["quantize.cu", "quantize_tma.cu", "quantize_tma_fp6_fp4.cu", "dequant
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC",
+    # static locals of template functions must stay private to each copy of the library that a process loads (the test
+    # build is loaded beside the product): GNU "unique" symbols would be shared across them
+    "-Xcompiler", "-fno-gnu-unique",
 ]
 
 

@@ -117,6 +117,15 @@ bool gemm_device(GemmDevice& out)
 }  // namespace gemm
 namespace {
 
+// D can be stored straight from registers when every row segment of 32 bytes is aligned (see GemmParams::d_direct);
+// MXFP8_GEMM_STAGED=1 forces the staged TMA path (testing aid)
+uint8_t* direct_output(void* D, int64_t N, int out_dtype)
+{
+    const int64_t pitch = N * (out_dtype == MXFP8_FP32 ? 4 : 2);
+    if (!D || (reinterpret_cast<uintptr_t>(D) & 31u) || (pitch & 31) || getenv("MXFP8_GEMM_STAGED")) return nullptr;
+    return static_cast<uint8_t*>(D);
+}
+
 int sm_count()
 {
     GemmDevice d;
@@ -197,8 +206,11 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
     p.M = M; p.N = N; p.K = K;
     p.a_mn = a_major; p.b_mn = b_major; p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
     p.store_d = D ? 1 : 0;
+    p.d_direct = direct_output(D, N, out_dtype);
     if (epi) {
         p.epi_orient = epi->orientation; p.epi_rule = epi->scale_rule; p.epi_elem = epi->elem;
+        p.epi_q_row = static_cast<uint8_t*>(epi->q_row);
+        p.epi_q_col = static_cast<uint8_t*>(epi->q_col);
         p.epi_s_row = static_cast<uint8_t*>(epi->s_row);
         p.epi_s_col = static_cast<uint8_t*>(epi->s_col);
     }
@@ -217,12 +229,9 @@ extern "C" int mxfp8_gemm(const void* Aq, const void* As, const void* Bq, const 
                      make_tmap_sf(&m.sfb, Bs, (uint64_t)((N + 127) / 128), (uint64_t)((K + 127) / 128));
     // maps that a launch does not use still have to be valid: point them at any output that exists
     void* q_any = epi ? ((epi->orientation & MXFP8_ROW) ? epi->q_row : epi->q_col) : D;
-    void* q_row = (epi && (epi->orientation & MXFP8_ROW)) ? epi->q_row : q_any;
-    void* q_col = (epi && (epi->orientation & MXFP8_COL)) ? epi->q_col : q_any;
     const bool okd = D ? make_tmap_d(&m.d, D, (uint64_t)M, (uint64_t)N, out_dtype) : make_tmap_q(&m.d, q_any, (uint64_t)M, (uint64_t)N);
-    bool okq = true;
-    if (epi) okq = make_tmap_q(&m.qrow, q_row, (uint64_t)M, (uint64_t)N) && make_tmap_q(&m.qcol, q_col, (uint64_t)M, (uint64_t)N);
-    else if (okd) { m.qrow = m.d; m.qcol = m.d; }   // never dereferenced without an epilogue, but must be valid maps
+    const bool okq = true;
+    if (okd) { m.qrow = m.d; m.qcol = m.d; }   // the fused output is stored from registers; these two only have to be valid maps
     if (getenv("MXFP8_LOG"))
         fprintf(stderr, "mxfp8_gemm M=%lld N=%lld K=%lld tile=%d%s maps: a=%d b=%d sf=%d d=%d q=%d\n", (long long)M, (long long)N,
                 (long long)K, best_bn, best_pair ? "p" : "", (int)oka, (int)okb, (int)oks, (int)okd, (int)okq);
@@ -266,6 +275,7 @@ extern "C" int mxfp8_grouped_gemm(const void* Aq, const void* As, const void* Bq
     p.M = M; p.N = N; p.K = K;
     p.a_elem = a_elem; p.b_elem = b_elem; p.out_dtype = out_dtype;
     p.store_d = 1;
+    p.d_direct = direct_output(D, N, out_dtype);
     p.group_offsets = group_offsets;
     p.num_groups = num_groups;
     const int sms = sm_count();
@@ -339,6 +349,7 @@ extern "C" int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, i
             if (!aligned16(g.Aq) || !aligned16(g.As) || !aligned16(g.Bq) || !aligned16(g.Bs) || !aligned16(g.D)) return MXFP8_ERR_ALIGN;
             MultiProblem& q = p.mp[i];
             q.M = (int)g.M; q.N = (int)g.N; q.num_kb = (int)((g.K + BK - 1) / BK);
+            q.d = direct_output(g.D, g.N, out_dtype);
             q.a_mn = g.a_major; q.b_mn = g.b_major; q.a_elem = g.a_elem; q.b_elem = g.b_elem;
         }
         ProblemMaps& pm = m.multi.p[i];

@@ -45,6 +45,16 @@ namespace gemm {
 constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 128;            // K bytes per pipeline stage = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 320;
+// Kernels with the fused MXFP8 output run 384 threads: warps 0-3 form a warp group of their own (producer, MMA issuer,
+// two idle warps) that hands most of its registers to the two warp groups of epilogue warps (setmaxnreg), because the
+// fused epilogue needs more than the 168 registers per thread that ten warps leave: with 168 it spilled 40 registers
+// per thread, and the spills missed the small L1 that 223 KB of shared memory leave (600 000 local loads per launch,
+// long-scoreboard the top stall, 4000 cycles per tile that nothing could hide).
+template <bool EPI> struct Roles {
+    static constexpr int THREADS = EPI ? 384 : GEMM_THREADS;
+    static constexpr int EPI_WARP0 = EPI ? 4 : 2;       // first of the eight epilogue warps
+    static constexpr int REGS_FEW = 104, REGS_MANY = 200;
+};
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 2048;   // 32 rows x 64 bytes per epilogue warp
 constexpr int TMEM_COLS = 512;
@@ -63,6 +73,7 @@ struct MultiProblem {
     int tiles_m, tiles_n, num_kb;
     int tile_start;       // first tile of this problem in the launch-wide numbering
     uint32_t stage_tx;
+    uint8_t* d;           // output of this problem when its rows can be stored straight from registers (see d_direct), else null
 };
 struct ProblemMaps { CUtensorMap a, b, sfa, sfb, d; };
 struct MultiMaps { ProblemMaps p[MAX_PROBLEMS]; };
@@ -78,6 +89,8 @@ struct GemmParams {
     int store_d;          // 0 when only the fused MXFP8 output is wanted
     int epi_orient;       // 0 = no fused MXFP8 output, else MXFP8_ROW / COL / BOTH
     int epi_rule, epi_elem;
+    uint8_t* epi_q_row;   // fused MXFP8 bytes [M, N] of the two orientations (stored straight from the epilogue registers)
+    uint8_t* epi_q_col;
     uint8_t* epi_s_row;   // swizzled scales of the row-blocked output, logical [M, N/32]
     uint8_t* epi_s_col;   // swizzled scales of the column-blocked output, logical [N, M/32]
     // grouped (per-expert) products: device array of num_groups + 1 token offsets, multiples of 128
@@ -86,6 +99,13 @@ struct GemmParams {
     int token_limit;      // offsets may not pass this (tokens in the grouped tensor)
     int num_problems;     // MULTI
     MultiProblem mp[MAX_PROBLEMS];
+    // Output rows stored straight from the epilogue registers (one 32-byte st.global.v8 per lane and 16 BF16 / 8 FP32
+    // columns) instead of through the shared-memory staging buffer and a TMA store: the K loop of the 256 x 256 pair
+    // tile keeps shared memory busy almost every cycle (33.5 KB of TMA writes + 32 KB of tensor-core reads per 512-cycle
+    // K block at 128 B/clk), and the staged epilogue's 128 KB per tile came on top of that.  Needs a 32-byte aligned D
+    // and a row pitch that is a multiple of 32 bytes; tiles that end beyond N, unaligned outputs and the adding
+    // (SCATTER) mode keep the TMA path.  Null = TMA path only.
+    uint8_t* d_direct;
     int kc_max;           // DEEP: longest run of K blocks accumulated inside the tensor core (see epoch_len)
     int test_skip_load;   // test builds only: 1 + index of the K block whose loads the producer leaves out (0 = none)
     int* status;          // device status word of this device (bounded waits and offset checks report here)
@@ -367,23 +387,16 @@ __device__ __forceinline__ uint32_t epi_inv_exp(uint32_t amax_bits, uint32_t rul
     const int e = (int)((amax_bits + rule_offset) >> 23);
     return (uint32_t)min(254 + ElemTraits<ELEM>::emax - e, 254);
 }
-// 64 bytes of one row (16 words) into the warp's 64-byte-swizzled staging buffer, then one TMA store
-// of the 32 x 64-byte box.  All lanes call it; lane 0 issues the store.
-__device__ __forceinline__ void epi_store_box(const CUtensorMap* map, uint32_t buf, uint32_t row_off, uint32_t sw, int lane,
-                                              const uint32_t (&w)[16], int c0, int c1)
+// This lane's 32 bytes of one output row, straight from registers to global memory: one 32-byte store where the
+// address allows it, two 16-byte ones otherwise (the outputs are 16-byte aligned and N is a multiple of 128).
+__device__ __forceinline__ void epi_store32(uint8_t* dst, const uint32_t (&w)[8])
 {
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-    __syncwarp();
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                     ::"r"(row_off + (((uint32_t)j ^ sw) << 4)), "r"(w[4 * j]), "r"(w[4 * j + 1]), "r"(w[4 * j + 2]), "r"(w[4 * j + 3]) : "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) {
-        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                     ::"l"(map), "r"(c0), "r"(c1), "r"(buf) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+    } else {
+        asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+        asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 16), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
     }
 }
 
@@ -391,86 +404,80 @@ __device__ __forceinline__ void epi_store_box(const CUtensorMap* map, uint32_t b
 // mxfp8_quantize would convert the FP32 output (Sec. 2: the FP32 output is quantized to MX format
 // when its consumer needs it): row blocks run along N inside a lane, column blocks are the warp's
 // 32 rows (one warp-wide integer max per column; |x| bit patterns of finite floats order like integers).
+//
+// The work is a rolled loop over 32-column chunks: every pass converts the chunk held in v[0..31], stores its 32 bytes
+// per row straight to global memory, and then moves the rest of the accumulator down by 32 registers (register files
+// have no indexed access, so the data moves instead of the index).  One chunk's body is a tenth of the code that
+// the straight-line form of both orientations over 128 columns took.  v is consumed.
 template <int CW, int ELEM>
-__device__ __forceinline__ void epi_mx(const uint32_t (&v)[CW], const GemmParams& p, const CUtensorMap* map_row,
-                                       const CUtensorMap* map_col, uint32_t buf, uint32_t row_off, uint32_t sw, int lane,
-                                       int row0, int col0)
+__device__ __forceinline__ void epi_mx(uint32_t (&v)[CW], const GemmParams& p, int lane, int row0, int col0)
 {
     const uint32_t rule_offset = (p.epi_rule == MXFP8_RULE_PAPER) ? paper_offset<ELEM>() : 0u;
     const int row = row0 + lane;
-    if (p.epi_orient & MXFP8_ROW) {
-        const int64_t nkb = p.N >> 5;
+    const bool do_row = (p.epi_orient & MXFP8_ROW) != 0, do_col = (p.epi_orient & MXFP8_COL) != 0;
+    const int64_t nkb_col = p.M >> 5, kb_col = row0 >> 5;
+    uint32_t srow = 0u;                   // this row's scale bytes of the warp's columns: adjacent bytes of one atom word
+#pragma unroll 1
+    for (int ch = 0; ch < CW / 32; ++ch) {
+        const int c0 = col0 + ch * 32;
+        if (do_row) {
+            uint32_t wr[8];
+            float m = 0.f;
 #pragma unroll
-        for (int ch = 0; ch < CW / 64; ++ch) {
-            uint32_t w[16];
+            for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(v[i])));   // NaN ignored
+            if (m == INFINITY) {   // rare: finite-only maximum
+                m = 0.f;
 #pragma unroll
-            for (int hb = 0; hb < 2; ++hb) {
-                const int b0 = ch * 64 + hb * 32;
-                float m = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(v[b0 + i])));   // NaN ignored
-                if (m == INFINITY) {   // rare: finite-only maximum
-                    m = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float a = fabsf(__uint_as_float(v[b0 + i]));
-                        if (a < INFINITY) m = fmaxf(m, a);
-                    }
+                for (int i = 0; i < 32; ++i) {
+                    const float a = fabsf(__uint_as_float(v[i]));
+                    if (a < INFINITY) m = fmaxf(m, a);
                 }
-                const uint32_t ie = epi_inv_exp<ELEM>(__float_as_uint(m), rule_offset);
-                const float inv = __uint_as_float(ie << 23);
-                p.epi_s_row[sf_swizzled_offset(row, (col0 + b0) >> 5, nkb)] = (uint8_t)(254u - ie);
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    w[hb * 8 + i] = cvt_fp8x4<ELEM>(__uint_as_float(v[b0 + 4 * i]) * inv, __uint_as_float(v[b0 + 4 * i + 1]) * inv,
-                                                    __uint_as_float(v[b0 + 4 * i + 2]) * inv, __uint_as_float(v[b0 + 4 * i + 3]) * inv);
             }
-            epi_store_box(map_row, buf, row_off, sw, lane, w, col0 + ch * 64, row0);
+            const uint32_t ie = epi_inv_exp<ELEM>(__float_as_uint(m), rule_offset);
+            const float inv = __uint_as_float(ie << 23);
+            srow |= (254u - ie) << (8 * ch);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                wr[i] = cvt_fp8x4<ELEM>(__uint_as_float(v[4 * i]) * inv, __uint_as_float(v[4 * i + 1]) * inv,
+                                        __uint_as_float(v[4 * i + 2]) * inv, __uint_as_float(v[4 * i + 3]) * inv);
+            epi_store32(p.epi_q_row + (int64_t)row * p.N + c0, wr);
         }
-    }
-    if (p.epi_orient & MXFP8_COL) {
-        const int64_t nkb = p.M >> 5;
-        const int64_t kb = row0 >> 5;
-        // Column c of this warp's CW columns is "owned" by lane c % 32 (slot c / 32): one warp-wide integer
-        // max per column, the owner keeps the result, computes scale and 1/X for its CW/32 columns, stores
-        // their scale bytes, and hands 1/X out again by shuffle when the column is cast.
-        // |x| bit patterns of finite floats order like integers; adding one exponent step makes the
-        // patterns of Inf and NaN wrap to negative numbers, so a SIGNED max leaves them out of the
-        // maximum without a second pass (all reductions issue back to back, nothing branches on them).
-        int own_biased[CW / 32];
+        if (do_col) {
+            // Column c of the chunk is "owned" by lane c: one warp-wide integer max per column, the owner keeps the
+            // result, derives scale and 1/X once, stores the scale byte, and hands 1/X out again by shuffle when the
+            // column is cast.  Adding one exponent step makes the patterns of Inf and NaN wrap to negative numbers,
+            // so a SIGNED max leaves them out of the maximum without a second pass.
+            int own_biased = 0;
 #pragma unroll
-        for (int c = 0; c < CW; ++c) {
-            const int a = (int)((v[c] & 0x7FFFFFFFu) + 0x00800000u);
-            int amax;
-            asm volatile("redux.sync.max.s32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
-            if ((c & 31) == 0) own_biased[c >> 5] = amax;          // every lane takes it, then the owner's survives
-            else if (lane == (c & 31)) own_biased[c >> 5] = amax;
-        }
-        uint32_t own[CW / 32];
+            for (int c = 0; c < 32; ++c) {
+                const int a = (int)((v[c] & 0x7FFFFFFFu) + 0x00800000u);
+                int amax;
+                asm volatile("redux.sync.max.s32 %0, %1, 0xffffffff;" : "=r"(amax) : "r"(a));
+                if (lane == c) own_biased = amax;
+            }
+            const uint32_t own = (uint32_t)(max(own_biased, 0x00800000) - 0x00800000);   // no finite element: 0
+            const uint32_t ie = epi_inv_exp<ELEM>(own, rule_offset);
+            const float own_inv = __uint_as_float(ie << 23);
+            uint32_t wc[8];
+            p.epi_s_col[sf_swizzled_offset(c0 + lane, kb_col, nkb_col)] = (uint8_t)(254u - ie);
 #pragma unroll
-        for (int j = 0; j < CW / 32; ++j) own[j] = (uint32_t)(max(own_biased[j], 0x00800000) - 0x00800000);   // no finite element: 0
-        float own_inv[CW / 32];
-#pragma unroll
-        for (int j = 0; j < CW / 32; ++j) {
-            const uint32_t ie = epi_inv_exp<ELEM>(own[j], rule_offset);
-            own_inv[j] = __uint_as_float(ie << 23);
-            p.epi_s_col[sf_swizzled_offset(col0 + j * 32 + lane, kb, nkb)] = (uint8_t)(254u - ie);
-        }
-#pragma unroll
-        for (int ch = 0; ch < CW / 64; ++ch) {
-            uint32_t w[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 float y[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = ch * 64 + i * 4 + e;
-                    y[e] = __uint_as_float(v[c]) * __shfl_sync(0xFFFFFFFFu, own_inv[c >> 5], c & 31);
-                }
-                w[i] = cvt_fp8x4<ELEM>(y[0], y[1], y[2], y[3]);
+                for (int e = 0; e < 4; ++e) y[e] = __uint_as_float(v[4 * i + e]) * __shfl_sync(0xFFFFFFFFu, own_inv, 4 * i + e);
+                wc[i] = cvt_fp8x4<ELEM>(y[0], y[1], y[2], y[3]);
             }
-            epi_store_box(map_col, buf, row_off, sw, lane, w, col0 + ch * 64, row0);
+            epi_store32(p.epi_q_col + (int64_t)row * p.N + c0, wc);
         }
+        // the next chunk moves down into v[0..31]
+#pragma unroll
+        for (int i = 0; i + 32 < CW; ++i) v[i] = v[i + 32];
+    }
+    if (do_row) {
+        // the scale bytes of 128 columns are the four bytes of one word of the atom (64 columns: half a word)
+        uint8_t* dst = p.epi_s_row + sf_swizzled_offset(row, col0 >> 5, p.N >> 5);
+        if (CW == 128) *reinterpret_cast<uint32_t*>(dst) = srow;
+        else *reinterpret_cast<uint16_t*>(dst) = (uint16_t)srow;
     }
 }
 
@@ -585,7 +592,7 @@ __device__ __forceinline__ int epoch_len(int nkb, int kc_max)
 // DEEP: reductions longer than kc_max K blocks, summed in epochs (separate instantiations again, so that the
 //       kernels of the common depths keep the straight-line epilogue)
 template <int BN, bool PAIR, int MODE, bool EPI, bool DEEP>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(Roles<EPI>::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
             const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_qrow,
@@ -636,7 +643,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // every CTA reads the offsets, checks them (non-negative, non-decreasing, multiples of 128,
         // inside the tensor) and, for GROUP_M, turns them into the first tile index of each group
         const int G = p.num_groups;
-        for (int i = threadIdx.x; i <= G; i += GEMM_THREADS) goff[i] = p.group_offsets[i];
+        for (int i = threadIdx.x; i <= G; i += Roles<EPI>::THREADS) goff[i] = p.group_offsets[i];
         __syncthreads();
         if (warp == 2) {
             bool bad = false;
@@ -698,7 +705,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int num_tiles = (MODE == DENSE || MODE == MULTI || MODE == SCATTER) ? p.num_tiles
                         : (*bad_groups ? 0 : (MODE == GROUP_M ? tstart[p.num_groups] : p.num_groups * p.tiles_m * p.tiles_n));
 
+    constexpr int EW0 = Roles<EPI>::EPI_WARP0;
+    // EPI: the first warp group shrinks to REGS_FEW registers per thread, the epilogue warp groups grow to REGS_MANY
     if (warp == 0) {
+        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
         // ------------------------------------------------------------------ TMA producer
         // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
         // ring-depth-unrolled loop as the MMA warp.
@@ -773,6 +783,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
+        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         // The whole warp walks the loop so that descriptors stay in uniform registers; one
         // elected lane issues the tcgen05 instructions.  The loop runs over all K blocks of all
@@ -880,12 +891,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 while (!mbar_try_wait(drain_bar, 0) && global_timer() - t0 < WAIT_LIMIT_NS) {}
             }
         }
-    } else {
+    } else if (warp >= EW0) {
+        if constexpr (EPI) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_MANY));
         // ------------------------------------------------------------------ epilogue warps
         constexpr int CW = BN / 2;               // accumulator columns per epilogue warp
         const int q = warp & 3;                  // TMEM lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;        // which half of the tile's columns
-        const uint32_t buf = base + C::SMEM_EPI + (warp - 2) * EPI_BUF_BYTES;
+        const int half = (warp - EW0) >> 2;      // which half of the tile's columns
+        const uint32_t buf = base + C::SMEM_EPI + (warp - EW0) * EPI_BUF_BYTES;
         // 64-byte swizzle of the staging buffer: 16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)
         const uint32_t row_off = buf + lane * 64;
         const uint32_t sw = (uint32_t)((lane >> 1) & 3);
@@ -957,12 +969,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             int row0 = t.row0 + t.d_row_extra + (tm * (PAIR ? 2 : 1) + (int)cta_rank) * BM + q * 32;
             const int col0 = tn * BN + half * CW;
             const bool rows_inside = row0 < t.rows_end;      // ragged last M tile / rows of the next expert: a 32-row box entirely outside stores nothing
-            if constexpr (EPI && CW % 64 == 0) {
-                if (p.epi_orient && rows_inside) {
-                    if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
-                    else epi_mx<CW, MXFP8_E5M2>(v, p, &tmap_qrow, &tmap_qcol, buf, row_off, sw, lane, row0, col0);
-                }
-            }
             if constexpr (MODE == SCATTER) {
                 if (rows_inside) {   // this 32-row box lies inside one owner's row range (ranges are multiples of 128 rows)
                     const int owner = row0 / p.rows_per_owner;
@@ -970,7 +976,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     row0 -= owner * p.rows_per_owner;
                 }
             }
+            uint8_t* d_base = nullptr;
+            if constexpr (MODE == MULTI) d_base = p.mp[t.prob].d;
+            else if constexpr (MODE != SCATTER) d_base = p.d_direct;
             if (!p.store_d || !rows_inside) {
+            } else if (MODE != SCATTER && d_base != nullptr && col0 + CW <= n_total) {
+                // the whole column range of this warp lies inside the output: every lane stores its own row
+                if (row0 + lane < t.rows_end) {
+                    if (p.out_dtype == MXFP8_BF16) {
+                        uint8_t* dst = d_base + ((int64_t)(row0 + lane) * n_total + col0) * 2;
+#pragma unroll
+                        for (int j = 0; j < CW / 16; ++j) {
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[j * 16 + 2 * e]),
+                                                                                __uint_as_float(v[j * 16 + 2 * e + 1]));
+                                pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+                            }
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                         ::"l"(dst + j * 32), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                           "r"(pk[6]), "r"(pk[7]) : "memory");
+                        }
+                    } else {
+                        uint8_t* dst = d_base + ((int64_t)(row0 + lane) * n_total + col0) * 4;
+#pragma unroll
+                        for (int j = 0; j < CW / 8; ++j)
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                         ::"l"(dst + j * 32), "r"(v[j * 8]), "r"(v[j * 8 + 1]), "r"(v[j * 8 + 2]), "r"(v[j * 8 + 3]),
+                                           "r"(v[j * 8 + 4]), "r"(v[j * 8 + 5]), "r"(v[j * 8 + 6]), "r"(v[j * 8 + 7]) : "memory");
+                    }
+                }
             } else if (p.out_dtype == MXFP8_BF16) {
 #pragma unroll
                 for (int ch = 0; ch < CW / 32; ++ch) {          // 32 columns = 64 bytes per row
@@ -1021,10 +1057,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     }
                 }
             }
+            // the fused MXFP8 output comes last: it consumes the accumulator registers
+            if constexpr (EPI && CW % 64 == 0) {
+                if (p.epi_orient && rows_inside && col0 < n_total) {   // N is a multiple of 128: a warp's columns are all inside or all outside
+                    if (p.epi_elem == MXFP8_E4M3) epi_mx<CW, MXFP8_E4M3>(v, p, lane, row0, col0);
+                    else epi_mx<CW, MXFP8_E5M2>(v, p, lane, row0, col0);
+                }
+            }
         }
         // all of this warp's stores must have left shared memory and reached global memory
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
+    } else {
+        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));   // the two idle warps of the first group
     }
 
     tc_fence_before();
@@ -1057,7 +1102,7 @@ int launch_kernel(const GemmMaps& m, const GemmParams& p, int workers, cudaStrea
     if (ensure_dynamic_smem(kernel, C::SMEM_TOTAL, smem_set) != cudaSuccess) return MXFP8_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * workers : workers));
-    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.blockDim = dim3(Roles<EPI>::THREADS);
     cfg.dynamicSmemBytes = C::SMEM_TOTAL;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -1069,7 +1114,7 @@ int launch_kernel(const GemmMaps& m, const GemmParams& p, int workers, cudaStrea
     cfg.numAttrs = 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, m.multi, p);
     if (getenv("MXFP8_LOG"))
-        fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d%s -> %s\n", cfg.gridDim.x, GEMM_THREADS,
+        fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d%s -> %s\n", cfg.gridDim.x, Roles<EPI>::THREADS,
                 C::SMEM_TOTAL, p.tiles_m, p.tiles_n, p.num_kb, DEEP ? " (epochs)" : "", cudaGetErrorString(err));
     count_launch(1);
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;

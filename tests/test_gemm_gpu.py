@@ -245,6 +245,42 @@ def test_fused_epilogue_against_fp64_oracle():
         assert (np.abs(dq) <= 448 * xfull).all()
 
 
+@pytest.mark.parametrize("shape", [(256, 384, 256), (384, 128, 128), (640, 896, 384)])
+@pytest.mark.parametrize("tile", ["256p", "256", "128"])
+def test_fused_epilogue_on_outputs_that_end_inside_a_tile(shape, tile, monkeypatch):
+    """M and N are multiples of 128 but not of the tile: the warps whose columns or rows lie beyond the output must
+    write nothing -- no element byte, no scale byte (guard bands around every buffer, pads zero)."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    from helpers import Guarded, swizzle_np
+    m, n, k = shape
+    if tile == "256p" and m < 256:
+        pytest.skip("a CTA pair needs 256 rows")
+    monkeypatch.setenv("MXFP8_GEMM_TILE", tile)
+    a = synth.gaussian((m, k), 21)
+    b = synth.student_t((n, k), 22)
+    aq, a_s = orc.quantize(a, orc.ROW)
+    bq, b_s = orc.quantize(b, orc.ROW)
+    dA, dB = torch.from_numpy(aq).cuda(), torch.from_numpy(bq).cuda()
+    dSA, dSB = torch.from_numpy(swizzle_np(a_s)).cuda(), torch.from_numpy(swizzle_np(b_s)).cuda()
+    g = [Guarded(m * n), Guarded(B.mxfp8_scale_bytes(m, n, B.ROW, B.SF_SWIZZLED)),
+         Guarded(m * n), Guarded(B.mxfp8_scale_bytes(m, n, B.COL, B.SF_SWIZZLED))]
+    for x in g:
+        x.view.zero_()
+    epi = B.make_epilogue(B.BOTH, B.RULE_PAPER, B.E4M3, g[0].view.view(m, n), g[1].view, g[2].view.view(m, n), g[3].view)
+    D = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    B.mxfp8_gemm(dA, dSA, dB, dSB, m, n, k, B.K_MAJOR, B.K_MAJOR, 0, 0, D, epi=epi)
+    assert B.mxfp8_device_status() == 0
+    ref = B.alloc_quantize_outputs(m, n, B.BOTH, B.SF_SWIZZLED)
+    for t in ref:
+        t.zero_()
+    B.mxfp8_quantize(D, B.BOTH, B.RULE_PAPER, B.E4M3, *ref, B.SF_SWIZZLED)
+    torch.cuda.synchronize()
+    for name, got, want in zip(("q_row", "s_row", "q_col", "s_col"), g, ref):
+        got.check(name)
+        assert np.array_equal(got.numpy(), want.cpu().numpy().reshape(-1)), name
+
+
 # ------------------------------------------------------------------------------- benchmark sizes
 
 def test_bench_step_shapes_sampled_rows():
