@@ -676,12 +676,14 @@ extern "C" int mxfp8_rmsnorm_quantize_static(const void* src, int src_dtype, int
                                              int sf_layout, void* stream)
 {
     using namespace mxfp8;
-    float* rstd = rstd_static_address();      // the array of the device that is current on this thread
-    if (!rstd) return MXFP8_ERR_CUDA;
-    // the same checks, in the same order, as the call with a caller's buffer; then this variant's own limit
-    const int bad = rmsnorm_check(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem, q_row, s_row, q_col, s_col, sf_layout);
+    // the same checks, in the same order, as the call with a caller's buffer (the array stands in for it: any aligned
+    // non-null address passes those two checks); then this variant's own limit; only then the device is asked
+    const int bad = rmsnorm_check(src, src_dtype, rows, cols, gamma, eps, reinterpret_cast<const float*>(uintptr_t(256)), orientation,
+                                  scale_rule, elem, q_row, s_row, q_col, s_col, sf_layout);
     if (bad != MXFP8_OK) return bad;
     if (rows > RSTD_STATIC_ROWS) return MXFP8_ERR_UNSUPPORTED;
+    float* rstd = rstd_static_address();      // the array of the device that is current on this thread
+    if (!rstd) return MXFP8_ERR_CUDA;
     return mxfp8_rmsnorm_quantize(src, src_dtype, rows, cols, gamma, eps, rstd, orientation, scale_rule, elem,
                                   q_row, s_row, q_col, s_col, sf_layout, stream);
 }
