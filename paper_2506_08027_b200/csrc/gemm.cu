@@ -334,8 +334,13 @@ extern "C" int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, i
     p.store_d = 1;
     p.num_problems = count;
     GemmMaps m;
+    // Deepest reductions first: the persistent workers take tiles round-robin in this order, so the launch ends on the
+    // shallow tiles and the workers finish within one short tile of each other instead of one long one.
+    int order[MAX_PROBLEMS] = {0, 1, 2};
+    for (int i = 1; i < count; ++i)
+        for (int j = i; j > 0 && problems[order[j]].K > problems[order[j - 1]].K; --j) { const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
     for (int i = 0; i < MAX_PROBLEMS; ++i) {
-        const mxfp8_gemm_problem& g = problems[i < count ? i : 0];   // unused slots repeat the first product: every map stays valid
+        const mxfp8_gemm_problem& g = problems[i < count ? order[i] : order[0]];   // unused slots repeat the first product: every map stays valid
         if (i < count) {
             if (g.a_major != MXFP8_K_MAJOR && g.a_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
             if (g.b_major != MXFP8_K_MAJOR && g.b_major != MXFP8_MN_MAJOR) return MXFP8_ERR_ENUM;
@@ -364,7 +369,7 @@ extern "C" int mxfp8_gemm_multi(const mxfp8_gemm_problem* problems, int count, i
         if (!ok) return MXFP8_ERR_CUDA;
     }
     // the single-product parameters and maps are unused in this mode but must be valid
-    p.M = problems[0].M; p.N = problems[0].N; p.K = problems[0].K;
+    p.M = problems[order[0]].M; p.N = problems[order[0]].N; p.K = problems[order[0]].K;
     m.a = m.multi.p[0].a; m.b = m.multi.p[0].b; m.sfa = m.multi.p[0].sfa; m.sfb = m.multi.p[0].sfb; m.d = m.multi.p[0].d;
     m.qrow = m.d; m.qcol = m.d;
     return launch_gemm<256, true, MULTI>(m, p, static_cast<cudaStream_t>(stream));
