@@ -44,9 +44,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # summarised under profiles/: the FPROP GEMM of this step, and the quantize kernel on a
 # 128 MB BF16 tensor (the size of dY, the largest cast of the step).  Writes still dirty in
 # L2 when the kernel ends are not counted by ncu, so both are below the algorithmic bytes.
-NCU_TRAFFIC_GEMM_FPROP = 49.8e6 + 85.3e6
-NCU_TRAFFIC_GEMM_MULTI = 293.4e6 + 189.0e6          # the three-product launch of the step (dram read + write, ncu)
-NCU_TRAFFIC_QUANTIZE_STEP = 201.4e6 + 152.5e6       # the batched cast of X, W, dY (408.9 MB algorithmic; part of the output still in L2)
+NCU_TRAFFIC_GEMM_FPROP = 49.3e6 + 84.8e6
+NCU_TRAFFIC_GEMM_MULTI = 325.3e6 + 153.5e6          # the three-product launch of the step (dram read + write, ncu)
+NCU_TRAFFIC_QUANTIZE_STEP = 201.4e6 + 153.0e6       # the batched cast of X, W, dY (408.9 MB algorithmic; part of the output still in L2)
 
 PASSES_PER_STEP = 64                                  # micro-batches per timed step (see the module docstring)
 STEP_FLOP = 3 * 2.0 * T * H * F                       # one pass: three GEMMs of 275 GFLOP
