@@ -45,14 +45,23 @@ namespace gemm {
 constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 128;            // K bytes per pipeline stage = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 320;
-// Kernels with the fused MXFP8 output run 384 threads: warps 0-3 form a warp group of their own (producer, MMA issuer,
-// two idle warps) that hands most of its registers to the two warp groups of epilogue warps (setmaxnreg), because the
-// fused epilogue needs more than the 168 registers per thread that ten warps leave: with 168 it spilled 40 registers
-// per thread, and the spills missed the small L1 that 223 KB of shared memory leave (600 000 local loads per launch,
-// long-scoreboard the top stall, 4000 cycles per tile that nothing could hide).
+// Every kernel runs 384 threads in three warp groups: warps 0-3 (producer, MMA issuer, two idle warps) and the
+// eight epilogue warps 4-11.  At launch each thread holds 168 registers (what twelve warps leave); the first group
+// then shrinks to 104 registers per thread and the epilogue groups grow to 200 (setmaxnreg, placed at the top of each
+// role's branch so that ptxas allocates every role against its own budget).  Why: the fused MXFP8 epilogue needs more
+// than 168 registers -- with ten warps of 168 it spilled 40 per thread and the reloads missed the 30 KB of L1 that
+// 223 KB of shared memory leave (600 000 local loads per launch, 4000 cycles per tile that nothing hid) -- and the
+// plain kernels turned out 7-13 % faster per K block in this layout as well (8192^3: 638 -> 565 cycles per K block in
+// an interleaved A/B run; the joint launch of the benchmark 0.485 -> 0.399 Mcycles).  MXFP8_GEMM_320 (compile time)
+// brings the ten-warp layout back for the plain kernels, for comparison.
 template <bool EPI> struct Roles {
-    static constexpr int THREADS = EPI ? 384 : GEMM_THREADS;
-    static constexpr int EPI_WARP0 = EPI ? 4 : 2;       // first of the eight epilogue warps
+#ifdef MXFP8_GEMM_320
+    static constexpr bool WIDE = EPI;
+#else
+    static constexpr bool WIDE = true;
+#endif
+    static constexpr int THREADS = WIDE ? 384 : GEMM_THREADS;
+    static constexpr int EPI_WARP0 = WIDE ? 4 : 2;      // first of the eight epilogue warps
     static constexpr int REGS_FEW = 104, REGS_MANY = 200;
 };
 constexpr int EPI_WARPS = 8;
@@ -708,7 +717,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     constexpr int EW0 = Roles<EPI>::EPI_WARP0;
     // EPI: the first warp group shrinks to REGS_FEW registers per thread, the epilogue warp groups grow to REGS_MANY
     if (warp == 0) {
-        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
+        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
         // ------------------------------------------------------------------ TMA producer
         // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
         // ring-depth-unrolled loop as the MMA warp.
@@ -783,7 +792,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
+        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         // The whole warp walks the loop so that descriptors stay in uniform registers; one
         // elected lane issues the tcgen05 instructions.  The loop runs over all K blocks of all
@@ -892,7 +901,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp >= EW0) {
-        if constexpr (EPI) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_MANY));
+        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_MANY));
         // ------------------------------------------------------------------ epilogue warps
         constexpr int CW = BN / 2;               // accumulator columns per epilogue warp
         const int q = warp & 3;                  // TMEM lane quadrant this warp may read
@@ -1069,7 +1078,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
     } else {
-        if constexpr (EPI) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));   // the two idle warps of the first group
+        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));   // the two idle warps of the first group
     }
 
     tc_fence_before();
