@@ -45,20 +45,20 @@ namespace gemm {
 constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 128;            // K bytes per pipeline stage = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 320;
-// Every kernel runs 384 threads in three warp groups: warps 0-3 (producer, MMA issuer, two idle warps) and the
+// The kernels run 384 threads in three warp groups: warps 0-3 (producer, MMA issuer, two idle warps) and the
 // eight epilogue warps 4-11.  At launch each thread holds 168 registers (what twelve warps leave); the first group
 // then shrinks to 104 registers per thread and the epilogue groups grow to 200 (setmaxnreg, placed at the top of each
 // role's branch so that ptxas allocates every role against its own budget).  Why: the fused MXFP8 epilogue needs more
 // than 168 registers -- with ten warps of 168 it spilled 40 per thread and the reloads missed the 30 KB of L1 that
 // 223 KB of shared memory leave (600 000 local loads per launch, 4000 cycles per tile that nothing hid) -- and the
 // plain kernels turned out 7-13 % faster per K block in this layout as well (8192^3: 638 -> 565 cycles per K block in
-// an interleaved A/B run; the joint launch of the benchmark 0.485 -> 0.399 Mcycles).  MXFP8_GEMM_320 (compile time)
-// brings the ten-warp layout back for the plain kernels, for comparison.
-template <bool EPI> struct Roles {
+// an interleaved A/B run; the joint launch of the benchmark 0.485 -> 0.399 Mcycles).  The one exception found is the
+// reduction-grouped WGRAD (tiles of 5-8 K blocks), 27 % slower in this layout: it keeps ten warps of 168 registers.
+template <bool EPI, int MODE> struct Roles {
 #ifdef MXFP8_GEMM_320
     static constexpr bool WIDE = EPI;
 #else
-    static constexpr bool WIDE = true;
+    static constexpr bool WIDE = EPI || MODE != 2 /* GROUP_K */;
 #endif
     static constexpr int THREADS = WIDE ? 384 : GEMM_THREADS;
     static constexpr int EPI_WARP0 = WIDE ? 4 : 2;      // first of the eight epilogue warps
@@ -135,12 +135,25 @@ enum { DENSE = 0, GROUP_M = 1, GROUP_K = 2, MULTI = 3, SCATTER = 4 };
 constexpr int MAX_OWNERS = 8;   // the owners' output maps take the place of MultiMaps (15 maps)
 static_assert(sizeof(MultiMaps) >= MAX_OWNERS * sizeof(CUtensorMap), "owner maps must fit where the MULTI maps go");
 
-// BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a
-// tile has 2*BM rows.  BN = 256 leaves room for one accumulator only (2 x 256 columns would fill
-// TMEM and the scales need columns too); BN = 192 and 128 double-buffer it, so the epilogue of
-// one tile runs under the MMAs of the next.
-template <int BN, bool PAIR> struct Cfg {
-    static constexpr int ACC_STAGES = (BN == 256) ? 1 : 2;
+// Modes whose 256-wide tiles use the two overlapping accumulators (see Cfg).  Measured in interleaved A/B runs, in
+// cycles: single products -6 % at K = 2048 and at 8192^3 and nothing lost elsewhere, token-grouped products -2 %; but
+// the joint launch of up to three products +14 % and the reduction-grouped WGRAD +36 %, so those (and the adding
+// mode, not measured) keep the single accumulator.
+__host__ __device__ constexpr bool overlap_for(int mode) { return mode == DENSE || mode == GROUP_M; }
+
+// BN = accumulator columns per CTA = N extent of one tile (256, 192 or 128).  In PAIR mode a tile has 2*BM rows.
+// BN = 192 and 128 have two accumulators side by side, so the epilogue of one tile runs under the MMAs of the next.
+// Two 256-column accumulators plus scale columns do not fit into the 512 columns of TMEM, so at BN = 256 there is
+// either one accumulator (OVL = false: every tile boundary waits for the whole drain) or two that OVERLAP (OVL = true):
+// accumulator 0 at columns [0, 256), accumulator 1 at [224, 480); the 32 shared columns are the last 32 of a tile on
+// accumulator 0 and the first 32 of a tile on accumulator 1.  The epilogue warps that own them drain them first and
+// signal a barrier of their own (ovl); the next tile's MMAs wait for that barrier (and for the long-finished full drain
+// of the tile before it).  The scales then alternate between two 12-column slots at [480, 504): tcgen05.cp and
+// tcgen05.mma execute in issue order.  Which modes overlap is decided by measurement (overlap_for).
+template <int BN, bool PAIR, bool OVL> struct Cfg {
+    static constexpr bool OVERLAP = OVL && (BN == 256);
+    static constexpr int ACC_STAGES = (BN == 256 && !OVERLAP) ? 1 : 2;
+    static constexpr int ACC_STRIDE = OVERLAP ? BN - 32 : BN;
     static constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // B rows (N indices) this CTA loads
     static constexpr int B_SLABS = (B_ROWS + 127) / 128;       // 128-wide slabs when B is MN-major
     static constexpr int A_BYTES = BM * BK;
@@ -151,18 +164,20 @@ template <int BN, bool PAIR> struct Cfg {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + 512 + 512 * SFB_ATOMS;
     static constexpr int STAGES = (206 * 1024) / STAGE_BYTES > 8 ? 8 : (206 * 1024) / STAGE_BYTES;
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;          // TMEM columns of scales per stage
-    static constexpr int SF_COL0 = ACC_STAGES * BN;            // first scale column
+    static constexpr int SF_COL0 = ACC_STRIDE * (ACC_STAGES - 1) + BN;   // first scale column
     static constexpr int SMEM_A = 0;
     static constexpr int SMEM_B = SMEM_A + STAGES * A_BYTES;
     static constexpr int SMEM_SFA = SMEM_B + STAGES * B_BYTES;
     static constexpr int SMEM_SFB = SMEM_SFA + STAGES * 512;
     static constexpr int SMEM_EPI = SMEM_SFB + STAGES * 512 * SFB_ATOMS;      // 8 x 2 KB, 512-aligned
-    static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES + 1;
+    static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES + 2;
     static constexpr int SMEM_BAR = SMEM_EPI + EPI_WARPS * EPI_BUF_BYTES;
     static constexpr int SMEM_MISC = SMEM_BAR + NUM_BARS * 8;  // tmem pointer, abort flag, bad-offsets flag
     static constexpr int SMEM_GROUPS = SMEM_MISC + 16;         // group offsets and first-tile indices, (MAX_GROUPS + 1) ints each
     static constexpr int SMEM_TOTAL = SMEM_GROUPS + 2 * (MAX_GROUPS + 1) * 4 + 4 + 1024;   // + slack to align the base to 1024
-    static_assert(SF_COL0 + STAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
+    static constexpr int SF_SLOTS = OVERLAP ? 2 : STAGES;      // scale slot of smem stage s: s % SF_SLOTS
+    static_assert(SF_COL0 + SF_SLOTS * SF_COLS <= TMEM_COLS, "TMEM budget");
+    static_assert(STAGES % SF_SLOTS == 0, "a stage keeps its scale slot from one pass over the ring to the next");
     static_assert(SMEM_TOTAL <= 227 * 1024, "shared memory budget");
     static_assert(SMEM_EPI % 512 == 0, "staging buffers need 512-byte alignment for the 64-byte swizzle");
     static_assert((BN / 2) % 32 == 0, "each epilogue warp owns whole 32-column chunks");
@@ -601,14 +616,14 @@ __device__ __forceinline__ int epoch_len(int nkb, int kc_max)
 // DEEP: reductions longer than kc_max K blocks, summed in epochs (separate instantiations again, so that the
 //       kernels of the common depths keep the straight-line epilogue)
 template <int BN, bool PAIR, int MODE, bool EPI, bool DEEP>
-__global__ void __launch_bounds__(Roles<EPI>::THREADS, 1)
+__global__ void __launch_bounds__(Roles<EPI, MODE>::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
             const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_qrow,
             const __grid_constant__ CUtensorMap tmap_qcol, const __grid_constant__ MultiMaps mmaps,
             const __grid_constant__ GemmParams p)
 {
-    using C = Cfg<BN, PAIR>;
+    using C = Cfg<BN, PAIR, overlap_for(MODE)>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;   // 128-byte swizzle needs 1024-byte alignment
@@ -620,6 +635,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * C::STAGES + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * C::STAGES + C::ACC_STAGES + a); };
     const uint32_t drain_bar = bar0 + 8u * (2 * C::STAGES + 2 * C::ACC_STAGES);
+    const uint32_t ovl_bar = drain_bar + 8u;   // OVERLAP: the columns that both accumulators use have been drained
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + C::SMEM_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::SMEM_MISC + 4);
     volatile int* bad_groups = reinterpret_cast<volatile int*>(base_ptr + C::SMEM_MISC + 8);
@@ -644,6 +660,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * EPI_WARPS);
         }
         mbar_init(drain_bar, 1);
+        mbar_init(ovl_bar, (PAIR ? 2 : 1) * (EPI_WARPS / 2));
         *abort_flag = 0;
         *bad_groups = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -652,7 +669,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // every CTA reads the offsets, checks them (non-negative, non-decreasing, multiples of 128,
         // inside the tensor) and, for GROUP_M, turns them into the first tile index of each group
         const int G = p.num_groups;
-        for (int i = threadIdx.x; i <= G; i += Roles<EPI>::THREADS) goff[i] = p.group_offsets[i];
+        for (int i = threadIdx.x; i <= G; i += Roles<EPI, MODE>::THREADS) goff[i] = p.group_offsets[i];
         __syncthreads();
         if (warp == 2) {
             bool bad = false;
@@ -714,10 +731,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int num_tiles = (MODE == DENSE || MODE == MULTI || MODE == SCATTER) ? p.num_tiles
                         : (*bad_groups ? 0 : (MODE == GROUP_M ? tstart[p.num_groups] : p.num_groups * p.tiles_m * p.tiles_n));
 
-    constexpr int EW0 = Roles<EPI>::EPI_WARP0;
+    constexpr int EW0 = Roles<EPI, MODE>::EPI_WARP0;
     // EPI: the first warp group shrinks to REGS_FEW registers per thread, the epilogue warp groups grow to REGS_MANY
     if (warp == 0) {
-        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
+        if constexpr (Roles<EPI, MODE>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI, MODE>::REGS_FEW));
         // ------------------------------------------------------------------ TMA producer
         // The whole warp walks the loop; one elected lane issues the copies.  Same flat,
         // ring-depth-unrolled loop as the MMA warp.
@@ -792,7 +809,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));
+        if constexpr (Roles<EPI, MODE>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI, MODE>::REGS_FEW));
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         // The whole warp walks the loop so that descriptors stay in uniform registers; one
         // elected lane issues the tcgen05 instructions.  The loop runs over all K blocks of all
@@ -849,7 +866,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                             const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
                             ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag, p.status);
                             if (!ok) break;
-                            d_tmem = tmem_base + as * BN;
+                            if (C::OVERLAP && acc_it > 0) {   // the shared columns: drained by the accumulator use just before
+                                ok = warp_wait(ovl_bar, (acc_it - 1u) & 1u, abort_flag, p.status);
+                                if (!ok) break;
+                            }
+                            d_tmem = tmem_base + as * C::ACC_STRIDE;
                         }
                     }
                     if constexpr (DEEP) {
@@ -858,13 +879,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                             const uint32_t aph = (acc_it / C::ACC_STAGES) & 1u;
                             ok = warp_wait(tempty_bar(as), aph ^ 1u, abort_flag, p.status);
                             if (!ok) break;
-                            d_tmem = tmem_base + as * BN;
+                            if (C::OVERLAP && acc_it > 0) {   // the shared columns: drained by the accumulator use just before
+                                ok = warp_wait(ovl_bar, (acc_it - 1u) & 1u, abort_flag, p.status);
+                                if (!ok) break;
+                            }
+                            d_tmem = tmem_base + as * C::ACC_STRIDE;
                         }
                     }
                     ok = warp_wait(full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS;
+                    const uint32_t sfa_t = tmem_base + C::SF_COL0 + (s % C::SF_SLOTS) * C::SF_COLS;
                     const uint32_t sfb_t = sfa_t + 4;
                     if (elect_one()) {
                         tc_cp_sf<PAIR>(sfa_t, desc64(sfa_lo0 + s * (512 >> 4), sf_hi));
@@ -901,7 +926,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else if (warp >= EW0) {
-        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_MANY));
+        if constexpr (Roles<EPI, MODE>::WIDE) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<EPI, MODE>::REGS_MANY));
         // ------------------------------------------------------------------ epilogue warps
         constexpr int CW = BN / 2;               // accumulator columns per epilogue warp
         const int q = warp & 3;                  // TMEM lane quadrant this warp may read
@@ -932,9 +957,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN + half * CW;
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + as * C::ACC_STRIDE + half * CW;
+                // OVERLAP: the warps of the upper half own the shared columns of a tile on accumulator 0 (its last chunk),
+                // the warps of the lower half those of a tile on accumulator 1 (its first chunk): drained first, signalled at once
+                const bool own_ovl = C::OVERLAP && half == (as ^ 1);
+                const int ovl_c = as == 0 ? CW / 32 - 1 : 0;
+                if (own_ovl) {
 #pragma unroll
-                for (int c = 0; c < CW / 32; ++c) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+                    for (int c = 0; c < CW / 32; ++c)
+                        if (c == ovl_c) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+                    tc_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR) mbar_arrive_cluster(map_to_cta(ovl_bar, 0));
+                        else mbar_arrive(ovl_bar);
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < CW / 32; ++c)
+                    if (!(own_ovl && c == ovl_c)) tc_ld32(t_row + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
                 tc_wait_ld();
                 // the accumulator now lives in registers: hand TMEM back to the MMA warp of the leader
                 tc_fence_before();
@@ -954,15 +996,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                         ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t t_row2 = tmem_base + ((uint32_t)(q * 32) << 16) + as2 * BN + half * CW;
+                        const uint32_t t_row2 = tmem_base + ((uint32_t)(q * 32) << 16) + as2 * C::ACC_STRIDE + half * CW;
+                        const bool own2 = C::OVERLAP && half == (as2 ^ 1);
+                        const int ovl2 = as2 == 0 ? CW / 32 - 1 : 0;
 #pragma unroll
-                        for (int c = 0; c < CW / 8; ++c) {
-                            uint32_t w[8];
-                            tc_ld8(t_row2 + c * 8, w);
-                            tc_wait_ld();
+                        for (int pass = 0; pass < 2; ++pass) {      // pass 0: the shared columns (their owner only), pass 1: the rest
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                v[c * 8 + i] = __float_as_uint(__fadd_rn(__uint_as_float(v[c * 8 + i]), __uint_as_float(w[i])));
+                            for (int c = 0; c < CW / 8; ++c) {
+                                if ((pass == 0) != (own2 && (c >> 2) == ovl2)) continue;
+                                uint32_t w[8];
+                                tc_ld8(t_row2 + c * 8, w);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    v[c * 8 + i] = __float_as_uint(__fadd_rn(__uint_as_float(v[c * 8 + i]), __uint_as_float(w[i])));
+                            }
+                            if (pass == 0 && own2) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    if (PAIR) mbar_arrive_cluster(map_to_cta(ovl_bar, 0));
+                                    else mbar_arrive(ovl_bar);
+                                }
+                            }
                         }
                         tc_fence_before();
                         __syncwarp();
@@ -1078,7 +1134,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
     } else {
-        if constexpr (Roles<EPI>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI>::REGS_FEW));   // the two idle warps of the first group
+        if constexpr (Roles<EPI, MODE>::WIDE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<EPI, MODE>::REGS_FEW));   // the two idle warps of the first group
     }
 
     tc_fence_before();
@@ -1105,13 +1161,13 @@ struct GemmMaps { CUtensorMap a, b, sfa, sfb, d, qrow, qcol; MultiMaps multi; };
 template <int BN, bool PAIR, int MODE, bool EPI, bool DEEP>
 int launch_kernel(const GemmMaps& m, const GemmParams& p, int workers, cudaStream_t stream)
 {
-    using C = Cfg<BN, PAIR>;
+    using C = Cfg<BN, PAIR, overlap_for(MODE)>;
     auto kernel = gemm_kernel<BN, PAIR, MODE, EPI, DEEP>;
     static unsigned long long smem_set = 0;
     if (ensure_dynamic_smem(kernel, C::SMEM_TOTAL, smem_set) != cudaSuccess) return MXFP8_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * workers : workers));
-    cfg.blockDim = dim3(Roles<EPI>::THREADS);
+    cfg.blockDim = dim3(Roles<EPI, MODE>::THREADS);
     cfg.dynamicSmemBytes = C::SMEM_TOTAL;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -1123,7 +1179,7 @@ int launch_kernel(const GemmMaps& m, const GemmParams& p, int workers, cudaStrea
     cfg.numAttrs = 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, m.a, m.b, m.sfa, m.sfb, m.d, m.qrow, m.qcol, m.multi, p);
     if (getenv("MXFP8_LOG"))
-        fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d%s -> %s\n", cfg.gridDim.x, Roles<EPI>::THREADS,
+        fprintf(stderr, "mxfp8_gemm launch grid=%u block=%d smem=%d tiles=%dx%d kblocks=%d%s -> %s\n", cfg.gridDim.x, Roles<EPI, MODE>::THREADS,
                 C::SMEM_TOTAL, p.tiles_m, p.tiles_n, p.num_kb, DEEP ? " (epochs)" : "", cudaGetErrorString(err));
     count_launch(1);
     return err == cudaSuccess ? MXFP8_OK : MXFP8_ERR_CUDA;
@@ -1142,7 +1198,7 @@ bool gemm_device(GemmDevice& out);
 template <int BN, bool PAIR, int MODE = DENSE, bool EPI = false>
 int launch_gemm(const GemmMaps& m, GemmParams p, cudaStream_t stream)
 {
-    using C = Cfg<BN, PAIR>;
+    using C = Cfg<BN, PAIR, overlap_for(MODE)>;
     p.tiles_m = (int)((p.M + (PAIR ? 2 * BM : BM) - 1) / (PAIR ? 2 * BM : BM));
     p.tiles_n = (int)((p.N + BN - 1) / BN);
     p.stage_tx = (PAIR ? 2u : 1u) * (uint32_t)(C::A_BYTES + (p.b_mn ? C::B_BYTES_MN : C::B_BYTES_K) + 512 + 512 * C::SFB_ATOMS);
