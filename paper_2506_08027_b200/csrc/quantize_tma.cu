@@ -104,6 +104,7 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
         QParams& q = p.t[i];
         q.rows = it.rows; q.cols = it.cols; q.rule = scale_rule; q.sf_layout = sf_layout;
         q.tiles_x = (int)((it.cols + t_cols - 1) / t_cols);
+        q.tiles_x_magic = div_magic((uint32_t)q.tiles_x);
         q.tiles_y = (int)((it.rows + T_ROWS - 1) / T_ROWS);
         q.q_row = static_cast<uint8_t*>(it.q_row);
         q.q_col = static_cast<uint8_t*>(it.q_col);

@@ -12,7 +12,9 @@
 //   pass A (column blocks): amax down the 32 rows inside the lane, packed bf16x2 max for BF16
 //   pass B (row blocks)   : amax across the lanes of a 32-column block by xor-shuffles; BF16 rows
 //                           go through the shuffles two at a time (one in each half of a register)
-//   scale: integer form of Algorithm 1 / App. A.1 on the amax bit pattern (see mxfp8_device.cuh)
+//   scale: integer form of Algorithm 1 / App. A.1 on the amax bit pattern (see mxfp8_device.cuh); the two BF16 rows of a
+//          pair keep sharing one register through it (16-bit lanes).  The bytes wait in shared memory in the order of a
+//          swizzled atom and leave once per tile: 16 bytes per lane for a whole BF16 tile, one word per row / column else
 //   cast : x * 2^-e in FP32 (exact), cvt.rn.satfinite to the element type (e4m3x2 / e5m2x2, or the
 //          6- / 4-bit types, whose codes are then packed 16 to a 16-byte slot across the lanes)
 //   One launch takes up to 8 tensors (their tiles form one pool); optional in-place prologues on the
@@ -32,6 +34,13 @@ constexpr int T_ROWS = 128;
 constexpr int T_BYTES = 256;                 // source bytes per tile row
 constexpr int IN_BYTES = T_ROWS * T_BYTES;   // 32 KB
 constexpr int QT_THREADS = 128;
+constexpr int RING = 2;                      // slots of the input ring
+constexpr int QT_CTAS_PER_SM = 3;            // by shared memory (2 x 32 KB + staging) and by registers (168)
+// Scale bytes of a tile wait in shared memory in the order of one swizzled 128 x 4 atom (see mxfp8.h): those of row
+// (or column) i of the tile start at stage_offset(i), one byte per block, 16 bytes from those of row i + 1.  A whole
+// BF16 tile's scales in the swizzled layout are exactly one atom, which then leaves as 32 16-byte stores.
+constexpr int STAGE_PITCH = 16;
+__device__ __forceinline__ int stage_offset(int i) { return (i & 31) * STAGE_PITCH + (i >> 5) * 4; }
 #ifdef MXFP8_TEST_HOOKS
 constexpr uint64_t QT_WAIT_LIMIT_NS = 5000000ull;      // test build: the bounded wait gives up after 5 ms
 #else
@@ -42,6 +51,7 @@ struct QParams {
     int64_t rows, cols;
     int rule, sf_layout;
     int tiles_x, tiles_y;
+    uint32_t tiles_x_magic;                  // div_magic(tiles_x)
     uint8_t* q_row;
     uint8_t* q_col;
     uint8_t* s_row;
@@ -216,6 +226,27 @@ __device__ __forceinline__ uint32_t hmax2(uint32_t a, uint32_t b)
 // flags a packed pair of bf16 magnitudes if either half is Inf or NaN
 __device__ __forceinline__ uint32_t nonfinite2(uint32_t z) { return (z + 0x00800080u) & 0x80008000u; }
 
+// inv_exp_field for two BF16 amax patterns at once (one per 16-bit half of z, both finite or flagged by the
+// caller).  A BF16 pattern is the upper half of the FP32 one, so the rule's offset acts through its upper
+// half alone (the lower half of the sum cannot carry), and every step stays inside its 16 bits:
+//   e = (h + off16) >> 7 (at most 0x100);  field = min(254 + emax - e, 254), never negative.
+template <int ELEM>
+__device__ __forceinline__ uint32_t inv_exp_field2(uint32_t z, uint32_t rule_offset16x2)
+{
+    const uint32_t e2 = ((z + rule_offset16x2) >> 7) & 0x01FF01FFu;
+    return __vminu2((254u + ElemTraits<ELEM>::emax) * 0x00010001u - e2, 0x00FE00FEu);
+}
+
+// n / d and n % d for 0 <= n < 2^31, 1 <= d: a multiply by magic = min(floor(2^32 / d), 2^32 - 1) gives the
+// quotient or one less, one correction settles it.
+__host__ __device__ __forceinline__ uint32_t div_magic(uint32_t d) { return d <= 1u ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / d); }
+__device__ __forceinline__ void divmod(uint32_t n, uint32_t d, uint32_t magic, int& q, int& r)
+{
+    uint32_t qq = __umulhi(n, magic), rr = n - qq * d;
+    if (rr >= d) { rr -= d; ++qq; }
+    q = (int)qq; r = (int)rr;
+}
+
 // X = 2^(b-127) as FP32 from the exponent field of 1/X (b = 254 - field; b = 0 is the subnormal 2^-127)
 __device__ __forceinline__ float scale_from_inv(float inv)
 {
@@ -302,7 +333,8 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
     constexpr bool BF = (DTYPE == MXFP8_BF16);
     constexpr int VEC = BF ? 4 : 2;
     constexpr int LPB = 32 / VEC;
-    uint32_t bad = 0u;
+    uint32_t bad = 0u, zall = 0u;
+    const uint32_t rule_offset16x2 = (rule_offset >> 16) * 0x00010001u;
     float col_inv[VEC], col_xs[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) { col_inv[i] = 1.f; col_xs[i] = 1.f; }
@@ -313,8 +345,8 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const uint2 w = *reinterpret_cast<const uint2*>(my_in + j * T_BYTES);
-                m0 = hmax2_abs(m0, w.x);
-                m1 = hmax2_abs(m1, w.y);
+                m0 = hmax2(m0, w.x & 0x7FFF7FFFu);     // the running maximum is a magnitude already
+                m1 = hmax2(m1, w.y & 0x7FFF7FFFu);
             }
             bad |= nonfinite2(m0) | nonfinite2(m1);
             cbits[0] = m0 << 16; cbits[1] = m0 & 0xFFFF0000u;
@@ -336,7 +368,7 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
             const uint32_t ie = inv_exp_field<ELEM>(cbits[i], rule_offset);
             col_inv[i] = __uint_as_float(ie << 23);
             col_xs[i] = scale_from_inv(col_inv[i]);
-            my_sm_col[i * 4] = (uint8_t)(254u - ie);
+            my_sm_col[i * STAGE_PITCH] = (uint8_t)(254u - ie);
         }
     }
 #pragma unroll
@@ -356,14 +388,14 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
                 uint32_t z = hmax2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));   // (amax_j, amax_j+1) of this lane
 #pragma unroll
                 for (int off = 1; off < LPB; off <<= 1) z = hmax2(z, __shfl_xor_sync(0xFFFFFFFFu, z, off));
-                bad |= nonfinite2(z);
-                const uint32_t ie0 = inv_exp_field<ELEM>(z << 16, rule_offset);
-                const uint32_t ie1 = inv_exp_field<ELEM>(z & 0xFFFF0000u, rule_offset);
-                inv0 = __uint_as_float(ie0 << 23);
-                inv1 = __uint_as_float(ie1 << 23);
+                zall = __vmaxu2(zall, z);            // magnitudes order as unsigned integers: finite < Inf < NaN
+                const uint32_t ie2 = inv_exp_field2<ELEM>(z, rule_offset16x2);   // both rows' fields, one per half
+                inv0 = __uint_as_float(ie2 << 23);
+                inv1 = __uint_as_float((ie2 & 0xFFFF0000u) << 7);
                 if ((lane & (LPB - 1)) == 0) {
-                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
-                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
+                    const uint32_t sb = 0x00FE00FEu - ie2;
+                    my_sm_row[j * STAGE_PITCH] = (uint8_t)sb;
+                    my_sm_row[(j + 1) * STAGE_PITCH] = (uint8_t)(sb >> 16);
                 }
             }
         } else {
@@ -384,8 +416,8 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
                 inv0 = __uint_as_float(ie0 << 23);
                 inv1 = __uint_as_float(ie1 << 23);
                 if ((lane & (LPB - 1)) == 0) {
-                    my_sm_row[j * 4] = (uint8_t)(254u - ie0);
-                    my_sm_row[(j + 1) * 4] = (uint8_t)(254u - ie1);
+                    my_sm_row[j * STAGE_PITCH] = (uint8_t)(254u - ie0);
+                    my_sm_row[(j + 1) * STAGE_PITCH] = (uint8_t)(254u - ie1);
                 }
             }
         }
@@ -404,7 +436,7 @@ __device__ __forceinline__ bool slab_fast(const uint8_t* __restrict__ my_in, uin
             emit<ELEM, VEC, EMU>(c0 + pitch, x1, col_inv, col_xs, lane);
         }
     }
-    return __any_sync(0xFFFFFFFFu, bad != 0u);
+    return __any_sync(0xFFFFFFFFu, (bad | nonfinite2(zall)) != 0u);
 }
 
 // The same slab with everything the fast path leaves out: Inf and NaN elements stay out of
@@ -450,7 +482,7 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
             const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(cmax[i]), rule_offset);
             col_inv[i] = __uint_as_float(ie << 23);
             col_xs[i] = scale_from_inv(col_inv[i]);
-            my_sm_col[i * 4] = (uint8_t)(254u - ie);
+            my_sm_col[i * STAGE_PITCH] = (uint8_t)(254u - ie);
         }
     }
 #pragma unroll 1
@@ -469,7 +501,7 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
             for (int off = 1; off < LPB; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
             const uint32_t ie = inv_exp_field<ELEM>(__float_as_uint(m), rule_offset);
             const float inv = __uint_as_float(ie << 23);
-            if ((lane & (LPB - 1)) == 0) my_sm_row[j * 4] = (uint8_t)(254u - ie);
+            if ((lane & (LPB - 1)) == 0) my_sm_row[j * STAGE_PITCH] = (uint8_t)(254u - ie);
             if (j < rows_here) {   // warp-uniform; lanes beyond the tensor's last column take part but do not store
                 float iv[VEC], sv[VEC];
 #pragma unroll
@@ -486,7 +518,7 @@ __device__ __noinline__ void slab_careful(const uint8_t* __restrict__ my_in, uin
 enum { PRO_NONE = 0, PRO_ELEMENTWISE = 1 /* activation or RMS normalisation */, PRO_GLU = 2 /* gated activation */ };
 
 template <int DTYPE, int ELEM, bool DO_ROW, bool DO_COL, bool EMU, int PRO>
-__global__ void __launch_bounds__(QT_THREADS, 3)
+__global__ void __launch_bounds__(QT_THREADS, QT_CTAS_PER_SM)
 quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QBatch batch)
 {
     constexpr bool BF = (DTYPE == MXFP8_BF16);
@@ -498,8 +530,8 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* in_ring = smem;                               // 2 x [128][256]
-    uint8_t* sm_scales = smem + 2 * IN_BYTES;              // 2 x ([128][4] row scales + [T_COLS][4] column scales)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);   // [0], [1]: ring slots; [2]: the up tile (gated mode)
+    uint8_t* sm_scales = smem + RING * IN_BYTES;           // 2 x (row scales + column scales of one tile, 512 bytes each)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_scales + 2048);   // [0 .. RING): ring slots; [RING]: the up tile (gated mode)
     uint8_t* up_buf = sm_scales + 2048 + 128;                         // gated mode only: [128][256], allocated by such launches
     const int glu_cols = GLU ? batch.glu_cols : 0;
 
@@ -507,9 +539,8 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     const uint32_t rule_offset = (batch.t[0].rule == MXFP8_RULE_PAPER) ? paper_offset<ELEM>() : 0u;
 
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[1])));
-        if (GLU) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[2])));
+        for (int k = 0; k < RING; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[k])));
+        if (GLU) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[RING])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -521,19 +552,21 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         if (batch.test_skip_tile && t == batch.test_skip_tile - 1) return;   // never issued: the consumer's bounded wait runs out
 #endif
         while (t >= batch.tile_start[load_ti + 1]) ++load_ti;
-        const int lt = t - batch.tile_start[load_ti], tx = batch.t[load_ti].tiles_x;
+        int lx, ly;
+        divmod((uint32_t)(t - batch.tile_start[load_ti]), (uint32_t)batch.t[load_ti].tiles_x, batch.t[load_ti].tiles_x_magic, ly, lx);
         const uint32_t b = smem_addr(&bars[buf]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&maps.m[load_ti]), "r"(b), "r"((lt % tx) * T_COLS), "r"((lt / tx) * T_ROWS)
+                     ::"r"(smem_addr(in_ring + buf * IN_BYTES)), "l"(&maps.m[load_ti]), "r"(b), "r"(lx * T_COLS), "r"(ly * T_ROWS)
                      : "memory");
     };
     auto issue_up = [&](int t) {              // gated mode (one tensor per launch): the up half of tile t
-        const int tx = batch.t[0].tiles_x;
-        const uint32_t b = smem_addr(&bars[2]);
+        int lx, ly;
+        divmod((uint32_t)t, (uint32_t)batch.t[0].tiles_x, batch.t[0].tiles_x_magic, ly, lx);
+        const uint32_t b = smem_addr(&bars[RING]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)IN_BYTES) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                     ::"r"(smem_addr(up_buf)), "l"(&maps.m[batch.up_map]), "r"(b), "r"(glu_cols + (t % tx) * T_COLS), "r"((t / tx) * T_ROWS)
+                     ::"r"(smem_addr(up_buf)), "l"(&maps.m[batch.up_map]), "r"(b), "r"(glu_cols + lx * T_COLS), "r"(ly * T_ROWS)
                      : "memory");
     };
     // bounded wait on one of the barriers: false when the limit passed
@@ -555,28 +588,28 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
     };
     int tile = blockIdx.x, ti = 0;
     if (tid == 0) {
-        if (tile < num_tiles) issue_load(tile, 0);
-        if (tile + (int)gridDim.x < num_tiles) issue_load(tile + gridDim.x, 1);
+        for (int k = 0; k < RING; ++k)
+            if (tile + k * (int)gridDim.x < num_tiles) issue_load(tile + k * gridDim.x, k);
         if (GLU && tile < num_tiles) issue_up(tile);
     }
 
     for (int it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
-        const int buf = it & 1;
-        const uint32_t phase = (uint32_t)(it >> 1) & 1u;
+        const int buf = it % RING;
+        const uint32_t phase = (uint32_t)(it / RING) & 1u;
         const uint32_t bar_a = smem_addr(&bars[buf]);
         uint8_t* in_tile = in_ring + buf * IN_BYTES;
-        uint8_t* sm_row = sm_scales + buf * 1024;          // [128][4]
-        uint8_t* sm_col = sm_row + 512;                    // [T_COLS][4]
+        uint8_t* sm_row = sm_scales + (it & 1) * 1024;          // 128 rows x 4 blocks, at stage_offset(row)
+        uint8_t* sm_col = sm_row + 512;                    // T_COLS columns x 4 blocks, at stage_offset(column)
         while (tile >= batch.tile_start[ti + 1]) ++ti;
         const QParams& p = batch.t[ti];
-        const int ltile = tile - batch.tile_start[ti];
-        const int tile_x = ltile % p.tiles_x, tile_y = ltile / p.tiles_x;
+        int tile_x, tile_y;
+        divmod((uint32_t)(tile - batch.tile_start[ti]), (uint32_t)p.tiles_x, p.tiles_x_magic, tile_y, tile_x);
         const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
 
         // wait for the tile (bounded: on expiry report through the status word and leave)
         {
             bool ok = wait_bar(bar_a, phase);
-            if constexpr (GLU) ok = wait_bar(smem_addr(&bars[2]), (uint32_t)it & 1u) && ok;
+            if constexpr (GLU) ok = wait_bar(smem_addr(&bars[RING]), (uint32_t)it & 1u) && ok;
             if (!__syncthreads_and((int)ok)) {
                 if (tid == 0) atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
                 return;
@@ -637,8 +670,8 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         uint8_t* my_qrow = p.q_row + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
         uint8_t* my_qcol = p.q_col + ((grow0 + warp * 32) * p.cols + my_col) * OUT_ESZ;
         const uint32_t pitch = (uint32_t)p.cols * OUT_ESZ;
-        uint8_t* my_sm_row = sm_row + warp * 128 + lane / LPB;
-        uint8_t* my_sm_col = sm_col + lane * VEC * 4 + warp;
+        uint8_t* my_sm_row = sm_row + warp * 4 + lane / LPB;                   // row 32 warp + j: + j * STAGE_PITCH
+        uint8_t* my_sm_col = sm_col + stage_offset(lane * VEC) + warp;         // column lane * VEC + i: + i * STAGE_PITCH
         const bool whole = __all_sync(0xFFFFFFFFu, col_ok) && rows_here == 32;
         bool special = !whole;
         if (whole)
@@ -650,46 +683,59 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         // every warp is done with this ring slot: refill it with the tile after next
         __syncthreads();
         if (tid == 0) {
-            const int next = tile + 2 * (int)gridDim.x;
+            const int next = tile + RING * (int)gridDim.x;
             if (next < num_tiles) issue_load(next, buf);
         }
 
-        // ---- scale bytes (1/32 of the output): plain stores from the staging arrays ----------
+        // ---- scale bytes (1/32 of the output) leave from the staging arrays ----------
+        // A BF16 tile wholly inside the tensor fills exactly one 512-byte atom of the swizzled layout per orientation,
+        // and the staging arrays are in the atom's order: one warp stores each atom, 16 bytes per lane.
+        if (BF && !EMU && p.sf_layout == MXFP8_SF_SWIZZLED && grow0 + T_ROWS <= p.rows && gcol0 + T_COLS <= p.cols &&
+            ((reinterpret_cast<uintptr_t>(p.s_row) | reinterpret_cast<uintptr_t>(p.s_col)) & 15) == 0) {
+            if (DO_ROW && warp == 0) {
+                const int64_t atoms_k = ((p.cols >> 5) + 3) >> 2;
+                *reinterpret_cast<uint4*>(p.s_row + ((int64_t)tile_y * atoms_k + tile_x) * 512 + lane * 16) =
+                    *reinterpret_cast<const uint4*>(sm_row + lane * 16);
+            }
+            if (DO_COL && warp == (DO_ROW ? 1 : 0)) {
+                const int64_t atoms_r = ((p.rows >> 5) + 3) >> 2;
+                *reinterpret_cast<uint4*>(p.s_col + ((int64_t)tile_x * atoms_r + tile_y) * 512 + lane * 16) =
+                    *reinterpret_cast<const uint4*>(sm_col + lane * 16);
+            }
+            continue;
+        }
+        // every other tile (ragged, FP32 source, linear layout): one thread per row / per column
+        auto first_bytes = [](uint32_t word, int n) { return n >= 4 ? word : (word & ((1u << (8 * max(n, 0))) - 1u)); };
         if (DO_ROW && !EMU && tid < T_ROWS) {
             const int64_t r = grow0 + tid, ncb = p.cols >> 5, kb0 = (int64_t)tile_x * NKB;
             const int nkb = (int)min((int64_t)NKB, ncb - kb0);
+            const uint32_t v = r < p.rows ? first_bytes(*reinterpret_cast<const uint32_t*>(sm_row + stage_offset(tid)), nkb) : 0u;
             if (p.sf_layout == MXFP8_SF_SWIZZLED) {
                 // every row of a started 128-row atom is written (pad rows / pad K-blocks get 0)
-                uint8_t* d = p.s_row + ((int64_t)tile_y * ((ncb + 3) >> 2) + (kb0 >> 2)) * 512 + (tid & 31) * 16 + (tid >> 5) * 4 + (kb0 & 3);
-                uint32_t v = 0u;
-                if (r < p.rows)
-                    for (int kb = 0; kb < nkb; ++kb) v |= (uint32_t)sm_row[tid * 4 + kb] << (8 * kb);
+                uint8_t* d = p.s_row + ((int64_t)tile_y * ((ncb + 3) >> 2) + (kb0 >> 2)) * 512 + stage_offset(tid) + (kb0 & 3);
                 // a 64-column FP32 tile owns half of the atom's 4 K-blocks; the left half also zeroes
                 // the right half when no tile exists there (pad K-blocks)
                 if (NKB == 4 || ((kb0 & 3) == 0 && kb0 + NKB >= ncb)) *reinterpret_cast<uint32_t*>(d) = v;
                 else *reinterpret_cast<uint16_t*>(d) = (uint16_t)v;
             } else if (r < p.rows) {
                 uint8_t* d = p.s_row + r * ncb + kb0;
-                for (int kb = 0; kb < nkb; ++kb) d[kb] = sm_row[tid * 4 + kb];
+                for (int kb = 0; kb < nkb; ++kb) d[kb] = (uint8_t)(v >> (8 * kb));
             }
         }
         if (DO_COL && !EMU && tid < T_COLS) {
             const int64_t c = gcol0 + tid, nrb = p.rows >> 5, rb0 = (int64_t)tile_y * 4;
             const int nrb_here = (int)min((int64_t)4, nrb - rb0);
+            const uint32_t v = c < p.cols ? first_bytes(*reinterpret_cast<const uint32_t*>(sm_col + stage_offset(tid)), nrb_here) : 0u;
             if (p.sf_layout == MXFP8_SF_SWIZZLED) {
                 const int64_t padded_cols = ((p.cols + 127) >> 7) << 7;
                 if (c < padded_cols) {
-                    uint8_t* d = p.s_col + ((c >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + (c & 31) * 16 + ((c >> 5) & 3) * 4;
-                    uint32_t v = 0u;
-                    if (c < p.cols)
-                        for (int w = 0; w < nrb_here; ++w) v |= (uint32_t)sm_col[tid * 4 + w] << (8 * w);
-                    *reinterpret_cast<uint32_t*>(d) = v;
+                    *reinterpret_cast<uint32_t*>(p.s_col + ((c >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + (c & 31) * 16 + ((c >> 5) & 3) * 4) = v;
                     // pad columns no tile covers (FP32 tiles are 64 wide, atoms 128 wide)
                     if (T_COLS == 64 && tile_x == p.tiles_x - 1 && c + 64 >= (int64_t)p.tiles_x * 64 && c + 64 < padded_cols)
                         *reinterpret_cast<uint32_t*>(p.s_col + (((c + 64) >> 7) * ((nrb + 3) >> 2) + tile_y) * 512 + ((c + 64) & 31) * 16 + (((c + 64) >> 5) & 3) * 4) = 0u;
                 }
             } else if (c < p.cols) {
-                for (int w = 0; w < nrb_here; ++w) p.s_col[(rb0 + w) * p.cols + c] = sm_col[tid * 4 + w];
+                for (int w = 0; w < nrb_here; ++w) p.s_col[(rb0 + w) * p.cols + c] = (uint8_t)(v >> (8 * w));
             }
         }
     }
@@ -709,7 +755,7 @@ template <int DTYPE, int ELEM, bool R, bool C, bool EMU, int PRO>
 cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
 {
     constexpr bool GLU = (PRO == PRO_GLU);
-    constexpr int SMEM = 2 * IN_BYTES + 2048 + 128;          // ring, scale staging, barriers
+    constexpr int SMEM = RING * IN_BYTES + 2048 + 128;          // ring, scale staging, barriers
     constexpr int SMEM_USED = GLU ? SMEM + IN_BYTES : SMEM;  // + the up tile of the gated mode
     auto kernel = quantize_tma_kernel<DTYPE, ELEM, R, C, EMU, PRO>;
     static unsigned long long smem_set = 0;
@@ -718,7 +764,7 @@ cudaError_t launch(const QMaps& ms, const QBatch& p, cudaStream_t stream)
     const int tiles = p.tile_start[p.count];
     const int sms = qt_sm_count();
     if (sms <= 0) return cudaErrorInvalidDevice;
-    const int max_ctas = sms * (GLU ? 2 : 3);
+    const int max_ctas = sms * (GLU ? 2 : QT_CTAS_PER_SM);
     const int grid = tiles < max_ctas ? tiles : max_ctas;
     kernel<<<grid, QT_THREADS, SMEM_USED, stream>>>(ms, p);
     count_launch(1);
