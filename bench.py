@@ -44,9 +44,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # summarised under profiles/: the FPROP GEMM of this step, and the quantize kernel on a
 # 128 MB BF16 tensor (the size of dY, the largest cast of the step).  Writes still dirty in
 # L2 when the kernel ends are not counted by ncu, so both are below the algorithmic bytes.
-NCU_TRAFFIC_GEMM_FPROP = 49.3e6 + 84.8e6
-NCU_TRAFFIC_GEMM_MULTI = 325.3e6 + 153.5e6          # the three-product launch of the step (dram read + write, ncu)
-NCU_TRAFFIC_QUANTIZE_STEP = 201.4e6 + 153.0e6       # the batched cast of X, W, dY (408.9 MB algorithmic; part of the output still in L2)
+NCU_TRAFFIC_GEMM_FPROP = 50.0e6 + 86.2e6
+NCU_TRAFFIC_GEMM_MULTI = 333.1e6 + 153.4e6          # the three-product launch of the step (dram read + write, ncu)
+NCU_TRAFFIC_QUANTIZE_STEP = 201.4e6 + 152.6e6       # the batched cast of X, W, dY (408.9 MB algorithmic; part of the output still in L2)
 
 PASSES_PER_STEP = 64                                  # micro-batches per timed step (see the module docstring)
 STEP_FLOP = 3 * 2.0 * T * H * F                       # one pass: three GEMMs of 275 GFLOP
@@ -569,6 +569,28 @@ def _time_calls(fn, n_bufs, min_iters=10, min_ms=30.0):
         iters *= 4
 
 
+def _time_graph(fn, n_bufs, calls=20, replays=20):
+    """Device time of fn(i) in ms with the host out of the picture: `calls` launches captured once in a CUDA graph,
+    the graph replayed `replays` times between two events."""
+    import torch
+    for i in range(3):
+        fn(i % n_bufs)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(calls):
+            fn(i % n_bufs)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (calls * replays)
+
+
 def run_sweep(args):
     """Tables for the cast sweep (sizes x shapes x dtypes x orientations) and the GEMM shape sweep
     (square sizes, the skinny wgrad, the 8B decoder-block GEMMs, with and without the fused MXFP8
@@ -600,17 +622,22 @@ def run_sweep(args):
                     torch.cuda.synchronize()
                     by = rows * cols * (esz + (2 if orient == B.BOTH else 1) * (1 + 1 / 32))
                     gbs = by / ms / 1e6
-                    print("| %s | %d MB | %d x %d | %s | %s | %s | %.1f | %.0f | %.2f | %s |" % (
+                    # the same launches replayed from a CUDA graph: what the kernel takes when the host is not the limit
+                    graph = ""
+                    if nbytes <= (64 << 20):
+                        gms = _time_graph(lambda i: B.mxfp8_quantize(srcs[i], orient, P, elem, *outs, S), n_bufs)
+                        graph = "%.1f us = %.2f" % (gms * 1e3, by / gms / 1e6 / peaks["hbm_gbs"])
+                    print("| %s | %d MB | %d x %d | %s | %s | %s | %.1f | %.0f | %.2f | %s | %s |" % (
                         dtype, nbytes >> 20, rows, cols, kind, oname, "e4m3" if elem == B.E4M3 else "e5m2",
-                        ms * 1e3, gbs, gbs / peaks["hbm_gbs"], "-" if host_us != host_us else "%.1f" % host_us), flush=True)
+                        ms * 1e3, gbs, gbs / peaks["hbm_gbs"], "-" if host_us != host_us else "%.1f" % host_us, graph or "-"), flush=True)
                     del outs
             del srcs
             torch.cuda.empty_cache()
 
         all_o = ((B.ROW, "row"), (B.COL, "col"), (B.BOTH, "both"))
         own_kind = {4096: "gaussian", 14336: "gradient_like", 8288: "student_t"}
-        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call |")
-        print("|---|---|---|---|---|---|---|---|---|---|")
+        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call | from a CUDA graph: us = of copy |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|")
         for dtype, esz in (("bf16", 2), ("fp32", 4)):
             for nbytes in (1 << 20, 4 << 20, 16 << 20, 64 << 20, 256 << 20, 1 << 30, 4 << 30):
                 for cols in (4096, 14336, 8288):
@@ -620,8 +647,8 @@ def run_sweep(args):
         print()
         print("Every distribution on every shape, both element types, 256 MB sources:")
         print()
-        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call |")
-        print("|---|---|---|---|---|---|---|---|---|---|")
+        print("| dtype | source bytes | rows x cols | dist | orient | elem | us | GB/s | of measured copy | host us/call | from a CUDA graph: us = of copy |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|")
         for dtype, esz in (("bf16", 2), ("fp32", 4)):
             for cols in (4096, 14336, 8288):
                 for kind in ("gaussian", "student_t", "gradient_like", "nonfinite"):

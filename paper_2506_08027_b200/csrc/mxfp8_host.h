@@ -31,6 +31,45 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long l
     return err;
 }
 
+// A small integer per (device, stream), handed out on first use and kept: the index of the stream's own words in a
+// device-side array (the conversion kernel's tile counter).  Kernels of one stream run one after the other, so words
+// that belong to a stream are never used by two kernels at once.  Returns -1 when no index can be given safely: the
+// per-thread default stream (one handle, many streams), a stream that is being captured (the captured launch may be
+// replayed on any stream later), more streams than slots.  The caller then takes its path that needs no such words.
+class StreamSlots {
+public:
+    static constexpr int SLOTS = 64;
+    int get(cudaStream_t stream)
+    {
+        if (stream == cudaStreamPerThread) return -1;
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return -1;
+        int device = 0;
+        if (cudaGetDevice(&device) != cudaSuccess) return -1;
+        const int used = __atomic_load_n(&used_, __ATOMIC_ACQUIRE);
+        for (int i = 0; i < used; ++i)
+            if (stream_[i] == stream && device_[i] == device) return i;
+        while (__atomic_exchange_n(&lock_, 1, __ATOMIC_ACQUIRE)) {}
+        int slot = -1;
+        for (int i = 0; i < used_; ++i)
+            if (stream_[i] == stream && device_[i] == device) slot = i;
+        if (slot < 0 && used_ < SLOTS) {
+            slot = used_;
+            stream_[slot] = stream;
+            device_[slot] = device;
+            __atomic_store_n(&used_, used_ + 1, __ATOMIC_RELEASE);
+        }
+        __atomic_store_n(&lock_, 0, __ATOMIC_RELEASE);
+        return slot;
+    }
+
+private:
+    cudaStream_t stream_[SLOTS] = {};
+    int device_[SLOTS] = {};
+    int used_ = 0;
+    int lock_ = 0;
+};
+
 // A value per device that costs driver calls to find (multiprocessor count, the address of a __device__ symbol:
 // every device holds its own copy of each symbol, at its own address).  get() fills the current device's slot on
 // first use, under a lock, and afterwards reads it without one.  `fill(device, value)` returns false on failure,

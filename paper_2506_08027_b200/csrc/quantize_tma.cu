@@ -5,6 +5,7 @@
 namespace mxfp8 {
 
 __device__ int g_quantize_status = 0;   // bounded TMA wait expired (read through mxfp8_device_status)
+__device__ unsigned int g_quantize_sched[2 * StreamSlots::SLOTS];   // tile counters, two words per stream slot, zero between launches
 
 int quantize_read_and_clear_status()
 {
@@ -63,7 +64,7 @@ bool quantize_tma_eligible(int src_dtype, int64_t rows, int64_t cols)
     if (cols % 16) return false;
     const int64_t t_cols = (src_dtype == MXFP8_BF16) ? 128 : 64;
     const int64_t tiles = ((cols + t_cols - 1) / t_cols) * ((rows + T_ROWS - 1) / T_ROWS);
-    return tiles < 0x7FFFFFFFLL && rows < 0x7FFFFFFFLL && cols < 0x7FFFFFFFLL && qt_encode_fn() != nullptr;
+    return tiles < 0x7FFF0000LL && rows < 0x7FFFFFFFLL && cols < 0x7FFFFFFFLL && qt_encode_fn() != nullptr;
 }
 
 int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int orientation, int scale_rule, int elem,
@@ -112,7 +113,7 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
         q.s_col = static_cast<uint8_t*>(it.s_col);
         p.tile_start[i] = (int)tiles;
         tiles += (int64_t)q.tiles_x * q.tiles_y;
-        if (tiles >= 0x7FFFFFFFLL) return MXFP8_ERR_UNSUPPORTED;
+        if (tiles >= 0x7FFF0000LL) return MXFP8_ERR_UNSUPPORTED;   // the tile counter runs a few thousand past the last tile
     }
     for (int i = count; i <= QT_MAX_TENSORS; ++i) p.tile_start[i] = (int)tiles;
     // every device holds its own copy of the status word, at its own address
@@ -124,6 +125,21 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
             return true;
         }))
         return MXFP8_ERR_CUDA;
+    // the tile counter: two words per stream in a per-device array (kernels of one stream never overlap, so the words are
+    // never shared); where no stream-owned words can be had the kernel deals tiles out by CTA index
+    {
+        static StreamSlots slots;
+        static PerDeviceCache<unsigned int*> sched_words;
+        unsigned int* base = nullptr;
+        const int slot = slots.get(stream);
+        if (slot >= 0 && sched_words.get(base, [](int, unsigned int*& addr) {
+                void* ptr = nullptr;
+                if (cudaGetSymbolAddress(&ptr, g_quantize_sched) != cudaSuccess) return false;
+                addr = static_cast<unsigned int*>(ptr);
+                return true;
+            }))
+            p.sched = base + 2 * slot;
+    }
 #ifdef MXFP8_TEST_HOOKS
     if (const char* skip = getenv("MXFP8_TEST_SKIP_TILE")) p.test_skip_tile = atoi(skip);
 #endif

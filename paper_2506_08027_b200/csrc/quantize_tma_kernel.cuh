@@ -184,6 +184,8 @@ __device__ __forceinline__ void glu_slab(uint8_t* gate, const uint8_t* up)
 constexpr int QT_MAX_TENSORS = 8;
 struct QBatch {
     int* status;                          // device status word of the library (bounded waits report here)
+    unsigned int* sched;                  // two words owned by the launch's stream, both zero between launches: [0] the next tile to
+                                          //   hand out, [1] CTAs that have left; null: tiles are dealt out by CTA index instead
     int test_skip_tile;                   // test builds only: 1 + index of the tile whose load is left out (0 = none)
     int act;                              // MXFP8_ACT_*: applied to every element before the conversion
     const float* rstd;                    // RMS normalisation ahead of the conversion (first tensor only): 1/rms per row,
@@ -586,15 +588,42 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         }
         return ok != 0;
     };
-    int tile = blockIdx.x, ti = 0;
+    // Tiles are handed out in order, one at a time (an atomic counter), as ring slots fall free: whatever the CTAs' relative
+    // speed, the tiles in flight stay a compact window of the row-major order, i.e. a few hundred long DRAM rows that all
+    // SMs read and write together.  Dealt out by CTA index (tile += gridDim.x) the window widens as soon as the kernel is
+    // memory-bound and CTAs drift apart, and the same bytes then move 15 % slower.  Without a counter (batch.sched null)
+    // the fixed order serves.
+    int* slot_tile = reinterpret_cast<int*>(bars + 8);       // the tile held by (or on its way into) each ring slot
+    auto next_tile = [&](int after) {                        // one thread
+        return batch.sched ? (int)atomicAdd(batch.sched, 1u) : after + (int)gridDim.x;
+    };
+    auto leave = [&]() {                                     // one thread, once: the last CTA out zeroes the words for the next launch
+        if (batch.sched == nullptr) return;
+        __threadfence();
+        if (atomicAdd(batch.sched + 1, 1u) == gridDim.x - 1) {
+            batch.sched[0] = 0u;
+            batch.sched[1] = 0u;
+        }
+    };
+    int tile = 0, ti = 0;
     if (tid == 0) {
-        for (int k = 0; k < RING; ++k)
-            if (tile + k * (int)gridDim.x < num_tiles) issue_load(tile + k * gridDim.x, k);
-        if (GLU && tile < num_tiles) issue_up(tile);
+        int t = (int)blockIdx.x - (int)gridDim.x;
+        for (int k = 0; k < RING; ++k) {
+            t = next_tile(t);
+            slot_tile[k] = t;
+            if (t < num_tiles) issue_load(t, k);
+        }
+        if (GLU && slot_tile[0] < num_tiles) issue_up(slot_tile[0]);
     }
-
-    for (int it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
+    __syncthreads();
+    for (int it = 0;; ++it) {
         const int buf = it % RING;
+        tile = slot_tile[buf];
+        if (tile >= num_tiles) break;
+        // the tile that will refill this slot: asked for now, needed after the slab (the counter's round trip hides under it);
+        // by CTA index it is RING strides on
+        int refill = 0;
+        if (tid == 0) refill = next_tile(batch.sched ? 0 : tile + (RING - 1) * (int)gridDim.x);
         const uint32_t phase = (uint32_t)(it / RING) & 1u;
         const uint32_t bar_a = smem_addr(&bars[buf]);
         uint8_t* in_tile = in_ring + buf * IN_BYTES;
@@ -611,7 +640,10 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
             bool ok = wait_bar(bar_a, phase);
             if constexpr (GLU) ok = wait_bar(smem_addr(&bars[RING]), (uint32_t)it & 1u) && ok;
             if (!__syncthreads_and((int)ok)) {
-                if (tid == 0) atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
+                if (tid == 0) {
+                    atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
+                    leave();
+                }
                 return;
             }
         }
@@ -633,7 +665,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncthreads();                     // every warp has consumed the up tile: fetch the next one under the conversion
-            if (tid == 0 && tile + (int)gridDim.x < num_tiles) issue_up(tile + gridDim.x);
+            if (tid == 0 && slot_tile[(it + 1) % RING] < num_tiles) issue_up(slot_tile[(it + 1) % RING]);
         }
         if (PRO == PRO_ELEMENTWISE && batch.rstd != nullptr) {
             // RMS normalisation in place (single-tensor launches only), then the unchanged conversion
@@ -683,8 +715,8 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         // every warp is done with this ring slot: refill it with the tile after next
         __syncthreads();
         if (tid == 0) {
-            const int next = tile + RING * (int)gridDim.x;
-            if (next < num_tiles) issue_load(next, buf);
+            slot_tile[buf] = refill;
+            if (refill < num_tiles) issue_load(refill, buf);
         }
 
         // ---- scale bytes (1/32 of the output) leave from the staging arrays ----------
@@ -739,6 +771,7 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
             }
         }
     }
+    if (tid == 0) leave();
 }
 
 // Multiprocessors of the current device (looked up once per device)
