@@ -35,7 +35,8 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long l
 // device-side array (the conversion kernel's tile counter).  Kernels of one stream run one after the other, so words
 // that belong to a stream are never used by two kernels at once.  Returns -1 when no index can be given safely: the
 // per-thread default stream (one handle, many streams), a stream that is being captured (the captured launch may be
-// replayed on any stream later), more streams than slots.  The caller then takes its path that needs no such words.
+// replayed on any stream later, or next to a second instance of its graph), more streams than slots, a failing
+// runtime call.  The caller then takes its path that needs no such words.
 class StreamSlots {
 public:
     static constexpr int SLOTS = 64;

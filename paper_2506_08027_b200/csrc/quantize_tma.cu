@@ -126,8 +126,10 @@ int quantize_tma_batch(const QuantizeItem* items, int count, int src_dtype, int 
         }))
         return MXFP8_ERR_CUDA;
     // the tile counter: two words per stream in a per-device array (kernels of one stream never overlap, so the words are
-    // never shared); where no stream-owned words can be had the kernel deals tiles out by CTA index
-    {
+    // never shared); where no stream-owned words can be had (a launch being captured, too many streams) the kernel deals
+    // tiles out by CTA index
+    // (a launch of a few tiles per CTA has nothing to gain from it and keeps the runtime calls of the lookup off its host path)
+    if (tiles > 4 * (int64_t)QT_CTAS_PER_SM * qt_sm_count()) {
         static StreamSlots slots;
         static PerDeviceCache<unsigned int*> sched_words;
         unsigned int* base = nullptr;

@@ -346,40 +346,40 @@ def test_more_than_2_to_31_elements_sampled():
 
 
 def test_conversions_on_many_streams_at_once():
-    """The conversion kernel hands its tiles out through a counter that belongs to the launch's stream.  Launches
-    that overlap on different streams must not disturb one another, a second launch on a stream must find the
-    counter as the first one left it, and streams beyond the number of counters (64) take the fixed tile order:
+    """A conversion of many tiles per CTA hands its tiles out through a counter that belongs to the launch's stream.
+    Launches that overlap on different streams must not disturb one another, a second launch on a stream must find
+    the counter as the first one left it, and streams beyond the number of counters (64) take the fixed tile order:
     the bytes are those of the oracle in every case."""
     import torch
     from paper_2506_08027_b200 import binding as B
+    from helpers import logical_scales_from_swizzled
     S = B.SF_SWIZZLED
-    shapes = [(1024, 2048), (640, 1024 + 128), (2048, 512)]
+    thr = os.cpu_count() or 1
+    shapes = [(4096, 8192), (2048 + 32, 16384 + 128)]        # 2048 and 2193 tiles of 128 x 128: more than 4 per CTA
     srcs, wants = [], []
     for k, shape in enumerate(shapes):
         bits = synth.f32_to_bf16_bits(synth.gaussian(shape, 400 + k))
         srcs.append(torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16))
         x = orc.bf16_bits_to_f32(bits)
-        wants.append((orc.quantize(x, orc.ROW), orc.quantize(x, orc.COL)))
+        wants.append((orc.quantize_threads(x, orc.ROW, orc.RULE_PAPER, orc.E4M3, thr),
+                      orc.quantize_threads(x, orc.COL, orc.RULE_PAPER, orc.E4M3, thr)))
     streams = [torch.cuda.Stream() for _ in range(70)]
-    outs = [[B.alloc_quantize_outputs(*shapes[k % 3], B.BOTH, S) for k in range(len(streams))] for _ in range(2)]
+    outs = [[B.alloc_quantize_outputs(*shapes[k % 2], B.BOTH, S) for k in range(len(streams))] for _ in range(2)]
     torch.cuda.synchronize()
     for rep in range(2):                                   # the second round reuses every stream's counter
         for k, st in enumerate(streams):
             with torch.cuda.stream(st):
-                B.mxfp8_quantize(srcs[k % 3], B.BOTH, B.RULE_PAPER, B.E4M3, *outs[rep][k], S)
+                B.mxfp8_quantize(srcs[k % 2], B.BOTH, B.RULE_PAPER, B.E4M3, *outs[rep][k], S)
     torch.cuda.synchronize()
     assert B.mxfp8_device_status() == 0
     for rep in range(2):
         for k in range(len(streams)):
-            (wq_r, ws_r), (wq_c, ws_c) = wants[k % 3]
+            (wq_r, ws_r), (wq_c, ws_c) = wants[k % 2]
+            rows, cols = shapes[k % 2]
             q_row, s_row, q_col, s_col = outs[rep][k]
             assert np.array_equal(q_row.cpu().numpy(), wq_r), "row bytes, stream %d" % k
             assert np.array_equal(q_col.cpu().numpy(), wq_c), "column bytes, stream %d" % k
-    # scale bytes once per shape (gathered out of the swizzled layout)
-    from helpers import logical_scales_from_swizzled
-    for k in range(3):
-        (wq_r, ws_r), (wq_c, ws_c) = wants[k]
-        rows, cols = shapes[k]
-        got_r = logical_scales_from_swizzled(outs[1][k][1].cpu().numpy(), rows, cols // 32)
-        got_c = logical_scales_from_swizzled(outs[1][k][3].cpu().numpy(), cols, rows // 32)
-        assert np.array_equal(got_r, ws_r) and np.array_equal(got_c.T, ws_c)
+            if k < 2 or k >= 68:
+                got_r = logical_scales_from_swizzled(s_row.cpu().numpy(), rows, cols // 32)
+                got_c = logical_scales_from_swizzled(s_col.cpu().numpy(), cols, rows // 32)
+                assert np.array_equal(got_r, ws_r) and np.array_equal(got_c.T, ws_c), "scale bytes, stream %d" % k
