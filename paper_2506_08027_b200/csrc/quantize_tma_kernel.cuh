@@ -635,18 +635,23 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         divmod((uint32_t)(tile - batch.tile_start[ti]), (uint32_t)p.tiles_x, p.tiles_x_magic, tile_y, tile_x);
         const int64_t gcol0 = (int64_t)tile_x * T_COLS, grow0 = (int64_t)tile_y * T_ROWS;
 
-        // wait for the tile (bounded: on expiry report through the status word and leave)
-        {
-            bool ok = wait_bar(bar_a, phase);
-            if constexpr (GLU) ok = wait_bar(smem_addr(&bars[RING]), (uint32_t)it & 1u) && ok;
-            if (!__syncthreads_and((int)ok)) {
-                if (tid == 0) {
-                    atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
-                    leave();
-                }
-                return;
+        // wait for the tile (bounded: on expiry report through the status word and leave).  A warp needs nothing from the
+        // other warps to start on its slab, so the CTA meets only once per tile, at the barrier that frees the ring slot:
+        // a warp whose wait ran out skips the tile and says so there.  (The gated mode meets in between for the up tile,
+        // so it settles the outcome of the wait first.)
+        bool ok = wait_bar(bar_a, phase);
+        if constexpr (GLU) ok = wait_bar(smem_addr(&bars[RING]), (uint32_t)it & 1u) && ok;
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        auto give_up = [&]() {
+            if (tid == 0) {
+                atomicExch(batch.status, (int)MXFP8_ERR_DEVICE_TIMEOUT);
+                leave();
             }
+        };
+        if constexpr (GLU) {
+            if (!__syncthreads_and((int)ok)) { give_up(); return; }
         }
+        if (ok) {
         if constexpr (GLU) {
             // gated activation: the slot holds the gate tile, up_buf the up tile; the slot becomes act(gate) * up
             uint8_t* mine = in_tile + warp * 32 * T_BYTES + lane * 8;
@@ -711,9 +716,10 @@ quantize_tma_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ 
         if (special && rows_here > 0)
             slab_careful<DTYPE, ELEM, DO_ROW, DO_COL, EMU>(my_in, my_qrow, my_qcol, pitch, my_sm_row, my_sm_col, lane, rule_offset,
                                                        rows_here, col_ok);
+        }
 
         // every warp is done with this ring slot: refill it with the tile after next
-        __syncthreads();
+        if (__syncthreads_or((int)!ok)) { give_up(); return; }
         if (tid == 0) {
             slot_tile[buf] = refill;
             if (refill < num_tiles) issue_load(refill, buf);
