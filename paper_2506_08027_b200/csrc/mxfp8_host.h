@@ -31,6 +31,22 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long l
     return err;
 }
 
+// n / d and n % d for 0 <= n < 2^31, 1 <= d, without a division on the device: a multiply by
+// magic = min(floor(2^32 / d), 2^32 - 1) gives the quotient or one less, one correction settles it.
+// (The conversion kernel turns a tile index into tile coordinates with it; the host computes the magic.)
+inline __host__ __device__ uint32_t div_magic(uint32_t d) { return d <= 1u ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / d); }
+inline __host__ __device__ void divmod(uint32_t n, uint32_t d, uint32_t magic, int& q, int& r)
+{
+#ifdef __CUDA_ARCH__
+    uint32_t qq = __umulhi(n, magic);
+#else
+    uint32_t qq = (uint32_t)(((uint64_t)n * magic) >> 32);
+#endif
+    uint32_t rr = n - qq * d;
+    if (rr >= d) { rr -= d; ++qq; }
+    q = (int)qq; r = (int)rr;
+}
+
 // A small integer per (device, stream), handed out on first use and kept: the index of the stream's own words in a
 // device-side array (the conversion kernel's tile counter).  Kernels of one stream run one after the other, so words
 // that belong to a stream are never used by two kernels at once.  Returns -1 when no index can be given safely: the

@@ -239,16 +239,6 @@ __device__ __forceinline__ uint32_t inv_exp_field2(uint32_t z, uint32_t rule_off
     return __vminu2((254u + ElemTraits<ELEM>::emax) * 0x00010001u - e2, 0x00FE00FEu);
 }
 
-// n / d and n % d for 0 <= n < 2^31, 1 <= d: a multiply by magic = min(floor(2^32 / d), 2^32 - 1) gives the
-// quotient or one less, one correction settles it.
-__host__ __device__ __forceinline__ uint32_t div_magic(uint32_t d) { return d <= 1u ? 0xFFFFFFFFu : (uint32_t)(0x100000000ull / d); }
-__device__ __forceinline__ void divmod(uint32_t n, uint32_t d, uint32_t magic, int& q, int& r)
-{
-    uint32_t qq = __umulhi(n, magic), rr = n - qq * d;
-    if (rr >= d) { rr -= d; ++qq; }
-    q = (int)qq; r = (int)rr;
-}
-
 // X = 2^(b-127) as FP32 from the exponent field of 1/X (b = 254 - field; b = 0 is the subnormal 2^-127)
 __device__ __forceinline__ float scale_from_inv(float inv)
 {

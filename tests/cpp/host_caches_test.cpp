@@ -1,5 +1,5 @@
-// Host-logic check of the two caches in csrc/mxfp8_host.h, with the device index given explicitly
-// (no GPU is touched): a value per device, filled once per device; tensor maps keyed by their arguments.
+// Host-logic check of csrc/mxfp8_host.h (no GPU is touched): a value per device, filled once per device, with the
+// device index given explicitly; tensor maps keyed by their arguments; division by a precomputed multiplier.
 #include <cstdio>
 #include <cstring>
 
@@ -54,6 +54,29 @@ int main()
     auto refuse = [&](FakeMap*) { return false; };
     check(!maps.get(tensor_map_key(buf_a, 7, 2, d1, s1, b1, 3, 2), &m, refuse), "a failed encode is reported");
     check(maps.get(tensor_map_key(buf_a, 7, 2, d1, s1, b1, 3, 2), &m, encode) && encodes == 5, "and not cached");
+
+    // ---- division by multiplication: every divisor a tile grid can have against tile indices around its multiples,
+    // around powers of two and at the top of the range
+    {
+        long bad = 0;
+        auto one = [&](uint32_t n, uint32_t d) {
+            int q = -1, r = -1;
+            divmod(n, d, div_magic(d), q, r);
+            if ((uint32_t)q != n / d || (uint32_t)r != n % d) ++bad;
+        };
+        for (uint32_t d = 1; d <= 70000; d += (d < 3000 ? 1 : 37)) {
+            for (uint32_t k = 0; k < 40; ++k) {
+                const uint64_t m = (uint64_t)d * (k * 53ull + (k > 30 ? 1000003ull * k : 0ull));
+                for (int off = -2; off <= 2; ++off) {
+                    const int64_t n = (int64_t)m + off;
+                    if (n >= 0 && n < 0x7FFFFFFFll) one((uint32_t)n, d);
+                }
+            }
+            for (int sh = 0; sh < 31; ++sh) { one((1u << sh) - 1u, d); one(1u << sh, d); one((1u << sh) + 1u, d); }
+            one(0x7FFEFFFFu, d); one(0x7FFFFFFEu, d);
+        }
+        check(bad == 0, "quotient and remainder by multiplication equal the division");
+    }
 
     std::printf(fails ? "%d checks failed\n" : "all checks passed\n", fails);
     return fails ? 1 : 0;
