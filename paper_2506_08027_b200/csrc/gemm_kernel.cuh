@@ -62,7 +62,11 @@ template <bool EPI, int MODE> struct Roles {
 #endif
     static constexpr int THREADS = WIDE ? 384 : GEMM_THREADS;
     static constexpr int EPI_WARP0 = WIDE ? 4 : 2;      // first of the eight epilogue warps
+    // 128 threads x 104 + 256 threads x 200 = 64 512 of the SM's 65 536 registers.  The split has to leave slack: the
+    // launch allocates 168 per thread, the first group's decrease frees 128 x 64, the epilogue warps then ask for
+    // 256 x 32, and a split that adds up to all 65 536 (112 / 200) left `setmaxnreg.inc` waiting for ever.
     static constexpr int REGS_FEW = 104, REGS_MANY = 200;
+    static_assert(128 * REGS_FEW + 256 * REGS_MANY <= 65536 - 1024, "register split without slack");
 };
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 2048;   // 32 rows x 64 bytes per epilogue warp

@@ -104,3 +104,37 @@ def test_conversion_wait_runs_out_once_and_the_next_conversion_is_right(hooks, m
     wq, ws = orc.quantize(orc.bf16_bits_to_f32(bits), orc.ROW)
     assert np.array_equal(q.cpu().numpy(), wq)
     assert np.array_equal(s.cpu().numpy().reshape(rows, cols // 32), ws)
+
+
+def test_conversion_wait_runs_out_with_the_tile_counter_in_use(hooks, monkeypatch):
+    """The same on a tensor large enough for tiles to be handed out through the stream's counter (more than four per
+    CTA): the CTA whose load is left out gives up, the others finish, the last one out leaves the counter at zero,
+    and the next conversion on the same stream is right."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    H = hooks
+    rows, cols = 4096, 8192                   # 2048 tiles of 128 x 128
+    bits = synth.f32_to_bf16_bits(synth.gaussian((rows, cols), 23))
+    src = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    q = torch.zeros((rows, cols), dtype=torch.uint8, device="cuda")
+    s = torch.zeros(B.mxfp8_scale_bytes(rows, cols, B.ROW, B.SF_LINEAR), dtype=torch.uint8, device="cuda")
+
+    def convert():
+        rc = H.mxfp8_quantize(src.data_ptr(), B.BF16, rows, cols, B.ROW, B.RULE_PAPER, B.E4M3, q.data_ptr(), s.data_ptr(),
+                              None, None, B.SF_LINEAR, None)
+        assert rc == 0
+
+    convert()                                                   # a clean run first: the counter is back at zero after it
+    assert H.mxfp8_device_status(None) == 0
+    monkeypatch.setenv("MXFP8_TEST_SKIP_TILE", "700")           # whichever CTA is handed tile 699 never gets its data
+    convert()
+    assert H.mxfp8_device_status(None) == TIMEOUT
+    assert H.mxfp8_device_status(None) == 0
+    monkeypatch.delenv("MXFP8_TEST_SKIP_TILE")
+    for _ in range(2):
+        q.zero_(); s.zero_()
+        convert()
+        assert H.mxfp8_device_status(None) == 0
+    wq, ws = orc.quantize_threads(orc.bf16_bits_to_f32(bits), orc.ROW, orc.RULE_PAPER, orc.E4M3, os.cpu_count() or 1)
+    assert np.array_equal(q.cpu().numpy(), wq)
+    assert np.array_equal(s.cpu().numpy().reshape(rows, cols // 32), ws)
