@@ -12,6 +12,11 @@
  *     every buffer; the library never allocates, frees or keeps a pointer after returning.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
  *     stream).  Nothing synchronises except mxfp8_device_status() and the *_host calls.
+ *     Calls may be made from several host threads and on several streams at once.  The
+ *     conversion kernels keep a few words of device state per stream (the first 64 streams
+ *     of a device that convert large tensors; later ones, the per-thread default stream and
+ *     launches inside a stream capture work without it, a little slower on tensors of
+ *     hundreds of megabytes); nothing a caller has to manage.
  *   - Return value: MXFP8_OK or a negative mxfp8_status.  Nothing is printed, nothing aborts.
  *   - Tensors are row-major.  A block is K = 32 consecutive elements (Sec. 2) along a row
  *     (MXFP8_ROW) or down a column (MXFP8_COL).  Quantized data keeps the shape and the
