@@ -335,6 +335,19 @@ def run_ours(args):
     steady_clock_mhz, _ = B.mxfp8_gemm_last_clock()
     cast_ms = statistics.median(s_cast)
     gemm_multi_ms = statistics.median(s_gemm)
+    # ---- the yardstick in the same place: a plain device-to-device copy that moves as many bytes as the cast does
+    # (half of them read, half written), launched where the cast is, in the same power state.  The measured copy rate of
+    # MEASURED_PEAKS.json is taken alone at the boost clock; behind the GEMM launch the memory system's clients run at
+    # the clock the power cap leaves, and this says how much of the cast's distance to that peak is the place it runs in.
+    copy_src = torch.empty(int(CAST_BYTES) // 2, dtype=torch.uint8, device=dev)
+    copy_dst = torch.empty_like(copy_src)
+    cev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(PASSES_PER_STEP)]
+    for k in range(PASSES_PER_STEP):
+        cev[k][0].record(); copy_dst.copy_(copy_src)
+        cev[k][1].record(); B.mxfp8_gemm_multi(gemms, B.BF16)
+    torch.cuda.synchronize()
+    copy_in_pass_ms = statistics.median(e[0].elapsed_time(e[1]) for e in cev)
+    del copy_src, copy_dst
     # ---- timed region 3: the three GEMMs launched one by one (per-product breakdown)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(PASSES_PER_STEP)]
     for k in range(PASSES_PER_STEP):
@@ -446,6 +459,10 @@ def run_ours(args):
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cast_gbs / peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "algorithmic_bytes_per_element": 4.0625,
                           "algorithmic_bytes_per_launch": CAST_BYTES, "frac_burst": gbs(b_cast_ms) / peaks["hbm_gbs"],
+                          "copy_of_the_same_bytes_in_the_pass_gbs": gbs(copy_in_pass_ms),
+                          "frac_of_that_copy": cast_gbs / gbs(copy_in_pass_ms),
+                          "copy_note": "a plain device-to-device copy of CAST_BYTES / 2 (read + written = the cast's bytes) launched in the cast's "
+                                       "place, between the GEMM launches of the steady state; torch's copy_, a yardstick, not part of the path",
                           "traffic": NCU_TRAFFIC_QUANTIZE_STEP,
                           "traffic_note": "ncu capture of this launch (X, W, dY in one), see profiles/"},
         "e2e": e2e, "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
