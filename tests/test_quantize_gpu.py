@@ -383,3 +383,55 @@ def test_conversions_on_many_streams_at_once():
                 got_r = logical_scales_from_swizzled(s_row.cpu().numpy(), rows, cols // 32)
                 got_c = logical_scales_from_swizzled(s_col.cpu().numpy(), cols, rows // 32)
                 assert np.array_equal(got_r, ws_r) and np.array_equal(got_c.T, ws_c), "scale bytes, stream %d" % k
+
+
+@pytest.mark.parametrize("dtype,elem,rule", [("bf16", orc.E5M2, orc.RULE_OCP), ("fp32", orc.E4M3, orc.RULE_PAPER)])
+def test_large_ragged_tensor_with_tiles_handed_out_by_the_counter(dtype, elem, rule):
+    """More than four tiles per CTA (the stream's tile counter is in use), the last tile of every row and the last
+    row of tiles ragged, linear scale layout (the per-row / per-column store path): bytes equal to the oracle's."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    rows, cols = 4096 + 32, (8192 + 32 if dtype == "bf16" else 4096 + 32)      # 33 x 65 tiles, the last of each ragged
+    thr = os.cpu_count() or 1
+    x32 = synth.gaussian((rows, cols), 77)
+    src_np = as_dtype(x32, dtype)
+    x = orc.bf16_bits_to_f32(src_np) if dtype == "bf16" else src_np
+    src = (torch.from_numpy(src_np.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(src_np).cuda())
+    q_row, s_row, _, _ = B.alloc_quantize_outputs(rows, cols, B.ROW, B.SF_LINEAR)
+    B.mxfp8_quantize(src, B.ROW, rule, elem, q_row, s_row, None, None, B.SF_LINEAR)
+    _, _, q_col, s_col = B.alloc_quantize_outputs(rows, cols, B.COL, B.SF_LINEAR)
+    B.mxfp8_quantize(src, B.COL, rule, elem, None, None, q_col, s_col, B.SF_LINEAR)
+    assert B.mxfp8_device_status() == 0
+    wq, ws = orc.quantize_threads(x, orc.ROW, rule, elem, thr)
+    assert_q_equal(q_row.cpu().numpy(), wq, elem, "row")
+    assert np.array_equal(s_row.cpu().numpy().reshape(rows, cols // 32), ws)
+    wq, ws = orc.quantize_threads(x, orc.COL, rule, elem, thr)
+    assert_q_equal(q_col.cpu().numpy(), wq, elem, "col")
+    assert np.array_equal(s_col.cpu().numpy().reshape(rows // 32, cols), ws)
+
+
+def test_conversion_captured_in_a_graph_equals_the_eager_one():
+    """A launch that is being captured cannot own a stream's tile counter and takes the fixed tile order: the replayed
+    graph must give the bytes of the eager call (which, at this size, uses the counter)."""
+    import torch
+    from paper_2506_08027_b200 import binding as B
+    S = B.SF_SWIZZLED
+    rows, cols = 4096, 8192
+    bits = synth.f32_to_bf16_bits(synth.gaussian((rows, cols), 91))
+    src = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    eager = B.alloc_quantize_outputs(rows, cols, B.BOTH, S)
+    graph = B.alloc_quantize_outputs(rows, cols, B.BOTH, S)
+    B.mxfp8_quantize(src, B.BOTH, B.RULE_PAPER, B.E4M3, *eager, S)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        B.mxfp8_quantize(src, B.BOTH, B.RULE_PAPER, B.E4M3, *graph, S)
+    for t in graph:
+        t.zero_()
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
+    for a, b in zip(eager, graph):
+        assert torch.equal(a, b)
+    wq, _ = orc.quantize_threads(orc.bf16_bits_to_f32(bits), orc.ROW, orc.RULE_PAPER, orc.E4M3, os.cpu_count() or 1)
+    assert np.array_equal(eager[0].cpu().numpy(), wq)
