@@ -104,19 +104,21 @@ def test_transcendental_gradients_match_up_to_rounding_boundaries(act, dtype):
         assert np.sqrt(((d_gpu - y) ** 2).sum()) <= 1.001 * np.sqrt(((d_orc - y) ** 2).sum())
 
 
-def test_equals_separate_gradient_then_quantize_on_device():
+@pytest.mark.parametrize("shape", [(1024, 2048), (8192, 4096 + 128)])   # the second: tiles handed out by the stream's counter, ragged last tile
+def test_equals_separate_gradient_then_quantize_on_device(shape):
     import torch
     from paper_2506_08027_b200 import binding as B
-    z = synth.device_tensor("activation", (1024, 2048), 9)
-    dh = synth.device_tensor("output_gradient", (1024, 2048), 10)
+    z = synth.device_tensor("activation", shape, 9)
+    dh = synth.device_tensor("output_gradient", shape, 10)
     y = (torch.where(z.float() > 0, 2.0 * z.float(), torch.zeros((), device="cuda")) * dh.float()).to(torch.bfloat16)
-    a = B.alloc_quantize_outputs(1024, 2048, B.BOTH, B.SF_SWIZZLED)
-    b = B.alloc_quantize_outputs(1024, 2048, B.BOTH, B.SF_SWIZZLED)
+    a = B.alloc_quantize_outputs(*shape, B.BOTH, B.SF_SWIZZLED)
+    b = B.alloc_quantize_outputs(*shape, B.BOTH, B.SF_SWIZZLED)
     for t in a + b:
         t.zero_()
     B.mxfp8_act_grad_quantize(dh, z, B.ACT_RELU2, B.BOTH, B.RULE_PAPER, B.E4M3, *a, B.SF_SWIZZLED)
     B.mxfp8_quantize(y, B.BOTH, B.RULE_PAPER, B.E4M3, *b, B.SF_SWIZZLED)
     torch.cuda.synchronize()
+    assert B.mxfp8_device_status() == 0
     for u, v in zip(a, b):
         assert torch.equal(u, v)
 

@@ -105,14 +105,15 @@ def test_transcendental_activations_match_up_to_rounding_boundaries(act, dtype):
         assert err_gpu <= 1.001 * err_orc
 
 
-def test_equals_separate_activation_then_quantize_on_device():
+@pytest.mark.parametrize("shape", [(1024, 2048), (8192, 4096 + 128)])   # the second: tiles handed out by the stream's counter, ragged last tile
+def test_equals_separate_activation_then_quantize_on_device(shape):
     # the fused call against mxfp8_quantize applied to a tensor that holds relu(x)^2 (computed by torch in FP32)
     import torch
     from paper_2506_08027_b200 import binding as B
-    x = synth.device_tensor("activation", (1024, 2048), 9)
+    x = synth.device_tensor("activation", shape, 9)
     y = (torch.relu(x.float()) ** 2).to(torch.bfloat16)
-    a = B.alloc_quantize_outputs(1024, 2048, B.BOTH, B.SF_SWIZZLED)
-    b = B.alloc_quantize_outputs(1024, 2048, B.BOTH, B.SF_SWIZZLED)
+    a = B.alloc_quantize_outputs(*shape, B.BOTH, B.SF_SWIZZLED)
+    b = B.alloc_quantize_outputs(*shape, B.BOTH, B.SF_SWIZZLED)
     for t in a + b:
         t.zero_()
     B.mxfp8_act_quantize(x, B.ACT_RELU2, B.BOTH, B.RULE_PAPER, B.E4M3, *a, B.SF_SWIZZLED)
