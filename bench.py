@@ -523,6 +523,22 @@ def run_case(args):
         off_d = torch.from_numpy(offs).cuda()
         for _ in range(reps):
             B.mxfp8_grouped_gemm(qx[0], qx[1], qw[0], qw[1], off_d, B.GROUP_M, Tt, Fe, Hd, B.K_MAJOR, E, E, yg)
+    elif args.case == "grouped_wgrad":
+        # per-expert wgrad of the same layer: dW_g = dY_g^T X_g over the expert's tokens (both operands token-major)
+        import numpy as np
+        Hd, Fe, G = 2048, 1408, 64
+        rng = np.random.default_rng(2506)
+        padded = (rng.multinomial(8192 * 6, np.full(G, 1.0 / G)) + 127) // 128 * 128
+        offs = np.concatenate([[0], np.cumsum(padded)]).astype(np.int32)
+        Tt = int(offs[-1])
+        xa = synth.device_tensor("activation", (Tt, Hd), 21)
+        dya = synth.device_tensor("output_gradient", (Tt, Fe), 22)
+        qx = B.alloc_quantize_outputs(Tt, Hd, B.COL, S); B.mxfp8_quantize(xa, B.COL, P, E, *qx, S)
+        qdy = B.alloc_quantize_outputs(Tt, Fe, B.COL, S); B.mxfp8_quantize(dya, B.COL, P, E, *qdy, S)
+        dwg = torch.empty((G * Fe, Hd), dtype=torch.bfloat16, device="cuda")
+        off_d = torch.from_numpy(offs).cuda()
+        for _ in range(reps):
+            B.mxfp8_grouped_gemm(qdy[2], qdy[3], qx[2], qx[3], off_d, B.GROUP_K, Fe, Hd, Tt, B.MN_MAJOR, E, E, dwg)
     elif args.case == "scatter":
         # the WGRAD product of the benchmark layer, its FP32 result added into 8 owner buffers (all on this device)
         xs = synth.device_tensor("activation", (T, H), 2)
@@ -910,7 +926,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "glu", "scatter"],
+    ap.add_argument("--case", default=None, choices=["quantize", "dequantize", "fake_quantize", "gemm", "gemm8k", "gemm_fused", "step", "grouped", "grouped_wgrad", "glu", "scatter"],
                     help="run one kernel on one small case and exit (for profiler captures)")
     ap.add_argument("--sweep", default=None, choices=["cast", "gemm", "emu", "moe", "dp", "rules"],
                     help="print the cast-bandwidth, GEMM-shape or round-trip (emu) sweep as a markdown table and exit")
